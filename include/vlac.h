@@ -1,0 +1,185 @@
+/*
+ * vlac.h -- C ABI of the VLA-Cache control-step library (CUDA, sm_100a).
+ *
+ * One control step of a vision-language-action decoder with cross-frame K/V reuse
+ * (VLA-Cache, arxiv 2502.02175): choose which vision tokens may keep last step's K/V
+ * (Algorithm 1 and Sec. 3.4), run every decoder layer over the remaining positions only
+ * (Algorithm 2, Sec. 4.1, Appendix "Inference Detail"), then generate the action tokens.
+ *
+ * General conventions
+ *   - Every pointer named "device" is a raw CUDA device pointer on the current device; "host"
+ *     pointers are ordinary host memory.  The library never takes ownership of caller memory.
+ *   - Work is enqueued on the CUDA stream passed as `void* stream` (a cudaStream_t; NULL is the
+ *     default stream).  Results are valid once the caller has synchronised that stream.
+ *   - Every call returns VLAC_OK (0) or a negative VLAC_ERR_* code; nothing throws or aborts.
+ *   - A context serves one call at a time; calls on the same context must be stream-ordered.
+ *   - The sequence is [n_text_pre text][n_cams*grid*grid vision][n_text_post text]; position p of
+ *     sequence b is row b*L+p of a [batch][L][hidden] buffer.  Vision token v (camera c, block
+ *     row i, block column j: v = c*grid*grid + i*grid + j) sits at position n_text_pre + v.
+ *   - bf16 means the upper 16 bits of an IEEE fp32.
+ */
+#ifndef VLAC_H_
+#define VLAC_H_
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define VLAC_OK                0
+#define VLAC_ERR_INVALID_ARG  -1
+#define VLAC_ERR_BAD_STATE    -2
+#define VLAC_ERR_OOM          -3
+#define VLAC_ERR_CUDA         -4
+#define VLAC_ERR_TIMEOUT      -5
+
+#define VLAC_MAX_LAYERS 64
+
+typedef struct vlac_ctx   vlac_ctx;    /* configuration, borrowed weight pointers, workspace         */
+typedef struct vlac_cache vlac_cache;  /* per-sequence K/V, previous frame, saved attention, selection */
+
+/* Decoder and sequence shape.  n_kv_heads must equal n_heads; head_dim must be a multiple of 32
+ * and at most 128, hidden and ffn multiples of 8; n_layers <= VLAC_MAX_LAYERS; patch*3 even. */
+typedef struct {
+  int n_layers, hidden, n_heads, n_kv_heads, head_dim, ffn, vocab;
+  int n_cams, grid, patch;            /* L_v = n_cams*grid*grid; a frame is (grid*patch)^2 RGB8 */
+  int n_text_pre, n_text_post;
+  int n_action;                       /* action tokens generated per step (the paper uses 7)    */
+  float rms_eps, rope_theta;          /* rope_theta is informational: the tables are inputs      */
+  int max_batch;
+} vlac_config;
+
+/* One layer's weights: device bf16, row-major [out_features][in_features]; gains [hidden]. */
+typedef struct {
+  const void *wq, *wk, *wv, *wo, *w_gate, *w_up, *w_down, *g_attn, *g_mlp;
+} vlac_layer_w;
+
+/* Whole model.  `layers` is a HOST array of n_layers structs (copied at create); all other
+ * pointers are device memory that must outlive the context.  rope_cos/rope_sin are fp32
+ * [L + n_action - 1][head_dim/2]: cos/sin(pos * theta^(-2i/head_dim)), rotate-half pairing. */
+typedef struct {
+  const vlac_layer_w* layers;
+  const void *embed;      /* bf16 [vocab][hidden]            */
+  const void *proj;       /* bf16 [hidden][hidden], vision feature projector */
+  const void *g_final;    /* bf16 [hidden]                   */
+  const void *lm_head;    /* bf16 [vocab][hidden]            */
+  const float *rope_cos, *rope_sin;
+} vlac_weights;
+
+/* Hyper-parameters of Algorithm 1 and Eq. (reuse_ratio).  Paper defaults (Appendix
+ * "Experimental Settings"): tau 0.996, top_k 100, tau_task 0.5.
+ *   task_mode 0: tau_task is a rank fraction -- the L_v - floor(tau_task*L_v) tokens with the
+ *                highest task-relevance score are recomputed;  1: the printed test S >= tau_task.
+ *   k_ent:       the k of Eq. (reuse_ratio) (the paper gives no value).
+ *   alpha_override: HOST pointer to n_layers doubles replacing the entropy-derived ratios, or NULL.
+ *   layer_mask:  bit l set = layer l enters the task-relevance mean (Sec. 3.3 "selected layers");
+ *                0 means all layers. */
+typedef struct {
+  double tau;
+  int    top_k;
+  double tau_task;
+  int    task_mode;
+  double k_ent;
+  const double* alpha_override;
+  unsigned long long layer_mask;
+} vlac_select_params;
+
+/* Views into the cache's selection state (device memory owned by the cache; valid until the
+ * cache is freed, contents overwritten by the next select/step).
+ *   M[b][l]            rows recomputed by layer l of sequence b
+ *   rows[b][l][0..M)   their positions, ascending; entries beyond M are unspecified
+ *   *_mask[b][v]       1/0 per vision token: P_static (Eq. topk), P_task (Eq. ptask), P_final (Eq. pfinal)
+ *   sim[b][v]          Eq. (sim);  S[b][v] task-relevance score (Sec. 3.3)
+ *   alpha[b][l]        reuse ratio actually applied (running maximum of Eq. reuse_ratio, or the override) */
+typedef struct {
+  int batch, n_layers, seq_len, n_vision;
+  int* M;
+  int* rows;
+  unsigned char *static_mask, *task_mask, *final_mask;
+  double *sim, *S, *alpha;
+} vlac_selection;
+
+/* Which part of a cache vlac_cache_read / vlac_cache_write address. */
+#define VLAC_PART_K          0   /* bf16 [max_seq][n_heads][head_dim] of (seq, layer), keys after rotation */
+#define VLAC_PART_V          1   /* same layout                                                           */
+#define VLAC_PART_PREV_FRAME 2   /* uint8 [n_cams][H][W][3] of seq (layer ignored)                         */
+#define VLAC_PART_ATTN_PREV  3   /* fp32 [n_layers][n_heads][L_v] of seq: scores saved by the previous step */
+#define VLAC_PART_ATTN_NEXT  4   /* same layout: scores being written by the current prefill               */
+#define VLAC_PART_WARM       5   /* int32 [1] of seq: 0 = cold (next select reuses nothing)                */
+
+/* Create a context.  Copies `cfg` and the layer table, borrows every weight pointer, allocates the
+ * workspace for max_batch sequences.  Errors: INVALID_ARG (bad shape, NULL), OOM, CUDA. */
+int vlac_create(const vlac_config* cfg, const vlac_weights* w, vlac_ctx** out);
+int vlac_destroy(vlac_ctx* ctx);
+
+/* Allocate the persistent state of `batch` (1..max_batch) independent sequences: per layer K/V
+ * caches of L + n_action - 1 positions (bf16, keys stored after rotation), the previous frame, the
+ * text-to-vision attention scores saved by the previous step (Sec. 3.3), and the selection buffers.
+ * The cache starts cold.  Library-owned device memory; release with vlac_cache_free. */
+int vlac_cache_alloc(vlac_ctx* ctx, int batch, vlac_cache** out);
+/* Make sequence `seq` (or all if seq < 0) cold: its next step recomputes every position. */
+int vlac_cache_reset(vlac_cache* cache, int seq, void* stream);
+int vlac_cache_free(vlac_cache* cache);
+/* Copy one part of the cache to / from caller DEVICE memory (device-to-device, stream-ordered).
+ * `bytes` must equal the part's size, else INVALID_ARG. */
+int vlac_cache_read (vlac_cache* cache, int part, int seq, int layer, void* dst_device, unsigned long long bytes, void* stream);
+int vlac_cache_write(vlac_cache* cache, int part, int seq, int layer, const void* src_device, unsigned long long bytes, void* stream);
+
+/* Token selection: Algorithm 1 (patch similarity Eq. sim, threshold + top-k Eq. topk, task
+ * relevance Eq. avistext/ptask from the saved scores, eviction Eq. pfinal) followed by the
+ * per-layer reuse ratio of Sec. 3.4 / Eq. (reuse_ratio) and the row lists each layer recomputes.
+ *   frames: device uint8 [batch][n_cams][H][W][3], the current camera frames (16-byte aligned).
+ * A cold sequence gets M = L for every layer.  `out` (may be NULL) receives views of the result.
+ * Runs entirely on the device; no host synchronisation. */
+int vlac_select(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames,
+                const vlac_select_params* params, vlac_selection* out, void* stream);
+
+/* Install a caller-made selection instead: HOST arrays M[batch][n_layers] and
+ * rows[batch][n_layers][L] (ascending positions).  For each sequence the row sets must shrink with
+ * depth (rows of layer l+1 a subset of layer l) and contain every text position; INVALID_ARG otherwise. */
+int vlac_select_import(vlac_ctx* ctx, vlac_cache* cache, const int* M_host, const int* rows_host, void* stream);
+
+/* One decoder layer over the selected rows only (Algorithm 2; Sec. 4.1; Appendix "Token Reuse
+ * Mechanism"): gather the rows of `hidden`, RMSNorm, Q/K/V projection, rotation at the rows' own
+ * positions, overwrite those positions of the layer's K/V cache, causal attention of the new
+ * queries over all cached positions (fresh and reused), output projection, SwiGLU MLP, both with
+ * residual; results are written back to the same rows of `hidden`.  Other rows are untouched.
+ * Also records, for the prompt-text queries behind the vision block, the mean attention
+ * probability on every vision key (readable as VLAC_PART_ATTN_NEXT).
+ *   hidden: device bf16 [batch][L][hidden], updated in place.
+ * Uses the selection currently held by the cache (from vlac_select / vlac_select_import);
+ * BAD_STATE if there is none. */
+int vlac_layer_forward(vlac_ctx* ctx, vlac_cache* cache, int layer, void* hidden, void* stream);
+
+/* One control step for every sequence of the cache: selection (skipped if force_full != 0 or the
+ * sequence is cold), input rows (token embeddings; projected vision features), all layers via the
+ * partial forward above, greedy first action token from the last prompt position, then
+ * n_action - 1 ordinary single-row passes that append K/V behind the prompt (Sec. 3.1).  Finally
+ * the frame and the recorded attention become "previous" and the sequences become warm.
+ *   frames        device uint8 [batch][n_cams][H][W][3]
+ *   vision_feats  device bf16  [batch][L_v][hidden]
+ *   prompt_ids    device int32 [batch][n_text_pre + n_text_post]
+ *   force_full    1 = recompute every position (the no-reuse step of the same library)
+ *   action_tokens device int32 [batch][n_action], ties in the argmax go to the lower id
+ *   all_logits    device fp32  [batch][n_action][vocab] or NULL: logits behind each action token
+ *   forced_tokens device int32 [batch][n_action] or NULL: tokens to feed back instead of the
+ *                 library's own choices (action_tokens still reports the library's choices). */
+int vlac_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, const void* vision_feats,
+              const int* prompt_ids, const vlac_select_params* params, int force_full,
+              int* action_tokens, float* all_logits, const int* forced_tokens, void* stream);
+
+/* Views of the selection held by the cache (after select / select_import / step). */
+int vlac_selection_view(vlac_cache* cache, vlac_selection* out);
+
+/* Number of kernels the library launched since the context was created (monotonic). */
+unsigned long long vlac_launch_count(const vlac_ctx* ctx);
+
+/* Nonzero if a device-side bounded wait gave up since the context was created (reads one int
+ * back; synchronises the stream). */
+int vlac_device_error(vlac_ctx* ctx, void* stream);
+
+const char* vlac_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* VLAC_H_ */
