@@ -1,0 +1,310 @@
+// Single-row passes: the action tokens after the first are produced by ordinary K/V-cache decoding
+// (Sec. 3.1, cache append; Appendix: "subsequent tokens are decoded autoregressively").
+//
+// With one row per sequence every projection is a matrix-vector product bound by streaming the
+// weights from HBM once.  One kernel serves all of them: each warp owns pairs of weight rows, the
+// (normalised) activations sit in shared memory as bf16, weights are read with 16-byte loads and
+// several loads are kept in flight per lane.  The pairing puts the two halves of a rotary pair, or
+// the gate and up rows of one FFN feature, in the same warp so the epilogue needs no exchange.
+#include "vlac_internal.h"
+
+namespace {
+
+__device__ __forceinline__ float bf2f(bf16 x) { return __bfloat162float(x); }
+
+enum { GV_QKV = 0, GV_RESID = 1, GV_SWIGLU = 2, GV_LOGITS = 3 };
+
+struct GemvArgs {
+  const float* x_f32;      // [nb][K] fp32 source (normalised with `gain`), or NULL
+  const bf16* x_bf16;      // [nb][K] bf16 source used as is, or NULL
+  const bf16* gain;        // [K]
+  const bf16 *w0, *w1, *w2;
+  int mode, nb, K, N;      // N: rows per matrix
+  float eps;
+  // epilogue targets
+  bf16* q_out;             // QKV: [nb][N]
+  bf16 *kc, *vc;           // QKV: [nb][max_seq][N]
+  const float *rope_cos, *rope_sin;
+  int pos, max_seq, d;
+  float* x_out;            // RESID: [nb][N] +=
+  bf16* h_out;             // SWIGLU: [nb][N]
+  float* logits;           // LOGITS: [nb][N]
+};
+
+__device__ __forceinline__ void fma8(float& acc, const uint4& w, const uint4& x) {
+  const __nv_bfloat162* wp = reinterpret_cast<const __nv_bfloat162*>(&w);
+  const __nv_bfloat162* xp = reinterpret_cast<const __nv_bfloat162*>(&x);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float2 wf = __bfloat1622float2(wp[e]);
+    const float2 xf = __bfloat1622float2(xp[e]);
+    acc = fmaf(wf.x, xf.x, acc);
+    acc = fmaf(wf.y, xf.y, acc);
+  }
+}
+
+template <int NB>
+__global__ void __launch_bounds__(256) gemv_pair_kernel(GemvArgs a) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  bf16* xs = reinterpret_cast<bf16*>(smem_raw);           // [NB][K]
+  __shared__ float red[8];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int K = a.K;
+
+  // ---- activations -> shared memory (RMSNorm here if a gain is given)
+  for (int b = 0; b < NB; ++b) {
+    if (b >= a.nb) {
+      for (int k = tid; k < K; k += 256) xs[(size_t)b * K + k] = __float2bfloat16(0.f);
+      continue;
+    }
+    if (a.x_f32) {
+      const float* x = a.x_f32 + (size_t)b * K;
+      float ss = 0.f;
+      for (int k = tid; k < K; k += 256) { const float v = x[k]; ss += v * v; }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+      __syncthreads();
+      if (lane == 0) red[warp] = ss;
+      __syncthreads();
+      float t = 0.f;
+      for (int w = 0; w < 8; ++w) t += red[w];
+      const float r = rsqrtf(t / (float)K + a.eps);
+      for (int k = tid; k < K; k += 256) xs[(size_t)b * K + k] = __float2bfloat16(x[k] * r * bf2f(a.gain[k]));
+    } else {
+      const uint4* src = reinterpret_cast<const uint4*>(a.x_bf16 + (size_t)b * K);
+      uint4* dst = reinterpret_cast<uint4*>(xs + (size_t)b * K);
+      for (int c = tid; c < K / 8; c += 256) dst[c] = src[c];
+    }
+  }
+  __syncthreads();
+
+  const int half = a.d / 2;
+  int n_units;
+  if (a.mode == GV_QKV) n_units = 3 * (a.N / 2);
+  else if (a.mode == GV_SWIGLU) n_units = a.N;
+  else n_units = (a.N + 1) / 2;
+  const int total_warps = gridDim.x * 8;
+  const int nchunk = K / 8;
+
+  for (int u = blockIdx.x * 8 + warp; u < n_units; u += total_warps) {
+    const bf16 *wa, *wb;
+    int rowA, rowB, mat = 0;
+    if (a.mode == GV_QKV) {
+      mat = u / (a.N / 2);
+      const int r = u - mat * (a.N / 2);
+      const int h = r / half, j = r - h * half;
+      rowA = h * a.d + j; rowB = rowA + half;
+      const bf16* W = mat == 0 ? a.w0 : (mat == 1 ? a.w1 : a.w2);
+      wa = W + (size_t)rowA * K; wb = W + (size_t)rowB * K;
+    } else if (a.mode == GV_SWIGLU) {
+      rowA = rowB = u;
+      wa = a.w0 + (size_t)u * K; wb = a.w1 + (size_t)u * K;
+    } else {
+      rowA = 2 * u; rowB = min(2 * u + 1, a.N - 1);
+      wa = a.w0 + (size_t)rowA * K; wb = a.w0 + (size_t)rowB * K;
+    }
+    float accA[NB], accB[NB];
+#pragma unroll
+    for (int b = 0; b < NB; ++b) accA[b] = accB[b] = 0.f;
+    const uint4* pa = reinterpret_cast<const uint4*>(wa);
+    const uint4* pb = reinterpret_cast<const uint4*>(wb);
+    for (int c0 = lane; c0 < nchunk; c0 += 128) {
+      uint4 va[4], vb[4];
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        const int c = c0 + 32 * t;
+        if (c < nchunk) { va[t] = __ldg(pa + c); vb[t] = __ldg(pb + c); }
+        else { va[t] = make_uint4(0, 0, 0, 0); vb[t] = make_uint4(0, 0, 0, 0); }
+      }
+#pragma unroll
+      for (int t = 0; t < 4; ++t) {
+        const int c = min(c0 + 32 * t, nchunk - 1);
+#pragma unroll
+        for (int b = 0; b < NB; ++b) {
+          const uint4 xv = *reinterpret_cast<const uint4*>(xs + (size_t)b * K + c * 8);
+          fma8(accA[b], va[t], xv);
+          fma8(accB[b], vb[t], xv);
+        }
+      }
+    }
+#pragma unroll
+    for (int b = 0; b < NB; ++b) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        accA[b] += __shfl_xor_sync(0xffffffffu, accA[b], o);
+        accB[b] += __shfl_xor_sync(0xffffffffu, accB[b], o);
+      }
+    }
+    if (lane == 0) {
+#pragma unroll
+      for (int b = 0; b < NB; ++b) {
+        if (b >= a.nb) break;
+        const float ya = accA[b], yb = accB[b];
+        if (a.mode == GV_QKV) {
+          if (mat == 2) {
+            bf16* dst = a.vc + ((size_t)b * a.max_seq + a.pos) * a.N;
+            dst[rowA] = __float2bfloat16(ya); dst[rowB] = __float2bfloat16(yb);
+          } else {
+            const int j = rowA % a.d;
+            const float c = a.rope_cos[(size_t)a.pos * half + j], s = a.rope_sin[(size_t)a.pos * half + j];
+            const float r1 = ya * c - yb * s, r2 = yb * c + ya * s;
+            bf16* dst = mat == 0 ? a.q_out + (size_t)b * a.N : a.kc + ((size_t)b * a.max_seq + a.pos) * a.N;
+            dst[rowA] = __float2bfloat16(r1); dst[rowB] = __float2bfloat16(r2);
+          }
+        } else if (a.mode == GV_SWIGLU) {
+          a.h_out[(size_t)b * a.N + rowA] = __float2bfloat16(ya / (1.f + __expf(-ya)) * yb);
+        } else if (a.mode == GV_RESID) {
+          a.x_out[(size_t)b * a.N + rowA] += ya;
+          if (rowB != rowA) a.x_out[(size_t)b * a.N + rowB] += yb;
+        } else {
+          a.logits[(size_t)b * a.N + rowA] = ya;
+          if (rowB != rowA) a.logits[(size_t)b * a.N + rowB] = yb;
+        }
+      }
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256) embed_token_kernel(const bf16* embed, const int* tokens, int tok_stride, int tok_index,
+                                                          float* x, int D, int vocab) {
+  const int b = blockIdx.x;
+  int id = tokens[(size_t)b * tok_stride + tok_index];
+  id = min(max(id, 0), vocab - 1);
+  for (int k = threadIdx.x; k < D; k += blockDim.x) x[(size_t)b * D + k] = bf2f(embed[(size_t)id * D + k]);
+}
+
+__global__ void __launch_bounds__(256) last_row_kernel(const bf16* hidden, float* x, int L, int D) {
+  const int b = blockIdx.x;
+  const bf16* src = hidden + ((size_t)b * L + (L - 1)) * D;
+  for (int k = threadIdx.x; k < D; k += blockDim.x) x[(size_t)b * D + k] = bf2f(src[k]);
+}
+
+// greedy choice; equal logits -> lower id
+__device__ __forceinline__ unsigned long long argmax_key(float v, int idx) {
+  unsigned int u = __float_as_uint(v);
+  u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);          // monotone map of float order onto unsigned order
+  return ((unsigned long long)u << 32) | (unsigned long long)(0xFFFFFFFFu - (unsigned int)idx);
+}
+
+__global__ void __launch_bounds__(256) argmax_partial_kernel(const float* logits, int vocab, unsigned long long* tmp) {
+  __shared__ unsigned long long red[8];
+  const int b = blockIdx.y;
+  const float* row = logits + (size_t)b * vocab;
+  unsigned long long best = 0ull;
+  for (int n = blockIdx.x * blockDim.x + threadIdx.x; n < vocab; n += gridDim.x * blockDim.x) {
+    const unsigned long long k = argmax_key(row[n], n);
+    best = k > best ? k : best;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) { const unsigned long long t = __shfl_xor_sync(0xffffffffu, best, o); best = t > best ? t : best; }
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = best;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < 8; ++w) best = red[w] > best ? red[w] : best;
+    tmp[(size_t)b * gridDim.x + blockIdx.x] = best;
+  }
+}
+
+__global__ void argmax_final_kernel(const unsigned long long* tmp, int n_part, int* tokens, int tok_stride, int tok_index) {
+  const int b = blockIdx.x;
+  if (threadIdx.x == 0) {
+    unsigned long long best = 0ull;
+    for (int i = 0; i < n_part; ++i) { const unsigned long long k = tmp[(size_t)b * n_part + i]; best = k > best ? k : best; }
+    tokens[(size_t)b * tok_stride + tok_index] = (int)(0xFFFFFFFFu - (unsigned int)(best & 0xFFFFFFFFull));
+  }
+}
+
+int launch_gemv(vlac_ctx* ctx, const GemvArgs& a, cudaStream_t s) {
+  const int nb = a.nb;
+  const int NB = nb <= 1 ? 1 : (nb <= 2 ? 2 : (nb <= 4 ? 4 : 8));
+  const size_t smem = (size_t)NB * a.K * sizeof(bf16);
+  const int grid = ctx->n_sm * 2;
+  switch (NB) {
+    case 1: gemv_pair_kernel<1><<<grid, 256, smem, s>>>(a); break;
+    case 2: gemv_pair_kernel<2><<<grid, 256, smem, s>>>(a); break;
+    case 4: gemv_pair_kernel<4><<<grid, 256, smem, s>>>(a); break;
+    default: gemv_pair_kernel<8><<<grid, 256, smem, s>>>(a); break;
+  }
+  VLAC_LAUNCH_CHECK(ctx);
+  return VLAC_OK;
+}
+
+}  // namespace
+
+int vlac_decode_setup(vlac_ctx* ctx) {
+  const int kmax = ctx->cfg.ffn > ctx->cfg.hidden ? ctx->cfg.ffn : ctx->cfg.hidden;
+  const int mb = ctx->cfg.max_batch;
+  if (mb > 8) return VLAC_ERR_INVALID_ARG;
+  const int NB = mb <= 1 ? 1 : (mb <= 2 ? 2 : (mb <= 4 ? 4 : 8));
+  const size_t smem = (size_t)NB * kmax * sizeof(bf16);
+  if (smem > 227 * 1024) return VLAC_ERR_INVALID_ARG;
+  VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_pair_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(1 * (size_t)kmax * 2)));
+  if (NB >= 2) VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_pair_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * (size_t)kmax * 2)));
+  if (NB >= 4) VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_pair_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(4 * (size_t)kmax * 2)));
+  if (NB >= 8) VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_pair_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(8 * (size_t)kmax * 2)));
+  return VLAC_OK;
+}
+
+int vlac_launch_last_row(vlac_ctx* ctx, vlac_cache* c, const bf16* hidden, cudaStream_t s) {
+  last_row_kernel<<<c->batch, 256, 0, s>>>(hidden, ctx->x_dec, ctx->L, ctx->cfg.hidden);
+  VLAC_LAUNCH_CHECK(ctx);
+  return VLAC_OK;
+}
+
+int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens, int tok_stride, int tok_index,
+                            int pos, cudaStream_t s) {
+  const vlac_config& g = ctx->cfg;
+  const int D = g.hidden, F = g.ffn, B = c->batch;
+  embed_token_kernel<<<B, 256, 0, s>>>((const bf16*)ctx->w.embed, fed_tokens, tok_stride, tok_index, ctx->x_dec, D, g.vocab);
+  VLAC_LAUNCH_CHECK(ctx);
+  for (int l = 0; l < g.n_layers; ++l) {
+    const vlac_layer_w& w = ctx->layers[l];
+    bf16* kc = c->k + (size_t)l * B * kv_layer_elems(ctx);
+    bf16* vc = c->v + (size_t)l * B * kv_layer_elems(ctx);
+    GemvArgs a = {};
+    a.x_f32 = ctx->x_dec; a.gain = (const bf16*)w.g_attn; a.eps = g.rms_eps;
+    a.w0 = (const bf16*)w.wq; a.w1 = (const bf16*)w.wk; a.w2 = (const bf16*)w.wv;
+    a.mode = GV_QKV; a.nb = B; a.K = D; a.N = D;
+    a.q_out = ctx->q_dec; a.kc = kc; a.vc = vc; a.rope_cos = ctx->w.rope_cos; a.rope_sin = ctx->w.rope_sin;
+    a.pos = pos; a.max_seq = ctx->max_seq; a.d = g.head_dim;
+    int rc = launch_gemv(ctx, a, s);
+    if (rc) return rc;
+    rc = vlac_launch_decode_attention(ctx, c, l, pos, s);
+    if (rc) return rc;
+    GemvArgs o = {};
+    o.x_bf16 = ctx->ao_dec; o.w0 = (const bf16*)w.wo; o.mode = GV_RESID; o.nb = B; o.K = D; o.N = D; o.x_out = ctx->x_dec; o.d = g.head_dim;
+    rc = launch_gemv(ctx, o, s);
+    if (rc) return rc;
+    GemvArgs gu = {};
+    gu.x_f32 = ctx->x_dec; gu.gain = (const bf16*)w.g_mlp; gu.eps = g.rms_eps;
+    gu.w0 = (const bf16*)w.w_gate; gu.w1 = (const bf16*)w.w_up; gu.mode = GV_SWIGLU; gu.nb = B; gu.K = D; gu.N = F;
+    gu.h_out = ctx->hm_dec; gu.d = g.head_dim;
+    rc = launch_gemv(ctx, gu, s);
+    if (rc) return rc;
+    GemvArgs dn = {};
+    dn.x_bf16 = ctx->hm_dec; dn.w0 = (const bf16*)w.w_down; dn.mode = GV_RESID; dn.nb = B; dn.K = F; dn.N = D; dn.x_out = ctx->x_dec; dn.d = g.head_dim;
+    rc = launch_gemv(ctx, dn, s);
+    if (rc) return rc;
+  }
+  return VLAC_OK;
+}
+
+int vlac_launch_logits_argmax(vlac_ctx* ctx, vlac_cache* c, int* tokens_out, int tok_stride, int tok_index,
+                              float* logits_copy, long long copy_stride, cudaStream_t s) {
+  const vlac_config& g = ctx->cfg;
+  const int B = c->batch;
+  GemvArgs a = {};
+  a.x_f32 = ctx->x_dec; a.gain = (const bf16*)ctx->w.g_final; a.eps = g.rms_eps;
+  a.w0 = (const bf16*)ctx->w.lm_head; a.mode = GV_LOGITS; a.nb = B; a.K = g.hidden; a.N = g.vocab; a.logits = ctx->logits; a.d = g.head_dim;
+  int rc = launch_gemv(ctx, a, s);
+  if (rc) return rc;
+  argmax_partial_kernel<<<dim3(VLAC_ARGMAX_BLOCKS, B), 256, 0, s>>>(ctx->logits, g.vocab, ctx->argmax_tmp);
+  VLAC_LAUNCH_CHECK(ctx);
+  argmax_final_kernel<<<B, 32, 0, s>>>(ctx->argmax_tmp, VLAC_ARGMAX_BLOCKS, tokens_out, tok_stride, tok_index);
+  VLAC_LAUNCH_CHECK(ctx);
+  if (logits_copy) {
+    VLAC_CUDA_CHECK(cudaMemcpy2DAsync(logits_copy, (size_t)copy_stride * sizeof(float), ctx->logits, (size_t)g.vocab * sizeof(float),
+                                      (size_t)g.vocab * sizeof(float), B, cudaMemcpyDeviceToDevice, s));
+  }
+  return VLAC_OK;
+}

@@ -1,0 +1,364 @@
+// C ABI: contexts, caches and the three calls of the control step (select, layer_forward, step).
+#include "vlac_internal.h"
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+#include <new>
+
+static char g_last_cuda_error[256] = "";
+
+void vlac_note_cuda_error(cudaError_t e, const char* file, int line) {
+  snprintf(g_last_cuda_error, sizeof(g_last_cuda_error), "%s (%s:%d)", cudaGetErrorString(e), file, line);
+  if (getenv("VLAC_VERBOSE")) fprintf(stderr, "[vlac] CUDA error: %s\n", g_last_cuda_error);
+}
+
+namespace {
+
+template <typename T>
+int dev_alloc(T** p, size_t n) {
+  *p = nullptr;
+  if (n == 0) n = 1;
+  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), n * sizeof(T));
+  if (e == cudaErrorMemoryAllocation) { cudaGetLastError(); return VLAC_ERR_OOM; }
+  if (e != cudaSuccess) { vlac_note_cuda_error(e, __FILE__, __LINE__); return VLAC_ERR_CUDA; }
+  e = cudaMemset(*p, 0, n * sizeof(T));
+  if (e != cudaSuccess) { vlac_note_cuda_error(e, __FILE__, __LINE__); return VLAC_ERR_CUDA; }
+  return VLAC_OK;
+}
+
+#define TRY(x) do { int rc__ = (x); if (rc__ != VLAC_OK) return rc__; } while (0)
+
+int fill_params(const vlac_ctx* ctx, const vlac_select_params* in, int force_full, SelectKernelParams* p) {
+  memset(p, 0, sizeof(*p));
+  p->force_full = force_full ? 1 : 0;
+  if (!in) {
+    if (!force_full) return VLAC_ERR_INVALID_ARG;
+    return VLAC_OK;
+  }
+  if (!(in->tau == in->tau) || !(in->tau_task == in->tau_task) || !(in->k_ent == in->k_ent)) return VLAC_ERR_INVALID_ARG;
+  if (in->task_mode != 0 && in->task_mode != 1) return VLAC_ERR_INVALID_ARG;
+  p->tau = in->tau; p->tau_task = in->tau_task; p->k_ent = in->k_ent;
+  p->top_k = in->top_k; p->task_mode = in->task_mode; p->layer_mask = in->layer_mask;
+  if (in->alpha_override) {
+    p->has_override = 1;
+    for (int l = 0; l < ctx->cfg.n_layers; ++l) p->alpha_override[l] = in->alpha_override[l];
+  }
+  return VLAC_OK;
+}
+
+void free_ctx_buffers(vlac_ctx* c) {
+  cudaFree(c->xn); cudaFree(c->q); cudaFree(c->ao); cudaFree(c->hm); cudaFree(c->part); cudaFree(c->scratch);
+  cudaFree(c->probs); cudaFree(c->hidden); cudaFree(c->x_dec); cudaFree(c->q_dec); cudaFree(c->ao_dec);
+  cudaFree(c->hm_dec); cudaFree(c->logits); cudaFree(c->argmax_tmp); cudaFree(c->dev_error);
+}
+
+void free_cache_buffers(vlac_cache* c) {
+  cudaFree(c->k); cudaFree(c->v); cudaFree(c->prev_frames); cudaFree(c->attn_prev); cudaFree(c->attn_next);
+  cudaFree(c->warm); cudaFree(c->sim); cudaFree(c->S_layer); cudaFree(c->S); cudaFree(c->alpha);
+  cudaFree(c->alpha_raw); cudaFree(c->entropy); cudaFree(c->static_mask); cudaFree(c->task_mask);
+  cudaFree(c->final_mask); cudaFree(c->rank); cudaFree(c->n_reuse); cudaFree(c->M); cudaFree(c->rows);
+  cudaFree(c->tot); cudaFree(c->rowmap); cudaFree(c->slot);
+}
+
+__global__ void set_warm_kernel(int* warm, int n, int value) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) warm[i] = value;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* vlac_status_string(int status) {
+  switch (status) {
+    case VLAC_OK: return "ok";
+    case VLAC_ERR_INVALID_ARG: return "invalid argument";
+    case VLAC_ERR_BAD_STATE: return "bad state";
+    case VLAC_ERR_OOM: return "out of device memory";
+    case VLAC_ERR_CUDA: return g_last_cuda_error[0] ? g_last_cuda_error : "CUDA error";
+    case VLAC_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+int vlac_create(const vlac_config* cfg, const vlac_weights* w, vlac_ctx** out) {
+  if (!cfg || !w || !out || !w->layers) return VLAC_ERR_INVALID_ARG;
+  *out = nullptr;
+  const vlac_config& g = *cfg;
+  if (g.n_layers < 1 || g.n_layers > VLAC_MAX_LAYERS || g.hidden < 8 || g.hidden % 8 || g.hidden > 8192 ||
+      g.n_heads < 1 || g.n_kv_heads != g.n_heads || g.head_dim < 32 || g.head_dim % 32 || g.head_dim > 128 ||
+      g.n_heads * g.head_dim != g.hidden || g.ffn < 8 || g.ffn % 8 || g.vocab < 2 || g.n_cams < 1 || g.grid < 1 ||
+      g.grid > 64 || g.patch < 1 || g.n_text_pre < 0 || g.n_text_post < 0 || g.n_action < 1 ||
+      g.max_batch < 1 || g.max_batch > 8 || !(g.rms_eps > 0.f))
+    return VLAC_ERR_INVALID_ARG;
+  if (!w->embed || !w->proj || !w->g_final || !w->lm_head || !w->rope_cos || !w->rope_sin) return VLAC_ERR_INVALID_ARG;
+  for (int l = 0; l < g.n_layers; ++l) {
+    const vlac_layer_w& lw = w->layers[l];
+    if (!lw.wq || !lw.wk || !lw.wv || !lw.wo || !lw.w_gate || !lw.w_up || !lw.w_down || !lw.g_attn || !lw.g_mlp)
+      return VLAC_ERR_INVALID_ARG;
+  }
+  vlac_ctx* c = new (std::nothrow) vlac_ctx();
+  if (!c) return VLAC_ERR_OOM;
+  memset(c, 0, sizeof(*c));
+  c->cfg = g; c->w = *w;
+  for (int l = 0; l < g.n_layers; ++l) c->layers[l] = w->layers[l];
+  c->w.layers = c->layers;
+  c->Lv = g.n_cams * g.grid * g.grid;
+  c->L = g.n_text_pre + c->Lv + g.n_text_post;
+  c->max_seq = c->L + g.n_action - 1;
+  c->frame_hw = g.grid * g.patch;
+  c->rows_max = g.max_batch * c->L;
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+    vlac_note_cuda_error(cudaGetLastError(), __FILE__, __LINE__);
+    delete c;
+    return VLAC_ERR_CUDA;
+  }
+  c->n_sm = prop.multiProcessorCount;
+  const size_t R = c->rows_max, D = g.hidden, F = g.ffn, B = g.max_batch;
+  const size_t wide = (3 * D > 2 * F ? 3 * D : 2 * F);
+  int rc = VLAC_OK;
+  if (rc == VLAC_OK) rc = dev_alloc(&c->xn, R * D);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->q, R * D);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->ao, R * D);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->hm, R * F);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->part, (size_t)VLAC_MAX_SPLITS * R * D);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->scratch, R * wide);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->probs, B * (size_t)g.n_text_post * g.n_heads * c->Lv);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->hidden, R * D);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->x_dec, B * D);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->q_dec, B * D);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->ao_dec, B * D);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->hm_dec, B * F);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->logits, B * (size_t)g.vocab);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->argmax_tmp, B * VLAC_ARGMAX_BLOCKS);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->dev_error, 1);
+  if (rc == VLAC_OK) rc = vlac_decode_setup(c);
+  if (rc != VLAC_OK) { free_ctx_buffers(c); delete c; return rc; }
+  *out = c;
+  return VLAC_OK;
+}
+
+int vlac_destroy(vlac_ctx* ctx) {
+  if (!ctx) return VLAC_ERR_INVALID_ARG;
+  cudaDeviceSynchronize();
+  free_ctx_buffers(ctx);
+  delete ctx;
+  return VLAC_OK;
+}
+
+int vlac_cache_alloc(vlac_ctx* ctx, int batch, vlac_cache** out) {
+  if (!ctx || !out || batch < 1 || batch > ctx->cfg.max_batch) return VLAC_ERR_INVALID_ARG;
+  *out = nullptr;
+  vlac_cache* c = new (std::nothrow) vlac_cache();
+  if (!c) return VLAC_ERR_OOM;
+  memset(c, 0, sizeof(*c));
+  c->ctx = ctx; c->batch = batch;
+  const vlac_config& g = ctx->cfg;
+  const size_t B = batch, nl = g.n_layers, Lv = ctx->Lv, L = ctx->L;
+  const size_t frame = (size_t)g.n_cams * ctx->frame_hw * ctx->frame_hw * 3;
+  int rc = VLAC_OK;
+  if (rc == VLAC_OK) rc = dev_alloc(&c->k, nl * B * kv_layer_elems(ctx));
+  if (rc == VLAC_OK) rc = dev_alloc(&c->v, nl * B * kv_layer_elems(ctx));
+  if (rc == VLAC_OK) rc = dev_alloc(&c->prev_frames, B * frame);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->attn_prev, B * nl * g.n_heads * Lv);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->attn_next, B * nl * g.n_heads * Lv);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->warm, B);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->sim, B * Lv);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->S_layer, B * nl * Lv);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->S, B * Lv);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->alpha, B * nl);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->alpha_raw, B * nl);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->entropy, B * (nl + 1));
+  if (rc == VLAC_OK) rc = dev_alloc(&c->static_mask, B * Lv);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->task_mask, B * Lv);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->final_mask, B * Lv);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->rank, B * Lv);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->n_reuse, B * nl);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->M, B * nl);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->rows, B * nl * L);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->tot, nl);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->rowmap, nl * B * L);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->slot, nl * B * L);
+  if (rc != VLAC_OK) { free_cache_buffers(c); delete c; return rc; }
+  *out = c;
+  return VLAC_OK;
+}
+
+int vlac_cache_reset(vlac_cache* cache, int seq, void* stream) {
+  if (!cache || seq >= cache->batch) return VLAC_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (seq < 0) VLAC_CUDA_CHECK(cudaMemsetAsync(cache->warm, 0, sizeof(int) * cache->batch, s));
+  else VLAC_CUDA_CHECK(cudaMemsetAsync(cache->warm + seq, 0, sizeof(int), s));
+  cache->has_selection = 0;
+  return VLAC_OK;
+}
+
+int vlac_cache_free(vlac_cache* cache) {
+  if (!cache) return VLAC_ERR_INVALID_ARG;
+  cudaDeviceSynchronize();
+  free_cache_buffers(cache);
+  delete cache;
+  return VLAC_OK;
+}
+
+static int cache_part(vlac_cache* c, int part, int seq, int layer, void** ptr, size_t* bytes) {
+  if (!c || seq < 0 || seq >= c->batch) return VLAC_ERR_INVALID_ARG;
+  vlac_ctx* ctx = c->ctx;
+  const vlac_config& g = ctx->cfg;
+  const size_t kv = kv_layer_elems(ctx);
+  const size_t attn = (size_t)g.n_layers * g.n_heads * ctx->Lv;
+  const size_t frame = (size_t)g.n_cams * ctx->frame_hw * ctx->frame_hw * 3;
+  switch (part) {
+    case VLAC_PART_K:
+    case VLAC_PART_V:
+      if (layer < 0 || layer >= g.n_layers) return VLAC_ERR_INVALID_ARG;
+      *ptr = (part == VLAC_PART_K ? c->k : c->v) + ((size_t)layer * c->batch + seq) * kv;
+      *bytes = kv * sizeof(bf16);
+      return VLAC_OK;
+    case VLAC_PART_PREV_FRAME: *ptr = c->prev_frames + seq * frame; *bytes = frame; return VLAC_OK;
+    case VLAC_PART_ATTN_PREV: *ptr = c->attn_prev + seq * attn; *bytes = attn * sizeof(float); return VLAC_OK;
+    case VLAC_PART_ATTN_NEXT: *ptr = c->attn_next + seq * attn; *bytes = attn * sizeof(float); return VLAC_OK;
+    case VLAC_PART_WARM: *ptr = c->warm + seq; *bytes = sizeof(int); return VLAC_OK;
+    default: return VLAC_ERR_INVALID_ARG;
+  }
+}
+
+int vlac_cache_read(vlac_cache* cache, int part, int seq, int layer, void* dst, unsigned long long bytes, void* stream) {
+  void* p; size_t n;
+  TRY(cache_part(cache, part, seq, layer, &p, &n));
+  if (!dst || bytes != n) return VLAC_ERR_INVALID_ARG;
+  VLAC_CUDA_CHECK(cudaMemcpyAsync(dst, p, n, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  return VLAC_OK;
+}
+
+int vlac_cache_write(vlac_cache* cache, int part, int seq, int layer, const void* src, unsigned long long bytes, void* stream) {
+  void* p; size_t n;
+  TRY(cache_part(cache, part, seq, layer, &p, &n));
+  if (!src || bytes != n) return VLAC_ERR_INVALID_ARG;
+  VLAC_CUDA_CHECK(cudaMemcpyAsync(p, src, n, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  return VLAC_OK;
+}
+
+int vlac_selection_view(vlac_cache* c, vlac_selection* out) {
+  if (!c || !out) return VLAC_ERR_INVALID_ARG;
+  out->batch = c->batch; out->n_layers = c->ctx->cfg.n_layers; out->seq_len = c->ctx->L; out->n_vision = c->ctx->Lv;
+  out->M = c->M; out->rows = c->rows;
+  out->static_mask = c->static_mask; out->task_mask = c->task_mask; out->final_mask = c->final_mask;
+  out->sim = c->sim; out->S = c->S; out->alpha = c->alpha;
+  return VLAC_OK;
+}
+
+int vlac_select(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, const vlac_select_params* params,
+                vlac_selection* out, void* stream) {
+  if (!ctx || !cache || cache->ctx != ctx || !frames || !params) return VLAC_ERR_INVALID_ARG;
+  SelectKernelParams p;
+  TRY(fill_params(ctx, params, 0, &p));
+  TRY(vlac_launch_select(ctx, cache, frames, p, (cudaStream_t)stream));
+  cache->has_selection = 1;
+  if (out) vlac_selection_view(cache, out);
+  return VLAC_OK;
+}
+
+int vlac_select_import(vlac_ctx* ctx, vlac_cache* cache, const int* M_host, const int* rows_host, void* stream) {
+  if (!ctx || !cache || cache->ctx != ctx || !M_host || !rows_host) return VLAC_ERR_INVALID_ARG;
+  const int nl = ctx->cfg.n_layers, L = ctx->L, B = cache->batch;
+  const int v0 = ctx->cfg.n_text_pre, v1 = v0 + ctx->Lv;
+  unsigned char* prev = (unsigned char*)malloc(L);
+  unsigned char* cur = (unsigned char*)malloc(L);
+  if (!prev || !cur) { free(prev); free(cur); return VLAC_ERR_OOM; }
+  int bad = 0;
+  for (int b = 0; b < B && !bad; ++b) {
+    memset(prev, 1, L);
+    for (int l = 0; l < nl && !bad; ++l) {
+      const int m = M_host[b * nl + l];
+      const int* r = rows_host + ((size_t)b * nl + l) * L;
+      if (m < 0 || m > L) { bad = 1; break; }
+      memset(cur, 0, L);
+      for (int i = 0; i < m; ++i) {
+        if (r[i] < 0 || r[i] >= L || (i > 0 && r[i] <= r[i - 1]) || !prev[r[i]]) { bad = 1; break; }
+        cur[r[i]] = 1;
+      }
+      for (int p = 0; p < L && !bad; ++p) if ((p < v0 || p >= v1) && !cur[p]) bad = 1;
+      memcpy(prev, cur, L);
+    }
+  }
+  free(prev); free(cur);
+  if (bad) return VLAC_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  VLAC_CUDA_CHECK(cudaMemcpyAsync(cache->M, M_host, sizeof(int) * B * nl, cudaMemcpyHostToDevice, s));
+  VLAC_CUDA_CHECK(cudaMemcpyAsync(cache->rows, rows_host, sizeof(int) * (size_t)B * nl * L, cudaMemcpyHostToDevice, s));
+  VLAC_CUDA_CHECK(cudaStreamSynchronize(s));     // the host arrays may be reused by the caller on return
+  TRY(vlac_launch_flatten(ctx, cache, s));
+  cache->has_selection = 1;
+  return VLAC_OK;
+}
+
+int vlac_layer_forward(vlac_ctx* ctx, vlac_cache* cache, int layer, void* hidden, void* stream) {
+  if (!ctx || !cache || cache->ctx != ctx || !hidden || layer < 0 || layer >= ctx->cfg.n_layers) return VLAC_ERR_INVALID_ARG;
+  if (!cache->has_selection) return VLAC_ERR_BAD_STATE;
+  cudaStream_t s = (cudaStream_t)stream;
+  bf16* h = (bf16*)hidden;
+  int n_splits = 0;
+  TRY(vlac_launch_finalize_norm(ctx, cache, h, layer, 0, layer, ctx->layers[layer].g_attn, s));
+  TRY(vlac_launch_layer_body(ctx, cache, layer, h, &n_splits, s));
+  TRY(vlac_launch_finalize_norm(ctx, cache, h, layer, n_splits, layer, nullptr, s));
+  return VLAC_OK;
+}
+
+int vlac_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, const void* vision_feats,
+              const int* prompt_ids, const vlac_select_params* params, int force_full,
+              int* action_tokens, float* all_logits, const int* forced_tokens, void* stream) {
+  if (!ctx || !cache || cache->ctx != ctx || !frames || !vision_feats || !action_tokens) return VLAC_ERR_INVALID_ARG;
+  const vlac_config& g = ctx->cfg;
+  if (!prompt_ids && g.n_text_pre + g.n_text_post > 0) return VLAC_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  SelectKernelParams p;
+  TRY(fill_params(ctx, params, force_full, &p));
+  const int B = cache->batch, nl = g.n_layers;
+  // 1. which rows each layer recomputes
+  TRY(vlac_launch_select(ctx, cache, frames, p, s));
+  cache->has_selection = 1;
+  // 2. rows entering layer 0
+  bf16* h = ctx->hidden;
+  TRY(vlac_launch_input_rows(ctx, cache, vision_feats, prompt_ids, h, s));
+  // 3. layers; the down-projection partials of layer l are folded into layer l+1's first kernel
+  int n_splits = 0;
+  for (int l = 0; l < nl; ++l) {
+    TRY(vlac_launch_finalize_norm(ctx, cache, h, l == 0 ? 0 : l - 1, l == 0 ? 0 : n_splits, l, ctx->layers[l].g_attn, s));
+    TRY(vlac_launch_layer_body(ctx, cache, l, h, &n_splits, s));
+  }
+  TRY(vlac_launch_finalize_norm(ctx, cache, h, nl - 1, n_splits, nl - 1, nullptr, s));
+  // 4. first action token
+  TRY(vlac_launch_last_row(ctx, cache, h, s));
+  const long long lstride = (long long)g.n_action * g.vocab;
+  TRY(vlac_launch_logits_argmax(ctx, cache, action_tokens, g.n_action, 0, all_logits, lstride, s));
+  // 5. remaining tokens, one single-row pass each
+  const int* fed = forced_tokens ? forced_tokens : action_tokens;
+  for (int i = 1; i < g.n_action; ++i) {
+    TRY(vlac_launch_decode_pass(ctx, cache, fed, g.n_action, i - 1, ctx->L - 1 + i, s));
+    TRY(vlac_launch_logits_argmax(ctx, cache, action_tokens, g.n_action, i,
+                                  all_logits ? all_logits + (size_t)i * g.vocab : nullptr, lstride, s));
+  }
+  // 6. this step becomes "previous"
+  const size_t frame = (size_t)B * g.n_cams * ctx->frame_hw * ctx->frame_hw * 3;
+  VLAC_CUDA_CHECK(cudaMemcpyAsync(cache->prev_frames, frames, frame, cudaMemcpyDeviceToDevice, s));
+  VLAC_CUDA_CHECK(cudaMemcpyAsync(cache->attn_prev, cache->attn_next, sizeof(float) * (size_t)B * nl * g.n_heads * ctx->Lv,
+                                  cudaMemcpyDeviceToDevice, s));
+  set_warm_kernel<<<1, 32, 0, s>>>(cache->warm, B, 1);
+  VLAC_LAUNCH_CHECK(ctx);
+  return VLAC_OK;
+}
+
+unsigned long long vlac_launch_count(const vlac_ctx* ctx) { return ctx ? ctx->launches : 0ull; }
+
+int vlac_device_error(vlac_ctx* ctx, void* stream) {
+  if (!ctx) return VLAC_ERR_INVALID_ARG;
+  int v = 0;
+  VLAC_CUDA_CHECK(cudaMemcpyAsync(&v, ctx->dev_error, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+  VLAC_CUDA_CHECK(cudaStreamSynchronize((cudaStream_t)stream));
+  return v ? VLAC_ERR_TIMEOUT : VLAC_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,97 @@
+// Internal declarations shared by the library's translation units.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "vlac.h"
+
+typedef __nv_bfloat16 bf16;
+
+void vlac_note_cuda_error(cudaError_t e, const char* file, int line);
+
+#define VLAC_CUDA_CHECK(expr)                                   \
+  do {                                                          \
+    cudaError_t e__ = (expr);                                   \
+    if (e__ != cudaSuccess) { vlac_note_cuda_error(e__, __FILE__, __LINE__); return VLAC_ERR_CUDA; } \
+  } while (0)
+
+#define VLAC_LAUNCH_CHECK(ctx)                                  \
+  do { (ctx)->launches++; VLAC_CUDA_CHECK(cudaGetLastError()); } while (0)
+
+// Largest split-K factor of the output / down projections (partials are reduced by the next kernel).
+#define VLAC_MAX_SPLITS 4
+
+struct SelectKernelParams {          // passed by value to the selection kernel
+  double tau, tau_task, k_ent;
+  int top_k, task_mode, has_override, force_full;
+  unsigned long long layer_mask;
+  double alpha_override[VLAC_MAX_LAYERS];
+};
+
+struct vlac_ctx {
+  vlac_config cfg;
+  vlac_weights w;
+  vlac_layer_w layers[VLAC_MAX_LAYERS];
+  int L, Lv, max_seq, frame_hw, rows_max, n_sm;
+  unsigned long long launches;
+  // workspace (device)
+  bf16 *xn, *q, *ao, *hm;            // [rows_max][hidden] x3, [rows_max][ffn]
+  float *part;                       // [VLAC_MAX_SPLITS][rows_max][hidden]
+  float *scratch;                    // [rows_max][max(3*hidden, 2*ffn)]   (generic GEMM output)
+  float *probs;                      // [max_batch][n_text_post][n_heads][Lv]
+  bf16 *hidden;                      // [max_batch][L][hidden]            (used by step)
+  float *x_dec;                      // [max_batch][hidden]
+  bf16 *q_dec, *ao_dec, *hm_dec;     // [max_batch][hidden] x2, [max_batch][ffn]
+  float *logits;                     // [max_batch][vocab]
+  unsigned long long *argmax_tmp;    // [max_batch][VLAC_ARGMAX_BLOCKS]
+  int *dev_error;                    // device int: nonzero if a bounded wait gave up
+};
+#define VLAC_ARGMAX_BLOCKS 64
+
+struct vlac_cache {
+  vlac_ctx* ctx;
+  int batch;
+  int has_selection;
+  // persistent state (device)
+  bf16 *k, *v;                       // [n_layers][batch][max_seq][n_heads][head_dim]
+  unsigned char* prev_frames;        // [batch][n_cams][H][W][3]
+  float *attn_prev, *attn_next;      // [batch][n_layers][n_heads][Lv]
+  int* warm;                         // [batch]
+  // selection state (device)
+  double *sim, *S_layer, *S, *alpha, *alpha_raw, *entropy;   // [b][Lv], [b][nl][Lv], [b][Lv], [b][nl] x2, [b][nl+1]
+  unsigned char *static_mask, *task_mask, *final_mask;       // [b][Lv]
+  int *rank, *n_reuse;               // [b][Lv], [b][nl]
+  int *M, *rows;                     // [b][nl], [b][nl][L]
+  int *tot;                          // [nl]                 total rows over the batch
+  int *rowmap;                       // [nl][batch*L]        compact index -> b*L + pos
+  int *slot;                         // [nl][batch*L]        b*L + pos -> compact index or -1
+};
+
+static inline size_t kv_layer_elems(const vlac_ctx* c) {
+  return (size_t)c->max_seq * c->cfg.n_heads * c->cfg.head_dim;
+}
+
+// ---- selection (select_kernels.cu)
+int vlac_launch_select(vlac_ctx* ctx, vlac_cache* c, const unsigned char* frames,
+                       const SelectKernelParams& p, cudaStream_t s);
+int vlac_launch_flatten(vlac_ctx* ctx, vlac_cache* c, cudaStream_t s);
+
+// ---- prefill (prefill_kernels.cu)
+int vlac_launch_input_rows(vlac_ctx* ctx, vlac_cache* c, const void* feats, const int* ids, bf16* hidden, cudaStream_t s);
+// If n_splits > 0: hidden[row] += sum of split-K partials, for the rows of layer l_prev.
+// If gain != NULL: RMSNorm the rows of layer l_next (after the update) into ctx->xn.
+int vlac_launch_finalize_norm(vlac_ctx* ctx, vlac_cache* c, bf16* hidden, int l_prev, int n_splits,
+                              int l_next, const void* gain, cudaStream_t s);
+// Everything of layer `layer` between its first RMSNorm (already in ctx->xn) and the down-projection
+// partials (left in ctx->part); returns the number of partials in *n_splits.
+int vlac_launch_layer_body(vlac_ctx* ctx, vlac_cache* c, int layer, bf16* hidden, int* n_splits, cudaStream_t s);
+
+int vlac_launch_decode_attention(vlac_ctx* ctx, vlac_cache* c, int layer, int pos, cudaStream_t s);
+
+// ---- decode (decode_kernels.cu)
+int vlac_decode_setup(vlac_ctx* ctx);
+int vlac_launch_last_row(vlac_ctx* ctx, vlac_cache* c, const bf16* hidden, cudaStream_t s);
+int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens, int tok_stride, int tok_index,
+                            int pos, cudaStream_t s);
+int vlac_launch_logits_argmax(vlac_ctx* ctx, vlac_cache* c, int* tokens_out, int tok_stride, int tok_index,
+                              float* logits_copy, long long copy_stride, cudaStream_t s);
