@@ -173,6 +173,15 @@ int vlac_selection_view(vlac_cache* cache, vlac_selection* out);
 /* Number of kernels the library launched since the context was created (monotonic). */
 unsigned long long vlac_launch_count(const vlac_ctx* ctx);
 
+/* Measurement aid (the paper has no counterpart): while enabled, the library brackets every launch of
+ * its single-row matrix-vector kernel (the kernel that streams the weights during the action-token
+ * passes) with CUDA events on the caller's stream, up to 4096 launches.  vlac_profile(ctx, 1) clears
+ * the record and starts; vlac_profile(ctx, 0) stops.  vlac_profile_read waits for the recorded events
+ * and returns the summed device time (ms), the summed weight bytes those launches streamed, and their
+ * count. */
+int vlac_profile(vlac_ctx* ctx, int enable);
+int vlac_profile_read(vlac_ctx* ctx, double* ms_total, unsigned long long* bytes_total, int* n_launches);
+
 /* Nonzero if a device-side bounded wait gave up since the context was created (reads one int
  * back; synchronises the stream). */
 int vlac_device_error(vlac_ctx* ctx, void* stream);

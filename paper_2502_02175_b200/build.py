@@ -34,7 +34,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [nvcc, "-shared", "-Xcompiler", "-fPIC", "-O3", "-std=c++17", "-lineinfo",
            "-gencode", "arch=compute_100a,code=sm_100a",
            "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-           "-o", LIB] + sources() + ["-lcuda"]
+           "-o", LIB] + sources()
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

@@ -219,11 +219,18 @@ int launch_gemv(vlac_ctx* ctx, const GemvArgs& a, cudaStream_t s) {
   const int NB = nb <= 1 ? 1 : (nb <= 2 ? 2 : (nb <= 4 ? 4 : 8));
   const size_t smem = (size_t)NB * a.K * sizeof(bf16);
   const int grid = ctx->n_sm * 2;
+  const bool timed = ctx->prof_on && ctx->prof_n < VLAC_PROF_CAP;
+  if (timed) VLAC_CUDA_CHECK(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n], s));
   switch (NB) {
     case 1: gemv_pair_kernel<1><<<grid, 256, smem, s>>>(a); break;
     case 2: gemv_pair_kernel<2><<<grid, 256, smem, s>>>(a); break;
     case 4: gemv_pair_kernel<4><<<grid, 256, smem, s>>>(a); break;
     default: gemv_pair_kernel<8><<<grid, 256, smem, s>>>(a); break;
+  }
+  if (timed) {
+    VLAC_CUDA_CHECK(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n + 1], s));
+    const unsigned long long mats = a.mode == GV_QKV ? 3ull : (a.mode == GV_SWIGLU ? 2ull : 1ull);
+    ctx->prof_bytes[ctx->prof_n++] = mats * (unsigned long long)a.N * a.K * sizeof(bf16);
   }
   VLAC_LAUNCH_CHECK(ctx);
   return VLAC_OK;

@@ -50,6 +50,11 @@ void free_ctx_buffers(vlac_ctx* c) {
   cudaFree(c->xn); cudaFree(c->q); cudaFree(c->ao); cudaFree(c->hm); cudaFree(c->part); cudaFree(c->scratch);
   cudaFree(c->probs); cudaFree(c->hidden); cudaFree(c->x_dec); cudaFree(c->q_dec); cudaFree(c->ao_dec);
   cudaFree(c->hm_dec); cudaFree(c->logits); cudaFree(c->argmax_tmp); cudaFree(c->dev_error);
+  if (c->prof_ev) {
+    for (int i = 0; i < 2 * VLAC_PROF_CAP; ++i) if (c->prof_ev[i]) cudaEventDestroy(c->prof_ev[i]);
+    free(c->prof_ev);
+  }
+  free(c->prof_bytes);
 }
 
 void free_cache_buffers(vlac_cache* c) {
@@ -352,6 +357,32 @@ int vlac_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, con
 }
 
 unsigned long long vlac_launch_count(const vlac_ctx* ctx) { return ctx ? ctx->launches : 0ull; }
+
+int vlac_profile(vlac_ctx* ctx, int enable) {
+  if (!ctx) return VLAC_ERR_INVALID_ARG;
+  if (enable && !ctx->prof_ev) {
+    ctx->prof_ev = (cudaEvent_t*)calloc(2 * VLAC_PROF_CAP, sizeof(cudaEvent_t));
+    ctx->prof_bytes = (unsigned long long*)calloc(VLAC_PROF_CAP, sizeof(unsigned long long));
+    if (!ctx->prof_ev || !ctx->prof_bytes) return VLAC_ERR_OOM;
+    for (int i = 0; i < 2 * VLAC_PROF_CAP; ++i) VLAC_CUDA_CHECK(cudaEventCreate(&ctx->prof_ev[i]));
+  }
+  ctx->prof_on = enable ? 1 : 0;
+  if (enable) ctx->prof_n = 0;
+  return VLAC_OK;
+}
+
+int vlac_profile_read(vlac_ctx* ctx, double* ms_total, unsigned long long* bytes_total, int* n_launches) {
+  if (!ctx || !ms_total || !bytes_total || !n_launches) return VLAC_ERR_INVALID_ARG;
+  double ms = 0.0; unsigned long long bytes = 0ull;
+  for (int i = 0; i < ctx->prof_n; ++i) {
+    VLAC_CUDA_CHECK(cudaEventSynchronize(ctx->prof_ev[2 * i + 1]));
+    float t = 0.f;
+    VLAC_CUDA_CHECK(cudaEventElapsedTime(&t, ctx->prof_ev[2 * i], ctx->prof_ev[2 * i + 1]));
+    ms += t; bytes += ctx->prof_bytes[i];
+  }
+  *ms_total = ms; *bytes_total = bytes; *n_launches = ctx->prof_n;
+  return VLAC_OK;
+}
 
 int vlac_device_error(vlac_ctx* ctx, void* stream) {
   if (!ctx) return VLAC_ERR_INVALID_ARG;

@@ -45,7 +45,12 @@ struct vlac_ctx {
   float *logits;                     // [max_batch][vocab]
   unsigned long long *argmax_tmp;    // [max_batch][VLAC_ARGMAX_BLOCKS]
   int *dev_error;                    // device int: nonzero if a bounded wait gave up
+  // optional per-launch timing of the matrix-vector kernel (vlac_profile)
+  int prof_on, prof_n;
+  cudaEvent_t* prof_ev;              // [2 * VLAC_PROF_CAP]
+  unsigned long long* prof_bytes;    // [VLAC_PROF_CAP] weight bytes streamed by each timed launch
 };
+#define VLAC_PROF_CAP 4096
 #define VLAC_ARGMAX_BLOCKS 64
 
 struct vlac_cache {

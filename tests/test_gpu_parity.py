@@ -1,0 +1,259 @@
+"""Parity of the CUDA library (through its C ABI) with the CPU checker on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import vla_cache_oracle as orc
+from paper_2502_02175_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def H():
+    import gpu_harness
+    return gpu_harness
+
+
+@pytest.fixture(scope="module")
+def vb():
+    from paper_2502_02175_b200 import binding
+    return binding
+
+
+def _tiny_inputs(seed=0):
+    cfg = synth.tiny_config()
+    model = synth.make_model(cfg, seed)
+    ids = synth.make_prompt_ids(cfg, seed)
+    rng = np.random.default_rng(seed + 1)
+    feats = synth.f32_to_bf16(rng.standard_normal((1, cfg.n_vision, cfg.hidden), dtype=np.float32))
+    return cfg, model, ids, feats
+
+
+class _DummyModel:
+    """Weight table whose pointers all alias one small buffer: enough for calls that never read weights."""
+
+    def __init__(self, vb, n_layers):
+        self.buf = torch.zeros(64, dtype=torch.float32, device="cuda")
+        p = self.buf.data_ptr()
+        self.layer_structs = (vb.vlac_layer_w * n_layers)()
+        for i in range(n_layers):
+            for name, _ in vb.vlac_layer_w._fields_:
+                setattr(self.layer_structs[i], name, p)
+        import ctypes as C
+        self.weights = vb.vlac_weights()
+        self.weights.layers = C.cast(self.layer_structs, C.POINTER(vb.vlac_layer_w))
+        for name in ("embed", "proj", "g_final", "lm_head", "rope_cos", "rope_sin"):
+            setattr(self.weights, name, p)
+
+
+# ------------------------------------------------------------------------------------- selection
+def _select_case(H, vb, cfg, prev, cur, attn, params, batch=1):
+    sess = H.Session(cfg, None, batch=batch, dev_model=_DummyModel(vb, cfg.n_layers))
+    try:
+        for b in range(batch):
+            sess.set_warm_state(prev[b], attn[b], seq=b)
+        gp, keep = H.gparams(params)
+        sel = vb.vlac_select(sess.ctx, sess.cache, torch.from_numpy(np.stack(cur)).to("cuda").contiguous(), gp)
+        got = vb.selection_to_host(sel)
+        for b in range(batch):
+            want = orc.select(cfg, cur[b], sess.ocache[b], params)
+            H.check_selection(got, want, b, cfg, where=f"seq {b}")
+        return got
+    finally:
+        sess.close()
+
+
+def test_select_tiny_tie_case(H, vb):
+    """51 bit-identical patches: the tie rule alone decides the top-k (Eq. topk)."""
+    cfg = synth.tiny_config()
+    prev, cur, _ = synth.rerandomised_pair(cfg, 0, 13)
+    attn = synth.scripted_attention(cfg, 0)
+    for params in (H.oparams(top_k=32), H.oparams(top_k=32, alpha_override=[0.5, 1.0]),
+                   H.oparams(top_k=32, k_ent=4.0), H.oparams(top_k=0), H.oparams(top_k=64, tau_task=1.0),
+                   H.oparams(top_k=32, tau_task=0.004, task_mode=1), H.oparams(top_k=40, layer_mask=[False, True])):
+        got = _select_case(H, vb, cfg, [prev], [cur], [attn], params)
+    assert got["M"].shape == (1, 2)
+
+
+@pytest.mark.parametrize("seed", [3, 4])
+def test_select_7b_shape_episode_frames(H, vb, seed):
+    """32 layers, 256 vision tokens, noisy frames with moving blobs, scripted attention (Alg. 1, Sec. 3.4)."""
+    cfg = synth.llama7b_config(n_layers=32)
+    ep = synth.make_episode(cfg.with_layers(1), seed, 3)
+    attn = synth.scripted_attention(cfg, seed, hot_tokens=ep.touched[1])
+    for params in (H.oparams(), H.oparams(k_ent=3.0), H.oparams(top_k=256, k_ent=1.5), H.oparams(tau=0.85, top_k=180, tau_task=0.7)):
+        got = _select_case(H, vb, cfg, [ep.frames[1]], [ep.frames[2]], [attn], params)
+    assert got["M"].min() >= cfg.n_text
+
+
+def test_select_dual_camera_batch(H, vb):
+    """Two cameras, three sequences with different change rates: one global top-k per sequence."""
+    cfg = synth.dual_camera_config(n_layers=8)
+    prevs, curs, attns = [], [], []
+    for b, frac in enumerate((0.1, 0.5, 0.9)):
+        ep = synth.make_episode(cfg.with_layers(1), 50 + b, 2, changed_fraction=[None, frac])
+        prevs.append(ep.frames[0]); curs.append(ep.frames[1])
+        attns.append(synth.scripted_attention(cfg, 50 + b, hot_tokens=ep.touched[1][:20]))
+    _select_case(H, vb, cfg, prevs, curs, attns, H.oparams(top_k=200, k_ent=2.0), batch=3)
+
+
+def test_select_cold_cache_recomputes_everything(H, vb):
+    cfg = synth.tiny_config()
+    sess = H.Session(cfg, None, dev_model=_DummyModel(vb, cfg.n_layers))
+    try:
+        _, cur, _ = synth.rerandomised_pair(cfg, 0, 13)
+        gp, _ = H.gparams(H.oparams())
+        got = vb.selection_to_host(vb.vlac_select(sess.ctx, sess.cache, torch.from_numpy(cur).to("cuda"), gp))
+        assert np.all(got["M"] == cfg.seq_len)
+        assert np.array_equal(got["rows"][0, 1], np.arange(cfg.seq_len))
+    finally:
+        sess.close()
+
+
+# ------------------------------------------------------------------------------------- one layer
+def _layer_case(H, vb, cfg, model, seed, reuse_count):
+    """Stale K/V from one set of hidden states, then a partial forward of other hidden states."""
+    L = cfg.seq_len
+    cos, sin = model["rope_cos"], model["rope_sin"]
+    lw = model["layers"][0]
+    h_old = orc.widen_bf16(synth.make_hidden(cfg, seed)[0])
+    h_new_bits = synth.make_hidden(cfg, seed + 1)[0]
+    # checker: full pass on the old states fills the cache, partial pass on the new ones
+    K = np.zeros((cfg.max_seq, cfg.n_heads, cfg.head_dim)); V = np.zeros_like(K)
+    hid = np.zeros((cfg.max_seq, cfg.hidden)); hid[:L] = h_old
+    orc.layer_forward(cfg, lw, K, V, hid, np.arange(L), cos, sin)
+    rng = np.random.default_rng(seed)
+    skipped = np.sort(rng.choice(cfg.n_vision, size=reuse_count, replace=False)) + cfg.n_text_pre
+    rows = np.setdiff1d(np.arange(L), skipped)
+    sess = H.Session(cfg, model)
+    try:
+        sess.write_kv(vb.PART_K, 0, K); sess.write_kv(vb.PART_V, 0, V)
+        # the checker continues from the bf16-rounded cache the library holds
+        K = sess.read_kv(vb.PART_K, 0); V = sess.read_kv(vb.PART_V, 0)
+        hid = np.zeros((cfg.max_seq, cfg.hidden)); hid[:L] = orc.widen_bf16(h_new_bits)
+        before = hid.copy()
+        emitted = orc.layer_forward(cfg, lw, K, V, hid, rows, cos, sin)
+        M = np.full((1, cfg.n_layers), len(rows), np.int32)
+        R = np.zeros((1, cfg.n_layers, L), np.int32); R[0, :, :len(rows)] = rows
+        vb.vlac_select_import(sess.ctx, sess.cache, M, R)
+        d_h = vb.upload_bf16(h_new_bits[None])
+        vb.vlac_layer_forward(sess.ctx, sess.cache, 0, d_h)
+        torch.cuda.synchronize()
+        g_h = H.bf16_tensor_to_f64(d_h)[0]
+        assert H.rel_err(g_h[rows], hid[rows]) <= H.TOL
+        if len(skipped):
+            assert np.array_equal(g_h[skipped], before[skipped])          # untouched rows
+        gK, gV = sess.read_kv(vb.PART_K, 0), sess.read_kv(vb.PART_V, 0)
+        assert H.rel_err(gK[:L], K[:L]) <= H.TOL and H.rel_err(gV[:L], V[:L]) <= H.TOL
+        if len(skipped):
+            assert np.array_equal(gK[skipped], K[skipped]) and np.array_equal(gV[skipped], V[skipped])   # reused entries kept
+        g_attn = sess.read_attn(vb.PART_ATTN_NEXT)[0]
+        assert H.rel_err(g_attn, emitted) <= H.TOL
+        return H.rel_err(g_h[rows], hid[rows])
+    finally:
+        sess.close()
+
+
+@pytest.mark.parametrize("reuse", [0, 1, 20, 64])
+def test_layer_forward_tiny(H, vb, reuse):
+    cfg = synth.tiny_config().with_layers(1)
+    model = synth.make_model(cfg, 5)
+    _layer_case(H, vb, cfg, model, 10 + reuse, reuse)
+
+
+@pytest.mark.parametrize("reuse", [0, 26, 100, 230])
+def test_layer_forward_7b_shape(H, vb, reuse):
+    """Single Llama-2-7B-shaped layer, 34 prompt + 256 vision tokens, reuse swept (M = 290 ... 60)."""
+    cfg = synth.llama7b_config(n_layers=1)
+    model = synth.make_model(cfg, 6)
+    _layer_case(H, vb, cfg, model, 20 + reuse, reuse)
+
+
+# ------------------------------------------------------------------------------------- whole step
+def test_step_tiny_episode(H, vb):
+    """Cold step, then cached steps with the tie-rule frames; selections bit-exact, logits within tolerance,
+    tokens identical wherever the checker's top-2 margin exceeds twice the logit error."""
+    cfg, model, ids, feats = _tiny_inputs()
+    prev, cur, changed = synth.rerandomised_pair(cfg, 0, 13)
+    sess = H.Session(cfg, model)
+    try:
+        rng = np.random.default_rng(3)
+        frames = [prev, cur, cur, prev]
+        total_guarded = 0
+        for t, fr in enumerate(frames):
+            f = feats.copy()
+            if t > 0:
+                for v in changed:
+                    f[0, v] = synth.f32_to_bf16(rng.standard_normal(cfg.hidden, dtype=np.float32))
+            params = H.oparams(top_k=32, alpha_override=[0.5, 1.0]) if t != 2 else H.oparams(top_k=32, k_ent=50.0)
+            r = H.run_step_pair(sess, fr[None], f, ids, params)[0]
+            assert r["logit_err"] <= H.TOL and r["attn_err"] <= H.TOL, (t, r)
+            if t == 0:
+                assert np.all(r["M"] == cfg.seq_len)
+            if t == 1:
+                assert r["M"][1] < cfg.seq_len
+            total_guarded += r["guarded"]
+        assert total_guarded <= 2 * len(frames)
+    finally:
+        sess.close()
+
+
+def test_step_force_full_equals_cold_step(H, vb):
+    """The no-reuse step of the same library equals a cold step on the same inputs, bit for bit."""
+    cfg, model, ids, feats = _tiny_inputs(1)
+    prev, cur, _ = synth.rerandomised_pair(cfg, 1, 13)
+    outs = []
+    for mode in ("cold", "full"):
+        sess = H.Session(cfg, model)
+        try:
+            gp, keep = H.gparams(H.oparams(top_k=32, alpha_override=[1.0, 1.0]))
+            tok = torch.zeros((1, cfg.n_action), dtype=torch.int32, device="cuda")
+            lg = torch.zeros((1, cfg.n_action, cfg.vocab), dtype=torch.float32, device="cuda")
+            args = (vb.upload_bf16(feats), torch.from_numpy(ids).to("cuda"))
+            if mode == "full":
+                vb.vlac_step(sess.ctx, sess.cache, torch.from_numpy(prev[None]).to("cuda"), *args, gp, False, tok, lg)
+            vb.vlac_step(sess.ctx, sess.cache, torch.from_numpy(cur[None]).to("cuda"), *args, gp, mode == "full", tok, lg)
+            torch.cuda.synchronize()
+            outs.append((tok.cpu().numpy().copy(), lg.cpu().numpy().copy()))
+        finally:
+            sess.close()
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+
+
+def test_step_7b_shape_two_layers(H, vb):
+    """7B-shaped layers, vocabulary 32000, 290 tokens: cold step then two cached steps of a blob episode."""
+    cfg = synth.llama7b_config(n_layers=2)
+    model = synth.make_model(cfg, 8)
+    ids = synth.make_prompt_ids(cfg, 8)
+    ep = synth.make_episode(cfg, 8, 3)
+    sess = H.Session(cfg, model)
+    try:
+        for t in range(3):
+            params = H.oparams(alpha_override=[0.6, 1.0]) if t < 2 else H.oparams(k_ent=2000.0)
+            r = H.run_step_pair(sess, ep.frames[t][None], ep.feats[t][None], ids, params)[0]
+            assert r["logit_err"] <= H.TOL and r["attn_err"] <= H.TOL, (t, r)
+            if t == 1:
+                assert r["M"][1] < cfg.seq_len, "the cached step must actually reuse tokens"
+    finally:
+        sess.close()
+
+
+def test_step_batch_of_three_ragged(H, vb):
+    """Three independent sequences per step with different changed fractions (ragged row counts)."""
+    cfg = synth.tiny_config()
+    model = synth.make_model(cfg, 2)
+    B = 3
+    ids = synth.make_prompt_ids(cfg, 2, batch=B)
+    pairs = [synth.rerandomised_pair(cfg, 20 + b, n) for b, n in enumerate((5, 30, 60))]
+    rng = np.random.default_rng(7)
+    feats = synth.f32_to_bf16(rng.standard_normal((B, cfg.n_vision, cfg.hidden), dtype=np.float32))
+    sess = H.Session(cfg, model, batch=B)
+    try:
+        r0 = H.run_step_pair(sess, np.stack([p[0] for p in pairs]), feats, ids, H.oparams(top_k=64, tau_task=1.0, alpha_override=[1.0, 1.0]))
+        r1 = H.run_step_pair(sess, np.stack([p[1] for p in pairs]), feats, ids, H.oparams(top_k=64, tau_task=1.0, alpha_override=[1.0, 1.0]))
+        assert [int(r["M"][0]) for r in r1] == [cfg.seq_len - (64 - n) for n in (5, 30, 60)]
+        for r in r0 + r1:
+            assert r["logit_err"] <= H.TOL and r["attn_err"] <= H.TOL
+    finally:
+        sess.close()
