@@ -1,0 +1,345 @@
+"""Benchmark of the cached control step (VLA-Cache, arxiv 2502.02175) on a 7B-shaped decoder.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--layers 32]
+
+A "step" is one control step: selection, partial prefill of all layers over the rows the
+selection keeps, and greedy generation of the 7 action tokens.  Workload: 32-layer Llama-2-7B
+shape (bf16, vocabulary 32000, random-init), 34 prompt + 256 vision tokens, a synthetic episode
+(static noise background, 1-3 moving blobs, Gaussian pixel noise sigma 2), paper defaults
+tau 0.996 / top-k 100 / tau_task 0.5.  The path does not shard: with N > 1 every rank runs an
+independent replica on its own GPU (no collective), and the value is the sum over replicas.
+
+One JSON line is printed by rank 0.  `value` is action tokens per second with all inputs already
+in HBM; `e2e` is the same through the C ABI with pinned-host inputs copied in and the tokens
+copied out inside the timed region.  `roofline` describes the kernel that dominates the step
+(the single-row matrix-vector kernel streaming the weights during the action-token passes).
+`--impl reference` times the CPU checker on the host cores instead (a bounded sample per step).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "cached_step_action_tokens_per_s"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.samples, self.stop_flag, self.thread = index, [], False, None
+
+    def _run(self):
+        while not self.stop_flag:
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-i", str(self.index)],
+                                     capture_output=True, text=True, timeout=5).stdout.strip()
+                if out:
+                    self.samples.append([x.strip() for x in out.split(",")])
+            except Exception:
+                pass
+            time.sleep(0.2)
+
+    def __enter__(self):
+        self.thread = threading.Thread(target=self._run, daemon=True)
+        self.thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self.stop_flag = True
+        self.thread.join(timeout=10)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        for s in self.samples:
+            try:
+                sm.append(float(s[0])); mx.append(float(s[1]))
+            except Exception:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), s[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def _workload(layers):
+    from paper_2502_02175_b200 import synth
+    return synth.llama7b_config(n_layers=layers)
+
+
+def _algorithmic_step_bytes(cfg, M_mean):
+    """Bytes one cached step must move: every weight once per pass (1 prefill + n_action-1 single-row
+    passes), the lm_head once per token, the K/V cache read once per pass."""
+    P = 4 * cfg.hidden * cfg.hidden + 3 * cfg.hidden * cfg.ffn
+    w_layers = 2 * P * cfg.n_layers
+    lm = 2 * cfg.vocab * cfg.hidden
+    kv = 2 * 2 * cfg.seq_len * cfg.hidden * cfg.n_layers
+    proj = 2 * cfg.hidden * cfg.hidden
+    return cfg.n_action * (w_layers + lm + kv) + proj
+
+
+def _cpu_sample(cfg, seed=0):
+    """One bounded sample of the workload on the CPU checker: selection + one 7B-shaped layer of the
+    cached prefill and of the six single-row passes + the seven lm_head products; the layer part is
+    scaled by n_layers.  Returns seconds for a whole step estimated that way and the thread count."""
+    from oracle import vla_cache_oracle as orc
+    from paper_2502_02175_b200 import synth
+    c1 = cfg.with_layers(1)
+    model = synth.make_model(c1, seed)
+    ids = synth.make_prompt_ids(c1, seed)[0]
+    ep = synth.make_episode(c1, seed, 2)
+    cache = orc.new_cache(c1)
+    params = orc.SelectParams(alpha_override=[1.0])
+    orc.step(c1, model, cache, ep.frames[0], ep.feats[0], ids, params)        # cold step: not timed
+    t0 = time.perf_counter()
+    sel = orc.select(c1, ep.frames[1], cache, params)
+    t_sel = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    hidden = orc.input_rows(c1, model, ep.feats[1], ids)
+    t_in = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    orc.layer_forward(c1, model["layers"][0], cache.K[0], cache.V[0], hidden, sel.rows[0], model["rope_cos"], model["rope_sin"])
+    for i in range(1, c1.n_action):
+        pos = c1.seq_len - 1 + i
+        hidden[pos] = orc.widen_bf16(model["embed"][int(ids[0])])
+        orc.layer_forward(c1, model["layers"][0], cache.K[0], cache.V[0], hidden, np.asarray([pos]),
+                          model["rope_cos"], model["rope_sin"], emit_attention=False)
+    t_layer = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    for i in range(c1.n_action):
+        orc._logits(c1, model, hidden[c1.seq_len - 1 + i])
+    t_head = time.perf_counter() - t0
+    total = t_sel + t_in + t_layer * cfg.n_layers + t_head
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    return total, threads, {"select_s": t_sel, "input_rows_s": t_in, "one_layer_all_passes_s": t_layer, "lm_head_x7_s": t_head,
+                            "rows_layer0": int(sel.M[0])}
+
+
+SAMPLE_TEXT = ("one cached control step estimated from: selection + input rows + ONE 7B-shaped layer run for the partial "
+               "prefill and the 6 single-row passes (time x n_layers) + 7 lm_head products")
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg = _workload(args.layers)
+    times = []
+    for i in range(args.warmup + args.steps):
+        if i >= args.warmup and len(times) and sum(times) > 150:
+            break
+        t, threads, parts = _cpu_sample(cfg, seed=i)
+        if i >= args.warmup or args.steps == 0:
+            times.append(t)
+        if i == 0 and t * (args.warmup + args.steps) > 240:          # keep the whole run within minutes
+            args.warmup = 0
+    ms = 1e3 * float(np.mean(times)) if times else float("nan")
+    value = cfg.n_action / (ms / 1e3)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": len(times),
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"cfg3: {cfg.n_layers}-layer Llama-2-7B shape, 34 prompt + 256 vision tokens, 7 action tokens", "batch": 1},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": SAMPLE_TEXT},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2502_02175_b200 import build
+    build.build()
+    from paper_2502_02175_b200 import binding as vb
+    from paper_2502_02175_b200 import synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    cfg = _workload(args.layers)
+    K, W = args.steps, args.warmup
+    dev = vb.DeviceModel.random(cfg, seed=1234 + rank)
+    ctx = vb.vlac_create(vb.make_config(cfg, 1), dev.weights)
+    cache = vb.vlac_cache_alloc(ctx, 1)
+    n_frames = 1 + W + K
+    ep = synth.make_episode(cfg, 3000 + rank, n_frames)
+    ids_h = synth.make_prompt_ids(cfg, 3000 + rank)
+    frames_d = torch.from_numpy(ep.frames).to("cuda")
+    feats_d = vb.upload_bf16(ep.feats)
+    ids_d = torch.from_numpy(ids_h).to("cuda")
+    tokens = torch.zeros((1, cfg.n_action), dtype=torch.int32, device="cuda")
+    # entropy-scaled ratios; the k of Eq. (reuse_ratio) has no published value: calibrated on the first
+    # cached step so that the median layer reuses 3/4 of P_final, then frozen
+    params, keep = vb.make_params(k_ent=1.0)
+
+    def step(t, p=params, full=False):
+        vb.vlac_step(ctx, cache, frames_d[t:t + 1], feats_d[t:t + 1], ids_d, p, full, tokens)
+
+    step(0)                                                     # cold step
+    step(1)
+    sel = vb.selection_to_host(vb.vlac_selection_view(cache))
+    k_ent = 1.0
+    # alpha^l = k * cum^l; choose k so that the median alpha over layers is 0.75 (clamped later to [0,1])
+    # cum^l is recovered from the applied ratios only when they are unclamped, so calibrate from a probe with tiny k
+    probe, keep2 = vb.make_params(k_ent=1e-6)
+    got = vb.selection_to_host(vb.vlac_select(ctx, cache, frames_d[1:2], probe))
+    cum = got["alpha"][0] / 1e-6
+    med = float(np.median(cum))
+    ratio_mode = "entropy (Eq. reuse_ratio), k calibrated once to a median ratio of 0.75"
+    if med > 0:
+        k_ent = 0.75 / med
+        params, keep = vb.make_params(k_ent=k_ent)
+    else:       # degenerate attention (no entropy drop anywhere): fixed ratio instead
+        ratio_mode = "fixed ratio 0.75 (entropy ratios were all <= 0)"
+        params, keep = vb.make_params(alpha_override=[0.75] * cfg.n_layers)
+
+    def timed(n, first, full=False):
+        step(first - 1, params, full)           # put the cache in the state the first timed frame expects
+        barrier()
+        l0 = vb.vlac_launch_count(ctx)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for i in range(n):
+            step(first + i, params, full)
+        ev1.record()
+        barrier()
+        return ev0.elapsed_time(ev1), vb.vlac_launch_count(ctx) - l0
+
+    for i in range(W):
+        step(1 + i, params)
+    with ClockSampler(local) as clocks:
+        ms_total, launches = timed(K, 1 + W)
+    sel = vb.selection_to_host(vb.vlac_selection_view(cache))
+    M = sel["M"][0].astype(float)
+    ms_step = ms_total / K
+
+    # roofline of the dominant kernel: same steps again with per-launch events on the library's stream
+    vb.vlac_profile(ctx, True)
+    timed(min(K, 4), 1 + W)
+    vb.vlac_profile(ctx, False)
+    k_ms, k_bytes, k_n = vb.vlac_profile_read(ctx)
+    # the same library with reuse off
+    for i in range(2):
+        step(1 + W + i, params, True)
+    ms_full, _ = timed(K, 1 + W, full=True)
+    ms_full /= K
+
+    # end to end through the C ABI: pinned host inputs in, tokens out, every step
+    frames_h = torch.from_numpy(ep.frames).pin_memory()
+    feats_h = torch.from_numpy(ep.feats.view(np.int16)).pin_memory()
+    ids_p = torch.from_numpy(ids_h).pin_memory()
+    tok_h = torch.zeros((1, cfg.n_action), dtype=torch.int32).pin_memory()
+    f_d = torch.empty_like(frames_d[0:1]); x_d = torch.empty((1, cfg.n_vision, cfg.hidden), dtype=torch.bfloat16, device="cuda")
+    i_d = torch.empty_like(ids_d)
+
+    def e2e_step(t):
+        f_d.copy_(frames_h[t:t + 1], non_blocking=True)
+        x_d.view(torch.int16).copy_(feats_h[t:t + 1], non_blocking=True)
+        i_d.copy_(ids_p, non_blocking=True)
+        vb.vlac_step(ctx, cache, f_d, x_d, i_d, params, False, tokens)
+        tok_h.copy_(tokens, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    e2e_step(W)
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(K):
+        e2e_step(1 + W + i)
+    barrier()
+    ms_e2e = 1e3 * (time.perf_counter() - t0) / K
+    h2d = int(frames_h[0:1].numel() + feats_h[0:1].numel() * 2 + ids_p.numel() * 4)
+    d2h = int(tok_h.numel() * 4)
+
+    # max over ranks
+    if world > 1:
+        t = torch.tensor([ms_step, ms_e2e, ms_full], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step, ms_e2e, ms_full = (float(x) for x in t.cpu())
+    if rank == 0:
+        peak, peak_kind = _peaks()
+        achieved = (k_bytes / 1e9) / (k_ms / 1e3) if k_ms > 0 else 0.0
+        step_bytes = _algorithmic_step_bytes(cfg, float(M.mean()))
+        cpu_s, cpu_threads, cpu_parts = _cpu_sample(cfg) if world == 1 else (None, None, None)
+        line = {
+            "metric": METRIC, "value": world * cfg.n_action / (ms_step / 1e3), "unit": UNIT, "n_gpus": world,
+            "steps": K, "warmup": W, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"cfg3: {cfg.n_layers}-layer Llama-2-7B shape, 34 prompt + 256 vision tokens, 7 action tokens",
+                       "batch": 1, "replicas": world, "tau": 0.996, "top_k": 100, "tau_task": 0.5, "k_ent": k_ent, "ratio_mode": ratio_mode,
+                       "rows_per_layer_mean": float(M.mean()), "rows_per_layer_min": float(M.min()), "seq_len": cfg.seq_len,
+                       "l2": "each step streams the 13 GB of weights 7 times: inputs far exceed the 126 MB L2"},
+            "e2e": {"value": world * cfg.n_action / (ms_e2e / 1e3), "unit": UNIT, "ms_per_step": ms_e2e,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": int(launches),
+            "clocks": clocks.summary(),
+            "roofline": {"bound": "hbm", "kernel": "gemv_pair_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                         "launches_timed": k_n, "avg_launch_us": 1e3 * k_ms / max(k_n, 1)},
+            "step_roofline": {"algorithmic_bytes": step_bytes, "floor_ms": step_bytes / (peak * 1e6),
+                              "frac": (step_bytes / (peak * 1e6)) / ms_step},
+            "full_recompute": {"ms_per_step": ms_full, "speedup_cached": ms_full / ms_step},
+            "control_hz": 1e3 / ms_step,
+            "cpu_baseline": None if cpu_s is None else {"value": cfg.n_action / cpu_s, "unit": UNIT, "cores": cpu_threads,
+                                                        "kind": "oracle", "sample": SAMPLE_TEXT, "parts": cpu_parts},
+            "paper_context": "paper: up to 1.7x CUDA latency, OpenVLA 51.91 -> 31.83 ms per step on one RTX 4090 (bf16, real weights)",
+        }
+        print(json.dumps(line), flush=True)
+    vb.vlac_cache_free(cache)
+    vb.vlac_destroy(ctx)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=32)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
