@@ -7,6 +7,7 @@
 // several loads are kept in flight per lane.  The pairing puts the two halves of a rotary pair, or
 // the gate and up rows of one FFN feature, in the same warp so the epilogue needs no exchange.
 #include "vlac_internal.h"
+#include "launch_util.h"
 
 namespace {
 
@@ -43,13 +44,75 @@ __device__ __forceinline__ void fma8(float& acc, const uint4& w, const uint4& x)
   }
 }
 
+struct UnitRows { const uint4 *pa, *pb; int rowA, rowB, mat; };
+
+__device__ __forceinline__ UnitRows unit_rows(const GemvArgs& a, int u) {
+  UnitRows r;
+  const int K = a.K;
+  if (a.mode == GV_QKV) {
+    const int half = a.d / 2;
+    r.mat = u / (a.N / 2);
+    const int q = u - r.mat * (a.N / 2);
+    const int h = q / half, j = q - h * half;
+    r.rowA = h * a.d + j; r.rowB = r.rowA + half;
+    const bf16* W = r.mat == 0 ? a.w0 : (r.mat == 1 ? a.w1 : a.w2);
+    r.pa = reinterpret_cast<const uint4*>(W + (size_t)r.rowA * K);
+    r.pb = reinterpret_cast<const uint4*>(W + (size_t)r.rowB * K);
+  } else if (a.mode == GV_SWIGLU) {
+    r.mat = 0; r.rowA = r.rowB = u;
+    r.pa = reinterpret_cast<const uint4*>(a.w0 + (size_t)u * K);
+    r.pb = reinterpret_cast<const uint4*>(a.w1 + (size_t)u * K);
+  } else {
+    r.mat = 0; r.rowA = 2 * u; r.rowB = min(2 * u + 1, a.N - 1);
+    r.pa = reinterpret_cast<const uint4*>(a.w0 + (size_t)r.rowA * K);
+    r.pb = reinterpret_cast<const uint4*>(a.w0 + (size_t)r.rowB * K);
+  }
+  return r;
+}
+
+// streaming loads: weights are read exactly once, keep them out of L1
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+
+#define GV_BATCH 4      // 16-byte chunks per row kept in flight per lane (two rows -> 8 loads)
+
+__device__ __forceinline__ void load_batch(uint4* va, uint4* vb, const UnitRows& r, int c0, int nchunk) {
+#pragma unroll
+  for (int t = 0; t < GV_BATCH; ++t) {
+    const int c = c0 + 32 * t;
+    if (c < nchunk) { va[t] = ld_stream(r.pa + c); vb[t] = ld_stream(r.pb + c); }
+    else { va[t] = make_uint4(0, 0, 0, 0); vb[t] = make_uint4(0, 0, 0, 0); }
+  }
+}
+
 template <int NB>
-__global__ void __launch_bounds__(256) gemv_pair_kernel(GemvArgs a) {
+__global__ void __launch_bounds__(256, 2) gemv_pair_kernel(GemvArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   bf16* xs = reinterpret_cast<bf16*>(smem_raw);           // [NB][K]
   __shared__ float red[8];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int K = a.K;
+  const int half = a.d / 2;
+  int n_units;
+  if (a.mode == GV_QKV) n_units = 3 * (a.N / 2);
+  else if (a.mode == GV_SWIGLU) n_units = a.N;
+  else n_units = (a.N + 1) / 2;
+  const int total_warps = gridDim.x * 8;
+  const int nchunk = K / 8;
+  const int bpu = (nchunk + 32 * GV_BATCH - 1) / (32 * GV_BATCH);      // load batches per unit
+  const int u0 = blockIdx.x * 8 + warp;
+  const int n_my = u0 < n_units ? (n_units - u0 + total_warps - 1) / total_warps : 0;
+  const int total_it = n_my * bpu;
+
+  // ---- first weights of this warp are requested before anything else: they depend on no earlier kernel
+  uint4 va[GV_BATCH], vb[GV_BATCH];
+  UnitRows ld_unit = unit_rows(a, min(u0, n_units - 1));
+  if (total_it > 0) load_batch(va, vb, ld_unit, lane, nchunk);
+  pdl_trigger();
+  pdl_wait();
 
   // ---- activations -> shared memory (RMSNorm here if a gain is given)
   for (int b = 0; b < NB; ++b) {
@@ -78,96 +141,87 @@ __global__ void __launch_bounds__(256) gemv_pair_kernel(GemvArgs a) {
   }
   __syncthreads();
 
-  const int half = a.d / 2;
-  int n_units;
-  if (a.mode == GV_QKV) n_units = 3 * (a.N / 2);
-  else if (a.mode == GV_SWIGLU) n_units = a.N;
-  else n_units = (a.N + 1) / 2;
-  const int total_warps = gridDim.x * 8;
-  const int nchunk = K / 8;
-
-  for (int u = blockIdx.x * 8 + warp; u < n_units; u += total_warps) {
-    const bf16 *wa, *wb;
-    int rowA, rowB, mat = 0;
-    if (a.mode == GV_QKV) {
-      mat = u / (a.N / 2);
-      const int r = u - mat * (a.N / 2);
-      const int h = r / half, j = r - h * half;
-      rowA = h * a.d + j; rowB = rowA + half;
-      const bf16* W = mat == 0 ? a.w0 : (mat == 1 ? a.w1 : a.w2);
-      wa = W + (size_t)rowA * K; wb = W + (size_t)rowB * K;
-    } else if (a.mode == GV_SWIGLU) {
-      rowA = rowB = u;
-      wa = a.w0 + (size_t)u * K; wb = a.w1 + (size_t)u * K;
-    } else {
-      rowA = 2 * u; rowB = min(2 * u + 1, a.N - 1);
-      wa = a.w0 + (size_t)rowA * K; wb = a.w0 + (size_t)rowB * K;
-    }
-    float accA[NB], accB[NB];
+  float accA[NB], accB[NB];
 #pragma unroll
-    for (int b = 0; b < NB; ++b) accA[b] = accB[b] = 0.f;
-    const uint4* pa = reinterpret_cast<const uint4*>(wa);
-    const uint4* pb = reinterpret_cast<const uint4*>(wb);
-    for (int c0 = lane; c0 < nchunk; c0 += 128) {
-      uint4 va[4], vb[4];
-#pragma unroll
-      for (int t = 0; t < 4; ++t) {
-        const int c = c0 + 32 * t;
-        if (c < nchunk) { va[t] = __ldg(pa + c); vb[t] = __ldg(pb + c); }
-        else { va[t] = make_uint4(0, 0, 0, 0); vb[t] = make_uint4(0, 0, 0, 0); }
-      }
-#pragma unroll
-      for (int t = 0; t < 4; ++t) {
-        const int c = min(c0 + 32 * t, nchunk - 1);
-#pragma unroll
-        for (int b = 0; b < NB; ++b) {
-          const uint4 xv = *reinterpret_cast<const uint4*>(xs + (size_t)b * K + c * 8);
-          fma8(accA[b], va[t], xv);
-          fma8(accB[b], vb[t], xv);
-        }
-      }
+  for (int b = 0; b < NB; ++b) accA[b] = accB[b] = 0.f;
+  UnitRows cu = ld_unit;                                    // unit being accumulated
+  int u_ld = u0, bi_ld = 0;                                 // unit / batch index of the loads in va, vb
+  for (int it = 0; it < total_it; ++it) {
+    const int c0 = lane + 32 * GV_BATCH * bi_ld;
+    const bool last_of_unit = (bi_ld == bpu - 1);
+    // request the next batch before computing on this one
+    uint4 na[GV_BATCH], nb2[GV_BATCH];
+    int u_nx = u_ld, bi_nx = bi_ld + 1;
+    if (last_of_unit) { u_nx = u_ld + total_warps; bi_nx = 0; }
+    const bool has_next = it + 1 < total_it;
+    if (has_next) {
+      if (last_of_unit) ld_unit = unit_rows(a, u_nx);
+      load_batch(na, nb2, ld_unit, lane + 32 * GV_BATCH * bi_nx, nchunk);
     }
 #pragma unroll
-    for (int b = 0; b < NB; ++b) {
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        accA[b] += __shfl_xor_sync(0xffffffffu, accA[b], o);
-        accB[b] += __shfl_xor_sync(0xffffffffu, accB[b], o);
-      }
-    }
-    if (lane == 0) {
+    for (int t = 0; t < GV_BATCH; ++t) {
+      const int c = min(c0 + 32 * t, nchunk - 1);
 #pragma unroll
       for (int b = 0; b < NB; ++b) {
-        if (b >= a.nb) break;
-        const float ya = accA[b], yb = accB[b];
-        if (a.mode == GV_QKV) {
-          if (mat == 2) {
-            bf16* dst = a.vc + ((size_t)b * a.max_seq + a.pos) * a.N;
-            dst[rowA] = __float2bfloat16(ya); dst[rowB] = __float2bfloat16(yb);
-          } else {
-            const int j = rowA % a.d;
-            const float c = a.rope_cos[(size_t)a.pos * half + j], s = a.rope_sin[(size_t)a.pos * half + j];
-            const float r1 = ya * c - yb * s, r2 = yb * c + ya * s;
-            bf16* dst = mat == 0 ? a.q_out + (size_t)b * a.N : a.kc + ((size_t)b * a.max_seq + a.pos) * a.N;
-            dst[rowA] = __float2bfloat16(r1); dst[rowB] = __float2bfloat16(r2);
-          }
-        } else if (a.mode == GV_SWIGLU) {
-          a.h_out[(size_t)b * a.N + rowA] = __float2bfloat16(ya / (1.f + __expf(-ya)) * yb);
-        } else if (a.mode == GV_RESID) {
-          a.x_out[(size_t)b * a.N + rowA] += ya;
-          if (rowB != rowA) a.x_out[(size_t)b * a.N + rowB] += yb;
-        } else {
-          a.logits[(size_t)b * a.N + rowA] = ya;
-          if (rowB != rowA) a.logits[(size_t)b * a.N + rowB] = yb;
-        }
+        const uint4 xv = *reinterpret_cast<const uint4*>(xs + (size_t)b * K + c * 8);
+        fma8(accA[b], va[t], xv);
+        fma8(accB[b], vb[t], xv);
       }
     }
+    if (last_of_unit) {
+#pragma unroll
+      for (int b = 0; b < NB; ++b) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          accA[b] += __shfl_xor_sync(0xffffffffu, accA[b], o);
+          accB[b] += __shfl_xor_sync(0xffffffffu, accB[b], o);
+        }
+      }
+      if (lane == 0) {
+        const int rowA = cu.rowA, rowB = cu.rowB, mat = cu.mat;
+#pragma unroll
+        for (int b = 0; b < NB; ++b) {
+          if (b >= a.nb) break;
+          const float ya = accA[b], yb = accB[b];
+          if (a.mode == GV_QKV) {
+            if (mat == 2) {
+              bf16* dst = a.vc + ((size_t)b * a.max_seq + a.pos) * a.N;
+              dst[rowA] = __float2bfloat16(ya); dst[rowB] = __float2bfloat16(yb);
+            } else {
+              const int j = rowA % a.d;
+              const float c = a.rope_cos[(size_t)a.pos * half + j], s = a.rope_sin[(size_t)a.pos * half + j];
+              const float r1 = ya * c - yb * s, r2 = yb * c + ya * s;
+              bf16* dst = mat == 0 ? a.q_out + (size_t)b * a.N : a.kc + ((size_t)b * a.max_seq + a.pos) * a.N;
+              dst[rowA] = __float2bfloat16(r1); dst[rowB] = __float2bfloat16(r2);
+            }
+          } else if (a.mode == GV_SWIGLU) {
+            a.h_out[(size_t)b * a.N + rowA] = __float2bfloat16(ya / (1.f + __expf(-ya)) * yb);
+          } else if (a.mode == GV_RESID) {
+            a.x_out[(size_t)b * a.N + rowA] += ya;
+            if (rowB != rowA) a.x_out[(size_t)b * a.N + rowB] += yb;
+          } else {
+            a.logits[(size_t)b * a.N + rowA] = ya;
+            if (rowB != rowA) a.logits[(size_t)b * a.N + rowB] = yb;
+          }
+        }
+      }
+#pragma unroll
+      for (int b = 0; b < NB; ++b) accA[b] = accB[b] = 0.f;
+      cu = ld_unit;
+    }
+    if (has_next) {
+#pragma unroll
+      for (int t = 0; t < GV_BATCH; ++t) { va[t] = na[t]; vb[t] = nb2[t]; }
+    }
+    u_ld = u_nx; bi_ld = bi_nx;
   }
 }
 
 __global__ void __launch_bounds__(256) embed_token_kernel(const bf16* embed, const int* tokens, int tok_stride, int tok_index,
                                                           float* x, int D, int vocab) {
   const int b = blockIdx.x;
+  pdl_trigger();
+  pdl_wait();
   int id = tokens[(size_t)b * tok_stride + tok_index];
   id = min(max(id, 0), vocab - 1);
   for (int k = threadIdx.x; k < D; k += blockDim.x) x[(size_t)b * D + k] = bf2f(embed[(size_t)id * D + k]);
@@ -189,6 +243,8 @@ __device__ __forceinline__ unsigned long long argmax_key(float v, int idx) {
 __global__ void __launch_bounds__(256) argmax_partial_kernel(const float* logits, int vocab, unsigned long long* tmp) {
   __shared__ unsigned long long red[8];
   const int b = blockIdx.y;
+  pdl_trigger();
+  pdl_wait();
   const float* row = logits + (size_t)b * vocab;
   unsigned long long best = 0ull;
   for (int n = blockIdx.x * blockDim.x + threadIdx.x; n < vocab; n += gridDim.x * blockDim.x) {
@@ -207,6 +263,8 @@ __global__ void __launch_bounds__(256) argmax_partial_kernel(const float* logits
 
 __global__ void argmax_final_kernel(const unsigned long long* tmp, int n_part, int* tokens, int tok_stride, int tok_index) {
   const int b = blockIdx.x;
+  pdl_trigger();
+  pdl_wait();
   if (threadIdx.x == 0) {
     unsigned long long best = 0ull;
     for (int i = 0; i < n_part; ++i) { const unsigned long long k = tmp[(size_t)b * n_part + i]; best = k > best ? k : best; }
@@ -222,10 +280,10 @@ int launch_gemv(vlac_ctx* ctx, const GemvArgs& a, cudaStream_t s) {
   const bool timed = ctx->prof_on && ctx->prof_n < VLAC_PROF_CAP;
   if (timed) VLAC_CUDA_CHECK(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n], s));
   switch (NB) {
-    case 1: gemv_pair_kernel<1><<<grid, 256, smem, s>>>(a); break;
-    case 2: gemv_pair_kernel<2><<<grid, 256, smem, s>>>(a); break;
-    case 4: gemv_pair_kernel<4><<<grid, 256, smem, s>>>(a); break;
-    default: gemv_pair_kernel<8><<<grid, 256, smem, s>>>(a); break;
+    case 1: VLAC_CUDA_CHECK(launch_pdl(gemv_pair_kernel<1>, dim3(grid), dim3(256), smem, s, a)); break;
+    case 2: VLAC_CUDA_CHECK(launch_pdl(gemv_pair_kernel<2>, dim3(grid), dim3(256), smem, s, a)); break;
+    case 4: VLAC_CUDA_CHECK(launch_pdl(gemv_pair_kernel<4>, dim3(grid), dim3(256), smem, s, a)); break;
+    default: VLAC_CUDA_CHECK(launch_pdl(gemv_pair_kernel<8>, dim3(grid), dim3(256), smem, s, a)); break;
   }
   if (timed) {
     VLAC_CUDA_CHECK(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n + 1], s));
@@ -262,7 +320,8 @@ int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens,
                             int pos, cudaStream_t s) {
   const vlac_config& g = ctx->cfg;
   const int D = g.hidden, F = g.ffn, B = c->batch;
-  embed_token_kernel<<<B, 256, 0, s>>>((const bf16*)ctx->w.embed, fed_tokens, tok_stride, tok_index, ctx->x_dec, D, g.vocab);
+  VLAC_CUDA_CHECK(launch_pdl(embed_token_kernel, dim3(B), dim3(256), 0, s, (const bf16*)ctx->w.embed, fed_tokens, tok_stride, tok_index,
+                             ctx->x_dec, D, g.vocab));
   VLAC_LAUNCH_CHECK(ctx);
   for (int l = 0; l < g.n_layers; ++l) {
     const vlac_layer_w& w = ctx->layers[l];
@@ -305,9 +364,11 @@ int vlac_launch_logits_argmax(vlac_ctx* ctx, vlac_cache* c, int* tokens_out, int
   a.w0 = (const bf16*)ctx->w.lm_head; a.mode = GV_LOGITS; a.nb = B; a.K = g.hidden; a.N = g.vocab; a.logits = ctx->logits; a.d = g.head_dim;
   int rc = launch_gemv(ctx, a, s);
   if (rc) return rc;
-  argmax_partial_kernel<<<dim3(VLAC_ARGMAX_BLOCKS, B), 256, 0, s>>>(ctx->logits, g.vocab, ctx->argmax_tmp);
+  VLAC_CUDA_CHECK(launch_pdl(argmax_partial_kernel, dim3(VLAC_ARGMAX_BLOCKS, B), dim3(256), 0, s, (const float*)ctx->logits, g.vocab,
+                             ctx->argmax_tmp));
   VLAC_LAUNCH_CHECK(ctx);
-  argmax_final_kernel<<<B, 32, 0, s>>>(ctx->argmax_tmp, VLAC_ARGMAX_BLOCKS, tokens_out, tok_stride, tok_index);
+  VLAC_CUDA_CHECK(launch_pdl(argmax_final_kernel, dim3(B), dim3(32), 0, s, (const unsigned long long*)ctx->argmax_tmp,
+                             (int)VLAC_ARGMAX_BLOCKS, tokens_out, tok_stride, tok_index));
   VLAC_LAUNCH_CHECK(ctx);
   if (logits_copy) {
     VLAC_CUDA_CHECK(cudaMemcpy2DAsync(logits_copy, (size_t)copy_stride * sizeof(float), ctx->logits, (size_t)g.vocab * sizeof(float),

@@ -5,7 +5,7 @@
 // Row counts live in device memory (written by the selection kernels); every grid is sized for the
 // worst case and CTAs beyond the live count exit at once, so the host never waits for a count.
 #include "vlac_internal.h"
-#include <mma.h>
+#include "launch_util.h"
 
 namespace {
 
@@ -244,6 +244,8 @@ __global__ void __launch_bounds__(128) attention_row_kernel(AttnArgs a) {
   float* p = sm + a.d;            // [max_seq]
   __shared__ float red[4];
   const int i = blockIdx.x, h = blockIdx.y, tid = threadIdx.x;
+  pdl_trigger();
+  pdl_wait();
   const int nq = a.tot ? *a.tot : a.nq_fixed;
   if (i >= nq) return;
   int b, pos;
@@ -355,7 +357,7 @@ int vlac_launch_decode_attention(vlac_ctx* ctx, vlac_cache* c, int layer, int po
   a.out = ctx->ao_dec; a.probs = nullptr;
   a.nq_fixed = B; a.fixed_pos = pos; a.L = ctx->L; a.max_seq = ctx->max_seq; a.H = g.n_heads; a.d = g.head_dim;
   a.v0 = g.n_text_pre; a.Lv = ctx->Lv; a.n_tp = g.n_text_post;
-  attention_row_kernel<<<dim3(B, g.n_heads), 128, (g.head_dim + ctx->max_seq) * sizeof(float), s>>>(a);
+  VLAC_CUDA_CHECK(launch_pdl(attention_row_kernel, dim3(B, g.n_heads), dim3(128), (g.head_dim + ctx->max_seq) * sizeof(float), s, a));
   VLAC_LAUNCH_CHECK(ctx);
   return VLAC_OK;
 }
