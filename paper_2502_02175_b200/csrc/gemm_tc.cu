@@ -1,0 +1,414 @@
+// Weight-streaming GEMM for the partial prefill on 5th-generation tensor cores (tcgen05, TMEM, TMA).
+//
+//   D[n, t] = sum_k W[n, k] * X[t, k]        W: weights [N][K] bf16, X: the recomputed rows [T][K] bf16
+//
+// The prefill multiplies every weight matrix with a few hundred rows (T = rows the selection kept), so
+// the weights are the big operand and each must cross HBM exactly once.  The operands are therefore
+// swapped: a CTA owns 128 rows of W as the M side of a 128 x T x 16 UMMA and ALL T tokens as the N
+// side; the fp32 accumulator [128 lanes][T columns] lives in tensor memory.  T is read from device
+// memory (the selection kernels wrote it); the instruction descriptor and the number of token boxes
+// are formed in the kernel, so no host round trip is needed.
+//
+// Warp roles (192 threads): warp 0 issues TMA loads into a ring of stages, warp 1 allocates TMEM and
+// issues the MMAs, warps 2-5 read the accumulator back (each its own quarter of the 128 lanes) and run
+// the epilogue.  The 128 weight rows of a tile are fetched as eight 16-row boxes whose order is chosen
+// per mode so that the two values an epilogue needs together sit 16 lanes apart in one warp:
+//   QKV     the two halves of a rotary pair  -> rotation at the row's own position, K/V scatter
+//   SWIGLU  gate row and up row of a feature -> silu(gate) * up
+//   PARTIAL plain order                      -> fp32 split-K partial (output / down projection)
+#include "vlac_internal.h"
+#include "launch_util.h"
+#include <cuda.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+namespace {
+
+constexpr int TG_QKV = 0, TG_PARTIAL = 1, TG_SWIGLU = 2;
+constexpr int TG_THREADS = 192;
+constexpr int TG_BK = 64;                       // bf16 elements per k-block = one 128-byte swizzle row
+constexpr int TG_A_BYTES = 128 * TG_BK * 2;     // 16 KB: 128 weight rows
+constexpr int TG_BOX_TOK = 64;                  // token rows per TMA box
+constexpr int TG_BOX_BYTES = TG_BOX_TOK * TG_BK * 2;   // 8 KB
+constexpr int TG_MAX_STAGES = 8;
+constexpr int TG_SMEM_RING = 208 * 1024;        // dynamic shared memory for the ring
+constexpr unsigned long long TG_WAIT_LIMIT_NS = 400000000ull;
+
+struct TcArgs {
+  const CUtensorMap* tm_a[3];     // weight matrices (16-row boxes)
+  const CUtensorMap* tm_b;        // activations [rows][K] (64-row boxes)
+  const int* tot;                 // live token count in device memory (NULL: tot_fixed)
+  int tot_fixed;
+  int K, N;                       // N = rows of one weight matrix
+  int mode, n_splits;
+  int d;                          // head_dim (QKV)
+  // epilogue operands
+  const int* rowmap;              // compact token -> b*L + pos
+  int L, max_seq;
+  const float *rope_cos, *rope_sin;
+  bf16 *q_out, *kc, *vc;          // QKV: [T][N], caches [B][max_seq][N]
+  float* part; size_t split_stride;   // PARTIAL: [split][T][N]
+  bf16* h_out;                    // SWIGLU: [T][N]
+  int* dev_error;
+};
+
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned parity) {
+  unsigned ok;
+  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+               : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait.  On expiry the CTA's abort flag is raised, `code` goes to the device error word and
+// every later wait of the CTA returns at once, so the kernel always terminates.
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, volatile int* abort_flag, int* dev_error, int code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (global_ns() - t0 > TG_WAIT_LIMIT_NS) break;
+  }
+  *abort_flag = 1;
+  if (dev_error) atomicCAS(dev_error, 0, code);
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, int x, int y, unsigned long long* bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(smem_u32(dst)), "l"(tm), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+// K-major operand, 128-byte swizzle: rows at a 128-byte pitch, 8-row groups 1024 bytes apart
+__device__ __forceinline__ unsigned long long umma_desc(const void* smem) {
+  unsigned long long d = 0;
+  d |= (unsigned long long)((smem_u32(smem) & 0x3FFFFu) >> 4);        // start address
+  d |= (unsigned long long)1 << 16;                                   // leading byte offset (unused for swizzled K-major)
+  d |= (unsigned long long)(1024 >> 4) << 32;                         // stride byte offset: 8 rows * 128 B
+  d |= (unsigned long long)1 << 46;                                   // descriptor version of this architecture
+  d |= (unsigned long long)2 << 61;                                   // SWIZZLE_128B
+  return d;
+}
+__device__ __forceinline__ unsigned umma_idesc_bf16(int M, int N) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((unsigned)(N >> 3) << 17) | ((unsigned)(M >> 4) << 24);   // f32 acc, bf16 x bf16, K-major both
+}
+__device__ __forceinline__ void umma_bf16(unsigned tmem_d, unsigned long long a, unsigned long long b, unsigned idesc, unsigned accumulate) {
+  asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+               ::"r"(tmem_d), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(unsigned long long* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(unsigned taddr, float* v) {
+  unsigned r[16];
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                 "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+               : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// First weight row of box g (16 rows) of tile `tile`, and which matrix it comes from.
+__device__ __forceinline__ void box_source(const TcArgs& a, int tile, int g, int* mat, int* row0) {
+  if (a.mode == TG_QKV) {
+    const int tiles_per_mat = (a.N + 127) / 128;
+    *mat = tile / tiles_per_mat;
+    const int base = (tile - *mat * tiles_per_mat) * 128;
+    const int half = a.d / 2;
+    const int p = 16 * (g >> 1);                       // first rotary pair of this warp quarter (64 pairs per tile)
+    const int r = base + (p / half) * a.d + (p % half);
+    *row0 = (g & 1) ? r + half : r;
+  } else if (a.mode == TG_SWIGLU) {
+    *mat = g & 1;                                      // even boxes: gate rows, odd boxes: up rows
+    *row0 = tile * 64 + 16 * (g >> 1);
+  } else {
+    *mat = 0;
+    *row0 = tile * 128 + 16 * g;
+  }
+}
+
+__global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(TcArgs a) {
+  extern __shared__ __align__(1024) unsigned char ring_raw[];
+  __shared__ __align__(8) unsigned long long full_bar[TG_MAX_STAGES], empty_bar[TG_MAX_STAGES], acc_bar;
+  __shared__ unsigned tmem_base_slot;
+  __shared__ int abort_flag;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // the ring must start on a 1024-byte boundary (swizzle atoms); dynamic smem is over-allocated by 1 KB
+  unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(ring_raw) + 1023) & ~(uintptr_t)1023);
+
+  const int tile = blockIdx.x, split = blockIdx.y;
+  if (tid == 0) {
+    for (int s = 0; s < TG_MAX_STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    mbar_init(&acc_bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+  pdl_trigger();
+  pdl_wait();                                                   // everything below may read what earlier kernels wrote
+  const int tokens = a.tot ? *a.tot : a.tot_fixed;
+  const int n_boxes = (tokens + TG_BOX_TOK - 1) / TG_BOX_TOK;
+  const int stage_bytes = TG_A_BYTES + n_boxes * TG_BOX_BYTES;
+  int n_stages = TG_SMEM_RING / stage_bytes;
+  if (n_stages > TG_MAX_STAGES) n_stages = TG_MAX_STAGES;
+  const int kb_total = (a.K + TG_BK - 1) / TG_BK;
+  const int kb0 = (int)(((long long)kb_total * split) / a.n_splits);
+  const int kb1 = (int)(((long long)kb_total * (split + 1)) / a.n_splits);
+  const int n_kb = (tokens > 0) ? kb1 - kb0 : 0;
+  const int n0 = min(((tokens + 15) / 16) * 16, 256);           // columns of the first MMA
+  const int n1 = tokens > 256 ? ((tokens - 256 + 15) / 16) * 16 : 0;
+  const unsigned tmem_cols = (n0 + n1) <= 32 ? 32u : ((n0 + n1) <= 64 ? 64u : ((n0 + n1) <= 128 ? 128u : ((n0 + n1) <= 256 ? 256u : 512u)));
+
+  if (warp == 1) {                                              // TMEM allocation (whole warp)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const unsigned tmem_base = tmem_base_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int mats[8], rows[8];
+#pragma unroll
+      for (int g = 0; g < 8; ++g) box_source(a, tile, g, &mats[g], &rows[g]);
+      for (int i = 0; i < n_kb; ++i) {
+        const int s = i % n_stages;
+        if (i >= n_stages && !mbar_wait(&empty_bar[s], ((i / n_stages) & 1) ^ 1, &abort_flag, a.dev_error, 0x40000 | (i & 0xffff))) break;
+        unsigned char* sa = ring + (size_t)s * stage_bytes;
+        unsigned char* sb = sa + TG_A_BYTES;
+        mbar_expect_tx(&full_bar[s], (unsigned)stage_bytes);
+        const int k = (kb0 + i) * TG_BK;
+#pragma unroll
+        for (int g = 0; g < 8; ++g) tma_load_2d(sa + g * 2048, a.tm_a[mats[g]], k, rows[g], &full_bar[s]);
+        for (int bx = 0; bx < n_boxes; ++bx) tma_load_2d(sb + bx * TG_BOX_BYTES, a.tm_b, k, bx * TG_BOX_TOK, &full_bar[s]);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const unsigned idesc0 = umma_idesc_bf16(128, n0);
+      const unsigned idesc1 = n1 ? umma_idesc_bf16(128, n1) : 0u;
+      bool ok = true;
+      for (int i = 0; i < n_kb && ok; ++i) {
+        const int s = i % n_stages;
+        ok = mbar_wait(&full_bar[s], (i / n_stages) & 1, &abort_flag, a.dev_error, 0x50000 | (i & 0xffff));
+        if (!ok) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const unsigned char* sa = ring + (size_t)s * stage_bytes;
+        const unsigned char* sb = sa + TG_A_BYTES;
+        const unsigned long long da = umma_desc(sa), db0 = umma_desc(sb), db1 = umma_desc(sb + 256 * 128);
+#pragma unroll
+        for (int k = 0; k < TG_BK / 16; ++k) {
+          const unsigned acc = (i > 0 || k > 0) ? 1u : 0u;
+          const unsigned long long koff = (unsigned long long)((k * 32) >> 4);        // 16 bf16 = 32 bytes along the swizzle row
+          umma_bf16(tmem_base, da + koff, db0 + koff, idesc0, acc);
+          if (n1) umma_bf16(tmem_base + 256, da + koff, db1 + koff, idesc1, acc);
+        }
+        umma_commit(&empty_bar[s]);                              // stage reusable once these MMAs have read it
+      }
+      if (ok) umma_commit(&acc_bar);                             // accumulator complete
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    const int q = warp & 3;                                      // TMEM lane quarter this warp may read
+    bool ok = n_kb > 0;
+    if (ok) ok = mbar_wait(&acc_bar, 0, &abort_flag, a.dev_error, 0x60000);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (ok) {
+      int mat, row0;
+      box_source(a, tile, 2 * q + (lane >> 4), &mat, &row0);
+      const int n = row0 + (lane & 15);                          // weight row (output feature) of this lane
+      const bool n_ok = n < a.N;
+      const int half = a.d / 2;
+      for (int c0 = 0; c0 < tokens; c0 += 16) {
+        float v[16];
+        tmem_ld16(tmem_base + ((unsigned)(32 * q) << 16) + (unsigned)c0, v);
+        if (a.mode == TG_PARTIAL) {
+          float* dst = a.part + (size_t)split * a.split_stride + n;
+#pragma unroll
+          for (int c = 0; c < 16; ++c)
+            if (c0 + c < tokens && n_ok) dst[(size_t)(c0 + c) * a.N] = v[c];
+        } else if (a.mode == TG_SWIGLU) {
+#pragma unroll
+          for (int c = 0; c < 16; ++c) {
+            const float pv = __shfl_xor_sync(0xffffffffu, v[c], 16);
+            const bool mine = ((c & 1) == 0) == (lane < 16);     // low half-warp finishes even columns, high half odd ones
+            const float g = lane < 16 ? v[c] : pv, u = lane < 16 ? pv : v[c];
+            if (mine && c0 + c < tokens && n_ok) a.h_out[(size_t)(c0 + c) * a.N + n] = __float2bfloat16(g / (1.f + __expf(-g)) * u);
+          }
+        } else {                                                 // TG_QKV
+#pragma unroll
+          for (int c = 0; c < 16; ++c) {
+            const float pv = __shfl_xor_sync(0xffffffffu, v[c], 16);
+            const int t = c0 + c;
+            if (t < tokens && n_ok) {
+              const int row = a.rowmap[t];
+              const int b = row / a.L, pos = row - b * a.L;
+              float y = v[c];
+              if (mat < 2) {
+                const int j = n % a.d % half;
+                const float cs = a.rope_cos[(size_t)pos * half + j], sn = a.rope_sin[(size_t)pos * half + j];
+                y = lane < 16 ? v[c] * cs - pv * sn : v[c] * cs + pv * sn;
+              }
+              if (mat == 0) a.q_out[(size_t)t * a.N + n] = __float2bfloat16(y);
+              else {
+                bf16* cache = mat == 1 ? a.kc : a.vc;
+                cache[((size_t)b * a.max_seq + pos) * a.N + n] = __float2bfloat16(y);
+              }
+            }
+          }
+        }
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+int encode_map(CUtensorMap* out, const void* base, int rows, int K, int box_rows) {
+  if (!g_encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn) return VLAC_ERR_CUDA;
+    g_encode = (EncodeTiledFn)fn;
+  }
+  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+  cuuint32_t box[2] = {(cuuint32_t)TG_BK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = g_encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? VLAC_OK : VLAC_ERR_CUDA;
+}
+
+}  // namespace
+
+// Tensor maps of one context: 7 per layer (weights, 16-row boxes) + 3 activation buffers (64-row boxes).
+enum { TM_WQ = 0, TM_WK, TM_WV, TM_WO, TM_GATE, TM_UP, TM_DOWN, TM_PER_LAYER };
+enum { TM_XN = 0, TM_AO, TM_HM, TM_ACT_COUNT };
+
+int vlac_tc_setup(vlac_ctx* ctx) {
+  const vlac_config& g = ctx->cfg;
+  ctx->tc_ok = 0;
+  // the TMA path needs 16-byte aligned rows and pointers
+  if (g.hidden % 8 || g.ffn % 8) return VLAC_OK;
+  const int n_maps = g.n_layers * TM_PER_LAYER + TM_ACT_COUNT;
+  CUtensorMap* host = (CUtensorMap*)malloc(sizeof(CUtensorMap) * n_maps);
+  if (!host) return VLAC_ERR_OOM;
+  int rc = VLAC_OK;
+  const int D = g.hidden, F = g.ffn;
+  for (int l = 0; l < g.n_layers && rc == VLAC_OK; ++l) {
+    const vlac_layer_w& w = ctx->layers[l];
+    const void* ptr[TM_PER_LAYER] = {w.wq, w.wk, w.wv, w.wo, w.w_gate, w.w_up, w.w_down};
+    const int rows[TM_PER_LAYER] = {D, D, D, D, F, F, D};
+    const int cols[TM_PER_LAYER] = {D, D, D, D, D, D, F};
+    for (int m = 0; m < TM_PER_LAYER && rc == VLAC_OK; ++m) {
+      if (reinterpret_cast<uintptr_t>(ptr[m]) & 15) { free(host); return VLAC_OK; }   // unaligned weights: stay on the generic path
+      rc = encode_map(&host[l * TM_PER_LAYER + m], ptr[m], rows[m], cols[m], 16);
+    }
+  }
+  CUtensorMap* act = host + g.n_layers * TM_PER_LAYER;
+  if (rc == VLAC_OK) rc = encode_map(&act[TM_XN], ctx->xn, ctx->rows_max, D, TG_BOX_TOK);
+  if (rc == VLAC_OK) rc = encode_map(&act[TM_AO], ctx->ao, ctx->rows_max, D, TG_BOX_TOK);
+  if (rc == VLAC_OK) rc = encode_map(&act[TM_HM], ctx->hm, ctx->rows_max, F, TG_BOX_TOK);
+  if (rc != VLAC_OK) { free(host); return rc; }
+  cudaError_t e = cudaMalloc(&ctx->tmaps, sizeof(CUtensorMap) * n_maps);
+  if (e != cudaSuccess) { free(host); cudaGetLastError(); return VLAC_ERR_OOM; }
+  e = cudaMemcpy(ctx->tmaps, host, sizeof(CUtensorMap) * n_maps, cudaMemcpyHostToDevice);
+  free(host);
+  if (e != cudaSuccess) { vlac_note_cuda_error(e, __FILE__, __LINE__); return VLAC_ERR_CUDA; }
+  e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TG_SMEM_RING + 1024);
+  if (e != cudaSuccess) { vlac_note_cuda_error(e, __FILE__, __LINE__); return VLAC_ERR_CUDA; }
+  // one CTA holds all tokens: at most 512 accumulator columns, and at least 2 ring stages
+  const int max_boxes = (ctx->rows_max + TG_BOX_TOK - 1) / TG_BOX_TOK;
+  if (ctx->rows_max > 512 || TG_SMEM_RING / (TG_A_BYTES + max_boxes * TG_BOX_BYTES) < 2) return VLAC_OK;
+  ctx->tc_ok = 1;
+  return VLAC_OK;
+}
+
+static int launch_tc(vlac_ctx* ctx, const TcArgs& a, int n_tiles, cudaStream_t s) {
+  VLAC_CUDA_CHECK(launch_pdl(gemm_tc_kernel, dim3(n_tiles, a.n_splits), dim3(TG_THREADS), (size_t)TG_SMEM_RING + 1024, s, a));
+  VLAC_LAUNCH_CHECK(ctx);
+  return VLAC_OK;
+}
+
+static void tc_common(vlac_ctx* ctx, vlac_cache* c, int layer, TcArgs* a) {
+  memset(a, 0, sizeof(*a));
+  a->tot = c->tot + layer;
+  a->d = ctx->cfg.head_dim;
+  a->rowmap = c->rowmap + (size_t)layer * c->batch * ctx->L;
+  a->L = ctx->L; a->max_seq = ctx->max_seq;
+  a->rope_cos = ctx->w.rope_cos; a->rope_sin = ctx->w.rope_sin;
+  a->dev_error = ctx->dev_error;
+  a->n_splits = 1;
+}
+
+int vlac_tc_qkv(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s) {
+  const vlac_config& g = ctx->cfg;
+  const CUtensorMap* tm = (const CUtensorMap*)ctx->tmaps + (size_t)layer * TM_PER_LAYER;
+  const CUtensorMap* act = (const CUtensorMap*)ctx->tmaps + (size_t)g.n_layers * TM_PER_LAYER;
+  TcArgs a; tc_common(ctx, c, layer, &a);
+  a.tm_a[0] = tm + TM_WQ; a.tm_a[1] = tm + TM_WK; a.tm_a[2] = tm + TM_WV; a.tm_b = act + TM_XN;
+  a.K = g.hidden; a.N = g.hidden; a.mode = TG_QKV;
+  a.q_out = ctx->q;
+  a.kc = c->k + (size_t)layer * c->batch * kv_layer_elems(ctx);
+  a.vc = c->v + (size_t)layer * c->batch * kv_layer_elems(ctx);
+  return launch_tc(ctx, a, 3 * ((g.hidden + 127) / 128), s);
+}
+
+int vlac_tc_partial(vlac_ctx* ctx, vlac_cache* c, int layer, int which, int* n_splits, cudaStream_t s) {
+  const vlac_config& g = ctx->cfg;
+  const CUtensorMap* tm = (const CUtensorMap*)ctx->tmaps + (size_t)layer * TM_PER_LAYER;
+  const CUtensorMap* act = (const CUtensorMap*)ctx->tmaps + (size_t)g.n_layers * TM_PER_LAYER;
+  TcArgs a; tc_common(ctx, c, layer, &a);
+  const bool down = which != 0;
+  a.tm_a[0] = tm + (down ? TM_DOWN : TM_WO); a.tm_b = act + (down ? TM_HM : TM_AO);
+  a.K = down ? g.ffn : g.hidden; a.N = g.hidden; a.mode = TG_PARTIAL;
+  const int tiles = (g.hidden + 127) / 128;
+  int splits = ctx->n_sm / tiles;                       // fill the SMs: the partial sums are folded by the next kernel
+  if (splits < 1) splits = 1;
+  if (splits > VLAC_MAX_SPLITS) splits = VLAC_MAX_SPLITS;
+  const int kb_total = (a.K + TG_BK - 1) / TG_BK;
+  if (splits > kb_total) splits = kb_total;
+  a.n_splits = splits;
+  a.part = ctx->part; a.split_stride = (size_t)ctx->rows_max * g.hidden;
+  *n_splits = splits;
+  return launch_tc(ctx, a, tiles, s);
+}
+
+int vlac_tc_gateup(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s) {
+  const vlac_config& g = ctx->cfg;
+  const CUtensorMap* tm = (const CUtensorMap*)ctx->tmaps + (size_t)layer * TM_PER_LAYER;
+  const CUtensorMap* act = (const CUtensorMap*)ctx->tmaps + (size_t)g.n_layers * TM_PER_LAYER;
+  TcArgs a; tc_common(ctx, c, layer, &a);
+  a.tm_a[0] = tm + TM_GATE; a.tm_a[1] = tm + TM_UP; a.tm_b = act + TM_XN;
+  a.K = g.hidden; a.N = g.ffn; a.mode = TG_SWIGLU;
+  a.h_out = ctx->hm;
+  return launch_tc(ctx, a, (g.ffn + 63) / 64, s);
+}

@@ -16,5 +16,8 @@ static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 b
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr; cfg.numAttrs = 1;
+#ifdef VLAC_NO_PDL
+  cfg.numAttrs = 0;
+#endif
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }

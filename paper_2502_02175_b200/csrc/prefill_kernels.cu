@@ -382,13 +382,18 @@ int vlac_launch_layer_body(vlac_ctx* ctx, vlac_cache* c, int layer, bf16* hidden
   bf16* kc = c->k + (size_t)layer * B * kv_layer_elems(ctx);
   bf16* vc = c->v + (size_t)layer * B * kv_layer_elems(ctx);
   int rc;
-  // Q/K/V projection of the normalised rows
-  rc = launch_gemm_generic(ctx, ctx->xn, (const bf16*)w.wq, (const bf16*)w.wk, (const bf16*)w.wv, 3, ctx->scratch,
-                           tot, 0, BL, D, D, 3 * D, s);
-  if (rc) return rc;
-  rope_scatter_kernel<<<BL, 256, 0, s>>>(ctx->scratch, tot, rowmap, ctx->w.rope_cos, ctx->w.rope_sin, ctx->q, kc, vc,
-                                         ctx->L, ctx->max_seq, g.n_heads, g.head_dim);
-  VLAC_LAUNCH_CHECK(ctx);
+  // Q/K/V projection of the normalised rows, rotation, K/V scatter
+  if (ctx->tc_ok) {
+    rc = vlac_tc_qkv(ctx, c, layer, s);
+    if (rc) return rc;
+  } else {
+    rc = launch_gemm_generic(ctx, ctx->xn, (const bf16*)w.wq, (const bf16*)w.wk, (const bf16*)w.wv, 3, ctx->scratch,
+                             tot, 0, BL, D, D, 3 * D, s);
+    if (rc) return rc;
+    rope_scatter_kernel<<<BL, 256, 0, s>>>(ctx->scratch, tot, rowmap, ctx->w.rope_cos, ctx->w.rope_sin, ctx->q, kc, vc,
+                                           ctx->L, ctx->max_seq, g.n_heads, g.head_dim);
+    VLAC_LAUNCH_CHECK(ctx);
+  }
   AttnArgs a;
   a.q = ctx->q; a.tot = tot; a.rowmap = rowmap; a.kc = kc; a.vc = vc; a.out = ctx->ao;
   a.probs = g.n_text_post > 0 ? ctx->probs : nullptr;
@@ -402,11 +407,18 @@ int vlac_launch_layer_body(vlac_ctx* ctx, vlac_cache* c, int layer, bf16* hidden
                                                                   g.n_text_post, g.n_heads, ctx->Lv);
     VLAC_LAUNCH_CHECK(ctx);
   }
-  // output projection -> partial; residual + RMSNorm for the MLP
-  rc = launch_gemm_generic(ctx, ctx->ao, (const bf16*)w.wo, nullptr, nullptr, 1, ctx->part, tot, 0, BL, D, D, D, s);
+  // output projection -> split-K partials; residual + RMSNorm for the MLP
+  int o_splits = 1;
+  if (ctx->tc_ok) rc = vlac_tc_partial(ctx, c, layer, 0, &o_splits, s);
+  else rc = launch_gemm_generic(ctx, ctx->ao, (const bf16*)w.wo, nullptr, nullptr, 1, ctx->part, tot, 0, BL, D, D, D, s);
   if (rc) return rc;
-  rc = vlac_launch_finalize_norm(ctx, c, hidden, layer, 1, layer, w.g_mlp, s);
+  rc = vlac_launch_finalize_norm(ctx, c, hidden, layer, o_splits, layer, w.g_mlp, s);
   if (rc) return rc;
+  if (ctx->tc_ok) {
+    rc = vlac_tc_gateup(ctx, c, layer, s);
+    if (rc) return rc;
+    return vlac_tc_partial(ctx, c, layer, 1, n_splits, s);
+  }
   rc = launch_gemm_generic(ctx, ctx->xn, (const bf16*)w.w_gate, (const bf16*)w.w_up, nullptr, 2, ctx->scratch,
                            tot, 0, BL, F, D, 2 * F, s);
   if (rc) return rc;

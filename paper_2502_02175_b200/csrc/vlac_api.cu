@@ -49,7 +49,7 @@ int fill_params(const vlac_ctx* ctx, const vlac_select_params* in, int force_ful
 void free_ctx_buffers(vlac_ctx* c) {
   cudaFree(c->xn); cudaFree(c->q); cudaFree(c->ao); cudaFree(c->hm); cudaFree(c->part); cudaFree(c->scratch);
   cudaFree(c->probs); cudaFree(c->hidden); cudaFree(c->x_dec); cudaFree(c->q_dec); cudaFree(c->ao_dec);
-  cudaFree(c->hm_dec); cudaFree(c->logits); cudaFree(c->argmax_tmp); cudaFree(c->dev_error);
+  cudaFree(c->hm_dec); cudaFree(c->logits); cudaFree(c->argmax_tmp); cudaFree(c->dev_error); cudaFree(c->tmaps);
   if (c->prof_ev) {
     for (int i = 0; i < 2 * VLAC_PROF_CAP; ++i) if (c->prof_ev[i]) cudaEventDestroy(c->prof_ev[i]);
     free(c->prof_ev);
@@ -138,8 +138,9 @@ int vlac_create(const vlac_config* cfg, const vlac_weights* w, vlac_ctx** out) {
   if (rc == VLAC_OK) rc = dev_alloc(&c->hm_dec, B * F);
   if (rc == VLAC_OK) rc = dev_alloc(&c->logits, B * (size_t)g.vocab);
   if (rc == VLAC_OK) rc = dev_alloc(&c->argmax_tmp, B * VLAC_ARGMAX_BLOCKS);
-  if (rc == VLAC_OK) rc = dev_alloc(&c->dev_error, 1);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->dev_error, 8);
   if (rc == VLAC_OK) rc = vlac_decode_setup(c);
+  if (rc == VLAC_OK) rc = vlac_tc_setup(c);
   if (rc != VLAC_OK) { free_ctx_buffers(c); delete c; return rc; }
   *out = c;
   return VLAC_OK;

@@ -44,7 +44,9 @@ struct vlac_ctx {
   bf16 *q_dec, *ao_dec, *hm_dec;     // [max_batch][hidden] x2, [max_batch][ffn]
   float *logits;                     // [max_batch][vocab]
   unsigned long long *argmax_tmp;    // [max_batch][VLAC_ARGMAX_BLOCKS]
-  int *dev_error;                    // device int: nonzero if a bounded wait gave up
+  int *dev_error;                    // device ints: [0] nonzero if a bounded wait gave up
+  void* tmaps;                       // device array of TMA tensor maps (weights per layer, activation buffers)
+  int tc_ok;                         // 1: shapes fit the tensor-memory GEMM
   // optional per-launch timing of the matrix-vector kernel (vlac_profile)
   int prof_on, prof_n;
   cudaEvent_t* prof_ev;              // [2 * VLAC_PROF_CAP]
@@ -92,6 +94,12 @@ int vlac_launch_finalize_norm(vlac_ctx* ctx, vlac_cache* c, bf16* hidden, int l_
 int vlac_launch_layer_body(vlac_ctx* ctx, vlac_cache* c, int layer, bf16* hidden, int* n_splits, cudaStream_t s);
 
 int vlac_launch_decode_attention(vlac_ctx* ctx, vlac_cache* c, int layer, int pos, cudaStream_t s);
+
+// ---- tensor-memory GEMM (gemm_tc.cu)
+int vlac_tc_setup(vlac_ctx* ctx);
+int vlac_tc_qkv(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s);
+int vlac_tc_partial(vlac_ctx* ctx, vlac_cache* c, int layer, int which /* 0: output proj, 1: down proj */, int* n_splits, cudaStream_t s);
+int vlac_tc_gateup(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s);
 
 // ---- decode (decode_kernels.cu)
 int vlac_decode_setup(vlac_ctx* ctx);
