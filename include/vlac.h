@@ -31,6 +31,7 @@ extern "C" {
 #define VLAC_ERR_OOM          -3
 #define VLAC_ERR_CUDA         -4
 #define VLAC_ERR_TIMEOUT      -5
+#define VLAC_ERR_TOO_LARGE    -6   /* a size exceeds a fixed capacity stated beside the call */
 
 #define VLAC_MAX_LAYERS 64
 
@@ -185,6 +186,26 @@ int vlac_profile_read(vlac_ctx* ctx, double* ms_total, unsigned long long* bytes
 /* Nonzero if a device-side bounded wait gave up since the context was created (reads one int
  * back; synchronises the stream). */
 int vlac_device_error(vlac_ctx* ctx, void* stream);
+
+/* Greedy token choice that allocates nothing (the paper has no counterpart; it is the last step of
+ * vlac_step offered on its own).  For each of `rows` logits rows it returns the index of the largest
+ * value, equal values going to the lower index, exactly as vlac_step picks action tokens.
+ *
+ * It exists for callers that may not allocate device memory at the time of the call: a control loop
+ * that reserved its whole memory budget at start-up and must not hit cudaMalloc (or the device-wide
+ * synchronisation it implies) afterwards, or a process whose GPU memory belongs to one pool.  It takes
+ * no context: its only scratch is a 32 KB array built into the library, which every GPU that loads
+ * the library holds until the process exits.  No cudaMalloc/cudaFree or allocating routine is called.
+ *
+ *   logits      device fp32, row r starts at logits + r*row_stride (row_stride >= vocab, in elements)
+ *   rows        1..64; more returns VLAC_ERR_TOO_LARGE and does nothing
+ *   tokens      device int32 [rows]
+ * The first call on each device looks up the array's device address (one runtime query); make that
+ * first call outside any stream capture.  All calls share the array and it keeps the previous call's
+ * contents; every slot is rewritten before it is read, so nothing needs clearing, but two calls whose
+ * kernels overlap on the GPU (different streams, no ordering) race on it: order them. */
+int vlac_greedy_tokens_static(const float* logits, int rows, int vocab, long long row_stride,
+                              int* tokens, void* stream);
 
 const char* vlac_status_string(int status);
 

@@ -55,7 +55,7 @@ class vlac_selection(C.Structure):
 EXPORTS = ("vlac_create", "vlac_destroy", "vlac_cache_alloc", "vlac_cache_reset", "vlac_cache_free",
            "vlac_cache_read", "vlac_cache_write", "vlac_select", "vlac_select_import", "vlac_layer_forward",
            "vlac_step", "vlac_selection_view", "vlac_launch_count", "vlac_device_error", "vlac_status_string",
-           "vlac_profile", "vlac_profile_read")
+           "vlac_profile", "vlac_profile_read", "vlac_greedy_tokens_static")
 
 lib.vlac_status_string.restype = C.c_char_p
 lib.vlac_status_string.argtypes = [C.c_int]
@@ -76,6 +76,7 @@ lib.vlac_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_vo
 lib.vlac_selection_view.argtypes = [C.c_void_p, C.POINTER(vlac_selection)]
 lib.vlac_device_error.argtypes = [C.c_void_p, C.c_void_p]
 lib.vlac_profile.argtypes = [C.c_void_p, C.c_int]
+lib.vlac_greedy_tokens_static.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_longlong, C.c_void_p, C.c_void_p]
 lib.vlac_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_ulonglong), C.POINTER(C.c_int)]
 
 
@@ -272,6 +273,16 @@ def vlac_profile_read(ctx: int):
     ms, by, n = C.c_double(), C.c_ulonglong(), C.c_int()
     _check(lib.vlac_profile_read(ctx, C.byref(ms), C.byref(by), C.byref(n)), "vlac_profile_read")
     return ms.value, by.value, n.value
+
+
+def vlac_greedy_tokens_static(logits: torch.Tensor, tokens: torch.Tensor) -> None:
+    """Argmax of each row of a 2-D fp32 device tensor into an int32 device tensor, ties to the lower
+    index, using only the scratch array built into the library (no allocation; at most 64 rows).
+    Meant for callers that may not allocate device memory when they run."""
+    assert logits.is_cuda and logits.dtype == torch.float32 and logits.dim() == 2 and logits.stride(1) == 1
+    assert tokens.is_cuda and tokens.dtype == torch.int32 and tokens.is_contiguous()
+    _check(lib.vlac_greedy_tokens_static(logits.data_ptr(), logits.shape[0], logits.shape[1], logits.stride(0),
+                                         tokens.data_ptr(), _stream()), "vlac_greedy_tokens_static")
 
 
 # --------------------------------------------------------------------------- reading views back

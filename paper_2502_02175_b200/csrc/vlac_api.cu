@@ -82,6 +82,7 @@ const char* vlac_status_string(int status) {
     case VLAC_ERR_OOM: return "out of device memory";
     case VLAC_ERR_CUDA: return g_last_cuda_error[0] ? g_last_cuda_error : "CUDA error";
     case VLAC_ERR_TIMEOUT: return "device-side wait timed out";
+    case VLAC_ERR_TOO_LARGE: return "size exceeds the fixed capacity of this call";
     default: return "unknown status";
   }
 }
