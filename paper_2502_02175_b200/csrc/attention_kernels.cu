@@ -1,0 +1,391 @@
+// Prefill attention of the recomputed rows over the position-indexed K/V cache (Sec. 3.1 attention;
+// Appendix "Position and Attention Masking": the mask follows original positions, so a recomputed
+// query at position p sees every cached key <= p, whether that key is fresh or reused).
+//
+// One CTA per (64-query tile of one sequence, head).  Warp 4 streams 64-key blocks of this head's
+// K and V through a shared-memory ring with TMA (128-byte swizzle); warps 0-3 each own 16 queries,
+// keep S and O in registers (warp-level MMA, online softmax) and read the swizzled tiles with
+// ldmatrix.  All four compute warps consume every block in order, so no waiter is ever more than one
+// phase ahead of a barrier.
+//
+// Text-to-vision scores (Eq. avistext, Sec. 3.3): tiles that hold prompt-text queries behind the
+// vision block run a second pass over the vision keys, now with the final row maxima and sums, and
+// leave the column sums of the normalised probabilities over their text rows in a per-tile partial;
+// a small kernel adds the tiles in order and divides by the number of text rows (fixed order: the
+// saved scores are bit-reproducible).
+#include "vlac_internal.h"
+#include <cuda.h>
+#include <stdlib.h>
+
+namespace {
+
+constexpr int AT_Q = 64;                  // queries per CTA
+constexpr int AT_KB = 64;                 // keys per block
+constexpr int AT_STAGES = 4;
+constexpr int AT_THREADS = 160;
+constexpr unsigned long long AT_WAIT_LIMIT_NS = 400000000ull;
+
+struct AttnTileArgs {
+  const CUtensorMap *tm_q, *tm_k, *tm_v;  // q [rows][H*d]; caches [B*max_seq][H*d]; 64x64 boxes
+  const int* M;                           // [B][nl] rows per sequence (this layer's column is used)
+  const int* rowmap;                      // [B*L] compact index -> b*L + pos (this layer)
+  bf16* out;                              // [rows][H*d]
+  float* partial;                         // [B][tiles][H][Lv] column sums over text rows, or NULL
+  int* dev_error;
+  int layer, nl, B, L, max_seq, H, v0, Lv, tiles;
+};
+
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned parity) {
+  unsigned ok;
+  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}\n"
+               : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, volatile int* abort_flag, int* dev_error, int code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (global_ns() - t0 > AT_WAIT_LIMIT_NS) break;
+  }
+  *abort_flag = 1;
+  if (dev_error) atomicCAS(dev_error, 0, code);
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, int x, int y, unsigned long long* bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(smem_u32(dst)), "l"(tm), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+// byte offset of element (row, col) in a [64 rows][64 bf16] box written by TMA with the 128-byte swizzle
+__device__ __forceinline__ unsigned swz(int row, int col) {
+  return (unsigned)(row * 128 + ((((col >> 3) ^ (row & 7)) & 7) << 4) + ((col & 7) << 1));
+}
+__device__ __forceinline__ void ldsm4(unsigned addr, unsigned* r) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm4t(unsigned addr, unsigned* r) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma16816(float* c, const unsigned* a, unsigned b0, unsigned b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ unsigned pack_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<unsigned*>(&v);
+}
+
+// S[16 x 64] = Q_warp K_block^T for one 64-key block (raw dot products)
+template <int DH>
+__device__ __forceinline__ void qk_block(const unsigned (*qf)[4], unsigned k_smem, int lane, float (*s)[4]) {
+#pragma unroll
+  for (int j = 0; j < 8; ++j) { s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.f; }
+#pragma unroll
+  for (int ks = 0; ks < DH / 16; ++ks) {
+    const int col = ks * 16 + ((lane >> 3) & 1) * 8;            // column inside the head
+    const unsigned base = k_smem + (unsigned)(col >> 6) * (AT_KB * 128);
+#pragma unroll
+    for (int jp = 0; jp < 4; ++jp) {
+      const int key = jp * 16 + (lane & 7) + ((lane >> 4) & 1) * 8;
+      unsigned b[4];
+      ldsm4(base + swz(key, col & 63), b);
+      mma16816(s[2 * jp], qf[ks], b[0], b[1]);
+      mma16816(s[2 * jp + 1], qf[ks], b[2], b[3]);
+    }
+  }
+}
+
+template <int DH>
+__global__ void __launch_bounds__(AT_THREADS, 1) attention_tile_kernel(AttnTileArgs a) {
+  extern __shared__ __align__(1024) unsigned char at_raw[];
+  __shared__ __align__(8) unsigned long long full_bar[AT_STAGES], empty_bar[AT_STAGES], q_bar;
+  __shared__ int abort_flag;
+  constexpr int HALVES = DH / 64;
+  constexpr int KV_BYTES = HALVES * AT_KB * 128;                // K (or V) of one key block
+  constexpr int STAGE_BYTES = 2 * KV_BYTES;
+  constexpr int Q_BYTES = HALVES * AT_Q * 128;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tile = blockIdx.x, b = blockIdx.y, h = blockIdx.z;
+
+  // rows of this tile: compact indices [row0, row0 + n_valid) of sequence b
+  int off = 0;
+  for (int bb = 0; bb < b; ++bb) off += a.M[(size_t)bb * a.nl + a.layer];
+  const int Mb = a.M[(size_t)b * a.nl + a.layer];
+  const int n_valid = min(AT_Q, Mb - tile * AT_Q);
+  if (n_valid <= 0) {
+    // no rows: the partial of this tile must still read as zero
+    if (a.partial)
+      for (int v = tid; v < a.Lv; v += AT_THREADS) a.partial[(((size_t)b * a.tiles + tile) * a.H + h) * a.Lv + v] = 0.f;
+    return;
+  }
+  const int row0 = off + tile * AT_Q;
+  const int pos_last = a.rowmap[row0 + n_valid - 1] - b * a.L;
+  const int n_kb = pos_last / AT_KB + 1;                         // key blocks any row of the tile can see
+  const int v1 = a.v0 + a.Lv;
+  const bool has_text = a.partial != nullptr && pos_last >= v1;  // rows ascend: text rows, if any, are last
+  const int e_kb0 = a.v0 / AT_KB, e_kb1 = (v1 - 1) / AT_KB + 1;  // key blocks covering the vision keys
+  const int n_eb = has_text ? (e_kb1 - e_kb0) : 0;
+  const int total = n_kb + n_eb;
+
+  unsigned char* base = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(at_raw) + 1023) & ~(uintptr_t)1023);
+  unsigned char* q_s = base;
+  unsigned char* ring = base + Q_BYTES;
+  float* colsum = reinterpret_cast<float*>(ring + AT_STAGES * STAGE_BYTES);     // [4 warps][Lv]
+
+  if (tid == 0) {
+    for (int s = 0; s < AT_STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 4); }
+    mbar_init(&q_bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+
+  if (warp == 4) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      mbar_expect_tx(&q_bar, Q_BYTES);
+#pragma unroll
+      for (int hf = 0; hf < HALVES; ++hf) tma_load_2d(q_s + hf * AT_Q * 128, a.tm_q, h * DH + hf * 64, row0, &q_bar);
+      for (int i = 0; i < total; ++i) {
+        const int s = i % AT_STAGES;
+        if (i >= AT_STAGES && !mbar_wait(&empty_bar[s], ((i / AT_STAGES) & 1) ^ 1, &abort_flag, a.dev_error, 0x70000 | i)) break;
+        const bool main_pass = i < n_kb;
+        const int kb = main_pass ? i : e_kb0 + (i - n_kb);
+        unsigned char* ks = ring + (size_t)s * STAGE_BYTES;
+        mbar_expect_tx(&full_bar[s], main_pass ? STAGE_BYTES : KV_BYTES);
+        const int y = b * a.max_seq + kb * AT_KB;
+#pragma unroll
+        for (int hf = 0; hf < HALVES; ++hf) tma_load_2d(ks + hf * AT_KB * 128, a.tm_k, h * DH + hf * 64, y, &full_bar[s]);
+        if (main_pass) {
+#pragma unroll
+          for (int hf = 0; hf < HALVES; ++hf) tma_load_2d(ks + KV_BYTES + hf * AT_KB * 128, a.tm_v, h * DH + hf * 64, y, &full_bar[s]);
+        }
+      }
+    }
+    return;
+  }
+
+  // -------------------------------------------------------------------- compute warps
+  const int g = lane >> 2, t = lane & 3;
+  const int r_lo = warp * 16 + g, r_hi = r_lo + 8;               // this thread's two query rows in the tile
+  const int pos_lo = r_lo < n_valid ? a.rowmap[row0 + r_lo] - b * a.L : -1;
+  const int pos_hi = r_hi < n_valid ? a.rowmap[row0 + r_hi] - b * a.L : -1;
+  const float scale = rsqrtf((float)DH) * 1.44269504088896f;     // softmax in base 2
+
+  bool ok = mbar_wait(&q_bar, 0, &abort_flag, a.dev_error, 0x71000);
+  unsigned qf[DH / 16][4];
+#pragma unroll
+  for (int ks = 0; ks < DH / 16; ++ks) {
+    const int row = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+    const int col = ks * 16 + (lane >> 4) * 8;
+    ldsm4(smem_u32(q_s) + (unsigned)(col >> 6) * (AT_Q * 128) + swz(row, col & 63), qf[ks]);
+  }
+  float o[DH / 8][4];
+#pragma unroll
+  for (int j = 0; j < DH / 8; ++j) { o[j][0] = o[j][1] = o[j][2] = o[j][3] = 0.f; }
+  float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+
+  int i = 0;
+  for (; i < n_kb && ok; ++i) {
+    const int s = i % AT_STAGES;
+    ok = mbar_wait(&full_bar[s], (i / AT_STAGES) & 1, &abort_flag, a.dev_error, 0x72000 | i);
+    if (!ok) break;
+    const unsigned k_smem = smem_u32(ring + (size_t)s * STAGE_BYTES);
+    const unsigned v_smem = k_smem + KV_BYTES;
+    float sc[8][4];
+    qk_block<DH>(qf, k_smem, lane, sc);
+    // scale, positional causal mask, block maxima
+    float bm_lo = -INFINITY, bm_hi = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int key = i * AT_KB + j * 8 + 2 * t;
+      sc[j][0] = key <= pos_lo ? sc[j][0] * scale : -INFINITY;
+      sc[j][1] = key + 1 <= pos_lo ? sc[j][1] * scale : -INFINITY;
+      sc[j][2] = key <= pos_hi ? sc[j][2] * scale : -INFINITY;
+      sc[j][3] = key + 1 <= pos_hi ? sc[j][3] * scale : -INFINITY;
+      bm_lo = fmaxf(bm_lo, fmaxf(sc[j][0], sc[j][1]));
+      bm_hi = fmaxf(bm_hi, fmaxf(sc[j][2], sc[j][3]));
+    }
+    bm_lo = fmaxf(bm_lo, __shfl_xor_sync(0xffffffffu, bm_lo, 1)); bm_lo = fmaxf(bm_lo, __shfl_xor_sync(0xffffffffu, bm_lo, 2));
+    bm_hi = fmaxf(bm_hi, __shfl_xor_sync(0xffffffffu, bm_hi, 1)); bm_hi = fmaxf(bm_hi, __shfl_xor_sync(0xffffffffu, bm_hi, 2));
+    const float mn_lo = fmaxf(m_lo, bm_lo), mn_hi = fmaxf(m_hi, bm_hi);
+    // rows without any visible key so far (padding rows) keep a finite reference to avoid inf - inf
+    const float ref_lo = mn_lo == -INFINITY ? 0.f : mn_lo, ref_hi = mn_hi == -INFINITY ? 0.f : mn_hi;
+    const float al_lo = exp2f(m_lo - ref_lo), al_hi = exp2f(m_hi - ref_hi);
+    m_lo = mn_lo; m_hi = mn_hi;
+    l_lo *= al_lo; l_hi *= al_hi;
+#pragma unroll
+    for (int j = 0; j < DH / 8; ++j) { o[j][0] *= al_lo; o[j][1] *= al_lo; o[j][2] *= al_hi; o[j][3] *= al_hi; }
+    unsigned pf[4][4];                                            // P as A fragments: 4 k-steps of 16 keys
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float p0 = exp2f(sc[j][0] - ref_lo), p1 = exp2f(sc[j][1] - ref_lo);
+      const float p2 = exp2f(sc[j][2] - ref_hi), p3 = exp2f(sc[j][3] - ref_hi);
+      l_lo += p0 + p1; l_hi += p2 + p3;
+      pf[j >> 1][(j & 1) * 2] = pack_bf16(p0, p1);
+      pf[j >> 1][(j & 1) * 2 + 1] = pack_bf16(p2, p3);
+    }
+    // O += P V
+#pragma unroll
+    for (int ks = 0; ks < 4; ++ks) {
+      const int key = ks * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+#pragma unroll
+      for (int np = 0; np < DH / 16; ++np) {
+        const int col = np * 16 + (lane >> 4) * 8;
+        unsigned bfr[4];
+        ldsm4t(v_smem + (unsigned)(col >> 6) * (AT_KB * 128) + swz(key, col & 63), bfr);
+        mma16816(o[2 * np], pf[ks], bfr[0], bfr[1]);
+        mma16816(o[2 * np + 1], pf[ks], bfr[2], bfr[3]);
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&empty_bar[s]);
+  }
+  // row sums over the four threads of a row
+  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1); l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+  l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1); l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+  const float inv_lo = l_lo > 0.f ? 1.f / l_lo : 0.f, inv_hi = l_hi > 0.f ? 1.f / l_hi : 0.f;
+  if (ok) {
+    const size_t D = (size_t)a.H * DH;
+#pragma unroll
+    for (int j = 0; j < DH / 8; ++j) {
+      const int col = h * DH + j * 8 + 2 * t;
+      if (r_lo < n_valid) *reinterpret_cast<unsigned*>(a.out + (size_t)(row0 + r_lo) * D + col) = pack_bf16(o[j][0] * inv_lo, o[j][1] * inv_lo);
+      if (r_hi < n_valid) *reinterpret_cast<unsigned*>(a.out + (size_t)(row0 + r_hi) * D + col) = pack_bf16(o[j][2] * inv_hi, o[j][3] * inv_hi);
+    }
+  }
+  if (a.partial == nullptr) return;                               // uniform over the CTA
+
+  // ---- second pass: normalised probabilities of the text rows over the vision keys
+  for (int v = tid; v < 4 * a.Lv; v += 128) colsum[v] = 0.f;
+  asm volatile("bar.sync 1, 128;");
+  const bool text_lo = pos_lo >= v1, text_hi = pos_hi >= v1;
+  for (int e = 0; e < n_eb && ok; ++e, ++i) {
+    const int s = i % AT_STAGES;
+    ok = mbar_wait(&full_bar[s], (i / AT_STAGES) & 1, &abort_flag, a.dev_error, 0x73000 | i);
+    if (!ok) break;
+    const unsigned k_smem = smem_u32(ring + (size_t)s * STAGE_BYTES);
+    float sc[8][4];
+    qk_block<DH>(qf, k_smem, lane, sc);
+    const int kb = e_kb0 + e;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int key = kb * AT_KB + j * 8 + 2 * t;
+      float c0 = 0.f, c1 = 0.f;
+      // text rows sit behind the vision block, so they see every vision key: no mask needed here
+      if (text_lo) { c0 += exp2f(sc[j][0] * scale - m_lo) * inv_lo; c1 += exp2f(sc[j][1] * scale - m_lo) * inv_lo; }
+      if (text_hi) { c0 += exp2f(sc[j][2] * scale - m_hi) * inv_hi; c1 += exp2f(sc[j][3] * scale - m_hi) * inv_hi; }
+#pragma unroll
+      for (int sh = 4; sh <= 16; sh <<= 1) { c0 += __shfl_xor_sync(0xffffffffu, c0, sh); c1 += __shfl_xor_sync(0xffffffffu, c1, sh); }
+      if (g == 0) {
+        const int v = key - a.v0;
+        if (v >= 0 && v < a.Lv) colsum[warp * a.Lv + v] = c0;
+        if (v + 1 >= 0 && v + 1 < a.Lv) colsum[warp * a.Lv + v + 1] = c1;
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&empty_bar[s]);
+  }
+  asm volatile("bar.sync 1, 128;");
+  float* dst = a.partial + (((size_t)b * a.tiles + tile) * a.H + h) * a.Lv;
+  for (int v = tid; v < a.Lv; v += 128) dst[v] = ((colsum[v] + colsum[a.Lv + v]) + colsum[2 * a.Lv + v]) + colsum[3 * a.Lv + v];
+}
+
+// sum of the per-tile partials in tile order, divided by the number of text rows
+__global__ void __launch_bounds__(256) emit_from_tiles_kernel(const float* partial, float* attn_next_layer, size_t seq_stride,
+                                                              int tiles, int n_tp, int H, int Lv) {
+  const int h = blockIdx.x, b = blockIdx.y;
+  float* dst = attn_next_layer + (size_t)b * seq_stride + (size_t)h * Lv;
+  for (int v = threadIdx.x; v < Lv; v += blockDim.x) {
+    float s = 0.f;
+    for (int tl = 0; tl < tiles; ++tl) s += partial[(((size_t)b * tiles + tl) * H + h) * Lv + v];
+    dst[v] = n_tp > 0 ? s / (float)n_tp : 0.f;
+  }
+}
+
+template <int DH>
+constexpr size_t at_smem(int Lv) {
+  return 1024 + (size_t)(DH / 64) * AT_Q * 128 + (size_t)AT_STAGES * 2 * (DH / 64) * AT_KB * 128 + (size_t)4 * Lv * sizeof(float);
+}
+
+}  // namespace
+
+int vlac_attention_setup(vlac_ctx* ctx) {
+  const vlac_config& g = ctx->cfg;
+  ctx->attn_tiles = 0;
+  if (!ctx->tc_ok) return VLAC_OK;
+  if (g.head_dim != 64 && g.head_dim != 128) return VLAC_OK;
+  const int tiles = (ctx->L + AT_Q - 1) / AT_Q;
+  if (g.n_text_post > 0 && tiles > g.n_text_post) return VLAC_OK;      // the partial buffer is sized by the text rows
+  cudaError_t e;
+  if (g.head_dim == 128) e = cudaFuncSetAttribute(attention_tile_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)at_smem<128>(ctx->Lv));
+  else e = cudaFuncSetAttribute(attention_tile_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)at_smem<64>(ctx->Lv));
+  if (e != cudaSuccess) { cudaGetLastError(); return VLAC_OK; }
+  if (cudaMalloc(&ctx->tmap_q, sizeof(CUtensorMap)) != cudaSuccess) { cudaGetLastError(); return VLAC_ERR_OOM; }
+  CUtensorMap m;
+  int rc = vlac_encode_map_2d(&m, ctx->q, ctx->rows_max, g.hidden, AT_Q);
+  if (rc != VLAC_OK) return rc;
+  VLAC_CUDA_CHECK(cudaMemcpy(ctx->tmap_q, &m, sizeof(m), cudaMemcpyHostToDevice));
+  ctx->attn_tiles = tiles;
+  return VLAC_OK;
+}
+
+int vlac_attention_cache_setup(vlac_ctx* ctx, vlac_cache* c) {
+  c->tmaps_kv = nullptr;
+  if (!ctx->attn_tiles) return VLAC_OK;
+  const vlac_config& g = ctx->cfg;
+  const int n = 2 * g.n_layers;
+  CUtensorMap* host = (CUtensorMap*)malloc(sizeof(CUtensorMap) * n);
+  if (!host) return VLAC_ERR_OOM;
+  int rc = VLAC_OK;
+  for (int l = 0; l < g.n_layers && rc == VLAC_OK; ++l) {
+    const size_t off = (size_t)l * c->batch * kv_layer_elems(ctx);
+    rc = vlac_encode_map_2d(&host[2 * l], c->k + off, c->batch * ctx->max_seq, g.hidden, AT_KB);
+    if (rc == VLAC_OK) rc = vlac_encode_map_2d(&host[2 * l + 1], c->v + off, c->batch * ctx->max_seq, g.hidden, AT_KB);
+  }
+  if (rc == VLAC_OK && cudaMalloc(&c->tmaps_kv, sizeof(CUtensorMap) * n) != cudaSuccess) { cudaGetLastError(); rc = VLAC_ERR_OOM; }
+  if (rc == VLAC_OK && cudaMemcpy(c->tmaps_kv, host, sizeof(CUtensorMap) * n, cudaMemcpyHostToDevice) != cudaSuccess) rc = VLAC_ERR_CUDA;
+  free(host);
+  return rc;
+}
+
+int vlac_launch_prefill_attention(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s) {
+  const vlac_config& g = ctx->cfg;
+  const int B = c->batch;
+  AttnTileArgs a;
+  a.tm_q = (const CUtensorMap*)ctx->tmap_q;
+  a.tm_k = (const CUtensorMap*)c->tmaps_kv + 2 * layer;
+  a.tm_v = a.tm_k + 1;
+  a.M = c->M; a.rowmap = c->rowmap + (size_t)layer * B * ctx->L;
+  a.out = ctx->ao;
+  a.partial = g.n_text_post > 0 ? ctx->probs : nullptr;
+  a.dev_error = ctx->dev_error;
+  a.layer = layer; a.nl = g.n_layers; a.B = B; a.L = ctx->L; a.max_seq = ctx->max_seq; a.H = g.n_heads;
+  a.v0 = g.n_text_pre; a.Lv = ctx->Lv; a.tiles = ctx->attn_tiles;
+  const dim3 grid(ctx->attn_tiles, B, g.n_heads);
+  if (g.head_dim == 128) attention_tile_kernel<128><<<grid, AT_THREADS, at_smem<128>(ctx->Lv), s>>>(a);
+  else attention_tile_kernel<64><<<grid, AT_THREADS, at_smem<64>(ctx->Lv), s>>>(a);
+  VLAC_LAUNCH_CHECK(ctx);
+  float* dst = c->attn_next + (size_t)layer * g.n_heads * ctx->Lv;
+  emit_from_tiles_kernel<<<dim3(g.n_heads, B), 256, 0, s>>>(ctx->probs, dst, (size_t)g.n_layers * g.n_heads * ctx->Lv,
+                                                            ctx->attn_tiles, g.n_text_post, g.n_heads, ctx->Lv);
+  VLAC_LAUNCH_CHECK(ctx);
+  return VLAC_OK;
+}

@@ -309,6 +309,10 @@ int encode_map(CUtensorMap* out, const void* base, int rows, int K, int box_rows
 
 }  // namespace
 
+int vlac_encode_map_2d(void* out, const void* base, int rows, int cols, int box_rows) {
+  return encode_map((CUtensorMap*)out, base, rows, cols, box_rows);
+}
+
 // Tensor maps of one context: 7 per layer (weights, 16-row boxes) + 3 activation buffers (64-row boxes).
 enum { TM_WQ = 0, TM_WK, TM_WV, TM_WO, TM_GATE, TM_UP, TM_DOWN, TM_PER_LAYER };
 enum { TM_XN = 0, TM_AO, TM_HM, TM_ACT_COUNT };

@@ -394,18 +394,23 @@ int vlac_launch_layer_body(vlac_ctx* ctx, vlac_cache* c, int layer, bf16* hidden
                                            ctx->L, ctx->max_seq, g.n_heads, g.head_dim);
     VLAC_LAUNCH_CHECK(ctx);
   }
-  AttnArgs a;
-  a.q = ctx->q; a.tot = tot; a.rowmap = rowmap; a.kc = kc; a.vc = vc; a.out = ctx->ao;
-  a.probs = g.n_text_post > 0 ? ctx->probs : nullptr;
-  a.nq_fixed = 0; a.fixed_pos = 0; a.L = ctx->L; a.max_seq = ctx->max_seq; a.H = g.n_heads; a.d = g.head_dim;
-  a.v0 = g.n_text_pre; a.Lv = ctx->Lv; a.n_tp = g.n_text_post;
-  attention_row_kernel<<<dim3(BL, g.n_heads), 128, (g.head_dim + ctx->max_seq) * sizeof(float), s>>>(a);
-  VLAC_LAUNCH_CHECK(ctx);
-  {
-    float* dst = c->attn_next + (size_t)layer * g.n_heads * ctx->Lv;
-    emit_attention_mean_kernel<<<dim3(g.n_heads, B), 256, 0, s>>>(ctx->probs, dst, (size_t)g.n_layers * g.n_heads * ctx->Lv,
-                                                                  g.n_text_post, g.n_heads, ctx->Lv);
+  if (ctx->attn_tiles) {
+    rc = vlac_launch_prefill_attention(ctx, c, layer, s);
+    if (rc) return rc;
+  } else {
+    AttnArgs a;
+    a.q = ctx->q; a.tot = tot; a.rowmap = rowmap; a.kc = kc; a.vc = vc; a.out = ctx->ao;
+    a.probs = g.n_text_post > 0 ? ctx->probs : nullptr;
+    a.nq_fixed = 0; a.fixed_pos = 0; a.L = ctx->L; a.max_seq = ctx->max_seq; a.H = g.n_heads; a.d = g.head_dim;
+    a.v0 = g.n_text_pre; a.Lv = ctx->Lv; a.n_tp = g.n_text_post;
+    attention_row_kernel<<<dim3(BL, g.n_heads), 128, (g.head_dim + ctx->max_seq) * sizeof(float), s>>>(a);
     VLAC_LAUNCH_CHECK(ctx);
+    {
+      float* dst = c->attn_next + (size_t)layer * g.n_heads * ctx->Lv;
+      emit_attention_mean_kernel<<<dim3(g.n_heads, B), 256, 0, s>>>(ctx->probs, dst, (size_t)g.n_layers * g.n_heads * ctx->Lv,
+                                                                    g.n_text_post, g.n_heads, ctx->Lv);
+      VLAC_LAUNCH_CHECK(ctx);
+    }
   }
   // output projection -> split-K partials; residual + RMSNorm for the MLP
   int o_splits = 1;

@@ -49,7 +49,7 @@ int fill_params(const vlac_ctx* ctx, const vlac_select_params* in, int force_ful
 void free_ctx_buffers(vlac_ctx* c) {
   cudaFree(c->xn); cudaFree(c->q); cudaFree(c->ao); cudaFree(c->hm); cudaFree(c->part); cudaFree(c->scratch);
   cudaFree(c->probs); cudaFree(c->hidden); cudaFree(c->x_dec); cudaFree(c->q_dec); cudaFree(c->ao_dec);
-  cudaFree(c->hm_dec); cudaFree(c->logits); cudaFree(c->argmax_tmp); cudaFree(c->dev_error); cudaFree(c->tmaps);
+  cudaFree(c->hm_dec); cudaFree(c->logits); cudaFree(c->argmax_tmp); cudaFree(c->dev_error); cudaFree(c->tmaps); cudaFree(c->tmap_q);
   if (c->prof_ev) {
     for (int i = 0; i < 2 * VLAC_PROF_CAP; ++i) if (c->prof_ev[i]) cudaEventDestroy(c->prof_ev[i]);
     free(c->prof_ev);
@@ -62,7 +62,7 @@ void free_cache_buffers(vlac_cache* c) {
   cudaFree(c->warm); cudaFree(c->sim); cudaFree(c->S_layer); cudaFree(c->S); cudaFree(c->alpha);
   cudaFree(c->alpha_raw); cudaFree(c->entropy); cudaFree(c->static_mask); cudaFree(c->task_mask);
   cudaFree(c->final_mask); cudaFree(c->rank); cudaFree(c->n_reuse); cudaFree(c->M); cudaFree(c->rows);
-  cudaFree(c->tot); cudaFree(c->rowmap); cudaFree(c->slot);
+  cudaFree(c->tot); cudaFree(c->rowmap); cudaFree(c->slot); cudaFree(c->tmaps_kv);
 }
 
 __global__ void set_warm_kernel(int* warm, int n, int value) {
@@ -142,6 +142,7 @@ int vlac_create(const vlac_config* cfg, const vlac_weights* w, vlac_ctx** out) {
   if (rc == VLAC_OK) rc = dev_alloc(&c->dev_error, 8);
   if (rc == VLAC_OK) rc = vlac_decode_setup(c);
   if (rc == VLAC_OK) rc = vlac_tc_setup(c);
+  if (rc == VLAC_OK) rc = vlac_attention_setup(c);
   if (rc != VLAC_OK) { free_ctx_buffers(c); delete c; return rc; }
   *out = c;
   return VLAC_OK;
@@ -188,6 +189,7 @@ int vlac_cache_alloc(vlac_ctx* ctx, int batch, vlac_cache** out) {
   if (rc == VLAC_OK) rc = dev_alloc(&c->tot, nl);
   if (rc == VLAC_OK) rc = dev_alloc(&c->rowmap, nl * B * L);
   if (rc == VLAC_OK) rc = dev_alloc(&c->slot, nl * B * L);
+  if (rc == VLAC_OK) rc = vlac_attention_cache_setup(ctx, c);
   if (rc != VLAC_OK) { free_cache_buffers(c); delete c; return rc; }
   *out = c;
   return VLAC_OK;

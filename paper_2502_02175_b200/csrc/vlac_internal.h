@@ -47,6 +47,8 @@ struct vlac_ctx {
   int *dev_error;                    // device ints: [0] nonzero if a bounded wait gave up
   void* tmaps;                       // device array of TMA tensor maps (weights per layer, activation buffers)
   int tc_ok;                         // 1: shapes fit the tensor-memory GEMM
+  void* tmap_q;                      // device tensor map of the query buffer (tiled attention)
+  int attn_tiles;                    // 64-query tiles per sequence, 0: tiled attention not usable
   // optional per-launch timing of the matrix-vector kernel (vlac_profile)
   int prof_on, prof_n;
   cudaEvent_t* prof_ev;              // [2 * VLAC_PROF_CAP]
@@ -72,6 +74,7 @@ struct vlac_cache {
   int *tot;                          // [nl]                 total rows over the batch
   int *rowmap;                       // [nl][batch*L]        compact index -> b*L + pos
   int *slot;                         // [nl][batch*L]        b*L + pos -> compact index or -1
+  void* tmaps_kv;                    // device tensor maps of the K and V cache of every layer
 };
 
 static inline size_t kv_layer_elems(const vlac_ctx* c) {
@@ -100,6 +103,12 @@ int vlac_tc_setup(vlac_ctx* ctx);
 int vlac_tc_qkv(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s);
 int vlac_tc_partial(vlac_ctx* ctx, vlac_cache* c, int layer, int which /* 0: output proj, 1: down proj */, int* n_splits, cudaStream_t s);
 int vlac_tc_gateup(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s);
+
+// ---- tiled prefill attention (attention_kernels.cu)
+int vlac_encode_map_2d(void* out, const void* base, int rows, int cols, int box_rows);
+int vlac_attention_setup(vlac_ctx* ctx);
+int vlac_attention_cache_setup(vlac_ctx* ctx, vlac_cache* c);
+int vlac_launch_prefill_attention(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s);
 
 // ---- decode (decode_kernels.cu)
 int vlac_decode_setup(vlac_ctx* ctx);
