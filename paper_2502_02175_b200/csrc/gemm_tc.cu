@@ -11,11 +11,13 @@
 //
 // Warp roles (192 threads): warp 0 issues TMA loads into a ring of stages, warp 1 allocates TMEM and
 // issues the MMAs, warps 2-5 read the accumulator back (each its own quarter of the 128 lanes) and run
-// the epilogue.  The 128 weight rows of a tile are fetched as eight 16-row boxes whose order is chosen
-// per mode so that the two values an epilogue needs together sit 16 lanes apart in one warp:
-//   QKV     the two halves of a rotary pair  -> rotation at the row's own position, K/V scatter
-//   SWIGLU  gate row and up row of a feature -> silu(gate) * up
-//   PARTIAL plain order                      -> fp32 split-K partial (output / down projection)
+// the epilogue.  Few, large TMA boxes are used (one 128-row box of weights, one box of up to 256 token
+// rows per k-block): the TMA unit works through requests one at a time, so many small boxes starve it.
+// Epilogues:
+//   QKV     rotation at the row's own position, K/V scatter into the cache, Q to the compact buffer;
+//           the two halves of a rotary pair sit in different warps and are exchanged through shared memory
+//   SWIGLU  the tile is 64 gate rows followed by the 64 up rows of the same features; silu(gate) * up
+//   PARTIAL fp32 split-K partial (output / down projection)
 #include "vlac_internal.h"
 #include "launch_util.h"
 #include <cuda.h>
@@ -36,13 +38,14 @@ constexpr int TG_SMEM_RING = 208 * 1024;        // dynamic shared memory for the
 constexpr unsigned long long TG_WAIT_LIMIT_NS = 400000000ull;
 
 struct TcArgs {
-  const CUtensorMap* tm_a[3];     // weight matrices (16-row boxes)
-  const CUtensorMap* tm_b;        // activations [rows][K] (64-row boxes)
+  const CUtensorMap* tm_a[3];     // weight matrices (128-row boxes; 64-row boxes for gate / up)
+  const CUtensorMap* tm_b;        // activations [rows][K]: 4 maps with boxes of 64, 128, 192, 256 rows
   const int* tot;                 // live token count in device memory (NULL: tot_fixed)
   int tot_fixed;
   int K, N;                       // N = rows of one weight matrix
   int mode, n_splits;
   int d;                          // head_dim (QKV)
+  int batch;                      // sequences sharing the compact row space
   // epilogue operands
   const int* rowmap;              // compact token -> b*L + pos
   int L, max_seq;
@@ -120,28 +123,10 @@ __device__ __forceinline__ void tmem_ld16(unsigned taddr, float* v) {
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-// First weight row of box g (16 rows) of tile `tile`, and which matrix it comes from.
-__device__ __forceinline__ void box_source(const TcArgs& a, int tile, int g, int* mat, int* row0) {
-  if (a.mode == TG_QKV) {
-    const int tiles_per_mat = (a.N + 127) / 128;
-    *mat = tile / tiles_per_mat;
-    const int base = (tile - *mat * tiles_per_mat) * 128;
-    const int half = a.d / 2;
-    const int p = 16 * (g >> 1);                       // first rotary pair of this warp quarter (64 pairs per tile)
-    const int r = base + (p / half) * a.d + (p % half);
-    *row0 = (g & 1) ? r + half : r;
-  } else if (a.mode == TG_SWIGLU) {
-    *mat = g & 1;                                      // even boxes: gate rows, odd boxes: up rows
-    *row0 = tile * 64 + 16 * (g >> 1);
-  } else {
-    *mat = 0;
-    *row0 = tile * 128 + 16 * g;
-  }
-}
-
 __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(TcArgs a) {
   extern __shared__ __align__(1024) unsigned char ring_raw[];
   __shared__ __align__(8) unsigned long long full_bar[TG_MAX_STAGES], empty_bar[TG_MAX_STAGES], acc_bar;
+  __shared__ float xch[2][4][16][32];                            // epilogue exchange between warp pairs (double-buffered)
   __shared__ unsigned tmem_base_slot;
   __shared__ int abort_flag;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -160,7 +145,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(TcArgs a) {
   pdl_trigger();
   pdl_wait();                                                   // everything below may read what earlier kernels wrote
   const int tokens = a.tot ? *a.tot : a.tot_fixed;
-  const int n_boxes = (tokens + TG_BOX_TOK - 1) / TG_BOX_TOK;
+  const int n_boxes = (tokens + TG_BOX_TOK - 1) / TG_BOX_TOK;    // token rows are staged in multiples of 64
   const int stage_bytes = TG_A_BYTES + n_boxes * TG_BOX_BYTES;
   int n_stages = TG_SMEM_RING / stage_bytes;
   if (n_stages > TG_MAX_STAGES) n_stages = TG_MAX_STAGES;
@@ -171,6 +156,10 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(TcArgs a) {
   const int n0 = min(((tokens + 15) / 16) * 16, 256);           // columns of the first MMA
   const int n1 = tokens > 256 ? ((tokens - 256 + 15) / 16) * 16 : 0;
   const unsigned tmem_cols = (n0 + n1) <= 32 ? 32u : ((n0 + n1) <= 64 ? 64u : ((n0 + n1) <= 128 ? 128u : ((n0 + n1) <= 256 ? 256u : 512u)));
+  // weight rows of this tile
+  const int tiles_per_mat = (a.N + 127) / 128;
+  const int mat = a.mode == TG_QKV ? tile / tiles_per_mat : 0;
+  const int row_base = a.mode == TG_QKV ? (tile - mat * tiles_per_mat) * 128 : (a.mode == TG_SWIGLU ? tile * 64 : tile * 128);
 
   if (warp == 1) {                                              // TMEM allocation (whole warp)
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
@@ -184,9 +173,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(TcArgs a) {
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      int mats[8], rows[8];
-#pragma unroll
-      for (int g = 0; g < 8; ++g) box_source(a, tile, g, &mats[g], &rows[g]);
+      const int rows0 = min(n_boxes, 4), rows1 = n_boxes - rows0;            // boxes of the first / second token request
       for (int i = 0; i < n_kb; ++i) {
         const int s = i % n_stages;
         if (i >= n_stages && !mbar_wait(&empty_bar[s], ((i / n_stages) & 1) ^ 1, &abort_flag, a.dev_error, 0x40000 | (i & 0xffff))) break;
@@ -194,9 +181,14 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(TcArgs a) {
         unsigned char* sb = sa + TG_A_BYTES;
         mbar_expect_tx(&full_bar[s], (unsigned)stage_bytes);
         const int k = (kb0 + i) * TG_BK;
-#pragma unroll
-        for (int g = 0; g < 8; ++g) tma_load_2d(sa + g * 2048, a.tm_a[mats[g]], k, rows[g], &full_bar[s]);
-        for (int bx = 0; bx < n_boxes; ++bx) tma_load_2d(sb + bx * TG_BOX_BYTES, a.tm_b, k, bx * TG_BOX_TOK, &full_bar[s]);
+        if (a.mode == TG_SWIGLU) {
+          tma_load_2d(sa, a.tm_a[0], k, row_base, &full_bar[s]);                // 64 gate rows
+          tma_load_2d(sa + 64 * 128, a.tm_a[1], k, row_base, &full_bar[s]);     // 64 up rows of the same features
+        } else {
+          tma_load_2d(sa, a.tm_a[mat], k, row_base, &full_bar[s]);
+        }
+        tma_load_2d(sb, a.tm_b + (rows0 - 1), k, 0, &full_bar[s]);
+        if (rows1 > 0) tma_load_2d(sb + 4 * TG_BOX_BYTES, a.tm_b + (rows1 - 1), k, 256, &full_bar[s]);
       }
     }
   } else if (warp == 1) {
@@ -230,48 +222,69 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(TcArgs a) {
     bool ok = n_kb > 0;
     if (ok) ok = mbar_wait(&acc_bar, 0, &abort_flag, a.dev_error, 0x60000);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (ok) {
-      int mat, row0;
-      box_source(a, tile, 2 * q + (lane >> 4), &mat, &row0);
-      const int n = row0 + (lane & 15);                          // weight row (output feature) of this lane
-      const bool n_ok = n < a.N;
-      const int half = a.d / 2;
-      for (int c0 = 0; c0 < tokens; c0 += 16) {
-        float v[16];
-        tmem_ld16(tmem_base + ((unsigned)(32 * q) << 16) + (unsigned)c0, v);
-        if (a.mode == TG_PARTIAL) {
-          float* dst = a.part + (size_t)split * a.split_stride + n;
+    const int r = 32 * q + lane;                                 // row of the tile held by this thread
+    const int half = a.d / 2;
+    // feature (weight row) this thread finishes, and the warp holding its partner value
+    int n, pq;
+    bool first;                                                  // QKV: first half of the rotary pair; SWIGLU: gate side
+    if (a.mode == TG_SWIGLU) { n = row_base + (r & 63); first = r < 64; pq = q ^ 2; }
+    else { n = row_base + r; first = ((r / half) & 1) == 0; pq = q ^ (half >> 5); }
+    const bool n_ok = n < a.N;
+    const bool exchange = a.mode == TG_SWIGLU || (a.mode == TG_QKV && mat < 2);
+    const int j = (n % a.d) % half;
+    const size_t N = (size_t)a.N;
+    int chunk = 0;
+    for (int c0 = 0; c0 < tokens; c0 += 16, ++chunk) {
+      float v[16], pv[16];
+      if (ok) tmem_ld16(tmem_base + ((unsigned)(32 * q) << 16) + (unsigned)c0, v);
+      else {
 #pragma unroll
-          for (int c = 0; c < 16; ++c)
-            if (c0 + c < tokens && n_ok) dst[(size_t)(c0 + c) * a.N] = v[c];
-        } else if (a.mode == TG_SWIGLU) {
+        for (int c = 0; c < 16; ++c) v[c] = 0.f;
+      }
+      if (exchange) {                                            // uniform over the four epilogue warps
+        float (*buf)[16][32] = xch[chunk & 1];
 #pragma unroll
-          for (int c = 0; c < 16; ++c) {
-            const float pv = __shfl_xor_sync(0xffffffffu, v[c], 16);
-            const bool mine = ((c & 1) == 0) == (lane < 16);     // low half-warp finishes even columns, high half odd ones
-            const float g = lane < 16 ? v[c] : pv, u = lane < 16 ? pv : v[c];
-            if (mine && c0 + c < tokens && n_ok) a.h_out[(size_t)(c0 + c) * a.N + n] = __float2bfloat16(g / (1.f + __expf(-g)) * u);
+        for (int c = 0; c < 16; ++c) buf[q][c][lane] = v[c];
+        asm volatile("bar.sync 2, 128;" ::: "memory");
+#pragma unroll
+        for (int c = 0; c < 16; ++c) pv[c] = buf[pq][c][lane];
+      }
+      const bool live = ok && n_ok;                               // no early exit: the warp shuffles below need every lane
+      if (a.mode == TG_PARTIAL) {
+        if (!live) continue;
+        float* dst = a.part + (size_t)split * a.split_stride + n;
+#pragma unroll
+        for (int c = 0; c < 16; ++c)
+          if (c0 + c < tokens) dst[(size_t)(c0 + c) * N] = v[c];
+      } else if (a.mode == TG_SWIGLU) {
+        // gate-side threads finish even columns, up-side threads odd columns
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          if (live && ((c & 1) == 0) == first && c0 + c < tokens) {
+            const float g = first ? v[c] : pv[c], u = first ? pv[c] : v[c];
+            a.h_out[(size_t)(c0 + c) * N + n] = __float2bfloat16(__fdividef(g, 1.f + __expf(-g)) * u);
           }
-        } else {                                                 // TG_QKV
+        }
+      } else {                                                   // TG_QKV
+        const int my_row = (c0 + (lane & 15) < tokens) ? __ldg(a.rowmap + c0 + (lane & 15)) : 0;
+        // all table reads of the chunk first (independent loads in flight together), then the arithmetic and stores
+        int bs[16], ps[16];
+        float cs[16], sn[16];
 #pragma unroll
-          for (int c = 0; c < 16; ++c) {
-            const float pv = __shfl_xor_sync(0xffffffffu, v[c], 16);
-            const int t = c0 + c;
-            if (t < tokens && n_ok) {
-              const int row = a.rowmap[t];
-              const int b = row / a.L, pos = row - b * a.L;
-              float y = v[c];
-              if (mat < 2) {
-                const int j = n % a.d % half;
-                const float cs = a.rope_cos[(size_t)pos * half + j], sn = a.rope_sin[(size_t)pos * half + j];
-                y = lane < 16 ? v[c] * cs - pv * sn : v[c] * cs + pv * sn;
-              }
-              if (mat == 0) a.q_out[(size_t)t * a.N + n] = __float2bfloat16(y);
-              else {
-                bf16* cache = mat == 1 ? a.kc : a.vc;
-                cache[((size_t)b * a.max_seq + pos) * a.N + n] = __float2bfloat16(y);
-              }
-            }
+        for (int c = 0; c < 16; ++c) {
+          const int row = __shfl_sync(0xffffffffu, my_row, c);
+          int b = 0, pos = row;
+          if (a.batch > 1) { b = row / a.L; pos = row - b * a.L; }
+          bs[c] = b; ps[c] = pos;
+          if (mat < 2) { cs[c] = __ldg(a.rope_cos + (size_t)pos * half + j); sn[c] = __ldg(a.rope_sin + (size_t)pos * half + j); }
+        }
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          if (live && c0 + c < tokens) {
+            float y = v[c];
+            if (mat < 2) y = first ? v[c] * cs[c] - pv[c] * sn[c] : v[c] * cs[c] + pv[c] * sn[c];
+            if (mat == 0) a.q_out[(size_t)(c0 + c) * N + n] = __float2bfloat16(y);
+            else (mat == 1 ? a.kc : a.vc)[((size_t)bs[c] * a.max_seq + ps[c]) * N + n] = __float2bfloat16(y);
           }
         }
       }
@@ -313,15 +326,15 @@ int vlac_encode_map_2d(void* out, const void* base, int rows, int cols, int box_
   return encode_map((CUtensorMap*)out, base, rows, cols, box_rows);
 }
 
-// Tensor maps of one context: 7 per layer (weights, 16-row boxes) + 3 activation buffers (64-row boxes).
+// Tensor maps of one context: 7 per layer (weights) + 3 activation buffers x 4 box heights.
 enum { TM_WQ = 0, TM_WK, TM_WV, TM_WO, TM_GATE, TM_UP, TM_DOWN, TM_PER_LAYER };
-enum { TM_XN = 0, TM_AO, TM_HM, TM_ACT_COUNT };
+enum { TM_XN = 0, TM_AO = 4, TM_HM = 8, TM_ACT_COUNT = 12 };   // 4 box heights (64..256 rows) per activation buffer
 
 int vlac_tc_setup(vlac_ctx* ctx) {
   const vlac_config& g = ctx->cfg;
   ctx->tc_ok = 0;
   // the TMA path needs 16-byte aligned rows and pointers
-  if (g.hidden % 8 || g.ffn % 8) return VLAC_OK;
+  if (g.hidden % 8 || g.ffn % 8 || (g.head_dim != 64 && g.head_dim != 128)) return VLAC_OK;
   const int n_maps = g.n_layers * TM_PER_LAYER + TM_ACT_COUNT;
   CUtensorMap* host = (CUtensorMap*)malloc(sizeof(CUtensorMap) * n_maps);
   if (!host) return VLAC_ERR_OOM;
@@ -334,13 +347,16 @@ int vlac_tc_setup(vlac_ctx* ctx) {
     const int cols[TM_PER_LAYER] = {D, D, D, D, D, D, F};
     for (int m = 0; m < TM_PER_LAYER && rc == VLAC_OK; ++m) {
       if (reinterpret_cast<uintptr_t>(ptr[m]) & 15) { free(host); return VLAC_OK; }   // unaligned weights: stay on the generic path
-      rc = encode_map(&host[l * TM_PER_LAYER + m], ptr[m], rows[m], cols[m], 16);
+      rc = encode_map(&host[l * TM_PER_LAYER + m], ptr[m], rows[m], cols[m], (m == TM_GATE || m == TM_UP) ? 64 : 128);
     }
   }
   CUtensorMap* act = host + g.n_layers * TM_PER_LAYER;
-  if (rc == VLAC_OK) rc = encode_map(&act[TM_XN], ctx->xn, ctx->rows_max, D, TG_BOX_TOK);
-  if (rc == VLAC_OK) rc = encode_map(&act[TM_AO], ctx->ao, ctx->rows_max, D, TG_BOX_TOK);
-  if (rc == VLAC_OK) rc = encode_map(&act[TM_HM], ctx->hm, ctx->rows_max, F, TG_BOX_TOK);
+  for (int hgt = 0; hgt < 4 && rc == VLAC_OK; ++hgt) {
+    const int box = 64 * (hgt + 1);
+    rc = encode_map(&act[TM_XN + hgt], ctx->xn, ctx->rows_max, D, box);
+    if (rc == VLAC_OK) rc = encode_map(&act[TM_AO + hgt], ctx->ao, ctx->rows_max, D, box);
+    if (rc == VLAC_OK) rc = encode_map(&act[TM_HM + hgt], ctx->hm, ctx->rows_max, F, box);
+  }
   if (rc != VLAC_OK) { free(host); return rc; }
   cudaError_t e = cudaMalloc(&ctx->tmaps, sizeof(CUtensorMap) * n_maps);
   if (e != cudaSuccess) { free(host); cudaGetLastError(); return VLAC_ERR_OOM; }
@@ -371,6 +387,7 @@ static void tc_common(vlac_ctx* ctx, vlac_cache* c, int layer, TcArgs* a) {
   a->rope_cos = ctx->w.rope_cos; a->rope_sin = ctx->w.rope_sin;
   a->dev_error = ctx->dev_error;
   a->n_splits = 1;
+  a->batch = c->batch;
 }
 
 int vlac_tc_qkv(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s) {
