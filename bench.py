@@ -208,6 +208,9 @@ def run_ours(args):
     # cached step so that the median layer reuses 3/4 of P_final, then frozen
     params, keep = vb.make_params(k_ent=1.0)
 
+    side = torch.cuda.Stream()          # the step replays as a CUDA graph on a non-default stream
+    torch.cuda.set_stream(side)
+
     def step(t, p=params, full=False):
         vb.vlac_step(ctx, cache, frames_d[t:t + 1], feats_d[t:t + 1], ids_d, p, full, tokens)
 

@@ -50,6 +50,8 @@ void free_ctx_buffers(vlac_ctx* c) {
   cudaFree(c->xn); cudaFree(c->q); cudaFree(c->ao); cudaFree(c->hm); cudaFree(c->part); cudaFree(c->scratch);
   cudaFree(c->probs); cudaFree(c->hidden); cudaFree(c->x_dec); cudaFree(c->q_dec); cudaFree(c->ao_dec);
   cudaFree(c->hm_dec); cudaFree(c->logits); cudaFree(c->argmax_tmp); cudaFree(c->dev_error); cudaFree(c->tmaps); cudaFree(c->tmap_q);
+  cudaFree(c->in_frames); cudaFree(c->in_feats); cudaFree(c->in_ids); cudaFree(c->in_forced); cudaFree(c->out_tokens); cudaFree(c->logits_all);
+  for (int i = 0; i < VLAC_MAX_GRAPHS; ++i) if (c->graphs[i].used) cudaGraphExecDestroy(c->graphs[i].exec);
   if (c->prof_ev) {
     for (int i = 0; i < 2 * VLAC_PROF_CAP; ++i) if (c->prof_ev[i]) cudaEventDestroy(c->prof_ev[i]);
     free(c->prof_ev);
@@ -140,6 +142,13 @@ int vlac_create(const vlac_config* cfg, const vlac_weights* w, vlac_ctx** out) {
   if (rc == VLAC_OK) rc = dev_alloc(&c->logits, B * (size_t)g.vocab);
   if (rc == VLAC_OK) rc = dev_alloc(&c->argmax_tmp, B * VLAC_ARGMAX_BLOCKS);
   if (rc == VLAC_OK) rc = dev_alloc(&c->dev_error, 8);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->in_frames, B * (size_t)g.n_cams * c->frame_hw * c->frame_hw * 3);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->in_feats, B * (size_t)c->Lv * D);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->in_ids, B * (size_t)(g.n_text_pre + g.n_text_post));
+  if (rc == VLAC_OK) rc = dev_alloc(&c->in_forced, B * (size_t)g.n_action);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->out_tokens, B * (size_t)g.n_action);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->logits_all, B * (size_t)g.n_action * g.vocab);
+  c->use_graph = getenv("VLAC_NO_GRAPH") ? 0 : 1;
   if (rc == VLAC_OK) rc = vlac_decode_setup(c);
   if (rc == VLAC_OK) rc = vlac_tc_setup(c);
   if (rc == VLAC_OK) rc = vlac_attention_setup(c);
@@ -207,6 +216,10 @@ int vlac_cache_reset(vlac_cache* cache, int seq, void* stream) {
 int vlac_cache_free(vlac_cache* cache) {
   if (!cache) return VLAC_ERR_INVALID_ARG;
   cudaDeviceSynchronize();
+  for (int i = 0; i < VLAC_MAX_GRAPHS; ++i) {
+    StepGraph& e = cache->ctx->graphs[i];
+    if (e.used && e.cache == cache) { cudaGraphExecDestroy(e.exec); e.used = 0; }
+  }
   free_cache_buffers(cache);
   delete cache;
   return VLAC_OK;
@@ -316,19 +329,14 @@ int vlac_layer_forward(vlac_ctx* ctx, vlac_cache* cache, int layer, void* hidden
   return VLAC_OK;
 }
 
-int vlac_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, const void* vision_feats,
-              const int* prompt_ids, const vlac_select_params* params, int force_full,
-              int* action_tokens, float* all_logits, const int* forced_tokens, void* stream) {
-  if (!ctx || !cache || cache->ctx != ctx || !frames || !vision_feats || !action_tokens) return VLAC_ERR_INVALID_ARG;
+// Enqueue every kernel of one control step on `s` (directly, or into a stream capture).
+static int enqueue_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, const void* vision_feats,
+                        const int* prompt_ids, const SelectKernelParams& p, int* action_tokens, float* all_logits,
+                        const int* forced_tokens, cudaStream_t s) {
   const vlac_config& g = ctx->cfg;
-  if (!prompt_ids && g.n_text_pre + g.n_text_post > 0) return VLAC_ERR_INVALID_ARG;
-  cudaStream_t s = (cudaStream_t)stream;
-  SelectKernelParams p;
-  TRY(fill_params(ctx, params, force_full, &p));
   const int B = cache->batch, nl = g.n_layers;
   // 1. which rows each layer recomputes
   TRY(vlac_launch_select(ctx, cache, frames, p, s));
-  cache->has_selection = 1;
   // 2. rows entering layer 0
   bf16* h = ctx->hidden;
   TRY(vlac_launch_input_rows(ctx, cache, vision_feats, prompt_ids, h, s));
@@ -357,6 +365,71 @@ int vlac_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, con
                                   cudaMemcpyDeviceToDevice, s));
   set_warm_kernel<<<1, 32, 0, s>>>(cache->warm, B, 1);
   VLAC_LAUNCH_CHECK(ctx);
+  return VLAC_OK;
+}
+
+int vlac_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, const void* vision_feats,
+              const int* prompt_ids, const vlac_select_params* params, int force_full,
+              int* action_tokens, float* all_logits, const int* forced_tokens, void* stream) {
+  if (!ctx || !cache || cache->ctx != ctx || !frames || !vision_feats || !action_tokens) return VLAC_ERR_INVALID_ARG;
+  const vlac_config& g = ctx->cfg;
+  const int n_text = g.n_text_pre + g.n_text_post;
+  if (!prompt_ids && n_text > 0) return VLAC_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  SelectKernelParams p;
+  TRY(fill_params(ctx, params, force_full, &p));
+  const int B = cache->batch;
+  cache->has_selection = 1;
+
+  // The step is replayed as a CUDA graph (about 1300 kernels with device-side shapes: the graph never
+  // changes).  A graph needs fixed addresses, so caller buffers are staged through library buffers.
+  // Not used on the legacy default stream, inside a caller's own capture, or while per-launch timing is on.
+  cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+  bool direct = !ctx->use_graph || ctx->prof_on || s == nullptr || s == cudaStreamLegacy;
+  if (!direct) {
+    VLAC_CUDA_CHECK(cudaStreamIsCapturing(s, &cap));
+    if (cap != cudaStreamCaptureStatusNone) direct = true;
+  }
+  if (direct)
+    return enqueue_step(ctx, cache, frames, vision_feats, prompt_ids, p, action_tokens, all_logits, forced_tokens, s);
+
+  const size_t frame = (size_t)B * g.n_cams * ctx->frame_hw * ctx->frame_hw * 3;
+  VLAC_CUDA_CHECK(cudaMemcpyAsync(ctx->in_frames, frames, frame, cudaMemcpyDeviceToDevice, s));
+  VLAC_CUDA_CHECK(cudaMemcpyAsync(ctx->in_feats, vision_feats, sizeof(bf16) * (size_t)B * ctx->Lv * g.hidden, cudaMemcpyDeviceToDevice, s));
+  if (n_text > 0) VLAC_CUDA_CHECK(cudaMemcpyAsync(ctx->in_ids, prompt_ids, sizeof(int) * (size_t)B * n_text, cudaMemcpyDeviceToDevice, s));
+  if (forced_tokens) VLAC_CUDA_CHECK(cudaMemcpyAsync(ctx->in_forced, forced_tokens, sizeof(int) * (size_t)B * g.n_action, cudaMemcpyDeviceToDevice, s));
+
+  StepGraph* entry = nullptr;
+  for (int i = 0; i < VLAC_MAX_GRAPHS; ++i) {
+    StepGraph& e = ctx->graphs[i];
+    if (e.used && e.cache == cache && e.force_full == (force_full ? 1 : 0) && e.use_forced == (forced_tokens ? 1 : 0) &&
+        memcmp(&e.p, &p, sizeof(p)) == 0) { entry = &e; break; }
+  }
+  if (!entry) {
+    StepGraph& e = ctx->graphs[ctx->graph_next];
+    ctx->graph_next = (ctx->graph_next + 1) % VLAC_MAX_GRAPHS;
+    if (e.used) { cudaGraphExecDestroy(e.exec); e.used = 0; }
+    const unsigned long long l0 = ctx->launches;
+    VLAC_CUDA_CHECK(cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal));
+    const int rc = enqueue_step(ctx, cache, ctx->in_frames, ctx->in_feats, ctx->in_ids, p, ctx->out_tokens, ctx->logits_all,
+                                forced_tokens ? ctx->in_forced : nullptr, s);
+    cudaGraph_t graph = nullptr;
+    const cudaError_t ce = cudaStreamEndCapture(s, &graph);
+    if (rc != VLAC_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
+    VLAC_CUDA_CHECK(ce);
+    const cudaError_t ie = cudaGraphInstantiate(&e.exec, graph, 0);
+    cudaGraphDestroy(graph);
+    VLAC_CUDA_CHECK(ie);
+    e.used = 1; e.cache = cache; e.force_full = force_full ? 1 : 0; e.use_forced = forced_tokens ? 1 : 0; e.p = p;
+    e.launches = ctx->launches - l0;
+    ctx->launches = l0;
+    entry = &e;
+  }
+  VLAC_CUDA_CHECK(cudaGraphLaunch(entry->exec, s));
+  ctx->launches += entry->launches;
+  VLAC_CUDA_CHECK(cudaMemcpyAsync(action_tokens, ctx->out_tokens, sizeof(int) * (size_t)B * g.n_action, cudaMemcpyDeviceToDevice, s));
+  if (all_logits)
+    VLAC_CUDA_CHECK(cudaMemcpyAsync(all_logits, ctx->logits_all, sizeof(float) * (size_t)B * g.n_action * g.vocab, cudaMemcpyDeviceToDevice, s));
   return VLAC_OK;
 }
 

@@ -28,6 +28,17 @@ struct SelectKernelParams {          // passed by value to the selection kernel
   double alpha_override[VLAC_MAX_LAYERS];
 };
 
+struct vlac_cache;
+struct StepGraph {                     // one captured control step (CUDA graph), keyed by what is baked into it
+  int used;
+  vlac_cache* cache;
+  int force_full, use_forced;
+  SelectKernelParams p;
+  cudaGraphExec_t exec;
+  unsigned long long launches;
+};
+#define VLAC_MAX_GRAPHS 4
+
 struct vlac_ctx {
   vlac_config cfg;
   vlac_weights w;
@@ -45,6 +56,10 @@ struct vlac_ctx {
   float *logits;                     // [max_batch][vocab]
   unsigned long long *argmax_tmp;    // [max_batch][VLAC_ARGMAX_BLOCKS]
   int *dev_error;                    // device ints: [0] nonzero if a bounded wait gave up
+  // step staging: the captured graph reads and writes only library-owned buffers
+  unsigned char* in_frames; bf16* in_feats; int *in_ids, *in_forced, *out_tokens; float* logits_all;
+  StepGraph graphs[VLAC_MAX_GRAPHS];
+  int graph_next, use_graph;
   void* tmaps;                       // device array of TMA tensor maps (weights per layer, activation buffers)
   int tc_ok;                         // 1: shapes fit the tensor-memory GEMM
   void* tmap_q;                      // device tensor map of the query buffer (tiled attention)

@@ -36,6 +36,7 @@ class Session:
         self.ctx = vb.vlac_create(vb.make_config(cfg, max_batch=batch), self.dev.weights)
         self.cache = vb.vlac_cache_alloc(self.ctx, batch)
         self.ocache = [orc.new_cache(cfg) for _ in range(batch)]
+        self.stream = torch.cuda.Stream()      # a non-default stream: vlac_step replays its CUDA graph there
 
     def close(self):
         vb.vlac_cache_free(self.cache)
@@ -114,7 +115,9 @@ def run_step_pair(sess: Session, frames: np.ndarray, feats: np.ndarray, ids: np.
     d_ids = torch.from_numpy(ids.astype(np.int32)).to("cuda").contiguous()
     tokens = torch.zeros((B, cfg.n_action), dtype=torch.int32, device="cuda")
     logits = torch.zeros((B, cfg.n_action, cfg.vocab), dtype=torch.float32, device="cuda")
-    vb.vlac_step(sess.ctx, sess.cache, d_frames, d_feats, d_ids, gp, force_full, tokens, logits)
+    torch.cuda.synchronize()
+    with torch.cuda.stream(sess.stream):
+        vb.vlac_step(sess.ctx, sess.cache, d_frames, d_feats, d_ids, gp, force_full, tokens, logits)
     torch.cuda.synchronize()
     assert vb.vlac_device_error(sess.ctx) == 0
     got_sel = vb.selection_to_host(vb.vlac_selection_view(sess.cache))

@@ -257,3 +257,38 @@ def test_step_batch_of_three_ragged(H, vb):
             assert r["logit_err"] <= H.TOL and r["attn_err"] <= H.TOL
     finally:
         sess.close()
+
+
+def test_step_graph_replay_equals_direct_launch(H, vb):
+    """On a non-default stream the step is captured once and replayed as a CUDA graph; on the default
+    stream every kernel is launched directly.  Both must give the same bits, step after step."""
+    cfg, model, ids, feats = _tiny_inputs(3)
+    prev, cur, _ = synth.rerandomised_pair(cfg, 3, 13)
+    side = torch.cuda.Stream()
+    outs = []
+    for use_side in (False, True):
+        sess = H.Session(cfg, model)
+        try:
+            gp, keep = H.gparams(H.oparams(top_k=32, alpha_override=[0.5, 1.0]))
+            args = (vb.upload_bf16(feats), torch.from_numpy(ids).to("cuda"))
+            res = []
+            torch.cuda.synchronize()
+            for fr in (prev, cur, cur, prev):
+                tok = torch.zeros((1, cfg.n_action), dtype=torch.int32, device="cuda")
+                lg = torch.zeros((1, cfg.n_action, cfg.vocab), dtype=torch.float32, device="cuda")
+                d_fr = torch.from_numpy(fr[None]).to("cuda")
+                torch.cuda.synchronize()
+                l0 = vb.vlac_launch_count(sess.ctx)
+                if use_side:
+                    with torch.cuda.stream(side):
+                        vb.vlac_step(sess.ctx, sess.cache, d_fr, *args, gp, False, tok, lg)
+                else:
+                    vb.vlac_step(sess.ctx, sess.cache, d_fr, *args, gp, False, tok, lg)
+                torch.cuda.synchronize()
+                res.append((tok.cpu().numpy().copy(), lg.cpu().numpy().copy(), vb.vlac_launch_count(sess.ctx) - l0))
+            outs.append(res)
+        finally:
+            sess.close()
+    for (t0, l0, n0), (t1, l1, n1) in zip(*outs):
+        assert np.array_equal(t0, t1) and np.array_equal(l0, l1)
+        assert n0 == n1 > 0                      # the replay reports the kernels it ran
