@@ -257,6 +257,7 @@ def run_ours(args):
     timed(min(K, 4), 1 + W)
     vb.vlac_profile(ctx, False)
     k_ms, k_bytes, k_n = vb.vlac_profile_read(ctx)
+    segments = vb.vlac_profile_segments(ctx)
     # the same library with reuse off
     for i in range(2):
         step(1 + W + i, params, True)
@@ -318,6 +319,9 @@ def run_ours(args):
                               "frac": (step_bytes / (peak * 1e6)) / ms_step},
             "full_recompute": {"ms_per_step": ms_full, "speedup_cached": ms_full / ms_step},
             "control_hz": 1e3 / ms_step,
+            "profiled_step_parts_ms": {"note": "direct launches with per-launch events, not the graph replay",
+                                       "select": segments[0], "input_rows": segments[1], "prefill_layers": segments[2],
+                                       "first_token": segments[3], "single_row_passes": segments[4:]} if len(segments) >= 5 else None,
             "cpu_baseline": None if cpu_s is None else {"value": cfg.n_action / cpu_s, "unit": UNIT, "cores": cpu_threads,
                                                         "kind": "oracle", "sample": SAMPLE_TEXT, "parts": cpu_parts},
             "paper_context": "paper: up to 1.7x CUDA latency, OpenVLA 51.91 -> 31.83 ms per step on one RTX 4090 (bf16, real weights)",

@@ -182,6 +182,11 @@ unsigned long long vlac_launch_count(const vlac_ctx* ctx);
  * count. */
 int vlac_profile(vlac_ctx* ctx, int enable);
 int vlac_profile_read(vlac_ctx* ctx, double* ms_total, unsigned long long* bytes_total, int* n_launches);
+/* Device time (ms) of the parts of the last step run while profiling was on, in order: selection,
+ * input rows, all prefill layers, first action token, then one entry per single-row pass.  Writes at
+ * most `cap` entries and their count to *n.  (A profiled step launches its kernels one by one; the
+ * graph replay is not used, so the parts include launch gaps the replay does not have.) */
+int vlac_profile_segments(vlac_ctx* ctx, double* ms, int cap, int* n);
 
 /* Nonzero if a device-side bounded wait gave up since the context was created (reads one int
  * back; synchronises the stream). */

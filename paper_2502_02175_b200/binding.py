@@ -55,7 +55,7 @@ class vlac_selection(C.Structure):
 EXPORTS = ("vlac_create", "vlac_destroy", "vlac_cache_alloc", "vlac_cache_reset", "vlac_cache_free",
            "vlac_cache_read", "vlac_cache_write", "vlac_select", "vlac_select_import", "vlac_layer_forward",
            "vlac_step", "vlac_selection_view", "vlac_launch_count", "vlac_device_error", "vlac_status_string",
-           "vlac_profile", "vlac_profile_read", "vlac_greedy_tokens_static")
+           "vlac_profile", "vlac_profile_read", "vlac_profile_segments", "vlac_greedy_tokens_static")
 
 lib.vlac_status_string.restype = C.c_char_p
 lib.vlac_status_string.argtypes = [C.c_int]
@@ -76,6 +76,7 @@ lib.vlac_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_vo
 lib.vlac_selection_view.argtypes = [C.c_void_p, C.POINTER(vlac_selection)]
 lib.vlac_device_error.argtypes = [C.c_void_p, C.c_void_p]
 lib.vlac_profile.argtypes = [C.c_void_p, C.c_int]
+lib.vlac_profile_segments.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.c_int, C.POINTER(C.c_int)]
 lib.vlac_greedy_tokens_static.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_longlong, C.c_void_p, C.c_void_p]
 lib.vlac_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_ulonglong), C.POINTER(C.c_int)]
 
@@ -266,6 +267,14 @@ def vlac_device_error(ctx: int) -> int:
 
 def vlac_profile(ctx: int, enable: bool) -> None:
     _check(lib.vlac_profile(ctx, int(bool(enable))), "vlac_profile")
+
+
+def vlac_profile_segments(ctx: int):
+    """Device ms of the parts of the last profiled step: [select, input rows, prefill, first token, pass 1, ...]."""
+    buf = (C.c_double * 16)()
+    n = C.c_int()
+    _check(lib.vlac_profile_segments(ctx, buf, 16, C.byref(n)), "vlac_profile_segments")
+    return [buf[i] for i in range(n.value)]
 
 
 def vlac_profile_read(ctx: int):

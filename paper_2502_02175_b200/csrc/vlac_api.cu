@@ -52,6 +52,7 @@ void free_ctx_buffers(vlac_ctx* c) {
   cudaFree(c->hm_dec); cudaFree(c->logits); cudaFree(c->argmax_tmp); cudaFree(c->dev_error); cudaFree(c->tmaps); cudaFree(c->tmap_q);
   cudaFree(c->in_frames); cudaFree(c->in_feats); cudaFree(c->in_ids); cudaFree(c->in_forced); cudaFree(c->out_tokens); cudaFree(c->logits_all);
   for (int i = 0; i < VLAC_MAX_GRAPHS; ++i) if (c->graphs[i].used) cudaGraphExecDestroy(c->graphs[i].exec);
+  for (int i = 0; i < VLAC_SEG_CAP; ++i) if (c->seg_ev[i]) cudaEventDestroy(c->seg_ev[i]);
   if (c->prof_ev) {
     for (int i = 0; i < 2 * VLAC_PROF_CAP; ++i) if (c->prof_ev[i]) cudaEventDestroy(c->prof_ev[i]);
     free(c->prof_ev);
@@ -329,17 +330,30 @@ int vlac_layer_forward(vlac_ctx* ctx, vlac_cache* cache, int layer, void* hidden
   return VLAC_OK;
 }
 
+// While profiling is on, mark a segment boundary of the step (select | input rows | prefill layers |
+// first token | one entry per single-row pass).
+static int seg_mark(vlac_ctx* ctx, cudaStream_t s) {
+  if (!ctx->prof_on || ctx->seg_n >= VLAC_SEG_CAP) return VLAC_OK;
+  if (!ctx->seg_ev[ctx->seg_n]) VLAC_CUDA_CHECK(cudaEventCreate(&ctx->seg_ev[ctx->seg_n]));
+  VLAC_CUDA_CHECK(cudaEventRecord(ctx->seg_ev[ctx->seg_n++], s));
+  return VLAC_OK;
+}
+
 // Enqueue every kernel of one control step on `s` (directly, or into a stream capture).
 static int enqueue_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, const void* vision_feats,
                         const int* prompt_ids, const SelectKernelParams& p, int* action_tokens, float* all_logits,
                         const int* forced_tokens, cudaStream_t s) {
   const vlac_config& g = ctx->cfg;
   const int B = cache->batch, nl = g.n_layers;
+  ctx->seg_n = 0;
+  TRY(seg_mark(ctx, s));
   // 1. which rows each layer recomputes
   TRY(vlac_launch_select(ctx, cache, frames, p, s));
+  TRY(seg_mark(ctx, s));
   // 2. rows entering layer 0
   bf16* h = ctx->hidden;
   TRY(vlac_launch_input_rows(ctx, cache, vision_feats, prompt_ids, h, s));
+  TRY(seg_mark(ctx, s));
   // 3. layers; the down-projection partials of layer l are folded into layer l+1's first kernel
   int n_splits = 0;
   for (int l = 0; l < nl; ++l) {
@@ -347,16 +361,19 @@ static int enqueue_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* f
     TRY(vlac_launch_layer_body(ctx, cache, l, h, &n_splits, s));
   }
   TRY(vlac_launch_finalize_norm(ctx, cache, h, nl - 1, n_splits, nl - 1, nullptr, s));
+  TRY(seg_mark(ctx, s));
   // 4. first action token
   TRY(vlac_launch_last_row(ctx, cache, h, s));
   const long long lstride = (long long)g.n_action * g.vocab;
   TRY(vlac_launch_logits_argmax(ctx, cache, action_tokens, g.n_action, 0, all_logits, lstride, s));
+  TRY(seg_mark(ctx, s));
   // 5. remaining tokens, one single-row pass each
   const int* fed = forced_tokens ? forced_tokens : action_tokens;
   for (int i = 1; i < g.n_action; ++i) {
     TRY(vlac_launch_decode_pass(ctx, cache, fed, g.n_action, i - 1, ctx->L - 1 + i, s));
     TRY(vlac_launch_logits_argmax(ctx, cache, action_tokens, g.n_action, i,
                                   all_logits ? all_logits + (size_t)i * g.vocab : nullptr, lstride, s));
+    TRY(seg_mark(ctx, s));
   }
   // 6. this step becomes "previous"
   const size_t frame = (size_t)B * g.n_cams * ctx->frame_hw * ctx->frame_hw * 3;
@@ -445,6 +462,19 @@ int vlac_profile(vlac_ctx* ctx, int enable) {
   }
   ctx->prof_on = enable ? 1 : 0;
   if (enable) ctx->prof_n = 0;
+  return VLAC_OK;
+}
+
+int vlac_profile_segments(vlac_ctx* ctx, double* ms, int cap, int* n) {
+  if (!ctx || !ms || !n) return VLAC_ERR_INVALID_ARG;
+  int k = 0;
+  for (int i = 0; i + 1 < ctx->seg_n && k < cap; ++i, ++k) {
+    VLAC_CUDA_CHECK(cudaEventSynchronize(ctx->seg_ev[i + 1]));
+    float t = 0.f;
+    VLAC_CUDA_CHECK(cudaEventElapsedTime(&t, ctx->seg_ev[i], ctx->seg_ev[i + 1]));
+    ms[k] = t;
+  }
+  *n = k;
   return VLAC_OK;
 }
 

@@ -28,6 +28,7 @@ struct SelectKernelParams {          // passed by value to the selection kernel
   double alpha_override[VLAC_MAX_LAYERS];
 };
 
+#define VLAC_SEG_CAP 16
 struct vlac_cache;
 struct StepGraph {                     // one captured control step (CUDA graph), keyed by what is baked into it
   int used;
@@ -68,6 +69,8 @@ struct vlac_ctx {
   int prof_on, prof_n;
   cudaEvent_t* prof_ev;              // [2 * VLAC_PROF_CAP]
   unsigned long long* prof_bytes;    // [VLAC_PROF_CAP] weight bytes streamed by each timed launch
+  cudaEvent_t seg_ev[VLAC_SEG_CAP];  // segment boundaries of the last profiled step
+  int seg_n;
 };
 #define VLAC_PROF_CAP 4096
 #define VLAC_ARGMAX_BLOCKS 64
