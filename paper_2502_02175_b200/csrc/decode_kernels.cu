@@ -217,6 +217,96 @@ __global__ void __launch_bounds__(256, 2) gemv_pair_kernel(GemvArgs a) {
   }
 }
 
+// Attention of one new row per sequence over the cache (Sec. 3.1): one CTA per (head, sequence).
+// Scores: one key per thread (whole 16-byte-vectorised dot product); P*V: keys dealt round-robin to the
+// eight warps, each lane owning d/32 consecutive dimensions, partial sums combined in warp order.
+template <int DPL>      // dimensions per lane = head_dim / 32
+__global__ void __launch_bounds__(256) decode_attention_kernel(const bf16* q, const bf16* kc, const bf16* vc, bf16* out,
+                                                               int pos, int max_seq, int H) {
+  extern __shared__ float dsm[];
+  constexpr int d = 32 * DPL;
+  float* qs = dsm;                 // [d]
+  float* p = dsm + d;              // [max_seq]
+  float* part = p + max_seq;       // [8][d]
+  __shared__ float red[8];
+  const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_trigger();
+  pdl_wait();
+  const int D = H * d, nkeys = pos + 1;
+  const float scale = rsqrtf((float)d);
+  if (tid < d) qs[tid] = bf2f(q[(size_t)b * D + h * d + tid]) * scale;
+  __syncthreads();
+  const bf16* kbase = kc + (size_t)b * max_seq * D + h * d;
+  float mx = -INFINITY;
+  for (int j = tid; j < nkeys; j += 256) {
+    const uint4* kp = reinterpret_cast<const uint4*>(kbase + (size_t)j * D);
+    uint4 raw[d / 8];
+#pragma unroll
+    for (int c = 0; c < d / 8; ++c) raw[c] = kp[c];
+    float dot = 0.f;
+#pragma unroll
+    for (int c = 0; c < d / 8; ++c) {
+      const bf16* kb = reinterpret_cast<const bf16*>(&raw[c]);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) dot += qs[c * 8 + e] * bf2f(kb[e]);
+    }
+    p[j] = dot;
+    mx = fmaxf(mx, dot);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  if (lane == 0) red[warp] = mx;
+  __syncthreads();
+  mx = red[0];
+#pragma unroll
+  for (int w = 1; w < 8; ++w) mx = fmaxf(mx, red[w]);
+  float sum = 0.f;
+  for (int j = tid; j < nkeys; j += 256) { const float e = __expf(p[j] - mx); p[j] = e; sum += e; }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  __syncthreads();
+  if (lane == 0) red[warp] = sum;
+  __syncthreads();
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) tot += red[w];
+  const float inv = 1.f / tot;
+  // P * V
+  const bf16* vbase = vc + (size_t)b * max_seq * D + h * d + lane * DPL;
+  float acc[DPL];
+#pragma unroll
+  for (int e = 0; e < DPL; ++e) acc[e] = 0.f;
+  for (int j0 = warp; j0 < nkeys; j0 += 32) {                  // four keys of this warp in flight
+    float pj[4];
+    __align__(8) bf16 vv[4][DPL];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int j = j0 + 8 * u;
+      pj[u] = j < nkeys ? p[j] : 0.f;
+      const bf16* vp = vbase + (size_t)min(j, nkeys - 1) * D;
+      if (DPL == 4) *reinterpret_cast<uint2*>(vv[u]) = *reinterpret_cast<const uint2*>(vp);
+      else if (DPL == 2) *reinterpret_cast<unsigned*>(vv[u]) = *reinterpret_cast<const unsigned*>(vp);
+      else {
+#pragma unroll
+        for (int e = 0; e < DPL; ++e) vv[u][e] = vp[e];
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+      for (int e = 0; e < DPL; ++e) acc[e] += pj[u] * bf2f(vv[u][e]);
+  }
+#pragma unroll
+  for (int e = 0; e < DPL; ++e) part[warp * d + lane * DPL + e] = acc[e];
+  __syncthreads();
+  if (tid < d) {
+    float o = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) o += part[w * d + tid];
+    out[(size_t)b * D + h * d + tid] = __float2bfloat16(o * inv);
+  }
+}
+
 __global__ void __launch_bounds__(256) embed_token_kernel(const bf16* embed, const int* tokens, int tok_stride, int tok_index,
                                                           float* x, int D, int vocab) {
   const int b = blockIdx.x;
@@ -335,8 +425,19 @@ int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens,
     a.pos = pos; a.max_seq = ctx->max_seq; a.d = g.head_dim;
     int rc = launch_gemv(ctx, a, s);
     if (rc) return rc;
-    rc = vlac_launch_decode_attention(ctx, c, l, pos, s);
-    if (rc) return rc;
+    {
+      const size_t smem = (size_t)(g.head_dim + ctx->max_seq + 8 * g.head_dim) * sizeof(float);
+      const dim3 grid(g.n_heads, B);
+      cudaError_t e;
+      switch (g.head_dim / 32) {
+        case 1: e = launch_pdl(decode_attention_kernel<1>, grid, dim3(256), smem, s, (const bf16*)ctx->q_dec, (const bf16*)kc, (const bf16*)vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads); break;
+        case 2: e = launch_pdl(decode_attention_kernel<2>, grid, dim3(256), smem, s, (const bf16*)ctx->q_dec, (const bf16*)kc, (const bf16*)vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads); break;
+        case 3: e = launch_pdl(decode_attention_kernel<3>, grid, dim3(256), smem, s, (const bf16*)ctx->q_dec, (const bf16*)kc, (const bf16*)vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads); break;
+        default: e = launch_pdl(decode_attention_kernel<4>, grid, dim3(256), smem, s, (const bf16*)ctx->q_dec, (const bf16*)kc, (const bf16*)vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads); break;
+      }
+      VLAC_CUDA_CHECK(e);
+      VLAC_LAUNCH_CHECK(ctx);
+    }
     GemvArgs o = {};
     o.x_bf16 = ctx->ao_dec; o.w0 = (const bf16*)w.wo; o.mode = GV_RESID; o.nb = B; o.K = D; o.N = D; o.x_out = ctx->x_dec; o.d = g.head_dim;
     rc = launch_gemv(ctx, o, s);
