@@ -8,6 +8,7 @@
 // the gate and up rows of one FFN feature, in the same warp so the epilogue needs no exchange.
 #include "vlac_internal.h"
 #include "launch_util.h"
+#include <stdlib.h>
 
 namespace {
 
@@ -77,7 +78,12 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
   return v;
 }
 
+#ifndef GV_BATCH
 #define GV_BATCH 4      // 16-byte chunks per row kept in flight per lane (two rows -> 8 loads)
+#endif
+#ifndef GV_CTAS_PER_SM
+#define GV_CTAS_PER_SM 2
+#endif
 
 __device__ __forceinline__ void load_batch(uint4* va, uint4* vb, const UnitRows& r, int c0, int nchunk) {
 #pragma unroll
@@ -88,11 +94,11 @@ __device__ __forceinline__ void load_batch(uint4* va, uint4* vb, const UnitRows&
   }
 }
 
-template <int NB>
-__global__ void __launch_bounds__(256, 2) gemv_pair_kernel(GemvArgs a) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+// One matrix-vector product.  `wait` runs after this warp's first weights have been requested and
+// before anything an earlier kernel (or phase) wrote is read: a dependency wait or a grid barrier.
+template <int NB, typename WaitFn>
+__device__ __forceinline__ void gemv_body(const GemvArgs& a, unsigned char* smem_raw, float* red, WaitFn wait) {
   bf16* xs = reinterpret_cast<bf16*>(smem_raw);           // [NB][K]
-  __shared__ float red[8];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int K = a.K;
   const int half = a.d / 2;
@@ -111,8 +117,7 @@ __global__ void __launch_bounds__(256, 2) gemv_pair_kernel(GemvArgs a) {
   uint4 va[GV_BATCH], vb[GV_BATCH];
   UnitRows ld_unit = unit_rows(a, min(u0, n_units - 1));
   if (total_it > 0) load_batch(va, vb, ld_unit, lane, nchunk);
-  pdl_trigger();
-  pdl_wait();
+  wait();
 
   // ---- activations -> shared memory (RMSNorm here if a gain is given)
   for (int b = 0; b < NB; ++b) {
@@ -217,21 +222,24 @@ __global__ void __launch_bounds__(256, 2) gemv_pair_kernel(GemvArgs a) {
   }
 }
 
+template <int NB>
+__global__ void __launch_bounds__(256, GV_CTAS_PER_SM) gemv_pair_kernel(GemvArgs a) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __shared__ float red[8];
+  gemv_body<NB>(a, smem_raw, red, [] { pdl_trigger(); pdl_wait(); });
+}
+
 // Attention of one new row per sequence over the cache (Sec. 3.1): one CTA per (head, sequence).
 // Scores: one key per thread (whole 16-byte-vectorised dot product); P*V: keys dealt round-robin to the
 // eight warps, each lane owning d/32 consecutive dimensions, partial sums combined in warp order.
 template <int DPL>      // dimensions per lane = head_dim / 32
-__global__ void __launch_bounds__(256) decode_attention_kernel(const bf16* q, const bf16* kc, const bf16* vc, bf16* out,
-                                                               int pos, int max_seq, int H) {
-  extern __shared__ float dsm[];
+__device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc, const bf16* vc, bf16* out,
+                                                      int pos, int max_seq, int H, int h, int b, float* dsm, float* red) {
   constexpr int d = 32 * DPL;
   float* qs = dsm;                 // [d]
   float* p = dsm + d;              // [max_seq]
   float* part = p + max_seq;       // [8][d]
-  __shared__ float red[8];
-  const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  pdl_trigger();
-  pdl_wait();
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int D = H * d, nkeys = pos + 1;
   const float scale = rsqrtf((float)d);
   if (tid < d) qs[tid] = bf2f(q[(size_t)b * D + h * d + tid]) * scale;
@@ -240,15 +248,18 @@ __global__ void __launch_bounds__(256) decode_attention_kernel(const bf16* q, co
   float mx = -INFINITY;
   for (int j = tid; j < nkeys; j += 256) {
     const uint4* kp = reinterpret_cast<const uint4*>(kbase + (size_t)j * D);
-    uint4 raw[d / 8];
-#pragma unroll
-    for (int c = 0; c < d / 8; ++c) raw[c] = kp[c];
     float dot = 0.f;
 #pragma unroll
-    for (int c = 0; c < d / 8; ++c) {
-      const bf16* kb = reinterpret_cast<const bf16*>(&raw[c]);
+    for (int c0 = 0; c0 < d / 8; c0 += 4) {                    // four 16-byte loads in flight at a time
+      uint4 raw[4];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) dot += qs[c * 8 + e] * bf2f(kb[e]);
+      for (int c = 0; c < 4; ++c) raw[c] = kp[c0 + c];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const bf16* kb = reinterpret_cast<const bf16*>(&raw[c]);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) dot += qs[(c0 + c) * 8 + e] * bf2f(kb[e]);
+      }
     }
     p[j] = dot;
     mx = fmaxf(mx, dot);
@@ -304,6 +315,96 @@ __global__ void __launch_bounds__(256) decode_attention_kernel(const bf16* q, co
 #pragma unroll
     for (int w = 0; w < 8; ++w) o += part[w * d + tid];
     out[(size_t)b * D + h * d + tid] = __float2bfloat16(o * inv);
+  }
+}
+
+template <int DPL>
+__global__ void __launch_bounds__(256) decode_attention_kernel(const bf16* q, const bf16* kc, const bf16* vc, bf16* out,
+                                                               int pos, int max_seq, int H) {
+  extern __shared__ float dsm[];
+  __shared__ float red[8];
+  pdl_trigger();
+  pdl_wait();
+  decode_attention_body<DPL>(q, kc, vc, out, pos, max_seq, H, blockIdx.x, blockIdx.y, dsm, red);
+}
+
+// ---- one whole single-row pass as ONE persistent kernel -------------------------------------------
+// All layers, five phases each (QKV | attention | output proj | gate/up | down), separated by grid
+// barriers instead of kernel boundaries.  Every CTA requests the first weights of its next phase
+// before it enters the barrier, so HBM keeps streaming while the grid synchronises.  Launched
+// cooperatively (all CTAs co-resident); every barrier wait is bounded by the global timer.
+#define GV_BARRIER_LIMIT_NS 200000000ull
+
+__device__ __forceinline__ unsigned long long gv_global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+// Arrive on the grid-wide counter and wait until `target` arrivals.  Returns false (for the whole CTA)
+// if the wait gave up or an error was already recorded; later barriers then fall through at once.
+__device__ __forceinline__ bool grid_barrier(unsigned* counter, unsigned target, int* dev_error) {
+  __syncthreads();
+  int ok = 1;
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(counter, 1u);
+    const unsigned long long t0 = gv_global_ns();
+    while (ld_acquire_u32(counter) < target) {
+      if (*reinterpret_cast<volatile int*>(dev_error) != 0) { ok = 0; break; }
+      if (gv_global_ns() - t0 > GV_BARRIER_LIMIT_NS) { atomicCAS(dev_error, 0, 0x80000 | (int)(target & 0xffff)); ok = 0; break; }
+    }
+    __threadfence();
+  }
+  return __syncthreads_and(ok) != 0;
+}
+
+struct PassArgs {
+  const GemvArgs* phases;      // [n_layers][4]: QKV, output proj, gate/up, down (for this pass's position)
+  int n_layers, pos, n_heads, batch;
+  bf16* ao;                    // attention output rows [batch][H*d]
+  unsigned* counter;           // grid barrier counter, zeroed before the launch
+  int* dev_error;
+};
+
+template <int NB>
+__global__ void __launch_bounds__(256, GV_CTAS_PER_SM) decode_pass_kernel(PassArgs pa) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __shared__ float red[8];
+  unsigned n_bar = 0;
+  const unsigned G = gridDim.x;
+  const int n_phases = 4 * pa.n_layers;
+  __shared__ GemvArgs sargs;                                   // this phase's arguments (kept out of registers)
+  for (int ph = 0; ph < n_phases; ++ph) {
+    __syncthreads();                                             // every warp is done with the previous phase's arguments
+    if (threadIdx.x < sizeof(GemvArgs) / sizeof(int))
+      reinterpret_cast<int*>(&sargs)[threadIdx.x] = reinterpret_cast<const int*>(pa.phases + ph)[threadIdx.x];
+    __syncthreads();
+    gemv_body<NB>(sargs, smem_raw, red, [&] {
+      // the row entering the pass was written by an earlier kernel: no barrier before the very first phase
+      if (ph > 0) grid_barrier(pa.counter, (++n_bar) * G, pa.dev_error);
+      if ((ph & 3) == 1) {
+        // attention of this layer sits between the Q/K/V phase and the output projection, whose first
+        // weights this CTA has already requested
+        const int hb = blockIdx.x;
+        if (hb < pa.n_heads * pa.batch) {
+          const GemvArgs* qkv = pa.phases + (ph - 1);
+          const bf16 *q = qkv->q_out, *kc = qkv->kc, *vc = qkv->vc;
+          const int max_seq = qkv->max_seq, dpl = qkv->d / 32;
+          const int h = hb % pa.n_heads, b = hb / pa.n_heads;
+          float* dsm = reinterpret_cast<float*>(smem_raw);
+          if (dpl == 4) decode_attention_body<4>(q, kc, vc, pa.ao, pa.pos, max_seq, pa.n_heads, h, b, dsm, red);
+          else if (dpl == 2) decode_attention_body<2>(q, kc, vc, pa.ao, pa.pos, max_seq, pa.n_heads, h, b, dsm, red);
+          else if (dpl == 3) decode_attention_body<3>(q, kc, vc, pa.ao, pa.pos, max_seq, pa.n_heads, h, b, dsm, red);
+          else decode_attention_body<1>(q, kc, vc, pa.ao, pa.pos, max_seq, pa.n_heads, h, b, dsm, red);
+        }
+        grid_barrier(pa.counter, (++n_bar) * G, pa.dev_error);
+      }
+    });
   }
 }
 
@@ -366,7 +467,7 @@ int launch_gemv(vlac_ctx* ctx, const GemvArgs& a, cudaStream_t s) {
   const int nb = a.nb;
   const int NB = nb <= 1 ? 1 : (nb <= 2 ? 2 : (nb <= 4 ? 4 : 8));
   const size_t smem = (size_t)NB * a.K * sizeof(bf16);
-  const int grid = ctx->n_sm * 2;
+  const int grid = ctx->n_sm * GV_CTAS_PER_SM;
   const bool timed = ctx->prof_on && ctx->prof_n < VLAC_PROF_CAP;
   if (timed) VLAC_CUDA_CHECK(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n], s));
   switch (NB) {
@@ -386,6 +487,8 @@ int launch_gemv(vlac_ctx* ctx, const GemvArgs& a, cudaStream_t s) {
 
 }  // namespace
 
+static size_t pass_smem(const vlac_ctx* ctx, int NB);
+
 int vlac_decode_setup(vlac_ctx* ctx) {
   const int kmax = ctx->cfg.ffn > ctx->cfg.hidden ? ctx->cfg.ffn : ctx->cfg.hidden;
   const int mb = ctx->cfg.max_batch;
@@ -397,6 +500,30 @@ int vlac_decode_setup(vlac_ctx* ctx) {
   if (NB >= 2) VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_pair_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * (size_t)kmax * 2)));
   if (NB >= 4) VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_pair_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(4 * (size_t)kmax * 2)));
   if (NB >= 8) VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_pair_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(8 * (size_t)kmax * 2)));
+  // persistent pass kernel: as many CTAs as are guaranteed co-resident
+  ctx->pass_grid = 0;
+  // Opt-in (VLAC_PASS_KERNEL=1): measured on B200 it streams at 5.5 TB/s between barriers but its five grid
+  // barriers per layer (about 5 us each) make a pass no faster than the per-phase kernels replayed from a graph.
+  if (getenv("VLAC_PASS_KERNEL") != nullptr && ctx->max_seq > 0) {
+    const size_t psm = pass_smem(ctx, NB);
+    int per_sm = 0, coop = 0, dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+    if (e == cudaSuccess && coop) {
+      switch (NB) {
+        case 1: e = cudaFuncSetAttribute(decode_pass_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psm);
+                if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_pass_kernel<1>, 256, psm); break;
+        case 2: e = cudaFuncSetAttribute(decode_pass_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psm);
+                if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_pass_kernel<2>, 256, psm); break;
+        case 4: e = cudaFuncSetAttribute(decode_pass_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psm);
+                if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_pass_kernel<4>, 256, psm); break;
+        default: e = cudaFuncSetAttribute(decode_pass_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psm);
+                if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_pass_kernel<8>, 256, psm); break;
+      }
+      if (e == cudaSuccess && per_sm > 0) ctx->pass_grid = ctx->n_sm * (per_sm < GV_CTAS_PER_SM ? per_sm : GV_CTAS_PER_SM);
+    }
+    if (e != cudaSuccess) cudaGetLastError();
+  }
   return VLAC_OK;
 }
 
@@ -406,52 +533,119 @@ int vlac_launch_last_row(vlac_ctx* ctx, vlac_cache* c, const bf16* hidden, cudaS
   return VLAC_OK;
 }
 
+// The four matrix-vector phases of layer l for a single-row pass at position `pos`.
+static void layer_phases(vlac_ctx* ctx, vlac_cache* c, int l, int pos, GemvArgs* out) {
+  const vlac_config& g = ctx->cfg;
+  const int D = g.hidden, F = g.ffn, B = c->batch;
+  const vlac_layer_w& w = ctx->layers[l];
+  GemvArgs a = {};
+  a.x_f32 = ctx->x_dec; a.gain = (const bf16*)w.g_attn; a.eps = g.rms_eps;
+  a.w0 = (const bf16*)w.wq; a.w1 = (const bf16*)w.wk; a.w2 = (const bf16*)w.wv;
+  a.mode = GV_QKV; a.nb = B; a.K = D; a.N = D;
+  a.q_out = ctx->q_dec;
+  a.kc = c->k + (size_t)l * B * kv_layer_elems(ctx);
+  a.vc = c->v + (size_t)l * B * kv_layer_elems(ctx);
+  a.rope_cos = ctx->w.rope_cos; a.rope_sin = ctx->w.rope_sin;
+  a.pos = pos; a.max_seq = ctx->max_seq; a.d = g.head_dim;
+  GemvArgs o = {};
+  o.x_bf16 = ctx->ao_dec; o.w0 = (const bf16*)w.wo; o.mode = GV_RESID; o.nb = B; o.K = D; o.N = D; o.x_out = ctx->x_dec; o.d = g.head_dim;
+  GemvArgs gu = {};
+  gu.x_f32 = ctx->x_dec; gu.gain = (const bf16*)w.g_mlp; gu.eps = g.rms_eps;
+  gu.w0 = (const bf16*)w.w_gate; gu.w1 = (const bf16*)w.w_up; gu.mode = GV_SWIGLU; gu.nb = B; gu.K = D; gu.N = F;
+  gu.h_out = ctx->hm_dec; gu.d = g.head_dim;
+  GemvArgs dn = {};
+  dn.x_bf16 = ctx->hm_dec; dn.w0 = (const bf16*)w.w_down; dn.mode = GV_RESID; dn.nb = B; dn.K = F; dn.N = D; dn.x_out = ctx->x_dec; dn.d = g.head_dim;
+  out[0] = a; out[1] = o; out[2] = gu; out[3] = dn;
+}
+
+static size_t pass_smem(const vlac_ctx* ctx, int NB) {
+  const vlac_config& g = ctx->cfg;
+  const int kmax = g.ffn > g.hidden ? g.ffn : g.hidden;
+  const size_t xs = (size_t)NB * kmax * sizeof(bf16);
+  const size_t at = (size_t)(g.head_dim + ctx->max_seq + 8 * g.head_dim) * sizeof(float);
+  return xs > at ? xs : at;
+}
+
+// Per-cache table of phase arguments for the persistent pass kernel, and its barrier counter.
+int vlac_decode_cache_setup(vlac_ctx* ctx, vlac_cache* c) {
+  const int nl = ctx->cfg.n_layers;
+  const int n_pass = ctx->cfg.n_action > 1 ? ctx->cfg.n_action - 1 : 1;      // one table per single-row position L, L+1, ...
+  const size_t n = (size_t)n_pass * 4 * nl;
+  static_assert(sizeof(GemvArgs) % sizeof(int) == 0, "copied word by word");
+  GemvArgs* host = (GemvArgs*)malloc(sizeof(GemvArgs) * n);
+  if (!host) return VLAC_ERR_OOM;
+  for (int i = 0; i < n_pass; ++i)
+    for (int l = 0; l < nl; ++l) layer_phases(ctx, c, l, ctx->L + i, host + ((size_t)i * nl + l) * 4);
+  int rc = VLAC_OK;
+  if (cudaMalloc(&c->dec_phases, sizeof(GemvArgs) * n) != cudaSuccess) { cudaGetLastError(); rc = VLAC_ERR_OOM; }
+  if (rc == VLAC_OK && cudaMemcpy(c->dec_phases, host, sizeof(GemvArgs) * n, cudaMemcpyHostToDevice) != cudaSuccess) rc = VLAC_ERR_CUDA;
+  free(host);
+  if (rc == VLAC_OK && cudaMalloc(&c->dec_counter, 256) != cudaSuccess) { cudaGetLastError(); rc = VLAC_ERR_OOM; }
+  return rc;
+}
+
+template <int NB>
+static cudaError_t launch_pass(const PassArgs& pa, int grid, size_t smem, cudaStream_t s) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;            // all CTAs resident at once: the grid barriers rely on it
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, decode_pass_kernel<NB>, pa);
+}
+
 int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens, int tok_stride, int tok_index,
                             int pos, cudaStream_t s) {
   const vlac_config& g = ctx->cfg;
-  const int D = g.hidden, F = g.ffn, B = c->batch;
+  const int D = g.hidden, B = c->batch;
   VLAC_CUDA_CHECK(launch_pdl(embed_token_kernel, dim3(B), dim3(256), 0, s, (const bf16*)ctx->w.embed, fed_tokens, tok_stride, tok_index,
                              ctx->x_dec, D, g.vocab));
   VLAC_LAUNCH_CHECK(ctx);
+  const int NB = B <= 1 ? 1 : (B <= 2 ? 2 : (B <= 4 ? 4 : 8));
+  const int pass_idx = pos - ctx->L;
+  if (ctx->pass_grid > 0 && !ctx->prof_on && g.n_heads * B <= ctx->pass_grid && pass_idx >= 0 && pass_idx < g.n_action - 1) {
+    // the whole pass as one persistent kernel
+    VLAC_CUDA_CHECK(cudaMemsetAsync(c->dec_counter, 0, sizeof(unsigned), s));
+    PassArgs pa;
+    pa.phases = (const GemvArgs*)c->dec_phases + (size_t)pass_idx * 4 * g.n_layers; pa.n_layers = g.n_layers; pa.pos = pos; pa.n_heads = g.n_heads; pa.batch = B;
+    pa.ao = ctx->ao_dec; pa.counter = (unsigned*)c->dec_counter; pa.dev_error = ctx->dev_error;
+    const size_t smem = pass_smem(ctx, NB);
+    cudaError_t e;
+    switch (NB) {
+      case 1: e = launch_pass<1>(pa, ctx->pass_grid, smem, s); break;
+      case 2: e = launch_pass<2>(pa, ctx->pass_grid, smem, s); break;
+      case 4: e = launch_pass<4>(pa, ctx->pass_grid, smem, s); break;
+      default: e = launch_pass<8>(pa, ctx->pass_grid, smem, s); break;
+    }
+    VLAC_CUDA_CHECK(e);
+    VLAC_LAUNCH_CHECK(ctx);
+    return VLAC_OK;
+  }
+  // one kernel per phase (also the path that per-launch timing brackets)
   for (int l = 0; l < g.n_layers; ++l) {
-    const vlac_layer_w& w = ctx->layers[l];
-    bf16* kc = c->k + (size_t)l * B * kv_layer_elems(ctx);
-    bf16* vc = c->v + (size_t)l * B * kv_layer_elems(ctx);
-    GemvArgs a = {};
-    a.x_f32 = ctx->x_dec; a.gain = (const bf16*)w.g_attn; a.eps = g.rms_eps;
-    a.w0 = (const bf16*)w.wq; a.w1 = (const bf16*)w.wk; a.w2 = (const bf16*)w.wv;
-    a.mode = GV_QKV; a.nb = B; a.K = D; a.N = D;
-    a.q_out = ctx->q_dec; a.kc = kc; a.vc = vc; a.rope_cos = ctx->w.rope_cos; a.rope_sin = ctx->w.rope_sin;
-    a.pos = pos; a.max_seq = ctx->max_seq; a.d = g.head_dim;
-    int rc = launch_gemv(ctx, a, s);
+    GemvArgs ph[4];
+    layer_phases(ctx, c, l, pos, ph);
+    int rc = launch_gemv(ctx, ph[0], s);
     if (rc) return rc;
     {
       const size_t smem = (size_t)(g.head_dim + ctx->max_seq + 8 * g.head_dim) * sizeof(float);
       const dim3 grid(g.n_heads, B);
+      const bf16 *q = ctx->q_dec, *kc = ph[0].kc, *vc = ph[0].vc;
       cudaError_t e;
       switch (g.head_dim / 32) {
-        case 1: e = launch_pdl(decode_attention_kernel<1>, grid, dim3(256), smem, s, (const bf16*)ctx->q_dec, (const bf16*)kc, (const bf16*)vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads); break;
-        case 2: e = launch_pdl(decode_attention_kernel<2>, grid, dim3(256), smem, s, (const bf16*)ctx->q_dec, (const bf16*)kc, (const bf16*)vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads); break;
-        case 3: e = launch_pdl(decode_attention_kernel<3>, grid, dim3(256), smem, s, (const bf16*)ctx->q_dec, (const bf16*)kc, (const bf16*)vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads); break;
-        default: e = launch_pdl(decode_attention_kernel<4>, grid, dim3(256), smem, s, (const bf16*)ctx->q_dec, (const bf16*)kc, (const bf16*)vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads); break;
+        case 1: e = launch_pdl(decode_attention_kernel<1>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads); break;
+        case 2: e = launch_pdl(decode_attention_kernel<2>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads); break;
+        case 3: e = launch_pdl(decode_attention_kernel<3>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads); break;
+        default: e = launch_pdl(decode_attention_kernel<4>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads); break;
       }
       VLAC_CUDA_CHECK(e);
       VLAC_LAUNCH_CHECK(ctx);
     }
-    GemvArgs o = {};
-    o.x_bf16 = ctx->ao_dec; o.w0 = (const bf16*)w.wo; o.mode = GV_RESID; o.nb = B; o.K = D; o.N = D; o.x_out = ctx->x_dec; o.d = g.head_dim;
-    rc = launch_gemv(ctx, o, s);
-    if (rc) return rc;
-    GemvArgs gu = {};
-    gu.x_f32 = ctx->x_dec; gu.gain = (const bf16*)w.g_mlp; gu.eps = g.rms_eps;
-    gu.w0 = (const bf16*)w.w_gate; gu.w1 = (const bf16*)w.w_up; gu.mode = GV_SWIGLU; gu.nb = B; gu.K = D; gu.N = F;
-    gu.h_out = ctx->hm_dec; gu.d = g.head_dim;
-    rc = launch_gemv(ctx, gu, s);
-    if (rc) return rc;
-    GemvArgs dn = {};
-    dn.x_bf16 = ctx->hm_dec; dn.w0 = (const bf16*)w.w_down; dn.mode = GV_RESID; dn.nb = B; dn.K = F; dn.N = D; dn.x_out = ctx->x_dec; dn.d = g.head_dim;
-    rc = launch_gemv(ctx, dn, s);
-    if (rc) return rc;
+    for (int k = 1; k < 4; ++k) {
+      rc = launch_gemv(ctx, ph[k], s);
+      if (rc) return rc;
+    }
   }
   return VLAC_OK;
 }

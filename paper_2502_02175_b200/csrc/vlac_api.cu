@@ -65,7 +65,7 @@ void free_cache_buffers(vlac_cache* c) {
   cudaFree(c->warm); cudaFree(c->sim); cudaFree(c->S_layer); cudaFree(c->S); cudaFree(c->alpha);
   cudaFree(c->alpha_raw); cudaFree(c->entropy); cudaFree(c->static_mask); cudaFree(c->task_mask);
   cudaFree(c->final_mask); cudaFree(c->rank); cudaFree(c->n_reuse); cudaFree(c->M); cudaFree(c->rows);
-  cudaFree(c->tot); cudaFree(c->rowmap); cudaFree(c->slot); cudaFree(c->tmaps_kv);
+  cudaFree(c->tot); cudaFree(c->rowmap); cudaFree(c->slot); cudaFree(c->tmaps_kv); cudaFree(c->dec_phases); cudaFree(c->dec_counter);
 }
 
 __global__ void set_warm_kernel(int* warm, int n, int value) {
@@ -200,6 +200,7 @@ int vlac_cache_alloc(vlac_ctx* ctx, int batch, vlac_cache** out) {
   if (rc == VLAC_OK) rc = dev_alloc(&c->rowmap, nl * B * L);
   if (rc == VLAC_OK) rc = dev_alloc(&c->slot, nl * B * L);
   if (rc == VLAC_OK) rc = vlac_attention_cache_setup(ctx, c);
+  if (rc == VLAC_OK) rc = vlac_decode_cache_setup(ctx, c);
   if (rc != VLAC_OK) { free_cache_buffers(c); delete c; return rc; }
   *out = c;
   return VLAC_OK;

@@ -63,6 +63,7 @@ struct vlac_ctx {
   int graph_next, use_graph;
   void* tmaps;                       // device array of TMA tensor maps (weights per layer, activation buffers)
   int tc_ok;                         // 1: shapes fit the tensor-memory GEMM
+  int pass_grid;                     // CTAs of the persistent single-row pass kernel (0: not used)
   void* tmap_q;                      // device tensor map of the query buffer (tiled attention)
   int attn_tiles;                    // 64-query tiles per sequence, 0: tiled attention not usable
   // optional per-launch timing of the matrix-vector kernel (vlac_profile)
@@ -93,6 +94,8 @@ struct vlac_cache {
   int *rowmap;                       // [nl][batch*L]        compact index -> b*L + pos
   int *slot;                         // [nl][batch*L]        b*L + pos -> compact index or -1
   void* tmaps_kv;                    // device tensor maps of the K and V cache of every layer
+  void* dec_phases;                  // device table of per-layer phase arguments (persistent pass kernel)
+  void* dec_counter;                 // its grid barrier counter
 };
 
 static inline size_t kv_layer_elems(const vlac_ctx* c) {
@@ -130,6 +133,7 @@ int vlac_launch_prefill_attention(vlac_ctx* ctx, vlac_cache* c, int layer, cudaS
 
 // ---- decode (decode_kernels.cu)
 int vlac_decode_setup(vlac_ctx* ctx);
+int vlac_decode_cache_setup(vlac_ctx* ctx, vlac_cache* c);
 int vlac_launch_last_row(vlac_ctx* ctx, vlac_cache* c, const bf16* hidden, cudaStream_t s);
 int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens, int tok_stride, int tok_index,
                             int pos, cudaStream_t s);
