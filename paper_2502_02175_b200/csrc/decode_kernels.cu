@@ -97,7 +97,7 @@ __device__ __forceinline__ void load_batch(uint4* va, uint4* vb, const UnitRows&
 // One matrix-vector product.  `wait` runs after this warp's first weights have been requested and
 // before anything an earlier kernel (or phase) wrote is read: a dependency wait or a grid barrier.
 template <int NB, typename WaitFn>
-__device__ __forceinline__ void gemv_body(const GemvArgs& a, unsigned char* smem_raw, float* red, WaitFn wait) {
+__device__ __forceinline__ void gemv_body(const GemvArgs& a, unsigned char* smem_raw, float* red, int* next_unit, WaitFn wait) {
   bf16* xs = reinterpret_cast<bf16*>(smem_raw);           // [NB][K]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int K = a.K;
@@ -106,17 +106,19 @@ __device__ __forceinline__ void gemv_body(const GemvArgs& a, unsigned char* smem
   if (a.mode == GV_QKV) n_units = 3 * (a.N / 2);
   else if (a.mode == GV_SWIGLU) n_units = a.N;
   else n_units = (a.N + 1) / 2;
-  const int total_warps = gridDim.x * 8;
   const int nchunk = K / 8;
   const int bpu = (nchunk + 32 * GV_BATCH - 1) / (32 * GV_BATCH);      // load batches per unit
-  const int u0 = blockIdx.x * 8 + warp;
-  const int n_my = u0 < n_units ? (n_units - u0 + total_warps - 1) / total_warps : 0;
-  const int total_it = n_my * bpu;
+  // This CTA owns a contiguous, balanced range of units.  Each warp starts on the unit of its own index
+  // and then takes the next free one from a shared ticket, so the CTA's warps finish together.
+  const int u_begin = (int)(((long long)n_units * blockIdx.x) / gridDim.x);
+  const int n_local = (int)(((long long)n_units * (blockIdx.x + 1)) / gridDim.x) - u_begin;
+  if (tid == 0) *next_unit = 8;                             // read only after the barriers of the prologue below
 
   // ---- first weights of this warp are requested before anything else: they depend on no earlier kernel
   uint4 va[GV_BATCH], vb[GV_BATCH];
-  UnitRows ld_unit = unit_rows(a, min(u0, n_units - 1));
-  if (total_it > 0) load_batch(va, vb, ld_unit, lane, nchunk);
+  int u_ld = warp < n_local ? warp : -1;                    // unit (local index) whose batch is in va, vb
+  UnitRows ld_unit = unit_rows(a, u_begin + max(u_ld, 0));
+  if (u_ld >= 0) load_batch(va, vb, ld_unit, lane, nchunk);
   wait();
 
   // ---- activations -> shared memory (RMSNorm here if a gain is given)
@@ -150,17 +152,23 @@ __device__ __forceinline__ void gemv_body(const GemvArgs& a, unsigned char* smem
 #pragma unroll
   for (int b = 0; b < NB; ++b) accA[b] = accB[b] = 0.f;
   UnitRows cu = ld_unit;                                    // unit being accumulated
-  int u_ld = u0, bi_ld = 0;                                 // unit / batch index of the loads in va, vb
-  for (int it = 0; it < total_it; ++it) {
+  int bi_ld = 0;                                            // batch index of the loads in va, vb
+  while (u_ld >= 0) {
     const int c0 = lane + 32 * GV_BATCH * bi_ld;
     const bool last_of_unit = (bi_ld == bpu - 1);
     // request the next batch before computing on this one
     uint4 na[GV_BATCH], nb2[GV_BATCH];
     int u_nx = u_ld, bi_nx = bi_ld + 1;
-    if (last_of_unit) { u_nx = u_ld + total_warps; bi_nx = 0; }
-    const bool has_next = it + 1 < total_it;
+    if (last_of_unit) {
+      int t = 0;
+      if (lane == 0) t = atomicAdd(next_unit, 1);
+      t = __shfl_sync(0xffffffffu, t, 0);
+      u_nx = t < n_local ? t : -1;
+      bi_nx = 0;
+    }
+    const bool has_next = u_nx >= 0;
     if (has_next) {
-      if (last_of_unit) ld_unit = unit_rows(a, u_nx);
+      if (last_of_unit) ld_unit = unit_rows(a, u_begin + u_nx);
       load_batch(na, nb2, ld_unit, lane + 32 * GV_BATCH * bi_nx, nchunk);
     }
 #pragma unroll
@@ -226,7 +234,8 @@ template <int NB>
 __global__ void __launch_bounds__(256, GV_CTAS_PER_SM) gemv_pair_kernel(GemvArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __shared__ float red[8];
-  gemv_body<NB>(a, smem_raw, red, [] { pdl_trigger(); pdl_wait(); });
+  __shared__ int next_unit;
+  gemv_body<NB>(a, smem_raw, red, &next_unit, [] { pdl_trigger(); pdl_wait(); });
 }
 
 // Attention of one new row per sequence over the cache (Sec. 3.1): one CTA per (head, sequence).
@@ -378,13 +387,14 @@ __global__ void __launch_bounds__(256, GV_CTAS_PER_SM) decode_pass_kernel(PassAr
   unsigned n_bar = 0;
   const unsigned G = gridDim.x;
   const int n_phases = 4 * pa.n_layers;
+  __shared__ int next_unit;
   __shared__ GemvArgs sargs;                                   // this phase's arguments (kept out of registers)
   for (int ph = 0; ph < n_phases; ++ph) {
     __syncthreads();                                             // every warp is done with the previous phase's arguments
     if (threadIdx.x < sizeof(GemvArgs) / sizeof(int))
       reinterpret_cast<int*>(&sargs)[threadIdx.x] = reinterpret_cast<const int*>(pa.phases + ph)[threadIdx.x];
     __syncthreads();
-    gemv_body<NB>(sargs, smem_raw, red, [&] {
+    gemv_body<NB>(sargs, smem_raw, red, &next_unit, [&] {
       // the row entering the pass was written by an earlier kernel: no barrier before the very first phase
       if (ph > 0) grid_barrier(pa.counter, (++n_bar) * G, pa.dev_error);
       if ((ph & 3) == 1) {
