@@ -53,6 +53,10 @@ struct TcArgs {
   bf16 *q_out, *kc, *vc;          // QKV: [T][N], caches [B][max_seq][N]
   float* part; size_t split_stride;   // PARTIAL: [split][T][N]
   bf16* h_out;                    // SWIGLU: [T][N]
+  // SWIGLU tail: tiles beyond the last full wave of CTAs are split along K so that they finish together;
+  // their raw gate/up sums go to tail_part[split][T][tail_ld] and a small kernel finishes them
+  int full_tiles, tail_splits, tail_ld;
+  float* tail_part; size_t tail_stride;
   int* dev_error;
 };
 
@@ -133,7 +137,12 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(TcArgs a) {
   // the ring must start on a 1024-byte boundary (swizzle atoms); dynamic smem is over-allocated by 1 KB
   unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(ring_raw) + 1023) & ~(uintptr_t)1023);
 
-  const int tile = blockIdx.x, split = blockIdx.y;
+  int tile = blockIdx.x, split = blockIdx.y, splits = a.n_splits;
+  bool tail = false;                                            // a K-split SWIGLU tile: epilogue stores raw sums
+  if (a.mode == TG_SWIGLU && a.tail_splits > 1 && tile >= a.full_tiles) {
+    const int u = tile - a.full_tiles;
+    tile = a.full_tiles + u / a.tail_splits; split = u % a.tail_splits; splits = a.tail_splits; tail = true;
+  }
   if (tid == 0) {
     for (int s = 0; s < TG_MAX_STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
     mbar_init(&acc_bar, 1);
@@ -150,8 +159,8 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(TcArgs a) {
   int n_stages = TG_SMEM_RING / stage_bytes;
   if (n_stages > TG_MAX_STAGES) n_stages = TG_MAX_STAGES;
   const int kb_total = (a.K + TG_BK - 1) / TG_BK;
-  const int kb0 = (int)(((long long)kb_total * split) / a.n_splits);
-  const int kb1 = (int)(((long long)kb_total * (split + 1)) / a.n_splits);
+  const int kb0 = (int)(((long long)kb_total * split) / splits);
+  const int kb1 = (int)(((long long)kb_total * (split + 1)) / splits);
   const int n_kb = (tokens > 0) ? kb1 - kb0 : 0;
   const int n0 = min(((tokens + 15) / 16) * 16, 256);           // columns of the first MMA
   const int n1 = tokens > 256 ? ((tokens - 256 + 15) / 16) * 16 : 0;
@@ -230,7 +239,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(TcArgs a) {
     if (a.mode == TG_SWIGLU) { n = row_base + (r & 63); first = r < 64; pq = q ^ 2; }
     else { n = row_base + r; first = ((r / half) & 1) == 0; pq = q ^ (half >> 5); }
     const bool n_ok = n < a.N;
-    const bool exchange = a.mode == TG_SWIGLU || (a.mode == TG_QKV && mat < 2);
+    const bool exchange = (a.mode == TG_SWIGLU && !tail) || (a.mode == TG_QKV && mat < 2);
     const int j = (n % a.d) % half;
     const size_t N = (size_t)a.N;
     int chunk = 0;
@@ -250,7 +259,13 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(TcArgs a) {
         for (int c = 0; c < 16; ++c) pv[c] = buf[pq][c][lane];
       }
       const bool live = ok && n_ok;                               // no early exit: the warp shuffles below need every lane
-      if (a.mode == TG_PARTIAL) {
+      if (tail) {
+        if (!ok) continue;
+        float* dst = a.tail_part + (size_t)split * a.tail_stride + (size_t)(tile - a.full_tiles) * 128 + r;
+#pragma unroll
+        for (int c = 0; c < 16; ++c)
+          if (c0 + c < tokens) dst[(size_t)(c0 + c) * a.tail_ld] = v[c];
+      } else if (a.mode == TG_PARTIAL) {
         if (!live) continue;
         float* dst = a.part + (size_t)split * a.split_stride + n;
 #pragma unroll
@@ -295,6 +310,26 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(TcArgs a) {
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+  }
+}
+
+// finishes the K-split SWIGLU tiles: sums the splits in order, silu(gate) * up
+__global__ void __launch_bounds__(256) swiglu_tail_kernel(const float* part, size_t stride, int ld, int splits, const int* tot,
+                                                          int full_tiles, int rem_tiles, int F, bf16* h_out) {
+  const int t = blockIdx.x;
+  pdl_trigger();
+  pdl_wait();
+  if (t >= *tot) return;
+  for (int i = threadIdx.x; i < rem_tiles * 64; i += blockDim.x) {
+    const int tl = i >> 6, fr = i & 63;
+    const int f = (full_tiles + tl) * 64 + fr;
+    if (f >= F) continue;
+    float g = 0.f, u = 0.f;
+    for (int s = 0; s < splits; ++s) {
+      const float* row = part + (size_t)s * stride + (size_t)t * ld + tl * 128;
+      g += row[fr]; u += row[64 + fr];
+    }
+    h_out[(size_t)t * F + f] = __float2bfloat16(__fdividef(g, 1.f + __expf(-g)) * u);
   }
 }
 
@@ -431,5 +466,24 @@ int vlac_tc_gateup(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s) {
   a.tm_a[0] = tm + TM_GATE; a.tm_a[1] = tm + TM_UP; a.tm_b = act + TM_XN;
   a.K = g.hidden; a.N = g.ffn; a.mode = TG_SWIGLU;
   a.h_out = ctx->hm;
-  return launch_tc(ctx, a, (g.ffn + 63) / 64, s);
+  const int tiles = (g.ffn + 63) / 64;
+  // tiles beyond the last full wave: split along K so that the second, short wave fills every SM
+  int full = tiles >= ctx->n_sm ? (tiles / ctx->n_sm) * ctx->n_sm : tiles;
+  int rem = tiles - full, splits = 1;
+  if (rem > 0) {
+    splits = ctx->n_sm / rem;
+    const int kb_total = (a.K + TG_BK - 1) / TG_BK;
+    if (splits > kb_total) splits = kb_total;
+    if (splits > 8) splits = 8;
+    const size_t wide = (size_t)(3 * g.hidden > 2 * g.ffn ? 3 * g.hidden : 2 * g.ffn);     // floats per row of ctx->scratch
+    if (splits < 2 || (size_t)splits * rem * 128 > wide) { splits = 1; full = tiles; rem = 0; }
+  }
+  a.full_tiles = full; a.tail_splits = splits; a.tail_ld = rem * 128;
+  a.tail_part = ctx->scratch; a.tail_stride = (size_t)ctx->rows_max * rem * 128;
+  int rc = launch_tc(ctx, a, full + rem * splits, s);
+  if (rc || rem == 0) return rc;
+  VLAC_CUDA_CHECK(launch_pdl(swiglu_tail_kernel, dim3(ctx->rows_max), dim3(256), 0, s, (const float*)a.tail_part, a.tail_stride, a.tail_ld,
+                             splits, a.tot, full, rem, g.ffn, ctx->hm));
+  VLAC_LAUNCH_CHECK(ctx);
+  return VLAC_OK;
 }
