@@ -42,6 +42,26 @@ def widen_bf16(bits: np.ndarray) -> np.ndarray:
     return (b.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
 
 
+# Optional memo of widened matrices (format conversion only, no arithmetic).  Off by default; tests that
+# call the same layer many times switch it on to avoid re-widening hundreds of MB per call.
+WIDEN_CACHE_MAX = 0
+_widen_cache: Dict[int, tuple] = {}
+
+
+def _widen_cached(bits: np.ndarray) -> np.ndarray:
+    if WIDEN_CACHE_MAX <= 0:
+        return widen_bf16(bits)
+    key = id(bits)
+    hit = _widen_cache.get(key)
+    if hit is not None and hit[0] is bits:
+        return hit[1]
+    if len(_widen_cache) >= WIDEN_CACHE_MAX:
+        _widen_cache.clear()
+    wide = widen_bf16(bits)
+    _widen_cache[key] = (bits, wide)
+    return wide
+
+
 @dataclass
 class SelectParams:
     """Hyper-parameters of Algorithm 1 and Eq. (reuse_ratio).
@@ -333,7 +353,7 @@ def layer_forward(cfg, layer_w: Dict[str, np.ndarray], K: np.ndarray, V: np.ndar
     """
     H, d = cfg.n_heads, cfg.head_dim
     rows = np.asarray(rows, dtype=np.int64)
-    W = {k: widen_bf16(v) for k, v in layer_w.items()}
+    W = {k: _widen_cached(v) for k, v in layer_w.items()}
     x = hidden[rows]
     xn = rms_norm(x, W["g_attn"], cfg.rms_eps)
     q = (xn @ W["wq"].T).reshape(len(rows), H, d)
@@ -397,7 +417,7 @@ def input_rows(cfg, model: Dict[str, object], feats_bf16: np.ndarray, prompt_ids
 
 def _logits(cfg, model, h_row: np.ndarray) -> np.ndarray:
     xn = rms_norm(h_row[None, :], widen_bf16(model["g_final"]), cfg.rms_eps)
-    return (xn @ widen_bf16(model["lm_head"]).T)[0]
+    return (xn @ _widen_cached(model["lm_head"]).T)[0]
 
 
 def step(cfg, model: Dict[str, object], cache: CacheState, frames_t: np.ndarray,

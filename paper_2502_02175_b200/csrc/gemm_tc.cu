@@ -153,7 +153,9 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(TcArgs a) {
   __syncthreads();
   pdl_trigger();
   pdl_wait();                                                   // everything below may read what earlier kernels wrote
-  const int tokens = a.tot ? *a.tot : a.tot_fixed;
+  // blockIdx.z selects a chunk of up to 512 tokens (one accumulator's worth of tensor-memory columns)
+  const int tok0 = blockIdx.z * 512;
+  const int tokens = min(max((a.tot ? *a.tot : a.tot_fixed) - tok0, 0), 512);
   const int n_boxes = (tokens + TG_BOX_TOK - 1) / TG_BOX_TOK;    // token rows are staged in multiples of 64
   const int stage_bytes = TG_A_BYTES + n_boxes * TG_BOX_BYTES;
   int n_stages = TG_SMEM_RING / stage_bytes;
@@ -196,8 +198,8 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(TcArgs a) {
         } else {
           tma_load_2d(sa, a.tm_a[mat], k, row_base, &full_bar[s]);
         }
-        tma_load_2d(sb, a.tm_b + (rows0 - 1), k, 0, &full_bar[s]);
-        if (rows1 > 0) tma_load_2d(sb + 4 * TG_BOX_BYTES, a.tm_b + (rows1 - 1), k, 256, &full_bar[s]);
+        tma_load_2d(sb, a.tm_b + (rows0 - 1), k, tok0, &full_bar[s]);
+        if (rows1 > 0) tma_load_2d(sb + 4 * TG_BOX_BYTES, a.tm_b + (rows1 - 1), k, tok0 + 256, &full_bar[s]);
       }
     }
   } else if (warp == 1) {
@@ -264,24 +266,24 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(TcArgs a) {
         float* dst = a.tail_part + (size_t)split * a.tail_stride + (size_t)(tile - a.full_tiles) * 128 + r;
 #pragma unroll
         for (int c = 0; c < 16; ++c)
-          if (c0 + c < tokens) dst[(size_t)(c0 + c) * a.tail_ld] = v[c];
+          if (c0 + c < tokens) dst[(size_t)(tok0 + c0 + c) * a.tail_ld] = v[c];
       } else if (a.mode == TG_PARTIAL) {
         if (!live) continue;
         float* dst = a.part + (size_t)split * a.split_stride + n;
 #pragma unroll
         for (int c = 0; c < 16; ++c)
-          if (c0 + c < tokens) dst[(size_t)(c0 + c) * N] = v[c];
+          if (c0 + c < tokens) dst[(size_t)(tok0 + c0 + c) * N] = v[c];
       } else if (a.mode == TG_SWIGLU) {
         // gate-side threads finish even columns, up-side threads odd columns
 #pragma unroll
         for (int c = 0; c < 16; ++c) {
           if (live && ((c & 1) == 0) == first && c0 + c < tokens) {
             const float g = first ? v[c] : pv[c], u = first ? pv[c] : v[c];
-            a.h_out[(size_t)(c0 + c) * N + n] = __float2bfloat16(__fdividef(g, 1.f + __expf(-g)) * u);
+            a.h_out[(size_t)(tok0 + c0 + c) * N + n] = __float2bfloat16(__fdividef(g, 1.f + __expf(-g)) * u);
           }
         }
       } else {                                                   // TG_QKV
-        const int my_row = (c0 + (lane & 15) < tokens) ? __ldg(a.rowmap + c0 + (lane & 15)) : 0;
+        const int my_row = (c0 + (lane & 15) < tokens) ? __ldg(a.rowmap + tok0 + c0 + (lane & 15)) : 0;
         // all table reads of the chunk first (independent loads in flight together), then the arithmetic and stores
         int bs[16], ps[16];
         float cs[16], sn[16];
@@ -298,7 +300,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(TcArgs a) {
           if (live && c0 + c < tokens) {
             float y = v[c];
             if (mat < 2) y = first ? v[c] * cs[c] - pv[c] * sn[c] : v[c] * cs[c] + pv[c] * sn[c];
-            if (mat == 0) a.q_out[(size_t)(c0 + c) * N + n] = __float2bfloat16(y);
+            if (mat == 0) a.q_out[(size_t)(tok0 + c0 + c) * N + n] = __float2bfloat16(y);
             else (mat == 1 ? a.kc : a.vc)[((size_t)bs[c] * a.max_seq + ps[c]) * N + n] = __float2bfloat16(y);
           }
         }
@@ -400,15 +402,14 @@ int vlac_tc_setup(vlac_ctx* ctx) {
   if (e != cudaSuccess) { vlac_note_cuda_error(e, __FILE__, __LINE__); return VLAC_ERR_CUDA; }
   e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TG_SMEM_RING + 1024);
   if (e != cudaSuccess) { vlac_note_cuda_error(e, __FILE__, __LINE__); return VLAC_ERR_CUDA; }
-  // one CTA holds all tokens: at most 512 accumulator columns, and at least 2 ring stages
-  const int max_boxes = (ctx->rows_max + TG_BOX_TOK - 1) / TG_BOX_TOK;
-  if (ctx->rows_max > 512 || TG_SMEM_RING / (TG_A_BYTES + max_boxes * TG_BOX_BYTES) < 2) return VLAC_OK;
+  // a CTA holds up to 512 tokens (accumulator columns); more tokens are further chunks along grid.z
   ctx->tc_ok = 1;
   return VLAC_OK;
 }
 
 static int launch_tc(vlac_ctx* ctx, const TcArgs& a, int n_tiles, cudaStream_t s) {
-  VLAC_CUDA_CHECK(launch_pdl(gemm_tc_kernel, dim3(n_tiles, a.n_splits), dim3(TG_THREADS), (size_t)TG_SMEM_RING + 1024, s, a));
+  VLAC_CUDA_CHECK(launch_pdl(gemm_tc_kernel, dim3(n_tiles, a.n_splits, (ctx->rows_max + 511) / 512), dim3(TG_THREADS),
+                             (size_t)TG_SMEM_RING + 1024, s, a));
   VLAC_LAUNCH_CHECK(ctx);
   return VLAC_OK;
 }

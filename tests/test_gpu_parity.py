@@ -292,3 +292,54 @@ def test_step_graph_replay_equals_direct_launch(H, vb):
     for (t0, l0, n0), (t1, l1, n1) in zip(*outs):
         assert np.array_equal(t0, t1) and np.array_equal(l0, l1)
         assert n0 == n1 > 0                      # the replay reports the kernels it ran
+
+
+def test_step_dual_camera_7b_shape(H, vb):
+    """Two cameras (2 x 256 vision tokens + 40 prompt tokens, L = 552): one nearly static stream, one with
+    30 % of its patches changing per step; 7B-shaped layer, more rows than one accumulator chunk holds."""
+    import dataclasses
+    orc.WIDEN_CACHE_MAX = 16
+    try:
+        cfg = dataclasses.replace(synth.dual_camera_config(n_layers=1), vocab=4096)
+        model = synth.make_model(cfg, 12)
+        ids = synth.make_prompt_ids(cfg, 12)
+        ep = synth.make_episode(cfg, 12, 2, changed_fraction=[0.0, 0.3])
+        sess = H.Session(cfg, model)
+        try:
+            for t in range(2):
+                r = H.run_step_pair(sess, ep.frames[t][None], ep.feats[t][None], ids, H.oparams(top_k=200, alpha_override=[1.0]))[0]
+                assert r["logit_err"] <= H.TOL and r["attn_err"] <= H.TOL, (t, r)
+            assert r["M"][0] < cfg.seq_len
+        finally:
+            sess.close()
+    finally:
+        orc.WIDEN_CACHE_MAX = 0
+        orc._widen_cache.clear()
+
+
+def test_step_batch_of_eight_7b_shape(H, vb):
+    """Eight independent sequences per step sharing the weights, each with its own cache and its own changed
+    fraction (10-90 %), so the recomputed row counts are ragged (uncapped top-k)."""
+    import dataclasses
+    orc.WIDEN_CACHE_MAX = 16
+    try:
+        cfg = dataclasses.replace(synth.llama7b_config(n_layers=1), vocab=4096)
+        model = synth.make_model(cfg, 13)
+        B = 8
+        ids = synth.make_prompt_ids(cfg, 13, batch=B)
+        fracs = np.random.default_rng(13).uniform(0.1, 0.9, size=B)
+        eps = [synth.make_episode(cfg, 130 + b, 2, changed_fraction=[float(fracs[b])]) for b in range(B)]
+        sess = H.Session(cfg, model, batch=B)
+        try:
+            for t in range(2):
+                frames = np.stack([e.frames[t] for e in eps]); feats = np.stack([e.feats[t] for e in eps])
+                res = H.run_step_pair(sess, frames, feats, ids, H.oparams(top_k=256, tau_task=0.8, alpha_override=[1.0]))
+                for r in res:
+                    assert r["logit_err"] <= H.TOL and r["attn_err"] <= H.TOL, (t, r)
+            Ms = [int(r["M"][0]) for r in res]
+            assert len(set(Ms)) > 1 and min(Ms) < cfg.seq_len
+        finally:
+            sess.close()
+    finally:
+        orc.WIDEN_CACHE_MAX = 0
+        orc._widen_cache.clear()
