@@ -138,29 +138,43 @@ __device__ void block_topk(const unsigned long long* keys, const unsigned char* 
     for (int v = tid; v < n; v += blockDim.x)
       if (cand[v] && (keys[v] & mask) == prefix) atomicAdd(&hist[(unsigned)(keys[v] >> shift) & 255u], 1u);
     __syncthreads();
-    if (tid == 0) {
-      int cum = 0, d = 255;
-      for (; d > 0; --d) {
-        if (cum + (int)hist[d] >= need) break;
-        cum += (int)hist[d];
+    // warp 0 finds the digit holding the last element taken: lane l owns bins 255-8l ... 248-8l (descending)
+    if (tid < 32) {
+      int local[8], lsum = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { local[i] = (int)hist[255 - 8 * tid - i]; lsum += local[i]; }
+      int incl = lsum;                                         // inclusive prefix over lanes (higher digits first)
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, incl, o); if (tid >= o) incl += t; }
+      const int excl = incl - lsum;
+      const bool here = excl < need && need <= incl;           // exactly one lane: need <= number of candidates
+      if (here) {
+        int cum = excl, d = 255 - 8 * tid;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (cum + local[i] >= need) { d = 255 - 8 * tid - i; sh[4] = local[i]; break; }
+          cum += local[i];
+        }
+        sh[1] = d;
+        sh[2] = need - cum;
       }
-      sh[1] = d;
-      sh[2] = need - cum;
     }
     __syncthreads();
     prefix |= (unsigned long long)sh[1] << shift;
     mask |= 255ull << shift;
     need = sh[2];
+    const bool whole_bin = sh[4] == need;                      // every candidate sharing these leading digits is taken
     __syncthreads();
+    if (whole_bin) break;
   }
-  // prefix is now the key of the last element taken; `need` of the elements equal to it are taken
+  // candidates above `prefix` (on the digits examined) are taken, and `need` of those equal to it
   for (int v = tid; v < n; v += blockDim.x) {
     unsigned char take = 0;
     if (cand[v]) {
-      if (keys[v] > prefix) take = 1;
-      else if (keys[v] == prefix) {
+      if ((keys[v] & mask) > prefix) take = 1;
+      else if ((keys[v] & mask) == prefix) {
         int before = 0;
-        for (int u = 0; u < v; ++u) before += (cand[u] && keys[u] == prefix) ? 1 : 0;
+        for (int u = 0; u < v; ++u) before += (cand[u] && (keys[u] & mask) == prefix) ? 1 : 0;
         take = before < need ? 1 : 0;
       }
     }
