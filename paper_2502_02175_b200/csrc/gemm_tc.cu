@@ -37,9 +37,11 @@ constexpr int TG_MAX_STAGES = 8;
 constexpr int TG_SMEM_RING = 208 * 1024;        // dynamic shared memory for the ring
 constexpr unsigned long long TG_WAIT_LIMIT_NS = 400000000ull;
 
-struct TcArgs {
-  const CUtensorMap* tm_a[3];     // weight matrices (128-row boxes; 64-row boxes for gate / up)
-  const CUtensorMap* tm_b;        // activations [rows][K]: 4 maps with boxes of 64, 128, 192, 256 rows
+struct alignas(64) TcArgs {
+  // Tensor maps travel by value inside the kernel parameters (constant bank): the TMA unit fetches the
+  // descriptor for every request, and from global memory that fetch limited it to ~4 requests per us.
+  CUtensorMap tm_a[3];            // weight matrices (128-row boxes; 64-row boxes for gate / up)
+  CUtensorMap tm_b[4];            // activations [rows][K]: boxes of 64, 128, 192, 256 rows
   const int* tot;                 // live token count in device memory (NULL: tot_fixed)
   int tot_fixed;
   int K, N;                       // N = rows of one weight matrix
@@ -127,7 +129,7 @@ __device__ __forceinline__ void tmem_ld16(unsigned taddr, float* v) {
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-__global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(TcArgs a) {
+__global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_constant__ TcArgs a) {
   extern __shared__ __align__(1024) unsigned char ring_raw[];
   __shared__ __align__(8) unsigned long long full_bar[TG_MAX_STAGES], empty_bar[TG_MAX_STAGES], acc_bar;
   __shared__ float xch[2][4][16][32];                            // epilogue exchange between warp pairs (double-buffered)
@@ -193,13 +195,13 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(TcArgs a) {
         mbar_expect_tx(&full_bar[s], (unsigned)stage_bytes);
         const int k = (kb0 + i) * TG_BK;
         if (a.mode == TG_SWIGLU) {
-          tma_load_2d(sa, a.tm_a[0], k, row_base, &full_bar[s]);                // 64 gate rows
-          tma_load_2d(sa + 64 * 128, a.tm_a[1], k, row_base, &full_bar[s]);     // 64 up rows of the same features
+          tma_load_2d(sa, &a.tm_a[0], k, row_base, &full_bar[s]);                // 64 gate rows
+          tma_load_2d(sa + 64 * 128, &a.tm_a[1], k, row_base, &full_bar[s]);     // 64 up rows of the same features
         } else {
-          tma_load_2d(sa, a.tm_a[mat], k, row_base, &full_bar[s]);
+          tma_load_2d(sa, &a.tm_a[mat], k, row_base, &full_bar[s]);
         }
-        tma_load_2d(sb, a.tm_b + (rows0 - 1), k, tok0, &full_bar[s]);
-        if (rows1 > 0) tma_load_2d(sb + 4 * TG_BOX_BYTES, a.tm_b + (rows1 - 1), k, tok0 + 256, &full_bar[s]);
+        tma_load_2d(sb, &a.tm_b[rows0 - 1], k, tok0, &full_bar[s]);
+        if (rows1 > 0) tma_load_2d(sb + 4 * TG_BOX_BYTES, &a.tm_b[rows1 - 1], k, tok0 + 256, &full_bar[s]);
       }
     }
   } else if (warp == 1) {
@@ -395,12 +397,8 @@ int vlac_tc_setup(vlac_ctx* ctx) {
     if (rc == VLAC_OK) rc = encode_map(&act[TM_HM + hgt], ctx->hm, ctx->rows_max, F, box);
   }
   if (rc != VLAC_OK) { free(host); return rc; }
-  cudaError_t e = cudaMalloc(&ctx->tmaps, sizeof(CUtensorMap) * n_maps);
-  if (e != cudaSuccess) { free(host); cudaGetLastError(); return VLAC_ERR_OOM; }
-  e = cudaMemcpy(ctx->tmaps, host, sizeof(CUtensorMap) * n_maps, cudaMemcpyHostToDevice);
-  free(host);
-  if (e != cudaSuccess) { vlac_note_cuda_error(e, __FILE__, __LINE__); return VLAC_ERR_CUDA; }
-  e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TG_SMEM_RING + 1024);
+  ctx->tmaps_host = host;                                        // copied into the kernel parameters at every launch
+  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TG_SMEM_RING + 1024);
   if (e != cudaSuccess) { vlac_note_cuda_error(e, __FILE__, __LINE__); return VLAC_ERR_CUDA; }
   // a CTA holds up to 512 tokens (accumulator columns); more tokens are further chunks along grid.z
   ctx->tc_ok = 1;
@@ -415,7 +413,7 @@ static int launch_tc(vlac_ctx* ctx, const TcArgs& a, int n_tiles, cudaStream_t s
 }
 
 static void tc_common(vlac_ctx* ctx, vlac_cache* c, int layer, TcArgs* a) {
-  memset(a, 0, sizeof(*a));
+  memset((void*)a, 0, sizeof(*a));
   a->tot = c->tot + layer;
   a->d = ctx->cfg.head_dim;
   a->rowmap = c->rowmap + (size_t)layer * c->batch * ctx->L;
@@ -428,10 +426,11 @@ static void tc_common(vlac_ctx* ctx, vlac_cache* c, int layer, TcArgs* a) {
 
 int vlac_tc_qkv(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s) {
   const vlac_config& g = ctx->cfg;
-  const CUtensorMap* tm = (const CUtensorMap*)ctx->tmaps + (size_t)layer * TM_PER_LAYER;
-  const CUtensorMap* act = (const CUtensorMap*)ctx->tmaps + (size_t)g.n_layers * TM_PER_LAYER;
+  const CUtensorMap* tm = (const CUtensorMap*)ctx->tmaps_host + (size_t)layer * TM_PER_LAYER;
+  const CUtensorMap* act = (const CUtensorMap*)ctx->tmaps_host + (size_t)g.n_layers * TM_PER_LAYER;
   TcArgs a; tc_common(ctx, c, layer, &a);
-  a.tm_a[0] = tm + TM_WQ; a.tm_a[1] = tm + TM_WK; a.tm_a[2] = tm + TM_WV; a.tm_b = act + TM_XN;
+  a.tm_a[0] = tm[TM_WQ]; a.tm_a[1] = tm[TM_WK]; a.tm_a[2] = tm[TM_WV];
+  for (int i = 0; i < 4; ++i) a.tm_b[i] = act[TM_XN + i];
   a.K = g.hidden; a.N = g.hidden; a.mode = TG_QKV;
   a.q_out = ctx->q;
   a.kc = c->k + (size_t)layer * c->batch * kv_layer_elems(ctx);
@@ -441,11 +440,12 @@ int vlac_tc_qkv(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s) {
 
 int vlac_tc_partial(vlac_ctx* ctx, vlac_cache* c, int layer, int which, int* n_splits, cudaStream_t s) {
   const vlac_config& g = ctx->cfg;
-  const CUtensorMap* tm = (const CUtensorMap*)ctx->tmaps + (size_t)layer * TM_PER_LAYER;
-  const CUtensorMap* act = (const CUtensorMap*)ctx->tmaps + (size_t)g.n_layers * TM_PER_LAYER;
+  const CUtensorMap* tm = (const CUtensorMap*)ctx->tmaps_host + (size_t)layer * TM_PER_LAYER;
+  const CUtensorMap* act = (const CUtensorMap*)ctx->tmaps_host + (size_t)g.n_layers * TM_PER_LAYER;
   TcArgs a; tc_common(ctx, c, layer, &a);
   const bool down = which != 0;
-  a.tm_a[0] = tm + (down ? TM_DOWN : TM_WO); a.tm_b = act + (down ? TM_HM : TM_AO);
+  a.tm_a[0] = tm[down ? TM_DOWN : TM_WO];
+  for (int i = 0; i < 4; ++i) a.tm_b[i] = act[(down ? TM_HM : TM_AO) + i];
   a.K = down ? g.ffn : g.hidden; a.N = g.hidden; a.mode = TG_PARTIAL;
   const int tiles = (g.hidden + 127) / 128;
   int splits = ctx->n_sm / tiles;                       // fill the SMs: the partial sums are folded by the next kernel
@@ -461,10 +461,11 @@ int vlac_tc_partial(vlac_ctx* ctx, vlac_cache* c, int layer, int which, int* n_s
 
 int vlac_tc_gateup(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s) {
   const vlac_config& g = ctx->cfg;
-  const CUtensorMap* tm = (const CUtensorMap*)ctx->tmaps + (size_t)layer * TM_PER_LAYER;
-  const CUtensorMap* act = (const CUtensorMap*)ctx->tmaps + (size_t)g.n_layers * TM_PER_LAYER;
+  const CUtensorMap* tm = (const CUtensorMap*)ctx->tmaps_host + (size_t)layer * TM_PER_LAYER;
+  const CUtensorMap* act = (const CUtensorMap*)ctx->tmaps_host + (size_t)g.n_layers * TM_PER_LAYER;
   TcArgs a; tc_common(ctx, c, layer, &a);
-  a.tm_a[0] = tm + TM_GATE; a.tm_a[1] = tm + TM_UP; a.tm_b = act + TM_XN;
+  a.tm_a[0] = tm[TM_GATE]; a.tm_a[1] = tm[TM_UP];
+  for (int i = 0; i < 4; ++i) a.tm_b[i] = act[TM_XN + i];
   a.K = g.hidden; a.N = g.ffn; a.mode = TG_SWIGLU;
   a.h_out = ctx->hm;
   const int tiles = (g.ffn + 63) / 64;

@@ -61,7 +61,8 @@ struct vlac_ctx {
   unsigned char* in_frames; bf16* in_feats; int *in_ids, *in_forced, *out_tokens; float* logits_all;
   StepGraph graphs[VLAC_MAX_GRAPHS];
   int graph_next, use_graph;
-  void* tmaps;                       // device array of TMA tensor maps (weights per layer, activation buffers)
+  void* tmaps;                       // (unused) device copy of the tensor maps
+  void* tmaps_host;                  // host array of TMA tensor maps (weights per layer, activation buffers)
   int tc_ok;                         // 1: shapes fit the tensor-memory GEMM
   int pass_grid;                     // CTAs of the persistent single-row pass kernel (0: not used)
   void* tmap_q;                      // device tensor map of the query buffer (tiled attention)
