@@ -58,9 +58,11 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, volatile int* abort_flag, int* dev_error, int code) {
   if (mbar_try_wait(bar, parity)) return true;
+  // The wall-clock timer is slow to read: poll the barrier many times between two looks at it.
   const unsigned long long t0 = global_ns();
   while (true) {
-    if (mbar_try_wait(bar, parity)) return true;
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
     if (global_ns() - t0 > AT_WAIT_LIMIT_NS) break;
   }

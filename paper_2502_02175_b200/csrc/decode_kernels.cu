@@ -363,7 +363,9 @@ __device__ __forceinline__ bool grid_barrier(unsigned* counter, unsigned target,
     __threadfence();
     atomicAdd(counter, 1u);
     const unsigned long long t0 = gv_global_ns();
+    unsigned polls = 0;
     while (ld_acquire_u32(counter) < target) {
+      if ((++polls & 255u) != 0) continue;                       // the error word and the wall clock are looked at rarely
       if (*reinterpret_cast<volatile int*>(dev_error) != 0) { ok = 0; break; }
       if (gv_global_ns() - t0 > GV_BARRIER_LIMIT_NS) { atomicCAS(dev_error, 0, 0x80000 | (int)(target & 0xffff)); ok = 0; break; }
     }

@@ -246,6 +246,23 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
     const bool exchange = (a.mode == TG_SWIGLU && !tail) || (a.mode == TG_QKV && mat < 2);
     const int j = (n % a.d) % half;
     const size_t N = (size_t)a.N;
+    // QKV: positions and rotary table entries of a 16-token chunk; fetched one chunk ahead of their use so
+    // that the table latency overlaps the previous chunk's exchange, arithmetic and stores
+    int bs[16], ps[16];
+    float cs[16], sn[16];
+    auto fetch_tables = [&](int c0, int* b_o, int* p_o, float* c_o, float* s_o) {
+      const int my_row = (c0 + (lane & 15) < tokens) ? __ldg(a.rowmap + tok0 + c0 + (lane & 15)) : 0;
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
+        const int row = __shfl_sync(0xffffffffu, my_row, c);
+        int b = 0, pos = row;
+        if (a.batch > 1) { b = row / a.L; pos = row - b * a.L; }
+        b_o[c] = b; p_o[c] = pos;
+        if (mat < 2) { c_o[c] = __ldg(a.rope_cos + (size_t)pos * half + j); s_o[c] = __ldg(a.rope_sin + (size_t)pos * half + j); }
+        else { c_o[c] = 1.f; s_o[c] = 0.f; }
+      }
+    };
+    if (a.mode == TG_QKV && tokens > 0) fetch_tables(0, bs, ps, cs, sn);
     int chunk = 0;
     for (int c0 = 0; c0 < tokens; c0 += 16, ++chunk) {
       float v[16], pv[16];
@@ -285,18 +302,10 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
           }
         }
       } else {                                                   // TG_QKV
-        const int my_row = (c0 + (lane & 15) < tokens) ? __ldg(a.rowmap + tok0 + c0 + (lane & 15)) : 0;
-        // all table reads of the chunk first (independent loads in flight together), then the arithmetic and stores
-        int bs[16], ps[16];
-        float cs[16], sn[16];
-#pragma unroll
-        for (int c = 0; c < 16; ++c) {
-          const int row = __shfl_sync(0xffffffffu, my_row, c);
-          int b = 0, pos = row;
-          if (a.batch > 1) { b = row / a.L; pos = row - b * a.L; }
-          bs[c] = b; ps[c] = pos;
-          if (mat < 2) { cs[c] = __ldg(a.rope_cos + (size_t)pos * half + j); sn[c] = __ldg(a.rope_sin + (size_t)pos * half + j); }
-        }
+        int bn[16], pn[16];
+        float cn[16], sn2[16];
+        const bool more = c0 + 16 < tokens;                     // uniform: next chunk's tables requested before this chunk's stores
+        if (more) fetch_tables(c0 + 16, bn, pn, cn, sn2);
 #pragma unroll
         for (int c = 0; c < 16; ++c) {
           if (live && c0 + c < tokens) {
@@ -305,6 +314,10 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
             if (mat == 0) a.q_out[(size_t)(tok0 + c0 + c) * N + n] = __float2bfloat16(y);
             else (mat == 1 ? a.kc : a.vc)[((size_t)bs[c] * a.max_seq + ps[c]) * N + n] = __float2bfloat16(y);
           }
+        }
+        if (more) {
+#pragma unroll
+          for (int c = 0; c < 16; ++c) { bs[c] = bn[c]; ps[c] = pn[c]; cs[c] = cn[c]; sn[c] = sn2[c]; }
         }
       }
     }
