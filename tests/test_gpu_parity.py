@@ -343,3 +343,86 @@ def test_step_batch_of_eight_7b_shape(H, vb):
     finally:
         orc.WIDEN_CACHE_MAX = 0
         orc._widen_cache.clear()
+
+
+def test_full_size_32_layers_properties_and_sampled_layer(H, vb):
+    """The bench configuration itself: 32 layers of the 7B shape, weights drawn on the device, graph replay
+    on a side stream.  Checked at this size: the selection against the checker (bit-exact, from the
+    library's own saved attention), run-to-run determinism, reuse ratio 0 == no-reuse step, and one
+    sampled layer's partial forward against the checker with that layer's weights copied to the host."""
+    cfg = synth.llama7b_config(n_layers=32)
+    dev = vb.DeviceModel.random(cfg, seed=77)
+    ep = synth.make_episode(cfg.with_layers(1), 77, 3)
+    ids = torch.from_numpy(synth.make_prompt_ids(cfg, 77)).to("cuda")
+    frames = torch.from_numpy(ep.frames).to("cuda")
+    feats = vb.upload_bf16(ep.feats)
+    side = torch.cuda.Stream()
+    ctx = vb.vlac_create(vb.make_config(cfg, 1), dev.weights)
+
+    def run(alpha, full_last=False):
+        cache = vb.vlac_cache_alloc(ctx, 1)
+        gp, keep = vb.make_params(alpha_override=alpha)
+        out = []
+        torch.cuda.synchronize()
+        with torch.cuda.stream(side):
+            for t in range(2):
+                tok = torch.zeros((1, cfg.n_action), dtype=torch.int32, device="cuda")
+                lg = torch.zeros((1, cfg.n_action, cfg.vocab), dtype=torch.float32, device="cuda")
+                attn_before = torch.empty((cfg.n_layers, cfg.n_heads, cfg.n_vision), dtype=torch.float32, device="cuda")
+                vb.vlac_cache_read(cache, vb.PART_ATTN_PREV, 0, 0, attn_before)
+                vb.vlac_step(ctx, cache, frames[t:t + 1], feats[t:t + 1], ids, gp, full_last and t == 1, tok, lg)
+                side.synchronize()
+                out.append((tok.cpu().numpy().copy(), lg.cpu().numpy().copy(), attn_before.cpu().numpy().copy()))
+        return cache, out
+
+    try:
+        alpha = [min(1.0, 0.25 + l / 24.0) for l in range(32)]
+        cache_a, out_a = run(alpha)
+        assert vb.vlac_device_error(ctx) == 0
+        # selection of the cached step, bit for bit, from the library's own saved scores
+        got = vb.selection_to_host(vb.vlac_selection_view(cache_a))
+        oc = orc.new_cache(cfg)
+        oc.prev_frames, oc.attn_tv, oc.warm = ep.frames[0], out_a[1][2].astype(np.float64), True
+        want = orc.select(cfg, ep.frames[1], oc, orc.SelectParams(alpha_override=alpha))
+        H.check_selection(got, want, 0, cfg, where="32 layers")
+        assert want.M[-1] < want.M[0] < cfg.seq_len
+        # determinism
+        cache_b, out_b = run(alpha)
+        for (t0, l0, _), (t1, l1, _) in zip(out_a, out_b):
+            assert np.array_equal(t0, t1) and np.array_equal(l0, l1)
+        # reuse ratio 0 is the no-reuse step
+        cache_c, out_c = run([0.0] * 32)
+        cache_d, out_d = run([0.0] * 32, full_last=True)
+        assert np.array_equal(out_c[1][1], out_d[1][1]) and np.array_equal(out_c[1][0], out_d[1][0])
+        assert not np.array_equal(out_a[1][1], out_c[1][1])          # reuse changes the result: it is an approximation
+        # one sampled layer against the checker, on the rows the cached step recomputed there
+        l = 17
+        lw = {}
+        for name, _ in vb.vlac_layer_w._fields_:
+            ptr = getattr(dev.layer_structs[l], name)
+            t = next(x for x in dev.tensors if x.data_ptr() == ptr)
+            lw[name] = t.view(torch.int16).cpu().numpy().view(np.uint16)
+        cos = next(x for x in dev.tensors if x.data_ptr() == dev.weights.rope_cos).cpu().numpy()
+        sin = next(x for x in dev.tensors if x.data_ptr() == dev.weights.rope_sin).cpu().numpy()
+        kt = torch.empty((cfg.max_seq, cfg.n_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda")
+        vt = torch.empty_like(kt)
+        vb.vlac_cache_read(cache_a, vb.PART_K, 0, l, kt); vb.vlac_cache_read(cache_a, vb.PART_V, 0, l, vt)
+        torch.cuda.synchronize()
+        K, V = H.bf16_tensor_to_f64(kt), H.bf16_tensor_to_f64(vt)
+        h_bits = synth.make_hidden(cfg, 5)
+        hid = np.zeros((cfg.max_seq, cfg.hidden)); hid[:cfg.seq_len] = orc.widen_bf16(h_bits[0])
+        rows = want.rows[l]
+        orc.layer_forward(cfg, lw, K, V, hid, rows, cos, sin)
+        d_h = vb.upload_bf16(h_bits)
+        with torch.cuda.stream(side):
+            vb.vlac_layer_forward(ctx, cache_a, l, d_h)
+        torch.cuda.synchronize()
+        g_h = H.bf16_tensor_to_f64(d_h)[0]
+        assert H.rel_err(g_h[rows], hid[rows]) <= H.TOL
+        vb.vlac_cache_read(cache_a, vb.PART_K, 0, l, kt)
+        torch.cuda.synchronize()
+        assert H.rel_err(H.bf16_tensor_to_f64(kt)[:cfg.seq_len], K[:cfg.seq_len]) <= H.TOL
+        for c in (cache_a, cache_b, cache_c, cache_d):
+            vb.vlac_cache_free(c)
+    finally:
+        vb.vlac_destroy(ctx)
