@@ -296,11 +296,12 @@ __device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc
   float acc[DPL];
 #pragma unroll
   for (int e = 0; e < DPL; ++e) acc[e] = 0.f;
-  for (int j0 = warp; j0 < nkeys; j0 += 32) {                  // four keys of this warp in flight
-    float pj[4];
-    __align__(8) bf16 vv[4][DPL];
+  constexpr int KF = 10;                                         // keys of this warp in flight (8 warps x 10 covers 80 keys per round)
+  for (int j0 = warp; j0 < nkeys; j0 += 8 * KF) {
+    float pj[KF];
+    __align__(8) bf16 vv[KF][DPL];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < KF; ++u) {
       const int j = j0 + 8 * u;
       pj[u] = j < nkeys ? p[j] : 0.f;
       const bf16* vp = vbase + (size_t)min(j, nkeys - 1) * D;
@@ -312,7 +313,7 @@ __device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc
       }
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u)
+    for (int u = 0; u < KF; ++u)
 #pragma unroll
       for (int e = 0; e < DPL; ++e) acc[e] += pj[u] * bf2f(vv[u][e]);
   }
