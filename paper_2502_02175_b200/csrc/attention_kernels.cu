@@ -14,6 +14,7 @@
 // a small kernel adds the tiles in order and divides by the number of text rows (fixed order: the
 // saved scores are bit-reproducible).
 #include "vlac_internal.h"
+#include "launch_util.h"
 #include <cuda.h>
 #include <stdlib.h>
 
@@ -124,6 +125,8 @@ __global__ void __launch_bounds__(AT_THREADS, 1) attention_tile_kernel(AttnTileA
   constexpr int Q_BYTES = HALVES * AT_Q * 128;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int tile = blockIdx.x, b = blockIdx.y, h = blockIdx.z;
+  pdl_trigger();
+  pdl_wait();                                                   // the row lists, Q and the caches come from earlier kernels
 
   // rows of this tile: compact indices [row0, row0 + n_valid) of sequence b
   int off = 0;
@@ -314,6 +317,8 @@ __global__ void __launch_bounds__(AT_THREADS, 1) attention_tile_kernel(AttnTileA
 __global__ void __launch_bounds__(256) emit_from_tiles_kernel(const float* partial, float* attn_next_layer, size_t seq_stride,
                                                               int tiles, int n_tp, int H, int Lv) {
   const int h = blockIdx.x, b = blockIdx.y;
+  pdl_trigger();
+  pdl_wait();
   float* dst = attn_next_layer + (size_t)b * seq_stride + (size_t)h * Lv;
   for (int v = threadIdx.x; v < Lv; v += blockDim.x) {
     float s = 0.f;
@@ -382,12 +387,12 @@ int vlac_launch_prefill_attention(vlac_ctx* ctx, vlac_cache* c, int layer, cudaS
   a.layer = layer; a.nl = g.n_layers; a.B = B; a.L = ctx->L; a.max_seq = ctx->max_seq; a.H = g.n_heads;
   a.v0 = g.n_text_pre; a.Lv = ctx->Lv; a.tiles = ctx->attn_tiles;
   const dim3 grid(ctx->attn_tiles, B, g.n_heads);
-  if (g.head_dim == 128) attention_tile_kernel<128><<<grid, AT_THREADS, at_smem<128>(ctx->Lv), s>>>(a);
-  else attention_tile_kernel<64><<<grid, AT_THREADS, at_smem<64>(ctx->Lv), s>>>(a);
+  if (g.head_dim == 128) VLAC_CUDA_CHECK(launch_pdl(attention_tile_kernel<128>, grid, dim3(AT_THREADS), at_smem<128>(ctx->Lv), s, a));
+  else VLAC_CUDA_CHECK(launch_pdl(attention_tile_kernel<64>, grid, dim3(AT_THREADS), at_smem<64>(ctx->Lv), s, a));
   VLAC_LAUNCH_CHECK(ctx);
   float* dst = c->attn_next + (size_t)layer * g.n_heads * ctx->Lv;
-  emit_from_tiles_kernel<<<dim3(g.n_heads, B), 256, 0, s>>>(ctx->probs, dst, (size_t)g.n_layers * g.n_heads * ctx->Lv,
-                                                            ctx->attn_tiles, g.n_text_post, g.n_heads, ctx->Lv);
+  VLAC_CUDA_CHECK(launch_pdl(emit_from_tiles_kernel, dim3(g.n_heads, B), dim3(256), 0, s, (const float*)ctx->probs, dst,
+                             (size_t)g.n_layers * g.n_heads * ctx->Lv, ctx->attn_tiles, g.n_text_post, g.n_heads, ctx->Lv));
   VLAC_LAUNCH_CHECK(ctx);
   return VLAC_OK;
 }

@@ -56,6 +56,8 @@ __global__ void __launch_bounds__(256) finalize_norm_kernel(bf16* hidden, const 
                                                             int D, float eps) {
   __shared__ float red[8];
   const int i = blockIdx.x;
+  pdl_trigger();
+  pdl_wait();
   if (i >= *tot_prev) return;
   const int row = rowmap_prev[i];
   const int j = slot_next ? slot_next[row] : i;
@@ -366,9 +368,10 @@ int vlac_launch_finalize_norm(vlac_ctx* ctx, vlac_cache* c, bf16* hidden, int l_
                               int l_next, const void* gain, cudaStream_t s) {
   const int BL = c->batch * ctx->L;
   const int* slot_next = (gain && l_next != l_prev) ? c->slot + (size_t)l_next * BL : nullptr;
-  finalize_norm_kernel<<<BL, 256, 0, s>>>(hidden, c->tot + l_prev, c->rowmap + (size_t)l_prev * BL, ctx->part, n_splits,
-                                          (size_t)ctx->rows_max * ctx->cfg.hidden, slot_next, (const bf16*)gain, ctx->xn,
-                                          ctx->cfg.hidden, ctx->cfg.rms_eps);
+  VLAC_CUDA_CHECK(launch_pdl(finalize_norm_kernel, dim3(BL), dim3(256), 0, s, hidden, (const int*)(c->tot + l_prev),
+                             (const int*)(c->rowmap + (size_t)l_prev * BL), (const float*)ctx->part, n_splits,
+                             (size_t)ctx->rows_max * ctx->cfg.hidden, slot_next, (const bf16*)gain, ctx->xn,
+                             ctx->cfg.hidden, ctx->cfg.rms_eps));
   VLAC_LAUNCH_CHECK(ctx);
   return VLAC_OK;
 }
