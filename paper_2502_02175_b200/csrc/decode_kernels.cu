@@ -16,6 +16,15 @@ __device__ __forceinline__ float bf2f(bf16 x) { return __bfloat162float(x); }
 
 enum { GV_QKV = 0, GV_RESID = 1, GV_SWIGLU = 2, GV_LOGITS = 3 };
 
+// Head of the weights the NEXT matrix-vector kernel on the stream will read: this kernel asks the L2 for
+// them while it is still streaming its own, so HBM stays busy across the kernel boundary.
+struct PfArgs {
+  const bf16 *w0, *w1, *w2;
+  int mode, K, N, d;
+  int units;               // units (row pairs) per CTA to request; 0: none
+  float frac;              // request them once this fraction of the CTA's own units has been handed out
+};
+
 struct GemvArgs {
   const float* x_f32;      // [nb][K] fp32 source (normalised with `gain`), or NULL
   const bf16* x_bf16;      // [nb][K] bf16 source used as is, or NULL
@@ -31,6 +40,7 @@ struct GemvArgs {
   float* x_out;            // RESID: [nb][N] +=
   bf16* h_out;             // SWIGLU: [nb][N]
   float* logits;           // LOGITS: [nb][N]
+  PfArgs pf;
 };
 
 __device__ __forceinline__ void fma8(float& acc, const uint4& w, const uint4& x) {
@@ -47,7 +57,8 @@ __device__ __forceinline__ void fma8(float& acc, const uint4& w, const uint4& x)
 
 struct UnitRows { const uint4 *pa, *pb; int rowA, rowB, mat; };
 
-__device__ __forceinline__ UnitRows unit_rows(const GemvArgs& a, int u) {
+template <typename A>
+__device__ __forceinline__ UnitRows unit_rows(const A& a, int u) {
   UnitRows r;
   const int K = a.K;
   if (a.mode == GV_QKV) {
@@ -71,6 +82,32 @@ __device__ __forceinline__ UnitRows unit_rows(const GemvArgs& a, int u) {
   return r;
 }
 
+// Epilogue of one unit (a pair of weight rows) for sequence b: ya, yb are the two finished dot products.
+__device__ __forceinline__ void store_unit(const GemvArgs& a, const UnitRows& cu, int b, float ya, float yb) {
+  const int rowA = cu.rowA, rowB = cu.rowB, mat = cu.mat;
+  if (a.mode == GV_QKV) {
+    if (mat == 2) {
+      bf16* dst = a.vc + ((size_t)b * a.max_seq + a.pos) * a.N;
+      dst[rowA] = __float2bfloat16(ya); dst[rowB] = __float2bfloat16(yb);
+    } else {
+      const int half = a.d / 2;
+      const int j = rowA % a.d;
+      const float c = a.rope_cos[(size_t)a.pos * half + j], s = a.rope_sin[(size_t)a.pos * half + j];
+      const float r1 = ya * c - yb * s, r2 = yb * c + ya * s;
+      bf16* dst = mat == 0 ? a.q_out + (size_t)b * a.N : a.kc + ((size_t)b * a.max_seq + a.pos) * a.N;
+      dst[rowA] = __float2bfloat16(r1); dst[rowB] = __float2bfloat16(r2);
+    }
+  } else if (a.mode == GV_SWIGLU) {
+    a.h_out[(size_t)b * a.N + rowA] = __float2bfloat16(ya / (1.f + __expf(-ya)) * yb);
+  } else if (a.mode == GV_RESID) {
+    a.x_out[(size_t)b * a.N + rowA] += ya;
+    if (rowB != rowA) a.x_out[(size_t)b * a.N + rowB] += yb;
+  } else {
+    a.logits[(size_t)b * a.N + rowA] = ya;
+    if (rowB != rowA) a.logits[(size_t)b * a.N + rowB] = yb;
+  }
+}
+
 // streaming loads: weights are read exactly once, keep them out of L1
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
   uint4 v;
@@ -84,6 +121,27 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
 #ifndef GV_CTAS_PER_SM
 #define GV_CTAS_PER_SM 2
 #endif
+
+__device__ __forceinline__ int unit_count(int mode, int N) {
+  if (mode == GV_QKV) return 3 * (N / 2);
+  if (mode == GV_SWIGLU) return N;
+  return (N + 1) / 2;
+}
+
+// One warp asks the L2 for the rows of the first `f.units` units that the CTA of the same index will own in
+// the next kernel (same grid size).  A hint only: nothing waits for it and nothing depends on it.
+__device__ __noinline__ void prefetch_next_rows(PfArgs f, int lane) {
+  const int nu = unit_count(f.mode, f.N);
+  const int ub = (int)(((long long)nu * blockIdx.x) / gridDim.x);
+  const int nloc = (int)(((long long)nu * (blockIdx.x + 1)) / gridDim.x) - ub;
+  const int cnt = min(f.units, nloc);
+  const unsigned bytes = (unsigned)f.K * (unsigned)sizeof(bf16);
+  for (int i = lane; i < 2 * cnt; i += 32) {
+    const UnitRows r = unit_rows(f, ub + (i >> 1));
+    const uint4* p = (i & 1) ? r.pb : r.pa;
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+  }
+}
 
 __device__ __forceinline__ void load_batch(uint4* va, uint4* vb, const UnitRows& r, int c0, int nchunk) {
 #pragma unroll
@@ -101,11 +159,7 @@ __device__ __forceinline__ void gemv_body(const GemvArgs& a, unsigned char* smem
   bf16* xs = reinterpret_cast<bf16*>(smem_raw);           // [NB][K]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int K = a.K;
-  const int half = a.d / 2;
-  int n_units;
-  if (a.mode == GV_QKV) n_units = 3 * (a.N / 2);
-  else if (a.mode == GV_SWIGLU) n_units = a.N;
-  else n_units = (a.N + 1) / 2;
+  const int n_units = unit_count(a.mode, a.N);
   const int nchunk = K / 8;
   const int bpu = (nchunk + 32 * GV_BATCH - 1) / (32 * GV_BATCH);      // load batches per unit
   // This CTA owns a contiguous, balanced range of units.  Each warp starts on the unit of its own index
@@ -119,6 +173,12 @@ __device__ __forceinline__ void gemv_body(const GemvArgs& a, unsigned char* smem
   int u_ld = warp < n_local ? warp : -1;                    // unit (local index) whose batch is in va, vb
   UnitRows ld_unit = unit_rows(a, u_begin + max(u_ld, 0));
   if (u_ld >= 0) load_batch(va, vb, ld_unit, lane, nchunk);
+  // ticket at which the next kernel's first rows are requested; a CTA with no tickets to draw asks now
+  int pf_at = -1;
+  if (a.pf.units > 0) {
+    pf_at = max(8, (int)((float)n_local * a.pf.frac));
+    if (pf_at >= n_local) { pf_at = -1; if (warp == 0) prefetch_next_rows(a.pf, lane); }
+  }
   wait();
 
   // ---- activations -> shared memory (RMSNorm here if a gain is given)
@@ -163,6 +223,7 @@ __device__ __forceinline__ void gemv_body(const GemvArgs& a, unsigned char* smem
       int t = 0;
       if (lane == 0) t = atomicAdd(next_unit, 1);
       t = __shfl_sync(0xffffffffu, t, 0);
+      if (t == pf_at) prefetch_next_rows(a.pf, lane);
       u_nx = t < n_local ? t : -1;
       bi_nx = 0;
     }
@@ -191,31 +252,10 @@ __device__ __forceinline__ void gemv_body(const GemvArgs& a, unsigned char* smem
         }
       }
       if (lane == 0) {
-        const int rowA = cu.rowA, rowB = cu.rowB, mat = cu.mat;
 #pragma unroll
         for (int b = 0; b < NB; ++b) {
           if (b >= a.nb) break;
-          const float ya = accA[b], yb = accB[b];
-          if (a.mode == GV_QKV) {
-            if (mat == 2) {
-              bf16* dst = a.vc + ((size_t)b * a.max_seq + a.pos) * a.N;
-              dst[rowA] = __float2bfloat16(ya); dst[rowB] = __float2bfloat16(yb);
-            } else {
-              const int j = rowA % a.d;
-              const float c = a.rope_cos[(size_t)a.pos * half + j], s = a.rope_sin[(size_t)a.pos * half + j];
-              const float r1 = ya * c - yb * s, r2 = yb * c + ya * s;
-              bf16* dst = mat == 0 ? a.q_out + (size_t)b * a.N : a.kc + ((size_t)b * a.max_seq + a.pos) * a.N;
-              dst[rowA] = __float2bfloat16(r1); dst[rowB] = __float2bfloat16(r2);
-            }
-          } else if (a.mode == GV_SWIGLU) {
-            a.h_out[(size_t)b * a.N + rowA] = __float2bfloat16(ya / (1.f + __expf(-ya)) * yb);
-          } else if (a.mode == GV_RESID) {
-            a.x_out[(size_t)b * a.N + rowA] += ya;
-            if (rowB != rowA) a.x_out[(size_t)b * a.N + rowB] += yb;
-          } else {
-            a.logits[(size_t)b * a.N + rowA] = ya;
-            if (rowB != rowA) a.logits[(size_t)b * a.N + rowB] = yb;
-          }
+          store_unit(a, cu, b, accA[b], accB[b]);
         }
       }
 #pragma unroll
@@ -236,6 +276,186 @@ __global__ void __launch_bounds__(256, GV_CTAS_PER_SM) gemv_pair_kernel(GemvArgs
   __shared__ float red[8];
   __shared__ int next_unit;
   gemv_body<NB>(a, smem_raw, red, &next_unit, [] { pdl_trigger(); pdl_wait(); });
+}
+
+// ---- the same product on the warp-level tensor cores, weights staged through shared memory --------------
+// A matrix-vector product has no reuse to offer the tensor cores, but it has instructions to save: read
+// with scalar code every 16 bytes of weights cost about twenty instructions (unpack, multiply-add), which
+// caps the bytes a thread can keep in flight.  Here a 16 x 16 tile of weights costs one ldmatrix and one
+// mma (the activations of up to 8 sequences are the 8 columns of B; unused columns are zero).
+//
+// One CTA of 16 warps per SM owns a contiguous range of units and walks it in groups of 8 units = 16 weight
+// rows (the A rows of the units on top, their partner rows below).  The warps split K into 64-wide
+// sub-stages dealt round-robin, so every warp streams the same share of every row and the CTA reads each
+// row front to back.  A warp copies a sub-stage (16 rows x 128 B, XOR-swizzled by row) with 16-byte
+// asynchronous copies into its own ring of GT_DEPTH slots and consumes it with ldmatrix; only warp-level
+// synchronisation guards the ring.  At the end of a group the 16 partial accumulator tiles meet in shared
+// memory and are added in warp order (bit-reproducible); one barrier per group, partials double-buffered.
+constexpr int GT_THREADS = 512;
+constexpr int GT_WARPS = GT_THREADS / 32;
+constexpr int GT_DEPTH = 5;
+constexpr int GT_SLOT_BYTES = 16 * 128;
+constexpr int GT_RING_BYTES = GT_WARPS * GT_DEPTH * GT_SLOT_BYTES;      // 160 KB
+constexpr int GT_PART_BYTES = 2 * GT_WARPS * 32 * 4 * (int)sizeof(float);  // 16 KB
+constexpr int GT_XR = 24;                                               // activations a thread keeps while it normalises a row
+
+__device__ __forceinline__ void cp_async16(unsigned smem_dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void ldmatrix_x4(unsigned addr, unsigned* r) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_16816(float* c, const unsigned* a, unsigned b0, unsigned b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+__global__ void __launch_bounds__(GT_THREADS, 1) gemv_mma_kernel(GemvArgs a) {
+  extern __shared__ __align__(128) unsigned char gt_smem[];
+  __shared__ float red[GT_WARPS];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int K = a.K, nb = a.nb;
+  const int n_units = unit_count(a.mode, a.N);
+  const int u_begin = (int)(((long long)n_units * blockIdx.x) / gridDim.x);
+  const int n_local = (int)(((long long)n_units * (blockIdx.x + 1)) / gridDim.x) - u_begin;
+  const int n_groups = (n_local + 7) / 8;
+  const int n_tab = ((n_units + (int)gridDim.x - 1) / (int)gridDim.x + 7) / 8 * 8;     // same for every CTA: sizes the table
+  const unsigned ring_w = (unsigned)__cvta_generic_to_shared(gt_smem) + (unsigned)warp * (GT_DEPTH * GT_SLOT_BYTES);
+  float* part = reinterpret_cast<float*>(gt_smem + GT_RING_BYTES);                      // [2][GT_WARPS][32][4]
+  const uint4** tab = reinterpret_cast<const uint4**>(gt_smem + GT_RING_BYTES + GT_PART_BYTES);   // [n_tab][2] row pointers
+  bf16* xs = reinterpret_cast<bf16*>(gt_smem + GT_RING_BYTES + GT_PART_BYTES + (size_t)n_tab * 16);  // [nb][K]
+
+  // row pointers of this CTA's units (the ragged end repeats the last unit: read, never stored)
+  if (n_local > 0)
+    for (int t = tid; t < n_groups * 8; t += GT_THREADS) {
+      const UnitRows r = unit_rows(a, u_begin + min(t, n_local - 1));
+      tab[2 * t] = r.pa; tab[2 * t + 1] = r.pb;
+    }
+  __syncthreads();
+
+  const int S = K / 64;                                                // sub-stages per row
+  const int ns_w = warp < S ? (S - warp + GT_WARPS - 1) / GT_WARPS : 0;   // ... of this warp
+  // ---- issue side: (group, sub-stage) in order; one copy group per item, empty once the work is exhausted
+  int ig = 0, ij = 0, islot = 0;
+  const char* rowptr[4];
+  auto load_rowptrs = [&](int g) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int row = (lane >> 3) + 4 * i;
+      rowptr[i] = reinterpret_cast<const char*>(tab[(g * 8 + (row & 7)) * 2 + (row >> 3)]);
+    }
+  };
+  if (n_groups > 0 && ns_w > 0) load_rowptrs(0);
+  auto issue = [&]() {
+    if (ig < n_groups && ns_w > 0) {
+      const unsigned slotp = ring_w + (unsigned)islot * GT_SLOT_BYTES;
+      const size_t koff = (size_t)(warp + GT_WARPS * ij) * 128 + (size_t)(lane & 7) * 16;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int row = (lane >> 3) + 4 * i;
+        cp_async16(slotp + (unsigned)(row * 128 + (((lane & 7) ^ (row & 7)) << 4)), rowptr[i] + koff);
+      }
+      if (++ij == ns_w) {
+        ij = 0;
+        if (++ig < n_groups) load_rowptrs(ig);
+      }
+    }
+    cp_async_commit();
+    islot = (islot + 1 == GT_DEPTH) ? 0 : islot + 1;
+  };
+  // weights depend on no earlier kernel: fill the ring before the dependency wait
+#pragma unroll
+  for (int i = 0; i < GT_DEPTH - 1; ++i) issue();
+  if (a.pf.units > 0 && warp == 0) prefetch_next_rows(a.pf, lane);
+  pdl_trigger();
+  pdl_wait();
+
+  // ---- activations -> shared memory as bf16 (RMSNorm here if a gain is given); each value is read once
+  for (int b = 0; b < nb; ++b) {
+    if (a.x_f32) {
+      const float* x = a.x_f32 + (size_t)b * K;
+      const bool cached = K <= GT_XR * GT_THREADS;
+      float xv[GT_XR];
+      float ss = 0.f;
+      if (cached) {
+#pragma unroll
+        for (int i = 0; i < GT_XR; ++i) {
+          const int k = tid + i * GT_THREADS;
+          xv[i] = k < K ? x[k] : 0.f;
+          ss += xv[i] * xv[i];
+        }
+      } else {
+        for (int k = tid; k < K; k += GT_THREADS) { const float v = x[k]; ss += v * v; }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+      __syncthreads();
+      if (lane == 0) red[warp] = ss;
+      __syncthreads();
+      float t = 0.f;
+#pragma unroll
+      for (int w = 0; w < GT_WARPS; ++w) t += red[w];
+      const float r = rsqrtf(t / (float)K + a.eps);
+      if (cached) {
+#pragma unroll
+        for (int i = 0; i < GT_XR; ++i) {
+          const int k = tid + i * GT_THREADS;
+          if (k < K) xs[(size_t)b * K + k] = __float2bfloat16(xv[i] * r * bf2f(a.gain[k]));
+        }
+      } else {
+        for (int k = tid; k < K; k += GT_THREADS) xs[(size_t)b * K + k] = __float2bfloat16(x[k] * r * bf2f(a.gain[k]));
+      }
+    } else {
+      const uint4* src = reinterpret_cast<const uint4*>(a.x_bf16 + (size_t)b * K);
+      uint4* dst = reinterpret_cast<uint4*>(xs + (size_t)b * K);
+      for (int c = tid; c < K / 8; c += GT_THREADS) dst[c] = src[c];
+    }
+  }
+  __syncthreads();
+
+  // ---- consume side
+  const int col_n = lane >> 2;                                         // B column (sequence) this lane feeds
+  const unsigned* xw = reinterpret_cast<const unsigned*>(xs + (size_t)min(col_n, max(nb - 1, 0)) * K) + (lane & 3);
+  const bool col_live = col_n < nb;
+  int cslot = 0;
+  for (int g = 0; g < n_groups; ++g) {
+    float c[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int j = 0; j < ns_w; ++j) {
+      issue();
+      cp_async_wait<GT_DEPTH - 1>();                                   // this lane's copies of the oldest item have landed
+      __syncwarp();                                                    // ... and so have the other lanes'
+      const unsigned slotp = ring_w + (unsigned)cslot * GT_SLOT_BYTES;
+      const int k0 = (warp + GT_WARPS * j) * 64;
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk) {
+        unsigned af[4];
+        const int row = lane & 15, kc = 2 * kk + (lane >> 4);
+        ldmatrix_x4(slotp + (unsigned)(row * 128 + ((kc ^ (row & 7)) << 4)), af);
+        unsigned b0 = 0u, b1 = 0u;
+        if (col_live) { b0 = xw[(k0 + kk * 16) / 2]; b1 = xw[(k0 + kk * 16) / 2 + 4]; }
+        mma_16816(c, af, b0, b1);
+      }
+      __syncwarp();                                                    // every lane has read the slot before it is refilled
+      cslot = (cslot + 1 == GT_DEPTH) ? 0 : cslot + 1;
+    }
+    *reinterpret_cast<float4*>(part + ((size_t)((g & 1) * GT_WARPS + warp) * 32 + lane) * 4) = make_float4(c[0], c[1], c[2], c[3]);
+    // The barrier that ends the next group also orders these reads before that half of `part` is rewritten.
+    __syncthreads();
+    if (tid < 64) {
+      const int uu = tid >> 3, col = tid & 7;
+      if (col < nb && g * 8 + uu < n_local) {
+        const float* src = part + ((size_t)(g & 1) * GT_WARPS * 32 + (uu * 4 + (col >> 1))) * 4 + (col & 1);
+        float ya = 0.f, yb = 0.f;
+#pragma unroll
+        for (int w = 0; w < GT_WARPS; ++w) { ya += src[(size_t)w * 32 * 4]; yb += src[(size_t)w * 32 * 4 + 2]; }
+        const UnitRows cu = unit_rows(a, u_begin + g * 8 + uu);
+        store_unit(a, cu, col, ya, yb);
+      }
+    }
+  }
 }
 
 // Attention of one new row per sequence over the cache (Sec. 3.1): one CTA per (head, sequence).
@@ -476,6 +696,13 @@ __global__ void argmax_final_kernel(const unsigned long long* tmp, int n_part, i
   }
 }
 
+constexpr size_t GT_SMEM_MAX = 226 * 1024;      // dynamic part; the kernel also has a little static shared memory
+size_t gt_smem_bytes(const vlac_ctx* ctx, const GemvArgs& a) {
+  const int n_units = a.mode == GV_QKV ? 3 * (a.N / 2) : (a.mode == GV_SWIGLU ? a.N : (a.N + 1) / 2);
+  const int n_tab = ((n_units + ctx->n_sm - 1) / ctx->n_sm + 7) / 8 * 8;
+  return (size_t)GT_RING_BYTES + GT_PART_BYTES + (size_t)n_tab * 16 + (size_t)a.nb * a.K * sizeof(bf16);
+}
+
 int launch_gemv(vlac_ctx* ctx, const GemvArgs& a, cudaStream_t s) {
   const int nb = a.nb;
   const int NB = nb <= 1 ? 1 : (nb <= 2 ? 2 : (nb <= 4 ? 4 : 8));
@@ -483,6 +710,10 @@ int launch_gemv(vlac_ctx* ctx, const GemvArgs& a, cudaStream_t s) {
   const int grid = ctx->n_sm * GV_CTAS_PER_SM;
   const bool timed = ctx->prof_on && ctx->prof_n < VLAC_PROF_CAP;
   if (timed) VLAC_CUDA_CHECK(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n], s));
+  const size_t gt_smem = gt_smem_bytes(ctx, a);
+  if (ctx->gemv_stream && a.K % 64 == 0 && nb <= 8 && gt_smem <= GT_SMEM_MAX) {
+    VLAC_CUDA_CHECK(launch_pdl(gemv_mma_kernel, dim3(ctx->n_sm), dim3(GT_THREADS), gt_smem, s, a));
+  } else
   switch (NB) {
     case 1: VLAC_CUDA_CHECK(launch_pdl(gemv_pair_kernel<1>, dim3(grid), dim3(256), smem, s, a)); break;
     case 2: VLAC_CUDA_CHECK(launch_pdl(gemv_pair_kernel<2>, dim3(grid), dim3(256), smem, s, a)); break;
@@ -513,6 +744,14 @@ int vlac_decode_setup(vlac_ctx* ctx) {
   if (NB >= 2) VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_pair_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * (size_t)kmax * 2)));
   if (NB >= 4) VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_pair_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(4 * (size_t)kmax * 2)));
   if (NB >= 8) VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_pair_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(8 * (size_t)kmax * 2)));
+  // tensor-core variant of the weight-streaming kernel (VLAC_GEMV_REG=1 keeps the register-pipelined one)
+  ctx->gemv_stream = getenv("VLAC_GEMV_REG") ? 0 : 1;
+  VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GT_SMEM_MAX));
+  // Cross-kernel L2 requests of the single-row kernels (VLAC_PF_KB=0 turns them off).
+  ctx->pf_kb = 0; ctx->pf_frac = 0.5f;
+  if (const char* e = getenv("VLAC_PF_KB")) ctx->pf_kb = atoi(e);
+  if (const char* e = getenv("VLAC_PF_FRAC")) ctx->pf_frac = (float)atof(e);
+  if (ctx->pf_kb < 0) ctx->pf_kb = 0;
   // persistent pass kernel: as many CTAs as are guaranteed co-resident
   ctx->pass_grid = 0;
   // Opt-in (VLAC_PASS_KERNEL=1): measured on B200 it streams at 5.5 TB/s between barriers but its five grid
@@ -569,6 +808,25 @@ static void layer_phases(vlac_ctx* ctx, vlac_cache* c, int l, int pos, GemvArgs*
   GemvArgs dn = {};
   dn.x_bf16 = ctx->hm_dec; dn.w0 = (const bf16*)w.w_down; dn.mode = GV_RESID; dn.nb = B; dn.K = F; dn.N = D; dn.x_out = ctx->x_dec; dn.d = g.head_dim;
   out[0] = a; out[1] = o; out[2] = gu; out[3] = dn;
+}
+
+static GemvArgs logits_phase(vlac_ctx* ctx, vlac_cache* c) {
+  const vlac_config& g = ctx->cfg;
+  GemvArgs a = {};
+  a.x_f32 = ctx->x_dec; a.gain = (const bf16*)ctx->w.g_final; a.eps = g.rms_eps;
+  a.w0 = (const bf16*)ctx->w.lm_head; a.mode = GV_LOGITS; a.nb = c->batch; a.K = g.hidden; a.N = g.vocab; a.logits = ctx->logits; a.d = g.head_dim;
+  return a;
+}
+
+// `cur` asks the L2 for the first rows `next` will read.
+static void chain_prefetch(const vlac_ctx* ctx, GemvArgs& cur, const GemvArgs& next) {
+  if (ctx->pf_kb <= 0) return;
+  PfArgs f;
+  f.w0 = next.w0; f.w1 = next.w1; f.w2 = next.w2; f.mode = next.mode; f.K = next.K; f.N = next.N; f.d = next.d;
+  const size_t unit_bytes = 2 * (size_t)next.K * sizeof(bf16);
+  f.units = (int)(((size_t)ctx->pf_kb * 1024 + unit_bytes - 1) / unit_bytes);
+  f.frac = ctx->pf_frac;
+  cur.pf = f;
 }
 
 static size_t pass_smem(const vlac_ctx* ctx, int NB) {
@@ -637,8 +895,14 @@ int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens,
   }
   // one kernel per phase (also the path that per-launch timing brackets)
   for (int l = 0; l < g.n_layers; ++l) {
-    GemvArgs ph[4];
+    GemvArgs ph[4], nx[4];
     layer_phases(ctx, c, l, pos, ph);
+    if (l + 1 < g.n_layers) layer_phases(ctx, c, l + 1, pos, nx);
+    else nx[0] = logits_phase(ctx, c);
+    chain_prefetch(ctx, ph[0], ph[1]);
+    chain_prefetch(ctx, ph[1], ph[2]);
+    chain_prefetch(ctx, ph[2], ph[3]);
+    chain_prefetch(ctx, ph[3], nx[0]);
     int rc = launch_gemv(ctx, ph[0], s);
     if (rc) return rc;
     {
@@ -664,12 +928,15 @@ int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens,
 }
 
 int vlac_launch_logits_argmax(vlac_ctx* ctx, vlac_cache* c, int* tokens_out, int tok_stride, int tok_index,
-                              float* logits_copy, long long copy_stride, cudaStream_t s) {
+                              float* logits_copy, long long copy_stride, int next_pos, cudaStream_t s) {
   const vlac_config& g = ctx->cfg;
   const int B = c->batch;
-  GemvArgs a = {};
-  a.x_f32 = ctx->x_dec; a.gain = (const bf16*)ctx->w.g_final; a.eps = g.rms_eps;
-  a.w0 = (const bf16*)ctx->w.lm_head; a.mode = GV_LOGITS; a.nb = B; a.K = g.hidden; a.N = g.vocab; a.logits = ctx->logits; a.d = g.head_dim;
+  GemvArgs a = logits_phase(ctx, c);
+  if (next_pos >= 0 && g.n_layers > 0) {
+    GemvArgs nx[4];
+    layer_phases(ctx, c, 0, next_pos, nx);
+    chain_prefetch(ctx, a, nx[0]);
+  }
   int rc = launch_gemv(ctx, a, s);
   if (rc) return rc;
   VLAC_CUDA_CHECK(launch_pdl(argmax_partial_kernel, dim3(VLAC_ARGMAX_BLOCKS, B), dim3(256), 0, s, (const float*)ctx->logits, g.vocab,
