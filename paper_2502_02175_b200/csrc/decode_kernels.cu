@@ -16,15 +16,6 @@ __device__ __forceinline__ float bf2f(bf16 x) { return __bfloat162float(x); }
 
 enum { GV_QKV = 0, GV_RESID = 1, GV_SWIGLU = 2, GV_LOGITS = 3 };
 
-// Head of the weights the NEXT matrix-vector kernel on the stream will read: this kernel asks the L2 for
-// them while it is still streaming its own, so HBM stays busy across the kernel boundary.
-struct PfArgs {
-  const bf16 *w0, *w1, *w2;
-  int mode, K, N, d;
-  int units;               // units (row pairs) per CTA to request; 0: none
-  float frac;              // request them once this fraction of the CTA's own units has been handed out
-};
-
 struct GemvArgs {
   const float* x_f32;      // [nb][K] fp32 source (normalised with `gain`), or NULL
   const bf16* x_bf16;      // [nb][K] bf16 source used as is, or NULL
@@ -40,7 +31,6 @@ struct GemvArgs {
   float* x_out;            // RESID: [nb][N] +=
   bf16* h_out;             // SWIGLU: [nb][N]
   float* logits;           // LOGITS: [nb][N]
-  PfArgs pf;
 };
 
 __device__ __forceinline__ void fma8(float& acc, const uint4& w, const uint4& x) {
@@ -128,21 +118,6 @@ __device__ __forceinline__ int unit_count(int mode, int N) {
   return (N + 1) / 2;
 }
 
-// One warp asks the L2 for the rows of the first `f.units` units that the CTA of the same index will own in
-// the next kernel (same grid size).  A hint only: nothing waits for it and nothing depends on it.
-__device__ __noinline__ void prefetch_next_rows(PfArgs f, int lane) {
-  const int nu = unit_count(f.mode, f.N);
-  const int ub = (int)(((long long)nu * blockIdx.x) / gridDim.x);
-  const int nloc = (int)(((long long)nu * (blockIdx.x + 1)) / gridDim.x) - ub;
-  const int cnt = min(f.units, nloc);
-  const unsigned bytes = (unsigned)f.K * (unsigned)sizeof(bf16);
-  for (int i = lane; i < 2 * cnt; i += 32) {
-    const UnitRows r = unit_rows(f, ub + (i >> 1));
-    const uint4* p = (i & 1) ? r.pb : r.pa;
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
-  }
-}
-
 __device__ __forceinline__ void load_batch(uint4* va, uint4* vb, const UnitRows& r, int c0, int nchunk) {
 #pragma unroll
   for (int t = 0; t < GV_BATCH; ++t) {
@@ -173,12 +148,6 @@ __device__ __forceinline__ void gemv_body(const GemvArgs& a, unsigned char* smem
   int u_ld = warp < n_local ? warp : -1;                    // unit (local index) whose batch is in va, vb
   UnitRows ld_unit = unit_rows(a, u_begin + max(u_ld, 0));
   if (u_ld >= 0) load_batch(va, vb, ld_unit, lane, nchunk);
-  // ticket at which the next kernel's first rows are requested; a CTA with no tickets to draw asks now
-  int pf_at = -1;
-  if (a.pf.units > 0) {
-    pf_at = max(8, (int)((float)n_local * a.pf.frac));
-    if (pf_at >= n_local) { pf_at = -1; if (warp == 0) prefetch_next_rows(a.pf, lane); }
-  }
   wait();
 
   // ---- activations -> shared memory (RMSNorm here if a gain is given)
@@ -223,7 +192,6 @@ __device__ __forceinline__ void gemv_body(const GemvArgs& a, unsigned char* smem
       int t = 0;
       if (lane == 0) t = atomicAdd(next_unit, 1);
       t = __shfl_sync(0xffffffffu, t, 0);
-      if (t == pf_at) prefetch_next_rows(a.pf, lane);
       u_nx = t < n_local ? t : -1;
       bi_nx = 0;
     }
@@ -289,15 +257,28 @@ __global__ void __launch_bounds__(256, GV_CTAS_PER_SM) gemv_pair_kernel(GemvArgs
 // sub-stages dealt round-robin, so every warp streams the same share of every row and the CTA reads each
 // row front to back.  A warp copies a sub-stage (16 rows x 128 B, XOR-swizzled by row) with 16-byte
 // asynchronous copies into its own ring of GT_DEPTH slots and consumes it with ldmatrix; only warp-level
-// synchronisation guards the ring.  At the end of a group the 16 partial accumulator tiles meet in shared
-// memory and are added in warp order (bit-reproducible); one barrier per group, partials double-buffered.
-constexpr int GT_THREADS = 512;
+// synchronisation guards the ring.  At the end of a group each warp leaves its partial accumulator tile in
+// shared memory; after a round of groups (8 for one sequence) one barrier lets the threads add the 16 tiles
+// in warp order (bit-reproducible) and run the epilogue.  Partials are double-buffered by round.
+#ifndef GT_THREADS_N
+#define GT_THREADS_N 512
+#endif
+#ifndef GT_DEPTH_N
+#define GT_DEPTH_N 4
+#endif
+#ifndef GT_GRID_PER_SM
+#define GT_GRID_PER_SM 1
+#endif
+#ifndef GT_MIN_CTAS
+#define GT_MIN_CTAS 1
+#endif
+constexpr int GT_THREADS = GT_THREADS_N;
 constexpr int GT_WARPS = GT_THREADS / 32;
-constexpr int GT_DEPTH = 5;
+constexpr int GT_DEPTH = GT_DEPTH_N;
 constexpr int GT_SLOT_BYTES = 16 * 128;
-constexpr int GT_RING_BYTES = GT_WARPS * GT_DEPTH * GT_SLOT_BYTES;      // 160 KB
-constexpr int GT_PART_BYTES = 2 * GT_WARPS * 32 * 4 * (int)sizeof(float);  // 16 KB
-constexpr int GT_XR = 24;                                               // activations a thread keeps while it normalises a row
+constexpr int GT_RING_BYTES = GT_WARPS * GT_DEPTH * GT_SLOT_BYTES;      // 128 KB
+constexpr int GT_PART_BYTES = 2 * 8 * GT_WARPS * 16 * (int)sizeof(float);  // partial tiles of two rounds: 16 KB
+constexpr int GT_XR = 8192 / GT_THREADS_N;                                              // activations a thread keeps while it normalises a row
 
 __device__ __forceinline__ void cp_async16(unsigned smem_dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(src) : "memory");
@@ -313,7 +294,7 @@ __device__ __forceinline__ void mma_16816(float* c, const unsigned* a, unsigned 
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-__global__ void __launch_bounds__(GT_THREADS, 1) gemv_mma_kernel(GemvArgs a) {
+__global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvArgs a) {
   extern __shared__ __align__(128) unsigned char gt_smem[];
   __shared__ float red[GT_WARPS];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -324,7 +305,7 @@ __global__ void __launch_bounds__(GT_THREADS, 1) gemv_mma_kernel(GemvArgs a) {
   const int n_groups = (n_local + 7) / 8;
   const int n_tab = ((n_units + (int)gridDim.x - 1) / (int)gridDim.x + 7) / 8 * 8;     // same for every CTA: sizes the table
   const unsigned ring_w = (unsigned)__cvta_generic_to_shared(gt_smem) + (unsigned)warp * (GT_DEPTH * GT_SLOT_BYTES);
-  float* part = reinterpret_cast<float*>(gt_smem + GT_RING_BYTES);                      // [2][GT_WARPS][32][4]
+  float* part = reinterpret_cast<float*>(gt_smem + GT_RING_BYTES);                      // [2][G][GT_WARPS][16][nbp], G * nbp = 8
   const uint4** tab = reinterpret_cast<const uint4**>(gt_smem + GT_RING_BYTES + GT_PART_BYTES);   // [n_tab][2] row pointers
   bf16* xs = reinterpret_cast<bf16*>(gt_smem + GT_RING_BYTES + GT_PART_BYTES + (size_t)n_tab * 16);  // [nb][K]
 
@@ -368,8 +349,7 @@ __global__ void __launch_bounds__(GT_THREADS, 1) gemv_mma_kernel(GemvArgs a) {
   };
   // weights depend on no earlier kernel: fill the ring before the dependency wait
 #pragma unroll
-  for (int i = 0; i < GT_DEPTH - 1; ++i) issue();
-  if (a.pf.units > 0 && warp == 0) prefetch_next_rows(a.pf, lane);
+  for (int i = 0; i < GT_DEPTH; ++i) issue();
   pdl_trigger();
   pdl_wait();
 
@@ -420,11 +400,13 @@ __global__ void __launch_bounds__(GT_THREADS, 1) gemv_mma_kernel(GemvArgs a) {
   const int col_n = lane >> 2;                                         // B column (sequence) this lane feeds
   const unsigned* xw = reinterpret_cast<const unsigned*>(xs + (size_t)min(col_n, max(nb - 1, 0)) * K) + (lane & 3);
   const bool col_live = col_n < nb;
+  // Partial tiles of G groups are collected before the CTA meets at a barrier: part[2][G][warp][16 rows][nbp]
+  const int nbp = nb <= 1 ? 1 : (nb <= 2 ? 2 : (nb <= 4 ? 4 : 8));
+  const int G = 8 / nbp;
   int cslot = 0;
   for (int g = 0; g < n_groups; ++g) {
     float c[4] = {0.f, 0.f, 0.f, 0.f};
     for (int j = 0; j < ns_w; ++j) {
-      issue();
       cp_async_wait<GT_DEPTH - 1>();                                   // this lane's copies of the oldest item have landed
       __syncwarp();                                                    // ... and so have the other lanes'
       const unsigned slotp = ring_w + (unsigned)cslot * GT_SLOT_BYTES;
@@ -438,20 +420,32 @@ __global__ void __launch_bounds__(GT_THREADS, 1) gemv_mma_kernel(GemvArgs a) {
         if (col_live) { b0 = xw[(k0 + kk * 16) / 2]; b1 = xw[(k0 + kk * 16) / 2 + 4]; }
         mma_16816(c, af, b0, b1);
       }
-      __syncwarp();                                                    // every lane has read the slot before it is refilled
+      __syncwarp();                                                    // every lane has read the slot: refill it
+      issue();
       cslot = (cslot + 1 == GT_DEPTH) ? 0 : cslot + 1;
     }
-    *reinterpret_cast<float4*>(part + ((size_t)((g & 1) * GT_WARPS + warp) * 32 + lane) * 4) = make_float4(c[0], c[1], c[2], c[3]);
-    // The barrier that ends the next group also orders these reads before that half of `part` is rewritten.
-    __syncthreads();
-    if (tid < 64) {
-      const int uu = tid >> 3, col = tid & 7;
-      if (col < nb && g * 8 + uu < n_local) {
-        const float* src = part + ((size_t)(g & 1) * GT_WARPS * 32 + (uu * 4 + (col >> 1))) * 4 + (col & 1);
+    const int round = g / G, gr = g - round * G;
+    {
+      float* dst = part + ((size_t)(((round & 1) * G + gr) * GT_WARPS + warp) * 16) * nbp;
+      const int r = lane >> 2, n0 = (lane & 3) * 2;
+      if (n0 < nb) { dst[r * nbp + n0] = c[0]; dst[(r + 8) * nbp + n0] = c[2]; }
+      if (n0 + 1 < nb) { dst[r * nbp + n0 + 1] = c[1]; dst[(r + 8) * nbp + n0 + 1] = c[3]; }
+    }
+    if (gr == G - 1 || g == n_groups - 1) {
+      // End of a round: add the warps' partial tiles in warp order and finish these units.  The other half of
+      // `part` takes the next round; the barrier that ends it also orders these reads before this half is reused.
+      __syncthreads();
+      const int n_items = (gr + 1) * 8 * nb;
+      for (int idx = tid; idx < n_items; idx += GT_THREADS) {
+        const int gi = idx / (8 * nb), rem = idx - gi * 8 * nb;
+        const int uu = rem / nb, col = rem - uu * nb;
+        const int ul = (round * G + gi) * 8 + uu;
+        if (ul >= n_local) continue;
+        const float* src = part + ((size_t)(((round & 1) * G + gi) * GT_WARPS) * 16) * nbp;
         float ya = 0.f, yb = 0.f;
 #pragma unroll
-        for (int w = 0; w < GT_WARPS; ++w) { ya += src[(size_t)w * 32 * 4]; yb += src[(size_t)w * 32 * 4 + 2]; }
-        const UnitRows cu = unit_rows(a, u_begin + g * 8 + uu);
+        for (int w = 0; w < GT_WARPS; ++w) { ya += src[((size_t)w * 16 + uu) * nbp + col]; yb += src[((size_t)w * 16 + uu + 8) * nbp + col]; }
+        const UnitRows cu = unit_rows(a, u_begin + ul);
         store_unit(a, cu, col, ya, yb);
       }
     }
@@ -699,7 +693,8 @@ __global__ void argmax_final_kernel(const unsigned long long* tmp, int n_part, i
 constexpr size_t GT_SMEM_MAX = 226 * 1024;      // dynamic part; the kernel also has a little static shared memory
 size_t gt_smem_bytes(const vlac_ctx* ctx, const GemvArgs& a) {
   const int n_units = a.mode == GV_QKV ? 3 * (a.N / 2) : (a.mode == GV_SWIGLU ? a.N : (a.N + 1) / 2);
-  const int n_tab = ((n_units + ctx->n_sm - 1) / ctx->n_sm + 7) / 8 * 8;
+  const int grid = ctx->n_sm * GT_GRID_PER_SM;
+  const int n_tab = ((n_units + grid - 1) / grid + 7) / 8 * 8;
   return (size_t)GT_RING_BYTES + GT_PART_BYTES + (size_t)n_tab * 16 + (size_t)a.nb * a.K * sizeof(bf16);
 }
 
@@ -712,7 +707,7 @@ int launch_gemv(vlac_ctx* ctx, const GemvArgs& a, cudaStream_t s) {
   if (timed) VLAC_CUDA_CHECK(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n], s));
   const size_t gt_smem = gt_smem_bytes(ctx, a);
   if (ctx->gemv_stream && a.K % 64 == 0 && nb <= 8 && gt_smem <= GT_SMEM_MAX) {
-    VLAC_CUDA_CHECK(launch_pdl(gemv_mma_kernel, dim3(ctx->n_sm), dim3(GT_THREADS), gt_smem, s, a));
+    VLAC_CUDA_CHECK(launch_pdl(gemv_mma_kernel, dim3(ctx->n_sm * GT_GRID_PER_SM), dim3(GT_THREADS), gt_smem, s, a));
   } else
   switch (NB) {
     case 1: VLAC_CUDA_CHECK(launch_pdl(gemv_pair_kernel<1>, dim3(grid), dim3(256), smem, s, a)); break;
@@ -747,11 +742,6 @@ int vlac_decode_setup(vlac_ctx* ctx) {
   // tensor-core variant of the weight-streaming kernel (VLAC_GEMV_REG=1 keeps the register-pipelined one)
   ctx->gemv_stream = getenv("VLAC_GEMV_REG") ? 0 : 1;
   VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GT_SMEM_MAX));
-  // Cross-kernel L2 requests of the single-row kernels (VLAC_PF_KB=0 turns them off).
-  ctx->pf_kb = 0; ctx->pf_frac = 0.5f;
-  if (const char* e = getenv("VLAC_PF_KB")) ctx->pf_kb = atoi(e);
-  if (const char* e = getenv("VLAC_PF_FRAC")) ctx->pf_frac = (float)atof(e);
-  if (ctx->pf_kb < 0) ctx->pf_kb = 0;
   // persistent pass kernel: as many CTAs as are guaranteed co-resident
   ctx->pass_grid = 0;
   // Opt-in (VLAC_PASS_KERNEL=1): measured on B200 it streams at 5.5 TB/s between barriers but its five grid
@@ -816,17 +806,6 @@ static GemvArgs logits_phase(vlac_ctx* ctx, vlac_cache* c) {
   a.x_f32 = ctx->x_dec; a.gain = (const bf16*)ctx->w.g_final; a.eps = g.rms_eps;
   a.w0 = (const bf16*)ctx->w.lm_head; a.mode = GV_LOGITS; a.nb = c->batch; a.K = g.hidden; a.N = g.vocab; a.logits = ctx->logits; a.d = g.head_dim;
   return a;
-}
-
-// `cur` asks the L2 for the first rows `next` will read.
-static void chain_prefetch(const vlac_ctx* ctx, GemvArgs& cur, const GemvArgs& next) {
-  if (ctx->pf_kb <= 0) return;
-  PfArgs f;
-  f.w0 = next.w0; f.w1 = next.w1; f.w2 = next.w2; f.mode = next.mode; f.K = next.K; f.N = next.N; f.d = next.d;
-  const size_t unit_bytes = 2 * (size_t)next.K * sizeof(bf16);
-  f.units = (int)(((size_t)ctx->pf_kb * 1024 + unit_bytes - 1) / unit_bytes);
-  f.frac = ctx->pf_frac;
-  cur.pf = f;
 }
 
 static size_t pass_smem(const vlac_ctx* ctx, int NB) {
@@ -895,14 +874,8 @@ int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens,
   }
   // one kernel per phase (also the path that per-launch timing brackets)
   for (int l = 0; l < g.n_layers; ++l) {
-    GemvArgs ph[4], nx[4];
+    GemvArgs ph[4];
     layer_phases(ctx, c, l, pos, ph);
-    if (l + 1 < g.n_layers) layer_phases(ctx, c, l + 1, pos, nx);
-    else nx[0] = logits_phase(ctx, c);
-    chain_prefetch(ctx, ph[0], ph[1]);
-    chain_prefetch(ctx, ph[1], ph[2]);
-    chain_prefetch(ctx, ph[2], ph[3]);
-    chain_prefetch(ctx, ph[3], nx[0]);
     int rc = launch_gemv(ctx, ph[0], s);
     if (rc) return rc;
     {
@@ -928,15 +901,10 @@ int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens,
 }
 
 int vlac_launch_logits_argmax(vlac_ctx* ctx, vlac_cache* c, int* tokens_out, int tok_stride, int tok_index,
-                              float* logits_copy, long long copy_stride, int next_pos, cudaStream_t s) {
+                              float* logits_copy, long long copy_stride, cudaStream_t s) {
   const vlac_config& g = ctx->cfg;
   const int B = c->batch;
   GemvArgs a = logits_phase(ctx, c);
-  if (next_pos >= 0 && g.n_layers > 0) {
-    GemvArgs nx[4];
-    layer_phases(ctx, c, 0, next_pos, nx);
-    chain_prefetch(ctx, a, nx[0]);
-  }
   int rc = launch_gemv(ctx, a, s);
   if (rc) return rc;
   VLAC_CUDA_CHECK(launch_pdl(argmax_partial_kernel, dim3(VLAC_ARGMAX_BLOCKS, B), dim3(256), 0, s, (const float*)ctx->logits, g.vocab,

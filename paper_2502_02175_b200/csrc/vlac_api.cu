@@ -366,15 +366,14 @@ static int enqueue_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* f
   // 4. first action token
   TRY(vlac_launch_last_row(ctx, cache, h, s));
   const long long lstride = (long long)g.n_action * g.vocab;
-  TRY(vlac_launch_logits_argmax(ctx, cache, action_tokens, g.n_action, 0, all_logits, lstride, g.n_action > 1 ? ctx->L : -1, s));
+  TRY(vlac_launch_logits_argmax(ctx, cache, action_tokens, g.n_action, 0, all_logits, lstride, s));
   TRY(seg_mark(ctx, s));
   // 5. remaining tokens, one single-row pass each
   const int* fed = forced_tokens ? forced_tokens : action_tokens;
   for (int i = 1; i < g.n_action; ++i) {
     TRY(vlac_launch_decode_pass(ctx, cache, fed, g.n_action, i - 1, ctx->L - 1 + i, s));
     TRY(vlac_launch_logits_argmax(ctx, cache, action_tokens, g.n_action, i,
-                                  all_logits ? all_logits + (size_t)i * g.vocab : nullptr, lstride,
-                                  i + 1 < g.n_action ? ctx->L + i : -1, s));
+                                  all_logits ? all_logits + (size_t)i * g.vocab : nullptr, lstride, s));
     TRY(seg_mark(ctx, s));
   }
   // 6. this step becomes "previous"

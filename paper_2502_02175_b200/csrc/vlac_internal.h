@@ -66,8 +66,6 @@ struct vlac_ctx {
   int tc_ok;                         // 1: shapes fit the tensor-memory GEMM
   int pass_grid;                     // CTAs of the persistent single-row pass kernel (0: not used)
   int gemv_stream;                   // single-row products use the shared-memory-staged kernel
-  int pf_kb;                         // single-row kernels: KB of the next kernel's weights each CTA asks the L2 for (0: none)
-  float pf_frac;                     // ... once this fraction of its own work has been handed out
   void* tmap_q;                      // device tensor map of the query buffer (tiled attention)
   int attn_tiles;                    // 64-query tiles per sequence, 0: tiled attention not usable
   // optional per-launch timing of the matrix-vector kernel (vlac_profile)
@@ -141,7 +139,5 @@ int vlac_decode_cache_setup(vlac_ctx* ctx, vlac_cache* c);
 int vlac_launch_last_row(vlac_ctx* ctx, vlac_cache* c, const bf16* hidden, cudaStream_t s);
 int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens, int tok_stride, int tok_index,
                             int pos, cudaStream_t s);
-// next_pos: position of the single-row pass that follows on the stream (its first weights are requested
-// ahead of time), or -1 if none does.
 int vlac_launch_logits_argmax(vlac_ctx* ctx, vlac_cache* c, int* tokens_out, int tok_stride, int tok_index,
-                              float* logits_copy, long long copy_stride, int next_pos, cudaStream_t s);
+                              float* logits_copy, long long copy_stride, cudaStream_t s);
