@@ -9,10 +9,12 @@
 // memory (the selection kernels wrote it); the instruction descriptor and the number of token boxes
 // are formed in the kernel, so no host round trip is needed.
 //
-// Warp roles (192 threads): warp 0 issues TMA loads into a ring of stages, warp 1 allocates TMEM and
-// issues the MMAs, warps 2-5 read the accumulator back (each its own quarter of the 128 lanes) and run
-// the epilogue.  Few, large TMA boxes are used (one 128-row box of weights, one box of up to 256 token
-// rows per k-block): the TMA unit works through requests one at a time, so many small boxes starve it.
+// Warp roles (256 threads): one lane each of warps 0, 6 and 7 issues TMA loads into a ring of stages (the
+// k-blocks dealt round-robin: a thread gets a tensor load accepted only every ~0.3 us whatever its size,
+// but threads of different warps are served in parallel), warp 1 allocates TMEM and issues the MMAs.  When
+// the accumulator is complete all eight warps read it back (two teams of four, one warp per quarter of
+// the 128 lanes, alternating 16-token chunks) and run the epilogue.  Few, large TMA boxes are used (one
+// 128-row box of weights, one box of up to 256 token rows per k-block).
 // Epilogues:
 //   QKV     rotation at the row's own position, K/V scatter into the cache, Q to the compact buffer;
 //           the two halves of a rotary pair sit in different warps and are exchanged through shared memory
@@ -28,13 +30,14 @@
 namespace {
 
 constexpr int TG_QKV = 0, TG_PARTIAL = 1, TG_SWIGLU = 2;
-constexpr int TG_THREADS = 192;
+constexpr int TG_THREADS = 256;
+constexpr int TG_PRODUCERS = 3;                // warps 0, 6, 7: one elected lane each issues TMA loads
 constexpr int TG_BK = 64;                       // bf16 elements per k-block = one 128-byte swizzle row
 constexpr int TG_A_BYTES = 128 * TG_BK * 2;     // 16 KB: 128 weight rows
 constexpr int TG_BOX_TOK = 64;                  // token rows per TMA box
 constexpr int TG_BOX_BYTES = TG_BOX_TOK * TG_BK * 2;   // 8 KB
 constexpr int TG_MAX_STAGES = 8;
-constexpr int TG_SMEM_RING = 208 * 1024;        // dynamic shared memory for the ring
+constexpr int TG_SMEM_RING = 192 * 1024;        // dynamic shared memory for the ring (four stages of 48 KB at up to 256 tokens)
 constexpr unsigned long long TG_WAIT_LIMIT_NS = 400000000ull;
 
 struct alignas(64) TcArgs {
@@ -132,7 +135,7 @@ __device__ __forceinline__ void tmem_ld16(unsigned taddr, float* v) {
 __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_constant__ TcArgs a) {
   extern __shared__ __align__(1024) unsigned char ring_raw[];
   __shared__ __align__(8) unsigned long long full_bar[TG_MAX_STAGES], empty_bar[TG_MAX_STAGES], acc_bar;
-  __shared__ float xch[2][4][16][32];                            // epilogue exchange between warp pairs (double-buffered)
+  __shared__ float xch[2][2][4][16][32];                         // epilogue exchange between warp pairs: [team][double buffer]
   __shared__ unsigned tmem_base_slot;
   __shared__ int abort_flag;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -183,11 +186,18 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const unsigned tmem_base = tmem_base_slot;
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+  if (warp == 0 || warp >= 6) {
+    // ------------------------------------------------------------------ TMA producers
+    // A thread gets a tensor load accepted only every ~0.3 us whatever the box size, but threads of
+    // different warps are served in parallel: the k-blocks are dealt round-robin to three producer lanes.
+    // Each producer waits for the ring slot of its own k-blocks only.  Its previous wait proved k-block
+    // i - P - n_stages consumed; the slot's previous phase (k-block i - 2 n_stages) must be complete by
+    // then, or the one-bit phase parity would alias: hence no more producers than stages.
+    const int n_prod = min(TG_PRODUCERS, n_stages);
+    const int pid = warp == 0 ? 0 : warp - 5;
+    if (lane == 0 && pid < n_prod) {
       const int rows0 = min(n_boxes, 4), rows1 = n_boxes - rows0;            // boxes of the first / second token request
-      for (int i = 0; i < n_kb; ++i) {
+      for (int i = pid; i < n_kb; i += n_prod) {
         const int s = i % n_stages;
         if (i >= n_stages && !mbar_wait(&empty_bar[s], ((i / n_stages) & 1) ^ 1, &abort_flag, a.dev_error, 0x40000 | (i & 0xffff))) break;
         unsigned char* sa = ring + (size_t)s * stage_bytes;
@@ -229,8 +239,13 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
       }
       if (ok) umma_commit(&acc_bar);                             // accumulator complete
     }
-  } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5)
+  }
+  __syncwarp();
+  {
+    // ------------------------------------------------------------------ epilogue (all eight warps)
+    // Once their loops are done the producer and MMA warps join: two teams of four warps (one warp per
+    // quarter of the 128 accumulator lanes in each) take the 16-token chunks alternately.
+    const int team = (warp >= 2 && warp <= 5) ? 0 : 1;
     const int q = warp & 3;                                      // TMEM lane quarter this warp may read
     bool ok = n_kb > 0;
     if (ok) ok = mbar_wait(&acc_bar, 0, &abort_flag, a.dev_error, 0x60000);
@@ -246,40 +261,45 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
     const bool exchange = (a.mode == TG_SWIGLU && !tail) || (a.mode == TG_QKV && mat < 2);
     const int j = (n % a.d) % half;
     const size_t N = (size_t)a.N;
-    // QKV: positions and rotary table entries of a 16-token chunk; fetched one chunk ahead of their use so
-    // that the table latency overlaps the previous chunk's exchange, arithmetic and stores
-    int bs[16], ps[16];
-    float cs[16], sn[16];
-    auto fetch_tables = [&](int c0, int* b_o, int* p_o, float* c_o, float* s_o) {
-      const int my_row = (c0 + (lane & 15) < tokens) ? __ldg(a.rowmap + tok0 + c0 + (lane & 15)) : 0;
-#pragma unroll
-      for (int c = 0; c < 16; ++c) {
-        const int row = __shfl_sync(0xffffffffu, my_row, c);
-        int b = 0, pos = row;
-        if (a.batch > 1) { b = row / a.L; pos = row - b * a.L; }
-        b_o[c] = b; p_o[c] = pos;
-        if (mat < 2) { c_o[c] = __ldg(a.rope_cos + (size_t)pos * half + j); s_o[c] = __ldg(a.rope_sin + (size_t)pos * half + j); }
-        else { c_o[c] = 1.f; s_o[c] = 0.f; }
+    // QKV: the ring is free once the accumulator is complete.  The row map of the tile's tokens and, for Q
+    // and K tiles, the rotary table rows of their positions are copied into it by all warps at once, so the
+    // chunk loop below reads them from shared memory instead of waiting on 32 global loads per chunk.
+    int* rows_s = reinterpret_cast<int*>(ring);                                  // [tokens]
+    float* tab_s = reinterpret_cast<float*>(ring + 2048);                        // [tokens][2 * half]: cos | sin
+    const bool staged = a.mode == TG_QKV && tokens > 0 &&
+                        (size_t)2048 + (size_t)tokens * 2 * half * sizeof(float) <= (size_t)TG_SMEM_RING && (half % 4) == 0;
+    if (staged) {                                                // uniform over the CTA
+      for (int t = tid; t < tokens; t += TG_THREADS) rows_s[t] = __ldg(a.rowmap + tok0 + t);
+      if (mat < 2) {
+        const int vec_per_tok = half / 2;                        // float4 per token: half/4 of cos, half/4 of sin
+        for (int idx = tid; idx < tokens * vec_per_tok; idx += TG_THREADS) {
+          const int t = idx / vec_per_tok, v = idx - t * vec_per_tok;
+          const int row = __ldg(a.rowmap + tok0 + t);
+          const int pos = a.batch > 1 ? row % a.L : row;
+          const float* src = (v < half / 4 ? a.rope_cos : a.rope_sin) + (size_t)pos * half + (size_t)(v % (half / 4)) * 4;
+          *reinterpret_cast<float4*>(tab_s + (size_t)t * 2 * half + (size_t)v * 4) = __ldg(reinterpret_cast<const float4*>(src));
+        }
       }
-    };
-    if (a.mode == TG_QKV && tokens > 0) fetch_tables(0, bs, ps, cs, sn);
+      __syncthreads();
+    }
+    const unsigned bar_id = 2u + (unsigned)team;
     int chunk = 0;
-    for (int c0 = 0; c0 < tokens; c0 += 16, ++chunk) {
+    for (int c0 = team * 16; c0 < tokens; c0 += 32, ++chunk) {
       float v[16], pv[16];
       if (ok) tmem_ld16(tmem_base + ((unsigned)(32 * q) << 16) + (unsigned)c0, v);
       else {
 #pragma unroll
         for (int c = 0; c < 16; ++c) v[c] = 0.f;
       }
-      if (exchange) {                                            // uniform over the four epilogue warps
-        float (*buf)[16][32] = xch[chunk & 1];
+      if (exchange) {                                            // uniform over the four warps of a team
+        float (*buf)[16][32] = xch[team][chunk & 1];
 #pragma unroll
         for (int c = 0; c < 16; ++c) buf[q][c][lane] = v[c];
-        asm volatile("bar.sync 2, 128;" ::: "memory");
+        asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
 #pragma unroll
         for (int c = 0; c < 16; ++c) pv[c] = buf[pq][c][lane];
       }
-      const bool live = ok && n_ok;                               // no early exit: the warp shuffles below need every lane
+      const bool live = ok && n_ok;
       if (tail) {
         if (!ok) continue;
         float* dst = a.tail_part + (size_t)split * a.tail_stride + (size_t)(tile - a.full_tiles) * 128 + r;
@@ -302,22 +322,22 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
           }
         }
       } else {                                                   // TG_QKV
-        int bn[16], pn[16];
-        float cn[16], sn2[16];
-        const bool more = c0 + 16 < tokens;                     // uniform: next chunk's tables requested before this chunk's stores
-        if (more) fetch_tables(c0 + 16, bn, pn, cn, sn2);
 #pragma unroll
         for (int c = 0; c < 16; ++c) {
           if (live && c0 + c < tokens) {
+            const int row = staged ? rows_s[c0 + c] : __ldg(a.rowmap + tok0 + c0 + c);
+            int b = 0, pos = row;
+            if (a.batch > 1) { b = row / a.L; pos = row - b * a.L; }
             float y = v[c];
-            if (mat < 2) y = first ? v[c] * cs[c] - pv[c] * sn[c] : v[c] * cs[c] + pv[c] * sn[c];
+            if (mat < 2) {
+              float cs, sn;
+              if (staged) { cs = tab_s[(size_t)(c0 + c) * 2 * half + j]; sn = tab_s[(size_t)(c0 + c) * 2 * half + half + j]; }
+              else { cs = __ldg(a.rope_cos + (size_t)pos * half + j); sn = __ldg(a.rope_sin + (size_t)pos * half + j); }
+              y = first ? v[c] * cs - pv[c] * sn : v[c] * cs + pv[c] * sn;
+            }
             if (mat == 0) a.q_out[(size_t)(tok0 + c0 + c) * N + n] = __float2bfloat16(y);
-            else (mat == 1 ? a.kc : a.vc)[((size_t)bs[c] * a.max_seq + ps[c]) * N + n] = __float2bfloat16(y);
+            else (mat == 1 ? a.kc : a.vc)[((size_t)b * a.max_seq + pos) * N + n] = __float2bfloat16(y);
           }
-        }
-        if (more) {
-#pragma unroll
-          for (int c = 0; c < 16; ++c) { bs[c] = bn[c]; ps[c] = pn[c]; cs[c] = cn[c]; sn[c] = sn2[c]; }
         }
       }
     }
