@@ -97,6 +97,17 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned pari
   if (dev_error) atomicCAS(dev_error, 0, code);
   return false;
 }
+__device__ __forceinline__ float lds_f32(unsigned addr) { float v; asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr)); return v; }
+__device__ __forceinline__ int lds_s32(unsigned addr) { int v; asm volatile("ld.shared.s32 %0, [%1];" : "=r"(v) : "r"(addr)); return v; }
+__device__ __forceinline__ uint4 lds_v4(unsigned addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void sts_f32(unsigned addr, float v) { asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory"); }
+__device__ __forceinline__ void sts_b16(unsigned addr, bf16 v) {
+  asm volatile("st.shared.b16 [%0], %1;" ::"r"(addr), "h"(*reinterpret_cast<unsigned short*>(&v)) : "memory");
+}
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, int x, int y, unsigned long long* bar) {
   asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                ::"r"(smem_u32(dst)), "l"(tm), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
@@ -140,7 +151,8 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
   __shared__ int abort_flag;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // the ring must start on a 1024-byte boundary (swizzle atoms); dynamic smem is over-allocated by 1 KB
-  unsigned char* ring = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(ring_raw) + 1023) & ~(uintptr_t)1023);
+  // (an offset from the array keeps the pointer in the shared address space for the compiler)
+  unsigned char* ring = ring_raw + ((1024u - (smem_u32(ring_raw) & 1023u)) & 1023u);
 
   int tile = blockIdx.x, split = blockIdx.y, splits = a.n_splits;
   bool tail = false;                                            // a K-split SWIGLU tile: epilogue stores raw sums
@@ -267,22 +279,45 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
     int* rows_s = reinterpret_cast<int*>(ring);                                  // [tokens]
     float* tab_s = reinterpret_cast<float*>(ring + 2048);                        // [tokens][2 * half]: cos | sin
     const bool staged = a.mode == TG_QKV && tokens > 0 &&
-                        (size_t)2048 + (size_t)tokens * 2 * half * sizeof(float) <= (size_t)TG_SMEM_RING && (half % 4) == 0;
+                        (size_t)2048 + (size_t)tokens * 2 * half * sizeof(float) <= (size_t)TG_SMEM_RING - 4 * 8192 && (half % 4) == 0;
     if (staged) {                                                // uniform over the CTA
       for (int t = tid; t < tokens; t += TG_THREADS) rows_s[t] = __ldg(a.rowmap + tok0 + t);
+      __syncthreads();
       if (mat < 2) {
         const int vec_per_tok = half / 2;                        // float4 per token: half/4 of cos, half/4 of sin
-        for (int idx = tid; idx < tokens * vec_per_tok; idx += TG_THREADS) {
-          const int t = idx / vec_per_tok, v = idx - t * vec_per_tok;
-          const int row = __ldg(a.rowmap + tok0 + t);
-          const int pos = a.batch > 1 ? row % a.L : row;
-          const float* src = (v < half / 4 ? a.rope_cos : a.rope_sin) + (size_t)pos * half + (size_t)(v % (half / 4)) * 4;
-          *reinterpret_cast<float4*>(tab_s + (size_t)t * 2 * half + (size_t)v * 4) = __ldg(reinterpret_cast<const float4*>(src));
+        const int total = tokens * vec_per_tok;
+        for (int base = tid; base < total; base += 8 * TG_THREADS) {             // eight independent loads in flight per thread
+          float4 tmp[8];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const int idx = min(base + u * TG_THREADS, total - 1);
+            const int t = idx / vec_per_tok, v = idx - t * vec_per_tok;
+            const int row = rows_s[t];
+            const int pos = a.batch > 1 ? row % a.L : row;
+            const float* src = (v < half / 4 ? a.rope_cos : a.rope_sin) + (size_t)pos * half + (size_t)(v % (half / 4)) * 4;
+            tmp[u] = __ldg(reinterpret_cast<const float4*>(src));
+          }
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+            const int idx = base + u * TG_THREADS;
+            if (idx < total) *reinterpret_cast<float4*>(tab_s + (size_t)idx * 4) = tmp[u];
+          }
         }
       }
       __syncthreads();
     }
     const unsigned bar_id = 2u + (unsigned)team;
+    // Results leave through shared memory: a team writes the 16 token rows of a chunk into its own buffer
+    // (end of the ring, double-buffered), meets at the team barrier and copies them out 16 bytes per thread,
+    // so that one store instruction of a warp carries 512 contiguous bytes instead of 64 or 128.  (The
+    // number of store requests an SM can have in flight, not their size, bounds the direct form.)
+    const int tteam = (q << 5) | lane;                            // thread index inside the team: also the tile row
+    const int out_cols = a.mode == TG_SWIGLU && !tail ? 64 : 128;
+    const int esz = (tail || a.mode == TG_PARTIAL) ? 4 : 2;       // fp32 partial sums, bf16 otherwise
+    const int row_bytes = out_cols * esz;
+    const bool vec_ok = (a.mode == TG_SWIGLU && !tail) ? (row_base + 64 <= a.N) : (tail ? true : (row_base + 128 <= a.N));
+    const unsigned out_base = smem_u32(ring) + (unsigned)TG_SMEM_RING - 4u * 8192u + (unsigned)team * 2u * 8192u;
+    const unsigned rows_a = smem_u32(rows_s), tab_a = smem_u32(tab_s) + (unsigned)j * 4u;
     int chunk = 0;
     for (int c0 = team * 16; c0 < tokens; c0 += 32, ++chunk) {
       float v[16], pv[16];
@@ -299,44 +334,90 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
 #pragma unroll
         for (int c = 0; c < 16; ++c) pv[c] = buf[pq][c][lane];
       }
-      const bool live = ok && n_ok;
-      if (tail) {
-        if (!ok) continue;
-        float* dst = a.tail_part + (size_t)split * a.tail_stride + (size_t)(tile - a.full_tiles) * 128 + r;
+      const unsigned out_a = out_base + (unsigned)(chunk & 1) * 8192u;
+      int rw[16];                                                // QKV: row map entries of the chunk's tokens
+      if (a.mode == TG_QKV) {
+        float cs[16], sn[16];
+        if (staged) {
 #pragma unroll
-        for (int c = 0; c < 16; ++c)
-          if (c0 + c < tokens) dst[(size_t)(tok0 + c0 + c) * a.tail_ld] = v[c];
-      } else if (a.mode == TG_PARTIAL) {
-        if (!live) continue;
-        float* dst = a.part + (size_t)split * a.split_stride + n;
+          for (int c = 0; c < 16; ++c) rw[c] = lds_s32(rows_a + (unsigned)min(c0 + c, tokens - 1) * 4u);
 #pragma unroll
-        for (int c = 0; c < 16; ++c)
-          if (c0 + c < tokens) dst[(size_t)(tok0 + c0 + c) * N] = v[c];
-      } else if (a.mode == TG_SWIGLU) {
+          for (int c = 0; c < 16; ++c) {
+            const unsigned ta = tab_a + (unsigned)min(c0 + c, tokens - 1) * (unsigned)(2 * half) * 4u;
+            if (mat < 2) { cs[c] = lds_f32(ta); sn[c] = lds_f32(ta + (unsigned)half * 4u); }
+            else { cs[c] = 1.f; sn[c] = 0.f; }
+          }
+        } else {
+#pragma unroll
+          for (int c = 0; c < 16; ++c) rw[c] = __ldg(a.rowmap + tok0 + min(c0 + c, tokens - 1));
+#pragma unroll
+          for (int c = 0; c < 16; ++c) {
+            const int pos = a.batch > 1 ? rw[c] % a.L : rw[c];
+            if (mat < 2) { cs[c] = __ldg(a.rope_cos + (size_t)pos * half + j); sn[c] = __ldg(a.rope_sin + (size_t)pos * half + j); }
+            else { cs[c] = 1.f; sn[c] = 0.f; }
+          }
+        }
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          float y = v[c];
+          if (mat < 2) y = first ? v[c] * cs[c] - pv[c] * sn[c] : v[c] * cs[c] + pv[c] * sn[c];
+          v[c] = y;
+        }
+      } else if (a.mode == TG_SWIGLU && !tail) {
         // gate-side threads finish even columns, up-side threads odd columns
 #pragma unroll
         for (int c = 0; c < 16; ++c) {
-          if (live && ((c & 1) == 0) == first && c0 + c < tokens) {
-            const float g = first ? v[c] : pv[c], u = first ? pv[c] : v[c];
-            a.h_out[(size_t)(tok0 + c0 + c) * N + n] = __float2bfloat16(__fdividef(g, 1.f + __expf(-g)) * u);
-          }
+          const float g = first ? v[c] : pv[c], u = first ? pv[c] : v[c];
+          v[c] = __fdividef(g, 1.f + __expf(-g)) * u;
         }
-      } else {                                                   // TG_QKV
+      }
+      if (vec_ok) {
+        // ---- rows of the chunk -> shared memory
+        if (esz == 4) {
 #pragma unroll
-        for (int c = 0; c < 16; ++c) {
-          if (live && c0 + c < tokens) {
-            const int row = staged ? rows_s[c0 + c] : __ldg(a.rowmap + tok0 + c0 + c);
+          for (int c = 0; c < 16; ++c) sts_f32(out_a + (unsigned)(c * 512 + r * 4), v[c]);
+        } else if (a.mode == TG_QKV) {
+#pragma unroll
+          for (int c = 0; c < 16; ++c) sts_b16(out_a + (unsigned)(c * 256 + r * 2), __float2bfloat16(v[c]));
+        } else {
+#pragma unroll
+          for (int c = 0; c < 16; ++c)
+            if (((c & 1) == 0) == first) sts_b16(out_a + (unsigned)(c * 128 + (r & 63) * 2), __float2bfloat16(v[c]));
+        }
+        asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+        // ---- shared memory -> global, 16 bytes per thread and request
+        const int spt = row_bytes >> 4;                          // 16-byte segments per token row: 32, 16 or 8
+        for (int seg = tteam; seg < 16 * spt; seg += 128) {
+          const int t = seg / spt, sx = seg - t * spt;
+          if (!ok || c0 + t >= tokens) continue;
+          const size_t tok = (size_t)(tok0 + c0 + t);
+          unsigned char* dst;
+          if (tail) dst = reinterpret_cast<unsigned char*>(a.tail_part + (size_t)split * a.tail_stride + tok * a.tail_ld + (size_t)(tile - a.full_tiles) * 128);
+          else if (a.mode == TG_PARTIAL) dst = reinterpret_cast<unsigned char*>(a.part + (size_t)split * a.split_stride + tok * N + row_base);
+          else if (a.mode == TG_SWIGLU) dst = reinterpret_cast<unsigned char*>(a.h_out + tok * N + row_base);
+          else if (mat == 0) dst = reinterpret_cast<unsigned char*>(a.q_out + tok * N + row_base);
+          else {
+            const int row = staged ? lds_s32(rows_a + (unsigned)(c0 + t) * 4u) : __ldg(a.rowmap + tok0 + c0 + t);
             int b = 0, pos = row;
             if (a.batch > 1) { b = row / a.L; pos = row - b * a.L; }
-            float y = v[c];
-            if (mat < 2) {
-              float cs, sn;
-              if (staged) { cs = tab_s[(size_t)(c0 + c) * 2 * half + j]; sn = tab_s[(size_t)(c0 + c) * 2 * half + half + j]; }
-              else { cs = __ldg(a.rope_cos + (size_t)pos * half + j); sn = __ldg(a.rope_sin + (size_t)pos * half + j); }
-              y = first ? v[c] * cs - pv[c] * sn : v[c] * cs + pv[c] * sn;
-            }
-            if (mat == 0) a.q_out[(size_t)(tok0 + c0 + c) * N + n] = __float2bfloat16(y);
-            else (mat == 1 ? a.kc : a.vc)[((size_t)b * a.max_seq + pos) * N + n] = __float2bfloat16(y);
+            dst = reinterpret_cast<unsigned char*>((mat == 1 ? a.kc : a.vc) + ((size_t)b * a.max_seq + pos) * N + row_base);
+          }
+          *reinterpret_cast<uint4*>(dst + sx * 16) = lds_v4(out_a + (unsigned)(t * row_bytes + sx * 16));
+        }
+      } else {
+        // ragged last tile of a matrix whose row count is no multiple of the tile: element by element
+        const bool live = ok && n_ok;
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          if (!live || c0 + c >= tokens) continue;
+          const size_t tok = (size_t)(tok0 + c0 + c);
+          if (a.mode == TG_PARTIAL) a.part[(size_t)split * a.split_stride + tok * N + n] = v[c];
+          else if (a.mode == TG_SWIGLU) { if (((c & 1) == 0) == first) a.h_out[tok * N + n] = __float2bfloat16(v[c]); }
+          else if (mat == 0) a.q_out[tok * N + n] = __float2bfloat16(v[c]);
+          else {
+            int b = 0, pos = rw[c];
+            if (a.batch > 1) { b = pos / a.L; pos -= b * a.L; }
+            (mat == 1 ? a.kc : a.vc)[((size_t)b * a.max_seq + pos) * N + n] = __float2bfloat16(v[c]);
           }
         }
       }
