@@ -452,6 +452,12 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
   }
 }
 
+#ifndef DA_KL
+#define DA_KL 4
+#endif
+#ifndef DA_KF
+#define DA_KF 20
+#endif
 // Attention of one new row per sequence over the cache (Sec. 3.1): one CTA per (head, sequence).
 // Scores: one key per thread (whole 16-byte-vectorised dot product); P*V: keys dealt round-robin to the
 // eight warps, each lane owning d/32 consecutive dimensions, partial sums combined in warp order.
@@ -473,12 +479,13 @@ __device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc
     const uint4* kp = reinterpret_cast<const uint4*>(kbase + (size_t)j * D);
     float dot = 0.f;
 #pragma unroll
-    for (int c0 = 0; c0 < d / 8; c0 += 4) {                    // four 16-byte loads in flight at a time
-      uint4 raw[4];
+    for (int c0 = 0; c0 < d / 8; c0 += DA_KL) {                // DA_KL 16-byte loads in flight at a time
+      uint4 raw[DA_KL];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) raw[c] = kp[c0 + c];
+      for (int c = 0; c < DA_KL; ++c) raw[c] = kp[min(c0 + c, d / 8 - 1)];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < DA_KL; ++c) {
+        if (c0 + c >= d / 8) break;
         const bf16* kb = reinterpret_cast<const bf16*>(&raw[c]);
 #pragma unroll
         for (int e = 0; e < 8; ++e) dot += qs[(c0 + c) * 8 + e] * bf2f(kb[e]);
@@ -510,7 +517,7 @@ __device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc
   float acc[DPL];
 #pragma unroll
   for (int e = 0; e < DPL; ++e) acc[e] = 0.f;
-  constexpr int KF = 10;                                         // keys of this warp in flight (8 warps x 10 covers 80 keys per round)
+  constexpr int KF = DA_KF;                                      // keys of this warp in flight
   for (int j0 = warp; j0 < nkeys; j0 += 8 * KF) {
     float pj[KF];
     __align__(8) bf16 vv[KF][DPL];
