@@ -461,21 +461,26 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
 // Attention of one new row per sequence over the cache (Sec. 3.1): one CTA per (head, sequence).
 // Scores: one key per thread (whole 16-byte-vectorised dot product); P*V: keys dealt round-robin to the
 // eight warps, each lane owning d/32 consecutive dimensions, partial sums combined in warp order.
-template <int DPL>      // dimensions per lane = head_dim / 32
+template <int DPL, int NT>      // dimensions per lane = head_dim / 32; threads of the CTA
 __device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc, const bf16* vc, bf16* out,
                                                       int pos, int max_seq, int H, int h, int b, float* dsm, float* red) {
   constexpr int d = 32 * DPL;
+  constexpr int NW = NT / 32;
   float* qs = dsm;                 // [d]
   float* p = dsm + d;              // [max_seq]
-  float* part = p + max_seq;       // [8][d]
+  float* part = p + max_seq;       // [NW][d]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int D = H * d, nkeys = pos + 1;
   const float scale = rsqrtf((float)d);
-  if (tid < d) qs[tid] = bf2f(q[(size_t)b * D + h * d + tid]) * scale;
+  // (q may have been written by another SM earlier in the same kernel: read it past the L1)
+  if (tid < d) {
+    const unsigned short raw = __ldcg(reinterpret_cast<const unsigned short*>(q) + (size_t)b * D + h * d + tid);
+    qs[tid] = __uint_as_float((unsigned)raw << 16) * scale;
+  }
   __syncthreads();
   const bf16* kbase = kc + (size_t)b * max_seq * D + h * d;
   float mx = -INFINITY;
-  for (int j = tid; j < nkeys; j += 256) {
+  for (int j = tid; j < nkeys; j += NT) {
     const uint4* kp = reinterpret_cast<const uint4*>(kbase + (size_t)j * D);
     float dot = 0.f;
 #pragma unroll
@@ -500,9 +505,9 @@ __device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc
   __syncthreads();
   mx = red[0];
 #pragma unroll
-  for (int w = 1; w < 8; ++w) mx = fmaxf(mx, red[w]);
+  for (int w = 1; w < NW; ++w) mx = fmaxf(mx, red[w]);
   float sum = 0.f;
-  for (int j = tid; j < nkeys; j += 256) { const float e = __expf(p[j] - mx); p[j] = e; sum += e; }
+  for (int j = tid; j < nkeys; j += NT) { const float e = __expf(p[j] - mx); p[j] = e; sum += e; }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
   __syncthreads();
@@ -510,7 +515,7 @@ __device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc
   __syncthreads();
   float tot = 0.f;
 #pragma unroll
-  for (int w = 0; w < 8; ++w) tot += red[w];
+  for (int w = 0; w < NW; ++w) tot += red[w];
   const float inv = 1.f / tot;
   // P * V
   const bf16* vbase = vc + (size_t)b * max_seq * D + h * d + lane * DPL;
@@ -518,12 +523,12 @@ __device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc
 #pragma unroll
   for (int e = 0; e < DPL; ++e) acc[e] = 0.f;
   constexpr int KF = DA_KF;                                      // keys of this warp in flight
-  for (int j0 = warp; j0 < nkeys; j0 += 8 * KF) {
+  for (int j0 = warp; j0 < nkeys; j0 += NW * KF) {
     float pj[KF];
     __align__(8) bf16 vv[KF][DPL];
 #pragma unroll
     for (int u = 0; u < KF; ++u) {
-      const int j = j0 + 8 * u;
+      const int j = j0 + NW * u;
       pj[u] = j < nkeys ? p[j] : 0.f;
       const bf16* vp = vbase + (size_t)min(j, nkeys - 1) * D;
       if (DPL == 4) *reinterpret_cast<uint2*>(vv[u]) = *reinterpret_cast<const uint2*>(vp);
@@ -544,7 +549,7 @@ __device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc
   if (tid < d) {
     float o = 0.f;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) o += part[w * d + tid];
+    for (int w = 0; w < NW; ++w) o += part[w * d + tid];
     out[(size_t)b * D + h * d + tid] = __float2bfloat16(o * inv);
   }
 }
@@ -556,7 +561,7 @@ __global__ void __launch_bounds__(256) decode_attention_kernel(const bf16* q, co
   __shared__ float red[8];
   pdl_trigger();
   pdl_wait();
-  decode_attention_body<DPL>(q, kc, vc, out, pos, max_seq, H, blockIdx.x, blockIdx.y, dsm, red);
+  decode_attention_body<DPL, 256>(q, kc, vc, out, pos, max_seq, H, blockIdx.x, blockIdx.y, dsm, red);
 }
 
 // ---- one whole single-row pass as ONE persistent kernel -------------------------------------------
@@ -604,41 +609,193 @@ struct PassArgs {
   int* dev_error;
 };
 
-template <int NB>
-__global__ void __launch_bounds__(256, GV_CTAS_PER_SM) decode_pass_kernel(PassArgs pa) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  __shared__ float red[8];
-  unsigned n_bar = 0;
-  const unsigned G = gridDim.x;
+// Phase parameters a warp derives from the arguments of a matrix-vector phase.
+struct PhaseGeom { int u_begin, n_local, n_groups, ns_w, K; };
+__device__ __forceinline__ PhaseGeom phase_geom(const GemvArgs& a, int warp) {
+  PhaseGeom g;
+  const int n_units = unit_count(a.mode, a.N);
+  g.u_begin = (int)(((long long)n_units * blockIdx.x) / gridDim.x);
+  g.n_local = (int)(((long long)n_units * (blockIdx.x + 1)) / gridDim.x) - g.u_begin;
+  g.n_groups = (g.n_local + 7) / 8;
+  const int S = a.K / 64;
+  g.ns_w = warp < S ? (S - warp + GT_WARPS - 1) / GT_WARPS : 0;
+  g.K = a.K;
+  return g;
+}
+
+// The tensor-core weight-streaming kernel as one persistent kernel per single-row pass.  The ring of
+// asynchronous copies does not stop at a phase boundary: while the CTA flushes a phase, waits at the grid
+// barrier and stages the next activations, its warps' copies of the NEXT phase's first weights (which depend
+// on nothing) are already in flight, so HBM keeps streaming across what would be a kernel boundary.
+// The issue side may run at most one phase ahead of the consume side; the arguments of phase p+1 are put in
+// shared memory when phase p begins.
+__global__ void __launch_bounds__(GT_THREADS, 1) decode_pass_kernel(PassArgs pa) {
+  extern __shared__ __align__(128) unsigned char gt_smem[];
+  __shared__ float red[GT_WARPS];
+  __shared__ GemvArgs sargs[2];                                 // arguments of phase p in slot p & 1
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const unsigned ring_w = (unsigned)__cvta_generic_to_shared(gt_smem) + (unsigned)warp * (GT_DEPTH * GT_SLOT_BYTES);
+  float* part = reinterpret_cast<float*>(gt_smem + GT_RING_BYTES);
+  bf16* xs = reinterpret_cast<bf16*>(gt_smem + GT_RING_BYTES + GT_PART_BYTES);
   const int n_phases = 4 * pa.n_layers;
-  __shared__ int next_unit;
-  __shared__ GemvArgs sargs;                                   // this phase's arguments (kept out of registers)
-  for (int ph = 0; ph < n_phases; ++ph) {
-    __syncthreads();                                             // every warp is done with the previous phase's arguments
-    if (threadIdx.x < sizeof(GemvArgs) / sizeof(int))
-      reinterpret_cast<int*>(&sargs)[threadIdx.x] = reinterpret_cast<const int*>(pa.phases + ph)[threadIdx.x];
-    __syncthreads();
-    gemv_body<NB>(sargs, smem_raw, red, &next_unit, [&] {
-      // the row entering the pass was written by an earlier kernel: no barrier before the very first phase
-      if (ph > 0) grid_barrier(pa.counter, (++n_bar) * G, pa.dev_error);
-      if ((ph & 3) == 1) {
-        // attention of this layer sits between the Q/K/V phase and the output projection, whose first
-        // weights this CTA has already requested
-        const int hb = blockIdx.x;
-        if (hb < pa.n_heads * pa.batch) {
-          const GemvArgs* qkv = pa.phases + (ph - 1);
-          const bf16 *q = qkv->q_out, *kc = qkv->kc, *vc = qkv->vc;
-          const int max_seq = qkv->max_seq, dpl = qkv->d / 32;
-          const int h = hb % pa.n_heads, b = hb / pa.n_heads;
-          float* dsm = reinterpret_cast<float*>(smem_raw);
-          if (dpl == 4) decode_attention_body<4>(q, kc, vc, pa.ao, pa.pos, max_seq, pa.n_heads, h, b, dsm, red);
-          else if (dpl == 2) decode_attention_body<2>(q, kc, vc, pa.ao, pa.pos, max_seq, pa.n_heads, h, b, dsm, red);
-          else if (dpl == 3) decode_attention_body<3>(q, kc, vc, pa.ao, pa.pos, max_seq, pa.n_heads, h, b, dsm, red);
-          else decode_attention_body<1>(q, kc, vc, pa.ao, pa.pos, max_seq, pa.n_heads, h, b, dsm, red);
-        }
-        grid_barrier(pa.counter, (++n_bar) * G, pa.dev_error);
+  const unsigned G_ctas = gridDim.x;
+  unsigned n_bar = 0;
+  auto load_args = [&](int ph) {
+    if (ph < n_phases && tid < (int)(sizeof(GemvArgs) / sizeof(int)))
+      reinterpret_cast<int*>(&sargs[ph & 1])[tid] = reinterpret_cast<const int*>(pa.phases + ph)[tid];
+  };
+  load_args(0);
+  load_args(1);
+  __syncthreads();
+
+  // ---- issue side
+  int pc = 0;                                                   // phase being consumed
+  int ip = 0, ig = 0, ij = 0, islot = 0;
+  bool i_ready = false;
+  unsigned real_mask = 0u;                                      // ring positions that hold an item (the rest were issued empty)
+  PhaseGeom igm = {0, 0, 0, 0, 0};
+  const char* rowptr[4];
+  auto load_rowptrs = [&](int g) {
+    const GemvArgs& a = sargs[ip & 1];
+    const UnitRows r0 = unit_rows(a, igm.u_begin + min(g * 8 + (lane >> 3), igm.n_local - 1));
+    const UnitRows r1 = unit_rows(a, igm.u_begin + min(g * 8 + (lane >> 3) + 4, igm.n_local - 1));
+    rowptr[0] = reinterpret_cast<const char*>(r0.pa); rowptr[1] = reinterpret_cast<const char*>(r1.pa);
+    rowptr[2] = reinterpret_cast<const char*>(r0.pb); rowptr[3] = reinterpret_cast<const char*>(r1.pb);
+  };
+  auto issue = [&]() {
+    if (!i_ready && ip < n_phases && ip <= pc + 1) {
+      igm = phase_geom(sargs[ip & 1], warp);
+      ig = 0; ij = 0;
+      if (igm.n_groups > 0 && igm.ns_w > 0) { load_rowptrs(0); i_ready = true; }
+      else ++ip;                                                // nothing for this warp in that phase
+    }
+    if (i_ready) real_mask |= 1u << islot; else real_mask &= ~(1u << islot);
+    if (i_ready) {
+      const unsigned slotp = ring_w + (unsigned)islot * GT_SLOT_BYTES;
+      const size_t koff = (size_t)(warp + GT_WARPS * ij) * 128 + (size_t)(lane & 7) * 16;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int row = (lane >> 3) + 4 * i;
+        cp_async16(slotp + (unsigned)(row * 128 + (((lane & 7) ^ (row & 7)) << 4)), rowptr[i] + koff);
       }
-    });
+      if (++ij == igm.ns_w) {
+        ij = 0;
+        if (++ig < igm.n_groups) load_rowptrs(ig);
+        else { ++ip; i_ready = false; }
+      }
+    }
+    cp_async_commit();
+    islot = (islot + 1 == GT_DEPTH) ? 0 : islot + 1;
+  };
+  // (the ring starts empty: the first positions the consume loop meets carry nothing and are filled there,
+  // which keeps the issue code at a single place)
+
+  int cslot = 0;
+  for (pc = 0; pc < n_phases; ++pc) {
+    // ---- phase start: next phase's arguments, dependencies, activations
+    load_args(pc + 1);
+    if (pc > 0) grid_barrier(pa.counter, (++n_bar) * G_ctas, pa.dev_error);   // the row entering the pass came from an earlier kernel
+    if ((pc & 3) == 1) {
+      // attention of this layer sits between the Q/K/V phase and the output projection
+      const int hb = blockIdx.x;
+      if (hb < pa.n_heads * pa.batch) {
+        const GemvArgs* qkv = pa.phases + (pc - 1);
+        const bf16 *q = qkv->q_out, *kc = qkv->kc, *vc = qkv->vc;
+        const int max_seq = qkv->max_seq, dpl = qkv->d / 32;
+        const int h = hb % pa.n_heads, b = hb / pa.n_heads;
+        float* dsm = reinterpret_cast<float*>(xs);
+        if (dpl == 4) decode_attention_body<4, GT_THREADS>(q, kc, vc, pa.ao, pa.pos, max_seq, pa.n_heads, h, b, dsm, red);
+        else if (dpl == 2) decode_attention_body<2, GT_THREADS>(q, kc, vc, pa.ao, pa.pos, max_seq, pa.n_heads, h, b, dsm, red);
+        else if (dpl == 3) decode_attention_body<3, GT_THREADS>(q, kc, vc, pa.ao, pa.pos, max_seq, pa.n_heads, h, b, dsm, red);
+        else decode_attention_body<1, GT_THREADS>(q, kc, vc, pa.ao, pa.pos, max_seq, pa.n_heads, h, b, dsm, red);
+      }
+      grid_barrier(pa.counter, (++n_bar) * G_ctas, pa.dev_error);
+    }
+    __syncthreads();                                            // sargs[pc & 1] and [(pc + 1) & 1] are in place
+    const GemvArgs& a = sargs[pc & 1];
+    const PhaseGeom gm = phase_geom(a, warp);
+    const int K = a.K, nb = a.nb;
+    for (int b = 0; b < nb; ++b) {
+      if (a.x_f32) {
+        // values an earlier phase of this kernel wrote on other SMs: read past the L1
+        const float* x = a.x_f32 + (size_t)b * K;
+        float ss = 0.f;
+        for (int k = tid; k < K; k += GT_THREADS) { const float v = __ldcg(x + k); ss += v * v; }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        __syncthreads();
+        if (lane == 0) red[warp] = ss;
+        __syncthreads();
+        float t = 0.f;
+#pragma unroll
+        for (int w = 0; w < GT_WARPS; ++w) t += red[w];
+        const float r = rsqrtf(t / (float)K + a.eps);
+        for (int k = tid; k < K; k += GT_THREADS) xs[(size_t)b * K + k] = __float2bfloat16(__ldcg(x + k) * r * bf2f(a.gain[k]));
+      } else {
+        const uint4* src = reinterpret_cast<const uint4*>(a.x_bf16 + (size_t)b * K);
+        uint4* dst = reinterpret_cast<uint4*>(xs + (size_t)b * K);
+        for (int c = tid; c < K / 8; c += GT_THREADS) dst[c] = __ldcg(src + c);
+      }
+    }
+    __syncthreads();
+
+    // ---- consume side of this phase
+    const int col_n = lane >> 2;
+    const unsigned* xw = reinterpret_cast<const unsigned*>(xs + (size_t)min(col_n, max(nb - 1, 0)) * K) + (lane & 3);
+    const bool col_live = col_n < nb;
+    const int nbp = nb <= 1 ? 1 : (nb <= 2 ? 2 : (nb <= 4 ? 4 : 8));
+    const int G = 8 / nbp;
+    for (int g = 0; g < gm.n_groups; ++g) {
+      float c[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int j = 0; j < gm.ns_w;) {
+        // the ring is consumed position by position; a position issued while the issue side had to hold
+        // back (it may not run two phases ahead) carries nothing and is simply handed back
+        cp_async_wait<GT_DEPTH - 1>();
+        __syncwarp();
+        const bool real = (real_mask >> cslot) & 1u;
+        if (real) {
+          const unsigned slotp = ring_w + (unsigned)cslot * GT_SLOT_BYTES;
+          const int k0 = (warp + GT_WARPS * j) * 64;
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {
+            unsigned af[4];
+            const int row = lane & 15, kc = 2 * kk + (lane >> 4);
+            ldmatrix_x4(slotp + (unsigned)(row * 128 + ((kc ^ (row & 7)) << 4)), af);
+            unsigned b0 = 0u, b1 = 0u;
+            if (col_live) { b0 = xw[(k0 + kk * 16) / 2]; b1 = xw[(k0 + kk * 16) / 2 + 4]; }
+            mma_16816(c, af, b0, b1);
+          }
+          ++j;
+        }
+        __syncwarp();
+        issue();
+        cslot = (cslot + 1 == GT_DEPTH) ? 0 : cslot + 1;
+      }
+      const int round = g / G, gr = g - round * G;
+      {
+        float* dst = part + ((size_t)(((round & 1) * G + gr) * GT_WARPS + warp) * 16) * nbp;
+        const int r = lane >> 2, n0 = (lane & 3) * 2;
+        if (n0 < nb) { dst[r * nbp + n0] = c[0]; dst[(r + 8) * nbp + n0] = c[2]; }
+        if (n0 + 1 < nb) { dst[r * nbp + n0 + 1] = c[1]; dst[(r + 8) * nbp + n0 + 1] = c[3]; }
+      }
+      if (gr == G - 1 || g == gm.n_groups - 1) {
+        __syncthreads();
+        const int n_items = (gr + 1) * 8 * nb;
+        for (int idx = tid; idx < n_items; idx += GT_THREADS) {
+          const int gi = idx / (8 * nb), rem = idx - gi * 8 * nb;
+          const int uu = rem / nb, col = rem - uu * nb;
+          const int ul = (round * G + gi) * 8 + uu;
+          if (ul >= gm.n_local) continue;
+          const float* src = part + ((size_t)(((round & 1) * G + gi) * GT_WARPS) * 16) * nbp;
+          float ya = 0.f, yb = 0.f;
+#pragma unroll
+          for (int w = 0; w < GT_WARPS; ++w) { ya += src[((size_t)w * 16 + uu) * nbp + col]; yb += src[((size_t)w * 16 + uu + 8) * nbp + col]; }
+          const UnitRows cu = unit_rows(a, gm.u_begin + ul);
+          store_unit(a, cu, col, ya, yb);
+        }
+      }
+    }
+    __syncthreads();                                            // the last flush has read `part` and the arguments
   }
 }
 
@@ -751,25 +908,19 @@ int vlac_decode_setup(vlac_ctx* ctx) {
   VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GT_SMEM_MAX));
   // persistent pass kernel: as many CTAs as are guaranteed co-resident
   ctx->pass_grid = 0;
-  // Opt-in (VLAC_PASS_KERNEL=1): measured on B200 it streams at 5.5 TB/s between barriers but its five grid
-  // barriers per layer (about 5 us each) make a pass no faster than the per-phase kernels replayed from a graph.
-  if (getenv("VLAC_PASS_KERNEL") != nullptr && ctx->max_seq > 0) {
+  // Opt-in (VLAC_PASS_KERNEL=1).  Needs every K to be a multiple of 64 (the tensor-core body) and room for
+  // the activations beside the ring.  Measured on B200: correct, but a pass takes 3.25 ms against 2.65 ms for
+  // the per-phase kernels replayed from a graph.  A grid barrier under a saturated memory system costs more
+  // than a programmatic kernel boundary, and the ring (19 MB over the GPU) covers under 3 us of streaming.
+  if (getenv("VLAC_PASS_KERNEL") != nullptr && ctx->max_seq > 0 && ctx->cfg.hidden % 64 == 0 && ctx->cfg.ffn % 64 == 0) {
     const size_t psm = pass_smem(ctx, NB);
     int per_sm = 0, coop = 0, dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
-    if (e == cudaSuccess && coop) {
-      switch (NB) {
-        case 1: e = cudaFuncSetAttribute(decode_pass_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psm);
-                if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_pass_kernel<1>, 256, psm); break;
-        case 2: e = cudaFuncSetAttribute(decode_pass_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psm);
-                if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_pass_kernel<2>, 256, psm); break;
-        case 4: e = cudaFuncSetAttribute(decode_pass_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psm);
-                if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_pass_kernel<4>, 256, psm); break;
-        default: e = cudaFuncSetAttribute(decode_pass_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psm);
-                if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_pass_kernel<8>, 256, psm); break;
-      }
-      if (e == cudaSuccess && per_sm > 0) ctx->pass_grid = ctx->n_sm * (per_sm < GV_CTAS_PER_SM ? per_sm : GV_CTAS_PER_SM);
+    if (e == cudaSuccess && coop && psm <= GT_SMEM_MAX) {
+      e = cudaFuncSetAttribute(decode_pass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psm);
+      if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_pass_kernel, GT_THREADS, psm);
+      if (e == cudaSuccess && per_sm > 0) ctx->pass_grid = ctx->n_sm;
     }
     if (e != cudaSuccess) cudaGetLastError();
   }
@@ -819,8 +970,8 @@ static size_t pass_smem(const vlac_ctx* ctx, int NB) {
   const vlac_config& g = ctx->cfg;
   const int kmax = g.ffn > g.hidden ? g.ffn : g.hidden;
   const size_t xs = (size_t)NB * kmax * sizeof(bf16);
-  const size_t at = (size_t)(g.head_dim + ctx->max_seq + 8 * g.head_dim) * sizeof(float);
-  return xs > at ? xs : at;
+  const size_t at = (size_t)(g.head_dim + ctx->max_seq + GT_WARPS * g.head_dim) * sizeof(float);   // attention scratch shares the activation area
+  return (size_t)GT_RING_BYTES + GT_PART_BYTES + (xs > at ? xs : at);
 }
 
 // Per-cache table of phase arguments for the persistent pass kernel, and its barrier counter.
@@ -841,15 +992,14 @@ int vlac_decode_cache_setup(vlac_ctx* ctx, vlac_cache* c) {
   return rc;
 }
 
-template <int NB>
 static cudaError_t launch_pass(const PassArgs& pa, int grid, size_t smem, cudaStream_t s) {
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(grid); cfg.blockDim = dim3(256); cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cfg.gridDim = dim3(grid); cfg.blockDim = dim3(GT_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = s;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeCooperative;            // all CTAs resident at once: the grid barriers rely on it
   attr[0].val.cooperative = 1;
   cfg.attrs = attr; cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, decode_pass_kernel<NB>, pa);
+  return cudaLaunchKernelEx(&cfg, decode_pass_kernel, pa);
 }
 
 int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens, int tok_stride, int tok_index,
@@ -868,14 +1018,7 @@ int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens,
     pa.phases = (const GemvArgs*)c->dec_phases + (size_t)pass_idx * 4 * g.n_layers; pa.n_layers = g.n_layers; pa.pos = pos; pa.n_heads = g.n_heads; pa.batch = B;
     pa.ao = ctx->ao_dec; pa.counter = (unsigned*)c->dec_counter; pa.dev_error = ctx->dev_error;
     const size_t smem = pass_smem(ctx, NB);
-    cudaError_t e;
-    switch (NB) {
-      case 1: e = launch_pass<1>(pa, ctx->pass_grid, smem, s); break;
-      case 2: e = launch_pass<2>(pa, ctx->pass_grid, smem, s); break;
-      case 4: e = launch_pass<4>(pa, ctx->pass_grid, smem, s); break;
-      default: e = launch_pass<8>(pa, ctx->pass_grid, smem, s); break;
-    }
-    VLAC_CUDA_CHECK(e);
+    VLAC_CUDA_CHECK(launch_pass(pa, ctx->pass_grid, smem, s));
     VLAC_LAUNCH_CHECK(ctx);
     return VLAC_OK;
   }
