@@ -73,7 +73,21 @@ __device__ __forceinline__ UnitRows unit_rows(const A& a, int u) {
 }
 
 // Epilogue of one unit (a pair of weight rows) for sequence b: ya, yb are the two finished dot products.
-__device__ __forceinline__ void store_unit(const GemvArgs& a, const UnitRows& cu, int b, float ya, float yb) {
+// What the epilogue of a unit reads besides the dot products (rotary table entry, or the residual values
+// it adds to): fetched ahead of time by unit_operands(), or by store_unit() itself when `pre` is NULL.
+__device__ __forceinline__ void unit_operands(const GemvArgs& a, const UnitRows& cu, int b, float* pre) {
+  pre[0] = pre[1] = 0.f;
+  if (a.mode == GV_QKV) {
+    if (cu.mat < 2) {
+      const int half = a.d / 2, j = cu.rowA % a.d;
+      pre[0] = a.rope_cos[(size_t)a.pos * half + j]; pre[1] = a.rope_sin[(size_t)a.pos * half + j];
+    }
+  } else if (a.mode == GV_RESID) {
+    pre[0] = a.x_out[(size_t)b * a.N + cu.rowA]; pre[1] = a.x_out[(size_t)b * a.N + cu.rowB];
+  }
+}
+
+__device__ __forceinline__ void store_unit(const GemvArgs& a, const UnitRows& cu, int b, float ya, float yb, const float* pre = nullptr) {
   const int rowA = cu.rowA, rowB = cu.rowB, mat = cu.mat;
   if (a.mode == GV_QKV) {
     if (mat == 2) {
@@ -82,7 +96,7 @@ __device__ __forceinline__ void store_unit(const GemvArgs& a, const UnitRows& cu
     } else {
       const int half = a.d / 2;
       const int j = rowA % a.d;
-      const float c = a.rope_cos[(size_t)a.pos * half + j], s = a.rope_sin[(size_t)a.pos * half + j];
+      const float c = pre ? pre[0] : a.rope_cos[(size_t)a.pos * half + j], s = pre ? pre[1] : a.rope_sin[(size_t)a.pos * half + j];
       const float r1 = ya * c - yb * s, r2 = yb * c + ya * s;
       bf16* dst = mat == 0 ? a.q_out + (size_t)b * a.N : a.kc + ((size_t)b * a.max_seq + a.pos) * a.N;
       dst[rowA] = __float2bfloat16(r1); dst[rowB] = __float2bfloat16(r2);
@@ -90,8 +104,13 @@ __device__ __forceinline__ void store_unit(const GemvArgs& a, const UnitRows& cu
   } else if (a.mode == GV_SWIGLU) {
     a.h_out[(size_t)b * a.N + rowA] = __float2bfloat16(ya / (1.f + __expf(-ya)) * yb);
   } else if (a.mode == GV_RESID) {
-    a.x_out[(size_t)b * a.N + rowA] += ya;
-    if (rowB != rowA) a.x_out[(size_t)b * a.N + rowB] += yb;
+    if (pre) {
+      a.x_out[(size_t)b * a.N + rowA] = pre[0] + ya;
+      if (rowB != rowA) a.x_out[(size_t)b * a.N + rowB] = pre[1] + yb;
+    } else {
+      a.x_out[(size_t)b * a.N + rowA] += ya;
+      if (rowB != rowA) a.x_out[(size_t)b * a.N + rowB] += yb;
+    }
   } else {
     a.logits[(size_t)b * a.N + rowA] = ya;
     if (rowB != rowA) a.logits[(size_t)b * a.N + rowB] = yb;
@@ -278,7 +297,6 @@ constexpr int GT_DEPTH = GT_DEPTH_N;
 constexpr int GT_SLOT_BYTES = 16 * 128;
 constexpr int GT_RING_BYTES = GT_WARPS * GT_DEPTH * GT_SLOT_BYTES;      // 128 KB
 constexpr int GT_PART_BYTES = 2 * 8 * GT_WARPS * 16 * (int)sizeof(float);  // partial tiles of two rounds: 16 KB
-constexpr int GT_XR = 8192 / GT_THREADS_N;                                              // activations a thread keeps while it normalises a row
 
 __device__ __forceinline__ void cp_async16(unsigned smem_dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(src) : "memory");
@@ -286,6 +304,7 @@ __device__ __forceinline__ void cp_async16(unsigned smem_dst, const void* src) {
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ unsigned lds_u32(unsigned addr) { unsigned v; asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr)); return v; }
 __device__ __forceinline__ void ldmatrix_x4(unsigned addr, unsigned* r) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
 }
@@ -350,6 +369,17 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
   // weights depend on no earlier kernel: fill the ring before the dependency wait
 #pragma unroll
   for (int i = 0; i < GT_DEPTH; ++i) issue();
+  // the norm gains are constants too: two 8-element chunks per thread cover K <= 8192
+  const int nchunk = K / 8;
+  const bool x_cached = a.x_f32 != nullptr && nchunk <= 2 * GT_THREADS;
+  uint4 gq[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
+  if (x_cached) {
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const int c = tid + i * GT_THREADS;
+      if (c < nchunk) gq[i] = __ldg(reinterpret_cast<const uint4*>(a.gain) + c);
+    }
+  }
   pdl_trigger();
   pdl_wait();
 
@@ -357,15 +387,20 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
   for (int b = 0; b < nb; ++b) {
     if (a.x_f32) {
       const float* x = a.x_f32 + (size_t)b * K;
-      const bool cached = K <= GT_XR * GT_THREADS;
-      float xv[GT_XR];
+      float4 xq[2][2];
       float ss = 0.f;
-      if (cached) {
+      if (x_cached) {
 #pragma unroll
-        for (int i = 0; i < GT_XR; ++i) {
-          const int k = tid + i * GT_THREADS;
-          xv[i] = k < K ? x[k] : 0.f;
-          ss += xv[i] * xv[i];
+        for (int i = 0; i < 2; ++i) {
+          const int c = tid + i * GT_THREADS;
+          if (c < nchunk) {
+            xq[i][0] = *reinterpret_cast<const float4*>(x + (size_t)c * 8);
+            xq[i][1] = *reinterpret_cast<const float4*>(x + (size_t)c * 8 + 4);
+          } else {
+            xq[i][0] = xq[i][1] = make_float4(0.f, 0.f, 0.f, 0.f);
+          }
+          ss += xq[i][0].x * xq[i][0].x + xq[i][0].y * xq[i][0].y + xq[i][0].z * xq[i][0].z + xq[i][0].w * xq[i][0].w;
+          ss += xq[i][1].x * xq[i][1].x + xq[i][1].y * xq[i][1].y + xq[i][1].z * xq[i][1].z + xq[i][1].w * xq[i][1].w;
         }
       } else {
         for (int k = tid; k < K; k += GT_THREADS) { const float v = x[k]; ss += v * v; }
@@ -379,11 +414,22 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
 #pragma unroll
       for (int w = 0; w < GT_WARPS; ++w) t += red[w];
       const float r = rsqrtf(t / (float)K + a.eps);
-      if (cached) {
+      if (x_cached) {
 #pragma unroll
-        for (int i = 0; i < GT_XR; ++i) {
-          const int k = tid + i * GT_THREADS;
-          if (k < K) xs[(size_t)b * K + k] = __float2bfloat16(xv[i] * r * bf2f(a.gain[k]));
+        for (int i = 0; i < 2; ++i) {
+          const int c = tid + i * GT_THREADS;
+          if (c < nchunk) {
+            const __nv_bfloat162* g2 = reinterpret_cast<const __nv_bfloat162*>(&gq[i]);
+            const float xv[8] = {xq[i][0].x, xq[i][0].y, xq[i][0].z, xq[i][0].w, xq[i][1].x, xq[i][1].y, xq[i][1].z, xq[i][1].w};
+            uint4 o;
+            __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float2 gf = __bfloat1622float2(g2[e]);
+              o2[e] = __floats2bfloat162_rn(xv[2 * e] * r * gf.x, xv[2 * e + 1] * r * gf.y);
+            }
+            *reinterpret_cast<uint4*>(xs + (size_t)b * K + (size_t)c * 8) = o;
+          }
         }
       } else {
         for (int k = tid; k < K; k += GT_THREADS) xs[(size_t)b * K + k] = __float2bfloat16(x[k] * r * bf2f(a.gain[k]));
@@ -398,13 +444,29 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
 
   // ---- consume side
   const int col_n = lane >> 2;                                         // B column (sequence) this lane feeds
-  const unsigned* xw = reinterpret_cast<const unsigned*>(xs + (size_t)min(col_n, max(nb - 1, 0)) * K) + (lane & 3);
+  const unsigned xw_a = (unsigned)__cvta_generic_to_shared(xs) + (unsigned)((size_t)min(col_n, max(nb - 1, 0)) * K * 2) + (unsigned)(lane & 3) * 4u;
   const bool col_live = col_n < nb;
   // Partial tiles of G groups are collected before the CTA meets at a barrier: part[2][G][warp][16 rows][nbp]
   const int nbp = nb <= 1 ? 1 : (nb <= 2 ? 2 : (nb <= 4 ? 4 : 8));
   const int G = 8 / nbp;
   int cslot = 0;
+  UnitRows fcu = {nullptr, nullptr, 0, 0, 0};                        // unit this thread finishes in the current round, if any
+  float fpre[2] = {0.f, 0.f};
+  int f_ul = -1, f_col = 0;
   for (int g = 0; g < n_groups; ++g) {
+    if (g % G == 0) {
+      // start of a round: the threads that will finish its units fetch what the epilogue needs now, so the
+      // last round does not end on a dependent global load
+      const int n_gr = min(G, n_groups - g);
+      f_ul = -1;
+      if (tid < n_gr * 8 * nb) {
+        const int gi = tid / (8 * nb), rem = tid - gi * 8 * nb;
+        const int uu = rem / nb;
+        f_col = rem - uu * nb;
+        const int ul = (g + gi) * 8 + uu;
+        if (ul < n_local) { f_ul = ul; fcu = unit_rows(a, u_begin + ul); unit_operands(a, fcu, f_col, fpre); }
+      }
+    }
     float c[4] = {0.f, 0.f, 0.f, 0.f};
     for (int j = 0; j < ns_w; ++j) {
       cp_async_wait<GT_DEPTH - 1>();                                   // this lane's copies of the oldest item have landed
@@ -417,7 +479,7 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
         const int row = lane & 15, kc = 2 * kk + (lane >> 4);
         ldmatrix_x4(slotp + (unsigned)(row * 128 + ((kc ^ (row & 7)) << 4)), af);
         unsigned b0 = 0u, b1 = 0u;
-        if (col_live) { b0 = xw[(k0 + kk * 16) / 2]; b1 = xw[(k0 + kk * 16) / 2 + 4]; }
+        if (col_live) { b0 = lds_u32(xw_a + (unsigned)(k0 + kk * 16) * 2u); b1 = lds_u32(xw_a + (unsigned)(k0 + kk * 16) * 2u + 16u); }
         mma_16816(c, af, b0, b1);
       }
       __syncwarp();                                                    // every lane has read the slot: refill it
@@ -435,18 +497,13 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
       // End of a round: add the warps' partial tiles in warp order and finish these units.  The other half of
       // `part` takes the next round; the barrier that ends it also orders these reads before this half is reused.
       __syncthreads();
-      const int n_items = (gr + 1) * 8 * nb;
-      for (int idx = tid; idx < n_items; idx += GT_THREADS) {
-        const int gi = idx / (8 * nb), rem = idx - gi * 8 * nb;
-        const int uu = rem / nb, col = rem - uu * nb;
-        const int ul = (round * G + gi) * 8 + uu;
-        if (ul >= n_local) continue;
+      if (f_ul >= 0) {                                           // at most 64 units x columns per round: one per thread
+        const int gi = f_ul / 8 - round * G, uu = f_ul & 7, col = f_col;
         const float* src = part + ((size_t)(((round & 1) * G + gi) * GT_WARPS) * 16) * nbp;
         float ya = 0.f, yb = 0.f;
 #pragma unroll
         for (int w = 0; w < GT_WARPS; ++w) { ya += src[((size_t)w * 16 + uu) * nbp + col]; yb += src[((size_t)w * 16 + uu + 8) * nbp + col]; }
-        const UnitRows cu = unit_rows(a, u_begin + ul);
-        store_unit(a, cu, col, ya, yb);
+        store_unit(a, fcu, col, ya, yb, fpre);
       }
     }
   }
