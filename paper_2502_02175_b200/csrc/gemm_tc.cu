@@ -31,6 +31,7 @@ namespace {
 
 constexpr int TG_QKV = 0, TG_PARTIAL = 1, TG_SWIGLU = 2;
 constexpr int TG_THREADS = 256;
+constexpr int TG_STG = 8;                       // table loads a thread keeps in flight while staging the rotary rows
 constexpr int TG_PRODUCERS = 3;                // warps 0, 6, 7: one elected lane each issues TMA loads
 constexpr int TG_BK = 64;                       // bf16 elements per k-block = one 128-byte swizzle row
 constexpr int TG_A_BYTES = 128 * TG_BK * 2;     // 16 KB: 128 weight rows
@@ -62,6 +63,7 @@ struct alignas(64) TcArgs {
   // their raw gate/up sums go to tail_part[split][T][tail_ld] and a small kernel finishes them
   int full_tiles, tail_splits, tail_ld;
   float* tail_part; size_t tail_stride;
+  int tmem_cols;                  // tensor-memory columns to allocate: covers the largest token chunk (power of two >= 32)
   int* dev_error;
 };
 
@@ -169,6 +171,12 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
   }
   __syncthreads();
   pdl_trigger();
+  // tensor memory does not depend on earlier kernels either: allocated (for the largest token chunk) before the wait
+  const unsigned tmem_cols = (unsigned)a.tmem_cols;
+  if (warp == 1) {                                              // whole warp
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
   pdl_wait();                                                   // everything below may read what earlier kernels wrote
   // blockIdx.z selects a chunk of up to 512 tokens (one accumulator's worth of tensor-memory columns)
   const int tok0 = blockIdx.z * 512;
@@ -183,16 +191,11 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
   const int n_kb = (tokens > 0) ? kb1 - kb0 : 0;
   const int n0 = min(((tokens + 15) / 16) * 16, 256);           // columns of the first MMA
   const int n1 = tokens > 256 ? ((tokens - 256 + 15) / 16) * 16 : 0;
-  const unsigned tmem_cols = (n0 + n1) <= 32 ? 32u : ((n0 + n1) <= 64 ? 64u : ((n0 + n1) <= 128 ? 128u : ((n0 + n1) <= 256 ? 256u : 512u)));
   // weight rows of this tile
   const int tiles_per_mat = (a.N + 127) / 128;
   const int mat = a.mode == TG_QKV ? tile / tiles_per_mat : 0;
   const int row_base = a.mode == TG_QKV ? (tile - mat * tiles_per_mat) * 128 : (a.mode == TG_SWIGLU ? tile * 64 : tile * 128);
 
-  if (warp == 1) {                                              // TMEM allocation (whole warp)
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -286,10 +289,10 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
       if (mat < 2) {
         const int vec_per_tok = half / 2;                        // float4 per token: half/4 of cos, half/4 of sin
         const int total = tokens * vec_per_tok;
-        for (int base = tid; base < total; base += 8 * TG_THREADS) {             // eight independent loads in flight per thread
-          float4 tmp[8];
+        for (int base = tid; base < total; base += TG_STG * TG_THREADS) {        // TG_STG independent loads in flight per thread
+          float4 tmp[TG_STG];
 #pragma unroll
-          for (int u = 0; u < 8; ++u) {
+          for (int u = 0; u < TG_STG; ++u) {
             const int idx = min(base + u * TG_THREADS, total - 1);
             const int t = idx / vec_per_tok, v = idx - t * vec_per_tok;
             const int row = rows_s[t];
@@ -298,7 +301,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
             tmp[u] = __ldg(reinterpret_cast<const float4*>(src));
           }
 #pragma unroll
-          for (int u = 0; u < 8; ++u) {
+          for (int u = 0; u < TG_STG; ++u) {
             const int idx = base + u * TG_THREADS;
             if (idx < total) *reinterpret_cast<float4*>(tab_s + (size_t)idx * 4) = tmp[u];
           }
@@ -488,7 +491,7 @@ int vlac_tc_setup(vlac_ctx* ctx) {
   ctx->tc_ok = 0;
   // the TMA path needs 16-byte aligned rows and pointers
   if (g.hidden % 8 || g.ffn % 8 || (g.head_dim != 64 && g.head_dim != 128)) return VLAC_OK;
-  const int n_maps = g.n_layers * TM_PER_LAYER + TM_ACT_COUNT;
+  const int n_maps = g.n_layers * TM_PER_LAYER + TM_ACT_COUNT + 1;      // + the vision projector
   CUtensorMap* host = (CUtensorMap*)malloc(sizeof(CUtensorMap) * n_maps);
   if (!host) return VLAC_ERR_OOM;
   int rc = VLAC_OK;
@@ -509,6 +512,11 @@ int vlac_tc_setup(vlac_ctx* ctx) {
     rc = encode_map(&act[TM_XN + hgt], ctx->xn, ctx->rows_max, D, box);
     if (rc == VLAC_OK) rc = encode_map(&act[TM_AO + hgt], ctx->ao, ctx->rows_max, D, box);
     if (rc == VLAC_OK) rc = encode_map(&act[TM_HM + hgt], ctx->hm, ctx->rows_max, F, box);
+  }
+  ctx->tc_proj = 0;
+  if (rc == VLAC_OK && ctx->w.proj && (reinterpret_cast<uintptr_t>(ctx->w.proj) & 15) == 0) {
+    rc = encode_map(&act[TM_ACT_COUNT], ctx->w.proj, D, D, 128);
+    if (rc == VLAC_OK) ctx->tc_proj = 1;
   }
   if (rc != VLAC_OK) { free(host); return rc; }
   ctx->tmaps_host = host;                                        // copied into the kernel parameters at every launch
@@ -535,6 +543,14 @@ static void tc_common(vlac_ctx* ctx, vlac_cache* c, int layer, TcArgs* a) {
   a->rope_cos = ctx->w.rope_cos; a->rope_sin = ctx->w.rope_sin;
   a->dev_error = ctx->dev_error;
   a->n_splits = 1;
+  {
+    const int chunk = ctx->rows_max < 512 ? ctx->rows_max : 512;          // largest token chunk a CTA can meet
+    const int n0 = ((chunk < 256 ? chunk : 256) + 15) / 16 * 16;
+    const int n1 = chunk > 256 ? (chunk - 256 + 15) / 16 * 16 : 0;
+    int cols = 32;
+    while (cols < n0 + n1) cols *= 2;
+    a->tmem_cols = cols;
+  }
   a->batch = c->batch;
 }
 
@@ -563,6 +579,33 @@ int vlac_tc_partial(vlac_ctx* ctx, vlac_cache* c, int layer, int which, int* n_s
   a.K = down ? g.ffn : g.hidden; a.N = g.hidden; a.mode = TG_PARTIAL;
   const int tiles = (g.hidden + 127) / 128;
   int splits = ctx->n_sm / tiles;                       // fill the SMs: the partial sums are folded by the next kernel
+  if (splits < 1) splits = 1;
+  if (splits > VLAC_MAX_SPLITS) splits = VLAC_MAX_SPLITS;
+  const int kb_total = (a.K + TG_BK - 1) / TG_BK;
+  if (splits > kb_total) splits = kb_total;
+  a.n_splits = splits;
+  a.part = ctx->part; a.split_stride = (size_t)ctx->rows_max * g.hidden;
+  *n_splits = splits;
+  return launch_tc(ctx, a, tiles, s);
+}
+
+// Vision projector (input rows of the vision positions): features [rows][D] x W_proj^T as K-split fp32
+// partial sums in ctx->part; the caller folds them.  The feature buffer is the caller's, so its tensor maps
+// are made here, per launch (inside a graph capture: once).
+int vlac_tc_projector(vlac_ctx* ctx, vlac_cache* c, const void* feats, int rows, int* n_splits, cudaStream_t s) {
+  const vlac_config& g = ctx->cfg;
+  if (!ctx->tc_ok || !ctx->tc_proj || (reinterpret_cast<uintptr_t>(feats) & 15) || rows > ctx->rows_max) return VLAC_ERR_INVALID_ARG;
+  const CUtensorMap* act = (const CUtensorMap*)ctx->tmaps_host + (size_t)g.n_layers * TM_PER_LAYER;
+  TcArgs a; tc_common(ctx, c, 0, &a);
+  a.tot = nullptr; a.tot_fixed = rows;
+  a.tm_a[0] = act[TM_ACT_COUNT];
+  for (int i = 0; i < 4; ++i) {
+    const int rc = encode_map(&a.tm_b[i], feats, rows, g.hidden, 64 * (i + 1));
+    if (rc != VLAC_OK) return rc;
+  }
+  a.K = g.hidden; a.N = g.hidden; a.mode = TG_PARTIAL;
+  const int tiles = (g.hidden + 127) / 128;
+  int splits = ctx->n_sm / tiles;
   if (splits < 1) splits = 1;
   if (splits > VLAC_MAX_SPLITS) splits = VLAC_MAX_SPLITS;
   const int kb_total = (a.K + TG_BK - 1) / TG_BK;

@@ -38,12 +38,17 @@ __global__ void __launch_bounds__(128) embed_rows_kernel(const bf16* embed, cons
   for (int c = threadIdx.x; c < D / 8; c += blockDim.x) dst[c] = src[c];
 }
 
-// fp32 [B*Lv][D] -> bf16 rows at the vision positions
-__global__ void __launch_bounds__(256) place_vision_rows_kernel(const float* src, bf16* hidden, int n_text_pre, int Lv, int L, int D) {
+// fp32 [splits][B*Lv][D] (K-split partial sums, added in split order) -> bf16 rows at the vision positions
+__global__ void __launch_bounds__(256) place_vision_rows_kernel(const float* src, int n_splits, size_t split_stride, bf16* hidden,
+                                                                int n_text_pre, int Lv, int L, int D) {
   const int r = blockIdx.x, b = r / Lv, v = r % Lv;
   const float* s = src + (size_t)r * D;
   bf16* d = hidden + ((size_t)b * L + n_text_pre + v) * D;
-  for (int c = threadIdx.x; c < D; c += blockDim.x) d[c] = __float2bfloat16(s[c]);
+  for (int c = threadIdx.x; c < D; c += blockDim.x) {
+    float acc = s[c];
+    for (int k = 1; k < n_splits; ++k) acc += s[(size_t)k * split_stride + c];
+    d[c] = __float2bfloat16(acc);
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -341,10 +346,18 @@ int vlac_launch_input_rows(vlac_ctx* ctx, vlac_cache* c, const void* feats, cons
                                                  ctx->Lv, ctx->L, D, g.vocab);
     VLAC_LAUNCH_CHECK(ctx);
   }
-  int rc = launch_gemm_generic(ctx, (const bf16*)feats, (const bf16*)ctx->w.proj, nullptr, nullptr, 1, ctx->scratch,
-                               nullptr, B * ctx->Lv, B * ctx->Lv, D, D, D, s);
-  if (rc) return rc;
-  place_vision_rows_kernel<<<B * ctx->Lv, 256, 0, s>>>(ctx->scratch, hidden, g.n_text_pre, ctx->Lv, ctx->L, D);
+  int n_splits = 1;
+  const float* src = ctx->scratch;
+  if (ctx->tc_ok && ctx->tc_proj && (reinterpret_cast<uintptr_t>(feats) & 15) == 0) {
+    const int rc = vlac_tc_projector(ctx, c, feats, B * ctx->Lv, &n_splits, s);
+    if (rc) return rc;
+    src = ctx->part;
+  } else {
+    const int rc = launch_gemm_generic(ctx, (const bf16*)feats, (const bf16*)ctx->w.proj, nullptr, nullptr, 1, ctx->scratch,
+                                       nullptr, B * ctx->Lv, B * ctx->Lv, D, D, D, s);
+    if (rc) return rc;
+  }
+  place_vision_rows_kernel<<<B * ctx->Lv, 256, 0, s>>>(src, n_splits, (size_t)ctx->rows_max * D, hidden, g.n_text_pre, ctx->Lv, ctx->L, D);
   VLAC_LAUNCH_CHECK(ctx);
   return VLAC_OK;
 }

@@ -64,6 +64,7 @@ struct vlac_ctx {
   void* tmaps;                       // (unused) device copy of the tensor maps
   void* tmaps_host;                  // host array of TMA tensor maps (weights per layer, activation buffers)
   int tc_ok;                         // 1: shapes fit the tensor-memory GEMM
+  int tc_proj;                       // the vision projector has a tensor map (tcgen05 path usable for the input rows)
   int pass_grid;                     // CTAs of the persistent single-row pass kernel (0: not used)
   int gemv_stream;                   // single-row products use the shared-memory-staged kernel
   void* tmap_q;                      // device tensor map of the query buffer (tiled attention)
@@ -126,6 +127,7 @@ int vlac_tc_setup(vlac_ctx* ctx);
 int vlac_tc_qkv(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s);
 int vlac_tc_partial(vlac_ctx* ctx, vlac_cache* c, int layer, int which /* 0: output proj, 1: down proj */, int* n_splits, cudaStream_t s);
 int vlac_tc_gateup(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s);
+int vlac_tc_projector(vlac_ctx* ctx, vlac_cache* c, const void* feats, int rows, int* n_splits, cudaStream_t s);
 
 // ---- tiled prefill attention (attention_kernels.cu)
 int vlac_encode_map_2d(void* out, const void* base, int rows, int cols, int box_rows);
