@@ -315,10 +315,13 @@ __global__ void __launch_bounds__(AT_THREADS, 1) attention_tile_kernel(AttnTileA
 
 // sum of the per-tile partials in tile order, divided by the number of text rows
 __global__ void __launch_bounds__(256) emit_from_tiles_kernel(const float* partial, float* attn_next_layer, size_t seq_stride,
-                                                              int tiles, int n_tp, int H, int Lv) {
+                                                              int tiles, int n_tp, int H, int Lv, size_t layer_stride_in) {
   const int h = blockIdx.x, b = blockIdx.y;
   pdl_trigger();
   pdl_wait();
+  // blockIdx.z: layer, when the partials of a whole step are folded at once
+  partial += (size_t)blockIdx.z * layer_stride_in;
+  attn_next_layer += (size_t)blockIdx.z * H * Lv;
   float* dst = attn_next_layer + (size_t)b * seq_stride + (size_t)h * Lv;
   for (int v = threadIdx.x; v < Lv; v += blockDim.x) {
     float s = 0.f;
@@ -350,6 +353,11 @@ int vlac_attention_setup(vlac_ctx* ctx) {
   int rc = vlac_encode_map_2d(&m, ctx->q, ctx->rows_max, g.hidden, AT_Q);
   if (rc != VLAC_OK) return rc;
   VLAC_CUDA_CHECK(cudaMemcpy(ctx->tmap_q, &m, sizeof(m), cudaMemcpyHostToDevice));
+  ctx->probs_all = nullptr; ctx->defer_emit = 0;
+  if (g.n_text_post > 0 &&
+      cudaMalloc(&ctx->probs_all, sizeof(float) * (size_t)g.n_layers * g.max_batch * tiles * g.n_heads * ctx->Lv) != cudaSuccess) {
+    cudaGetLastError(); return VLAC_ERR_OOM;
+  }
   ctx->attn_tiles = tiles;
   return VLAC_OK;
 }
@@ -382,7 +390,9 @@ int vlac_launch_prefill_attention(vlac_ctx* ctx, vlac_cache* c, int layer, cudaS
   a.tm_v = a.tm_k + 1;
   a.M = c->M; a.rowmap = c->rowmap + (size_t)layer * B * ctx->L;
   a.out = ctx->ao;
-  a.partial = g.n_text_post > 0 ? ctx->probs : nullptr;
+  const bool defer = ctx->defer_emit && ctx->probs_all;
+  const size_t layer_stride = (size_t)B * ctx->attn_tiles * g.n_heads * ctx->Lv;
+  a.partial = g.n_text_post > 0 ? (defer ? ctx->probs_all + (size_t)layer * layer_stride : ctx->probs) : nullptr;
   a.dev_error = ctx->dev_error;
   a.layer = layer; a.nl = g.n_layers; a.B = B; a.L = ctx->L; a.max_seq = ctx->max_seq; a.H = g.n_heads;
   a.v0 = g.n_text_pre; a.Lv = ctx->Lv; a.tiles = ctx->attn_tiles;
@@ -390,9 +400,23 @@ int vlac_launch_prefill_attention(vlac_ctx* ctx, vlac_cache* c, int layer, cudaS
   if (g.head_dim == 128) VLAC_CUDA_CHECK(launch_pdl(attention_tile_kernel<128>, grid, dim3(AT_THREADS), at_smem<128>(ctx->Lv), s, a));
   else VLAC_CUDA_CHECK(launch_pdl(attention_tile_kernel<64>, grid, dim3(AT_THREADS), at_smem<64>(ctx->Lv), s, a));
   VLAC_LAUNCH_CHECK(ctx);
+  if (defer) return VLAC_OK;
   float* dst = c->attn_next + (size_t)layer * g.n_heads * ctx->Lv;
   VLAC_CUDA_CHECK(launch_pdl(emit_from_tiles_kernel, dim3(g.n_heads, B), dim3(256), 0, s, (const float*)ctx->probs, dst,
-                             (size_t)g.n_layers * g.n_heads * ctx->Lv, ctx->attn_tiles, g.n_text_post, g.n_heads, ctx->Lv));
+                             (size_t)g.n_layers * g.n_heads * ctx->Lv, ctx->attn_tiles, g.n_text_post, g.n_heads, ctx->Lv, (size_t)0));
+  VLAC_LAUNCH_CHECK(ctx);
+  return VLAC_OK;
+}
+
+// Text-to-vision scores of all layers from the per-tile partials a step left in probs_all: off the critical
+// path of the layers (nothing in the step reads them; the next step's selection does).
+int vlac_launch_emit_all(vlac_ctx* ctx, vlac_cache* c, cudaStream_t s) {
+  const vlac_config& g = ctx->cfg;
+  if (!ctx->attn_tiles || !ctx->probs_all || g.n_text_post <= 0) return VLAC_OK;
+  const int B = c->batch;
+  VLAC_CUDA_CHECK(launch_pdl(emit_from_tiles_kernel, dim3(g.n_heads, B, g.n_layers), dim3(256), 0, s, (const float*)ctx->probs_all,
+                             c->attn_next, (size_t)g.n_layers * g.n_heads * ctx->Lv, ctx->attn_tiles, g.n_text_post, g.n_heads, ctx->Lv,
+                             (size_t)B * ctx->attn_tiles * g.n_heads * ctx->Lv));
   VLAC_LAUNCH_CHECK(ctx);
   return VLAC_OK;
 }

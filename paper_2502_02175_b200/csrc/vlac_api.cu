@@ -49,7 +49,7 @@ int fill_params(const vlac_ctx* ctx, const vlac_select_params* in, int force_ful
 void free_ctx_buffers(vlac_ctx* c) {
   cudaFree(c->xn); cudaFree(c->q); cudaFree(c->ao); cudaFree(c->hm); cudaFree(c->part); cudaFree(c->scratch);
   cudaFree(c->probs); cudaFree(c->hidden); cudaFree(c->x_dec); cudaFree(c->q_dec); cudaFree(c->ao_dec);
-  cudaFree(c->hm_dec); cudaFree(c->logits); cudaFree(c->argmax_tmp); cudaFree(c->dev_error); cudaFree(c->tmaps); cudaFree(c->tmap_q); free(c->tmaps_host);
+  cudaFree(c->hm_dec); cudaFree(c->logits); cudaFree(c->argmax_tmp); cudaFree(c->dev_error); cudaFree(c->tmaps); cudaFree(c->tmap_q); cudaFree(c->probs_all); free(c->tmaps_host);
   cudaFree(c->in_frames); cudaFree(c->in_feats); cudaFree(c->in_ids); cudaFree(c->in_forced); cudaFree(c->out_tokens); cudaFree(c->logits_all);
   for (int i = 0; i < VLAC_MAX_GRAPHS; ++i) if (c->graphs[i].used) cudaGraphExecDestroy(c->graphs[i].exec);
   for (int i = 0; i < VLAC_SEG_CAP; ++i) if (c->seg_ev[i]) cudaEventDestroy(c->seg_ev[i]);
@@ -357,11 +357,16 @@ static int enqueue_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* f
   TRY(seg_mark(ctx, s));
   // 3. layers; the down-projection partials of layer l are folded into layer l+1's first kernel
   int n_splits = 0;
+  ctx->defer_emit = ctx->attn_tiles > 0 && ctx->probs_all != nullptr;
   for (int l = 0; l < nl; ++l) {
-    TRY(vlac_launch_finalize_norm(ctx, cache, h, l == 0 ? 0 : l - 1, l == 0 ? 0 : n_splits, l, ctx->layers[l].g_attn, s));
-    TRY(vlac_launch_layer_body(ctx, cache, l, h, &n_splits, s));
+    int rc = vlac_launch_finalize_norm(ctx, cache, h, l == 0 ? 0 : l - 1, l == 0 ? 0 : n_splits, l, ctx->layers[l].g_attn, s);
+    if (rc == VLAC_OK) rc = vlac_launch_layer_body(ctx, cache, l, h, &n_splits, s);
+    if (rc != VLAC_OK) { ctx->defer_emit = 0; return rc; }
   }
+  const bool deferred = ctx->defer_emit != 0;
+  ctx->defer_emit = 0;
   TRY(vlac_launch_finalize_norm(ctx, cache, h, nl - 1, n_splits, nl - 1, nullptr, s));
+  if (deferred) TRY(vlac_launch_emit_all(ctx, cache, s));
   TRY(seg_mark(ctx, s));
   // 4. first action token
   TRY(vlac_launch_last_row(ctx, cache, h, s));

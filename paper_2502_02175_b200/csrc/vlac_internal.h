@@ -69,6 +69,8 @@ struct vlac_ctx {
   int gemv_stream;                   // single-row products use the shared-memory-staged kernel
   void* tmap_q;                      // device tensor map of the query buffer (tiled attention)
   int attn_tiles;                    // 64-query tiles per sequence, 0: tiled attention not usable
+  float* probs_all;                  // [n_layers][max_batch][tiles][n_heads][Lv]: per-tile column sums of every layer of a step
+  int defer_emit;                    // set while a whole step is enqueued: text-to-vision scores of all layers are formed by one kernel at its end
   // optional per-launch timing of the matrix-vector kernel (vlac_profile)
   int prof_on, prof_n;
   cudaEvent_t* prof_ev;              // [2 * VLAC_PROF_CAP]
@@ -134,6 +136,7 @@ int vlac_encode_map_2d(void* out, const void* base, int rows, int cols, int box_
 int vlac_attention_setup(vlac_ctx* ctx);
 int vlac_attention_cache_setup(vlac_ctx* ctx, vlac_cache* c);
 int vlac_launch_prefill_attention(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s);
+int vlac_launch_emit_all(vlac_ctx* ctx, vlac_cache* c, cudaStream_t s);   // after a step enqueued with defer_emit
 
 // ---- decode (decode_kernels.cu)
 int vlac_decode_setup(vlac_ctx* ctx);

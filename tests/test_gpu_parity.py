@@ -239,6 +239,25 @@ def test_step_7b_shape_two_layers(H, vb):
         sess.close()
 
 
+@pytest.mark.parametrize("env", [{"VLAC_PASS_KERNEL": "1"}, {"VLAC_GEMV_REG": "1"}])
+def test_step_alternative_single_row_paths(H, vb, env, monkeypatch):
+    """The opt-in single-row paths (one persistent kernel per pass; the register-pipelined matrix-vector kernel)
+    pass the same check as the default path.  The library reads the switches when a context is created."""
+    for k, v in env.items():
+        monkeypatch.setenv(k, v)
+    cfg = synth.llama7b_config(n_layers=2)
+    model = synth.make_model(cfg, 8)
+    ids = synth.make_prompt_ids(cfg, 8)
+    ep = synth.make_episode(cfg, 8, 2)
+    sess = H.Session(cfg, model)
+    try:
+        for t in range(2):
+            r = H.run_step_pair(sess, ep.frames[t][None], ep.feats[t][None], ids, H.oparams(alpha_override=[0.6, 1.0]))[0]
+            assert r["logit_err"] <= H.TOL and r["attn_err"] <= H.TOL, (t, r)
+    finally:
+        sess.close()
+
+
 def test_step_batch_of_three_ragged(H, vb):
     """Three independent sequences per step with different changed fractions (ragged row counts)."""
     cfg = synth.tiny_config()
