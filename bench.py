@@ -284,6 +284,34 @@ def run_ours(args):
     ms_full, _ = timed(K, 1 + W, full=True)
     ms_full /= K
 
+    # the part the method changes: selection + partial prefill + first action token, timed through the same
+    # entry point on a context of the same weights that generates one token per step
+    import dataclasses
+    cfg1 = dataclasses.replace(cfg, n_action=1)
+    ctx1 = vb.vlac_create(vb.make_config(cfg1, 1), dev.weights)
+    cache1 = vb.vlac_cache_alloc(ctx1, 1)
+    tok1 = torch.zeros((1, 1), dtype=torch.int32, device="cuda")
+
+    def step1(t, full=False):
+        vb.vlac_step(ctx1, cache1, frames_d[t:t + 1], feats_d[t:t + 1], ids_d, params, full, tok1)
+
+    def timed1(n, first, full):
+        for i in range(3):
+            step1(max(first - 3 + i, 0), full)
+        barrier()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for i in range(n):
+            step1(first + i, full)
+        ev1.record()
+        barrier()
+        return ev0.elapsed_time(ev1) / n
+
+    ms_prefill = timed1(K, 1 + W, False)
+    ms_prefill_full = timed1(K, 1 + W, True)
+    vb.vlac_cache_free(cache1)
+    vb.vlac_destroy(ctx1)
+
     # end to end through the C ABI: pinned host inputs in, tokens out, every step
     frames_h = torch.from_numpy(ep.frames).pin_memory()
     feats_h = torch.from_numpy(ep.feats.view(np.int16)).pin_memory()
@@ -312,7 +340,7 @@ def run_ours(args):
 
     # max over ranks
     if world > 1:
-        ms_step, ms_e2e, ms_full = max_over_ranks([ms_step, ms_e2e, ms_full], "cuda")
+        ms_step, ms_e2e, ms_full, ms_prefill, ms_prefill_full = max_over_ranks([ms_step, ms_e2e, ms_full, ms_prefill, ms_prefill_full], "cuda")
     if rank == 0:
         peak, peak_kind = _peaks()
         achieved = (k_bytes / 1e9) / (k_ms / 1e3) if k_ms > 0 else 0.0
@@ -338,6 +366,9 @@ def run_ours(args):
             "step_roofline": {"algorithmic_bytes": step_bytes, "floor_ms": step_bytes / (peak * 1e6),
                               "frac": (step_bytes / (peak * 1e6)) / ms_step},
             "full_recompute": {"ms_per_step": ms_full, "speedup_cached": ms_full / ms_step},
+            "prefill": {"note": "selection + partial prefill + first action token (a one-token context on the same weights)",
+                        "cached_ms": ms_prefill, "full_recompute_ms": ms_prefill_full, "speedup_cached": ms_prefill_full / ms_prefill,
+                        "prompt_tokens_per_s": cfg.seq_len / (ms_prefill / 1e3)},
             "control_hz": 1e3 / ms_step,
             "profiled_step_parts_ms": {"note": "direct launches with per-launch events, not the graph replay",
                                        "select": segments[0], "input_rows": segments[1], "prefill_layers": segments[2],
