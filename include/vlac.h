@@ -108,7 +108,14 @@ typedef struct {
 #define VLAC_PART_WARM       5   /* int32 [1] of seq: 0 = cold (next select reuses nothing)                */
 
 /* Create a context.  Copies `cfg` and the layer table, borrows every weight pointer, allocates the
- * workspace for max_batch sequences.  Errors: INVALID_ARG (bad shape, NULL), OOM, CUDA. */
+ * workspace for max_batch sequences.  Errors: INVALID_ARG (bad shape, NULL), OOM, CUDA.
+ *
+ * Environment switches, read here once per context (all off by default; results stay within the same
+ * tolerance, timings differ):
+ *   VLAC_NO_GRAPH=1     vlac_step launches its kernels one by one instead of replaying a captured graph
+ *   VLAC_PASS_KERNEL=1  each single-row pass (action tokens 2..n) runs as one persistent cooperative kernel
+ *   VLAC_GEMV_REG=1     single-row products use the register-pipelined kernel instead of the tensor-core one
+ *   VLAC_VERBOSE=1      CUDA errors noted by the library are also printed to stderr */
 int vlac_create(const vlac_config* cfg, const vlac_weights* w, vlac_ctx** out);
 int vlac_destroy(vlac_ctx* ctx);
 
