@@ -322,31 +322,23 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
   const int u_begin = (int)(((long long)n_units * blockIdx.x) / gridDim.x);
   const int n_local = (int)(((long long)n_units * (blockIdx.x + 1)) / gridDim.x) - u_begin;
   const int n_groups = (n_local + 7) / 8;
-  const int n_tab = ((n_units + (int)gridDim.x - 1) / (int)gridDim.x + 7) / 8 * 8;     // same for every CTA: sizes the table
   const unsigned ring_w = (unsigned)__cvta_generic_to_shared(gt_smem) + (unsigned)warp * (GT_DEPTH * GT_SLOT_BYTES);
   float* part = reinterpret_cast<float*>(gt_smem + GT_RING_BYTES);                      // [2][G][GT_WARPS][16][nbp], G * nbp = 8
-  const uint4** tab = reinterpret_cast<const uint4**>(gt_smem + GT_RING_BYTES + GT_PART_BYTES);   // [n_tab][2] row pointers
-  bf16* xs = reinterpret_cast<bf16*>(gt_smem + GT_RING_BYTES + GT_PART_BYTES + (size_t)n_tab * 16);  // [nb][K]
-
-  // row pointers of this CTA's units (the ragged end repeats the last unit: read, never stored)
-  if (n_local > 0)
-    for (int t = tid; t < n_groups * 8; t += GT_THREADS) {
-      const UnitRows r = unit_rows(a, u_begin + min(t, n_local - 1));
-      tab[2 * t] = r.pa; tab[2 * t + 1] = r.pb;
-    }
-  __syncthreads();
+  bf16* xs = reinterpret_cast<bf16*>(gt_smem + GT_RING_BYTES + GT_PART_BYTES);            // [nb][K]
 
   const int S = K / 64;                                                // sub-stages per row
   const int ns_w = warp < S ? (S - warp + GT_WARPS - 1) / GT_WARPS : 0;   // ... of this warp
   // ---- issue side: (group, sub-stage) in order; one copy group per item, empty once the work is exhausted
   int ig = 0, ij = 0, islot = 0;
   const char* rowptr[4];
+  // A lane copies rows (lane >> 3) + 4 i of a group: both rows of units (lane >> 3) and (lane >> 3) + 4.  Their
+  // addresses are worked out per group (a group is 128 KB of weights and more: the few divisions do not show);
+  // the ragged end repeats the last unit (read, never stored).
   auto load_rowptrs = [&](int g) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int row = (lane >> 3) + 4 * i;
-      rowptr[i] = reinterpret_cast<const char*>(tab[(g * 8 + (row & 7)) * 2 + (row >> 3)]);
-    }
+    const UnitRows r0 = unit_rows(a, u_begin + min(g * 8 + (lane >> 3), n_local - 1));
+    const UnitRows r1 = unit_rows(a, u_begin + min(g * 8 + (lane >> 3) + 4, n_local - 1));
+    rowptr[0] = reinterpret_cast<const char*>(r0.pa); rowptr[1] = reinterpret_cast<const char*>(r1.pa);
+    rowptr[2] = reinterpret_cast<const char*>(r0.pb); rowptr[3] = reinterpret_cast<const char*>(r1.pb);
   };
   if (n_groups > 0 && ns_w > 0) load_rowptrs(0);
   auto issue = [&]() {
@@ -913,10 +905,8 @@ __global__ void argmax_final_kernel(const unsigned long long* tmp, int n_part, i
 
 constexpr size_t GT_SMEM_MAX = 226 * 1024;      // dynamic part; the kernel also has a little static shared memory
 size_t gt_smem_bytes(const vlac_ctx* ctx, const GemvArgs& a) {
-  const int n_units = a.mode == GV_QKV ? 3 * (a.N / 2) : (a.mode == GV_SWIGLU ? a.N : (a.N + 1) / 2);
-  const int grid = ctx->n_sm * GT_GRID_PER_SM;
-  const int n_tab = ((n_units + grid - 1) / grid + 7) / 8 * 8;
-  return (size_t)GT_RING_BYTES + GT_PART_BYTES + (size_t)n_tab * 16 + (size_t)a.nb * a.K * sizeof(bf16);
+  (void)ctx;
+  return (size_t)GT_RING_BYTES + GT_PART_BYTES + (size_t)a.nb * a.K * sizeof(bf16);
 }
 
 int launch_gemv(vlac_ctx* ctx, const GemvArgs& a, cudaStream_t s) {
