@@ -115,6 +115,8 @@ typedef struct {
  *   VLAC_NO_GRAPH=1     vlac_step launches its kernels one by one instead of replaying a captured graph
  *   VLAC_PASS_KERNEL=1  each single-row pass (action tokens 2..n) runs as one persistent cooperative kernel
  *   VLAC_GEMV_REG=1     single-row products use the register-pipelined kernel instead of the tensor-core one
+ *   VLAC_GEMM_PAIR=1    Q/K/V, output and down projections of the prefill run as clusters of two CTAs that share
+ *                       the activation tile (tcgen05 cta_group::2)
  *   VLAC_VERBOSE=1      CUDA errors noted by the library are also printed to stderr */
 int vlac_create(const vlac_config* cfg, const vlac_weights* w, vlac_ctx** out);
 int vlac_destroy(vlac_ctx* ctx);

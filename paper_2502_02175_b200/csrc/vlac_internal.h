@@ -64,6 +64,7 @@ struct vlac_ctx {
   void* tmaps;                       // (unused) device copy of the tensor maps
   void* tmaps_host;                  // host array of TMA tensor maps (weights per layer, activation buffers)
   int tc_ok;                         // 1: shapes fit the tensor-memory GEMM
+  int gemm_pair;                     // prefill GEMMs with an even tile count run as two-CTA clusters (cta_group::2)
   int tc_proj;                       // the vision projector has a tensor map (tcgen05 path usable for the input rows)
   int pass_grid;                     // CTAs of the persistent single-row pass kernel (0: not used)
   int gemv_stream;                   // single-row products use the shared-memory-staged kernel

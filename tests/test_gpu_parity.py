@@ -239,10 +239,10 @@ def test_step_7b_shape_two_layers(H, vb):
         sess.close()
 
 
-@pytest.mark.parametrize("env", [{"VLAC_PASS_KERNEL": "1"}, {"VLAC_GEMV_REG": "1"}])
+@pytest.mark.parametrize("env", [{"VLAC_PASS_KERNEL": "1"}, {"VLAC_GEMV_REG": "1"}, {"VLAC_GEMM_PAIR": "1"}])
 def test_step_alternative_single_row_paths(H, vb, env, monkeypatch):
-    """The opt-in single-row paths (one persistent kernel per pass; the register-pipelined matrix-vector kernel)
-    pass the same check as the default path.  The library reads the switches when a context is created."""
+    """The opt-in paths (one persistent kernel per single-row pass; the register-pipelined matrix-vector kernel;
+    prefill GEMMs as two-CTA clusters sharing the activation tile) pass the same check as the default path.  The library reads the switches when a context is created."""
     for k, v in env.items():
         monkeypatch.setenv(k, v)
     cfg = synth.llama7b_config(n_layers=2)
