@@ -363,6 +363,13 @@ def run_ours(args):
                          # dram read+write per launch from profiles/gemv_mma_kernel_7b_shape_2layers.md: 1.029 x algorithmic
                          "traffic": 1.029 * k_bytes / max(k_n, 1), "algorithmic_bytes_per_launch": k_bytes / max(k_n, 1),
                          "launches_timed": k_n, "avg_launch_us": 1e3 * k_ms / max(k_n, 1)},
+            "single_row_pass": {"note": "one pass = 4 weight-streaming launches per layer + lm_head, with the single-row attention, argmax and "
+                                        "kernel boundaries between them; time = (step - one-token step) / (n_action - 1), graph replay",
+                                "ms": (ms_step - ms_prefill) / max(cfg.n_action - 1, 1),
+                                "weight_gbs": (2.0 * (4 * cfg.hidden * cfg.hidden + 3 * cfg.hidden * cfg.ffn) * cfg.n_layers + 2.0 * cfg.vocab * cfg.hidden)
+                                              / 1e9 / max((ms_step - ms_prefill) / max(cfg.n_action - 1, 1) / 1e3, 1e-9),
+                                "frac_of_peak": (2.0 * (4 * cfg.hidden * cfg.hidden + 3 * cfg.hidden * cfg.ffn) * cfg.n_layers + 2.0 * cfg.vocab * cfg.hidden)
+                                                / 1e9 / max((ms_step - ms_prefill) / max(cfg.n_action - 1, 1) / 1e3, 1e-9) / peak},
             "step_roofline": {"algorithmic_bytes": step_bytes, "floor_ms": step_bytes / (peak * 1e6),
                               "frac": (step_bytes / (peak * 1e6)) / ms_step},
             "full_recompute": {"ms_per_step": ms_full, "speedup_cached": ms_full / ms_step},
