@@ -210,7 +210,8 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
       asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
   }
-  pdl_wait();                                                   // everything below may read what earlier kernels wrote
+  // The live token count was written by the selection kernels, which never release their dependents early, so
+  // it is complete before any kernel launched after them starts: it may be read ahead of the dependency wait.
   // blockIdx.z selects a chunk of up to 512 tokens (one accumulator's worth of tensor-memory columns)
   const int tok0 = blockIdx.z * 512;
   const int tokens = min(max((a.tot ? *a.tot : a.tot_fixed) - tok0, 0), 512);
@@ -233,6 +234,29 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
   const int mat = a.mode == TG_QKV ? tile / tiles_per_mat : 0;
   const int row_base = a.mode == TG_QKV ? (tile - mat * tiles_per_mat) * 128 : (a.mode == TG_SWIGLU ? tile * 64 : tile * 128);
 
+  // ---- the weights depend on no earlier kernel: the weight boxes of the first ring round are requested before
+  // the dependency wait (their bytes announced without an arrival; the activation boxes follow after the wait)
+  const int n_prod = min(TG_PRODUCERS, n_stages);
+  const int pid = warp == 0 ? 0 : warp - 5;
+  const bool producer = lane == 0 && (warp == 0 || warp >= 6) && pid < n_prod;
+  auto load_weights = [&](int i, int s) {
+    unsigned char* sa = ring + (size_t)s * stage_bytes;
+    const int k = (kb0 + i) * TG_BK;
+    if (a.mode == TG_SWIGLU) {
+      tma_load_2d(sa, &a.tm_a[0], k, row_base, &full_bar[s]);                // 64 gate rows
+      tma_load_2d(sa + 64 * 128, &a.tm_a[1], k, row_base, &full_bar[s]);     // 64 up rows of the same features
+    } else {
+      tma_load_2d(sa, &a.tm_a[mat], k, row_base, &full_bar[s]);
+    }
+  };
+  const int n_early = PAIR ? 0 : min(n_kb, n_stages);           // k-blocks whose weights go out early
+  if (producer)
+    for (int i = pid; i < n_early; i += n_prod) {
+      asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&full_bar[i])), "r"((unsigned)TG_A_BYTES) : "memory");
+      load_weights(i, i);
+    }
+  pdl_wait();                                                   // everything below may read what earlier kernels wrote
+
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -245,9 +269,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
     // Each producer waits for the ring slot of its own k-blocks only.  Its previous wait proved k-block
     // i - P - n_stages consumed; the slot's previous phase (k-block i - 2 n_stages) must be complete by
     // then, or the one-bit phase parity would alias: hence no more producers than stages.
-    const int n_prod = min(TG_PRODUCERS, n_stages);
-    const int pid = warp == 0 ? 0 : warp - 5;
-    if (lane == 0 && pid < n_prod) {
+    if (producer) {
       const int rows0 = min(n_boxes, 4), rows1 = n_boxes - rows0;            // boxes of the first / second token request
       for (int i = pid; i < n_kb; i += n_prod) {
         const int s = i % n_stages;
@@ -269,12 +291,11 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
           }
           continue;
         }
-        mbar_expect_tx(&full_bar[s], (unsigned)stage_bytes);
-        if (a.mode == TG_SWIGLU) {
-          tma_load_2d(sa, &a.tm_a[0], k, row_base, &full_bar[s]);                // 64 gate rows
-          tma_load_2d(sa + 64 * 128, &a.tm_a[1], k, row_base, &full_bar[s]);     // 64 up rows of the same features
+        if (i < n_early) {
+          mbar_expect_tx(&full_bar[s], (unsigned)(stage_bytes - TG_A_BYTES));     // the weights of this k-block are on their way
         } else {
-          tma_load_2d(sa, &a.tm_a[mat], k, row_base, &full_bar[s]);
+          mbar_expect_tx(&full_bar[s], (unsigned)stage_bytes);
+          load_weights(i, s);
         }
         tma_load_2d(sb, &a.tm_b[rows0 - 1], k, tok0, &full_bar[s]);
         if (rows1 > 0) tma_load_2d(sb + 4 * TG_BOX_BYTES, &a.tm_b[rows1 - 1], k, tok0 + 256, &full_bar[s]);
