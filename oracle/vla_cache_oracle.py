@@ -337,7 +337,7 @@ def silu(x: np.ndarray) -> np.ndarray:
 
 def layer_forward(cfg, layer_w: Dict[str, np.ndarray], K: np.ndarray, V: np.ndarray,
                   hidden: np.ndarray, rows: np.ndarray, cos: np.ndarray, sin: np.ndarray,
-                  emit_attention: bool = True) -> Optional[np.ndarray]:
+                  emit_attention: bool = True, block_start: Optional[int] = None) -> Optional[np.ndarray]:
     """One decoder layer over the positions in ``rows`` only (Algorithm 2, Sec. 4.1).
 
     ``K``/``V`` are this layer's cache ``[max_seq, heads, d]`` and are updated in place at
@@ -345,7 +345,9 @@ def layer_forward(cfg, layer_w: Dict[str, np.ndarray], K: np.ndarray, V: np.ndar
     is ``[>= max(rows)+1, hidden]`` and is updated in place at ``rows``.  A recomputed query
     at position ``p`` attends to all cache positions ``<= p`` (Sec. 3.1 attention; the mask
     follows original positions, Appendix "Position and Attention Masking"), whether their
-    K/V are fresh or reused.  Keys are stored after rotation.
+    K/V are fresh or reused.  Keys are stored after rotation.  With ``block_start`` the rows
+    at positions ``>= block_start`` form one block that is decoded in parallel: each of them
+    also sees the block's later positions (see ``step_chunk``).
 
     Returns, if asked, ``[heads, L_v]``: the softmax probability on each vision key averaged
     over the prompt-text query rows that follow the vision block (Eq. avistext, read as
@@ -367,6 +369,8 @@ def layer_forward(cfg, layer_w: Dict[str, np.ndarray], K: np.ndarray, V: np.ndar
     n_keys = int(rows.max()) + 1
     key_pos = np.arange(n_keys)
     visible = key_pos[None, :] <= rows[:, None]                      # [rows, keys]
+    if block_start is not None:
+        visible = visible | ((rows[:, None] >= block_start) & (key_pos[None, :] >= block_start))
     v0 = cfg.n_text_pre
     v1 = v0 + cfg.n_vision
     text_q = (rows >= v1) & (rows < cfg.seq_len)
@@ -462,4 +466,48 @@ def step(cfg, model: Dict[str, object], cache: CacheState, frames_t: np.ndarray,
     cache.prev_frames = np.array(frames_t, copy=True)
     cache.warm = True
     return StepResult(tokens=tokens, fed_tokens=fed, logits=logits, margins=margins,
+                      selection=sel, hidden=hidden, attn_tv=attn_next)
+
+
+def step_chunk(cfg, model: Dict[str, object], cache: CacheState, frames_t: np.ndarray,
+               feats_bf16: np.ndarray, prompt_ids: np.ndarray, params: SelectParams,
+               act_embed_bf16: np.ndarray, force_full: bool = False,
+               selection: Optional[Selection] = None) -> StepResult:
+    """Selection and partial prefill as in ``step``, then ALL action tokens from one pass.
+
+    The paper applies the method unchanged to OpenVLA-OFT, "a faster variant with action
+    chunking" (main LIBERO results), and gives no equations for that decoder.  Reading taken
+    here: behind the prompt sit ``n_action`` placeholder rows at positions ``L .. L+n_action-1``
+    whose input is the fixed embedding ``act_embed_bf16[i]`` (a weight, not a fed-back token).
+    They run through every layer together: each sees the whole prompt (reused or fresh K/V, as
+    the prefill left it) and every row of the chunk, in both directions; their K/V are written
+    behind the prompt and overwritten by the next step.  Token ``i`` is the argmax (ties to the
+    lower id) of the logits of row ``L+i``.  The prefill's own last-row logits are not used.
+    ``fed_tokens`` of the result equals ``tokens``: nothing is fed back.
+    """
+    sel = selection if selection is not None else select(cfg, frames_t, cache, params, force_full)
+    cos, sin = model["rope_cos"], model["rope_sin"]
+    hidden = input_rows(cfg, model, feats_bf16, prompt_ids)
+    attn_next = np.zeros((cfg.n_layers, cfg.n_heads, cfg.n_vision), dtype=np.float64)
+    for l in range(cfg.n_layers):
+        attn_next[l] = layer_forward(cfg, model["layers"][l], cache.K[l], cache.V[l], hidden,
+                                     sel.rows[l], cos, sin, emit_attention=True)
+    L, n = cfg.seq_len, cfg.n_action
+    chunk_rows = np.arange(L, L + n, dtype=np.int64)
+    hidden[chunk_rows] = widen_bf16(np.asarray(act_embed_bf16).reshape(n, cfg.hidden))
+    for l in range(cfg.n_layers):
+        layer_forward(cfg, model["layers"][l], cache.K[l], cache.V[l], hidden, chunk_rows, cos, sin,
+                      emit_attention=False, block_start=L)
+    tokens = np.zeros(n, dtype=np.int64)
+    logits = np.zeros((n, cfg.vocab), dtype=np.float64)
+    margins = np.zeros(n, dtype=np.float64)
+    for i in range(n):
+        logits[i] = _logits(cfg, model, hidden[L + i])
+        tokens[i] = int(np.argmax(logits[i]))
+        top2 = np.partition(logits[i], -2)[-2:]
+        margins[i] = float(top2[1] - top2[0])
+    cache.attn_tv = attn_next
+    cache.prev_frames = np.array(frames_t, copy=True)
+    cache.warm = True
+    return StepResult(tokens=tokens, fed_tokens=tokens.copy(), logits=logits, margins=margins,
                       selection=sel, hidden=hidden, attn_tv=attn_next)

@@ -78,8 +78,9 @@ class ModelConfig:
 
     @property
     def max_seq(self) -> int:
-        """Prefill length plus room for the K/V of the fed-back action tokens."""
-        return self.seq_len + max(self.n_action - 1, 0)
+        """Prefill length plus room for the K/V of the action rows (one per action token: the fed-back
+        tokens use all but the last, a chunk decoded in parallel uses all)."""
+        return self.seq_len + self.n_action
 
     @property
     def frame_hw(self) -> int:
@@ -173,6 +174,13 @@ def make_prompt_ids(cfg: ModelConfig, seed: int, batch: int = 1) -> np.ndarray:
     """Random token ids ``[batch, n_text]`` (pre-vision tokens first, then post-vision)."""
     rng = np.random.default_rng(seed + 7919)
     return rng.integers(0, cfg.vocab, size=(batch, cfg.n_text), dtype=np.int32)
+
+
+def make_action_embed(cfg: ModelConfig, seed: int) -> np.ndarray:
+    """Placeholder embeddings ``[n_action, hidden]`` (bf16 bits) of the action rows that a chunk
+    decoded in parallel starts from; same distribution as the token embeddings."""
+    rng = np.random.default_rng(seed + 15485863)
+    return _normal_bf16(rng, (cfg.n_action, cfg.hidden), 0.02)
 
 
 def make_hidden(cfg: ModelConfig, seed: int, batch: int = 1, std: float = 1.0) -> np.ndarray:

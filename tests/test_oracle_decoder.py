@@ -37,15 +37,18 @@ def _torch_rope(x, cos, sin):
     return x * c + rot * s
 
 
-def _torch_layer(cfg, lw, h, cos, sin):
-    """Textbook Llama layer over a full causal sequence in fp64."""
+def _torch_layer(cfg, lw, h, cos, sin, mask=None):
+    """Textbook Llama layer over a full sequence in fp64: causal, or with a boolean mask [L, L]."""
     L, H, d = h.shape[0], cfg.n_heads, cfg.head_dim
     F = torch.nn.functional
     xn = F.rms_norm(h, (cfg.hidden,), _t(lw["g_attn"]), cfg.rms_eps)
     q = _torch_rope(F.linear(xn, _t(lw["wq"])).view(L, H, d), cos, sin)
     k = _torch_rope(F.linear(xn, _t(lw["wk"])).view(L, H, d), cos, sin)
     v = F.linear(xn, _t(lw["wv"])).view(L, H, d)
-    o = F.scaled_dot_product_attention(q.transpose(0, 1), k.transpose(0, 1), v.transpose(0, 1), is_causal=True)
+    if mask is None:
+        o = F.scaled_dot_product_attention(q.transpose(0, 1), k.transpose(0, 1), v.transpose(0, 1), is_causal=True)
+    else:
+        o = F.scaled_dot_product_attention(q.transpose(0, 1), k.transpose(0, 1), v.transpose(0, 1), attn_mask=mask)
     h = h + F.linear(o.transpose(0, 1).reshape(L, H * d), _t(lw["wo"]))
     xn = F.rms_norm(h, (cfg.hidden,), _t(lw["g_mlp"]), cfg.rms_eps)
     return h + F.linear(F.silu(F.linear(xn, _t(lw["w_gate"]))) * F.linear(xn, _t(lw["w_up"])), _t(lw["w_down"])), k, v
@@ -164,6 +167,59 @@ def test_decode_pass_equals_longer_prefill():
     assert int(torch.argmax(logits)) == int(res.tokens[1])
     logits0 = F.linear(F.rms_norm(ht[L - 1], (cfg.hidden,), _t(model["g_final"]), cfg.rms_eps), _t(model["lm_head"]))
     np.testing.assert_allclose(res.logits[0], logits0.numpy(), atol=1e-9)
+
+
+def test_chunk_pass_equals_joint_forward_with_block_mask():
+    """A chunk of action rows decoded in parallel behind a full prefill equals ONE forward of
+    textbook layers over prompt + chunk under the mask "causal, except that chunk rows see the
+    whole chunk": the prompt rows never see the chunk, so prefill-then-chunk and the joint pass
+    are the same function.  Pins the mask, the positions of the chunk rows and the K/V append."""
+    cfg, model, ids, feats = _tiny()
+    L, n = cfg.seq_len, cfg.n_action
+    act = synth.make_action_embed(cfg, 3)
+    cache = orc.new_cache(cfg)
+    res = orc.step_chunk(cfg, model, cache, np.zeros((1, 112, 112, 3), np.uint8), feats, ids, orc.SelectParams(), act)
+    h = orc.input_rows(cfg, model, feats, ids)
+    h[L:L + n] = orc.widen_bf16(act)
+    ht = torch.from_numpy(h[:L + n].copy())
+    cos = torch.from_numpy(model["rope_cos"][:L + n].astype(np.float64)); sin = torch.from_numpy(model["rope_sin"][:L + n].astype(np.float64))
+    mask = torch.tril(torch.ones(L + n, L + n, dtype=torch.bool))
+    mask[L:, L:] = True
+    for l in range(cfg.n_layers):
+        ht, k, v = _torch_layer(cfg, model["layers"][l], ht, cos, sin, mask=mask)
+        np.testing.assert_allclose(cache.K[l][:L + n], k.numpy(), atol=1e-10)
+        np.testing.assert_allclose(cache.V[l][:L + n], v.numpy(), atol=1e-10)
+    F = torch.nn.functional
+    logits = F.linear(F.rms_norm(ht[L:], (cfg.hidden,), _t(model["g_final"]), cfg.rms_eps), _t(model["lm_head"]))
+    np.testing.assert_allclose(res.logits, logits.numpy(), atol=1e-9)
+    assert torch.argmax(logits, dim=1).tolist() == res.tokens.tolist()
+    # the mask matters: a purely causal pass gives other logits for every row but the last
+    hc = torch.from_numpy(h[:L + n].copy())
+    for l in range(cfg.n_layers):
+        hc, _, _ = _torch_layer(cfg, model["layers"][l], hc, cos, sin)
+    lc = F.linear(F.rms_norm(hc[L:], (cfg.hidden,), _t(model["g_final"]), cfg.rms_eps), _t(model["lm_head"])).numpy()
+    assert np.abs(lc[:-1] - res.logits[:-1]).max() > 1e-6
+
+
+def test_chunk_step_leaves_the_prompt_state_of_an_ordinary_step():
+    """The chunk pass writes only behind the prompt: selection, prompt K/V, prompt hidden rows and the
+    emitted text-to-vision attention of a chunk step equal those of an ordinary step on the same
+    inputs, cold and cached."""
+    cfg, model, ids, feats = _tiny()
+    L = cfg.seq_len
+    act = synth.make_action_embed(cfg, 3)
+    prev, cur, _ = synth.rerandomised_pair(cfg, 0, 13)
+    params = orc.SelectParams(top_k=32, alpha_override=[0.5, 1.0])
+    ca, cb = orc.new_cache(cfg), orc.new_cache(cfg)
+    for frame in (prev, cur):
+        ra = orc.step(cfg, model, ca, frame, feats, ids, params)
+        rb = orc.step_chunk(cfg, model, cb, frame, feats, ids, params, act)
+        assert [r.tolist() for r in ra.selection.rows] == [r.tolist() for r in rb.selection.rows]
+        np.testing.assert_array_equal(ca.K[:, :L], cb.K[:, :L])
+        np.testing.assert_array_equal(ca.V[:, :L], cb.V[:, :L])
+        np.testing.assert_array_equal(ra.hidden[:L], rb.hidden[:L])
+        np.testing.assert_array_equal(ra.attn_tv, rb.attn_tv)
+    assert rb.selection.M[1] < L
 
 
 def _two_steps(cfg, model, ids, feats0, feats1, prev, cur, params, force_full=False):
