@@ -56,7 +56,7 @@ typedef struct {
 
 /* Whole model.  `layers` is a HOST array of n_layers structs (copied at create); all other
  * pointers are device memory that must outlive the context.  rope_cos/rope_sin are fp32
- * [L + n_action - 1][head_dim/2]: cos/sin(pos * theta^(-2i/head_dim)), rotate-half pairing. */
+ * [L + n_action][head_dim/2]: cos/sin(pos * theta^(-2i/head_dim)), rotate-half pairing. */
 typedef struct {
   const vlac_layer_w* layers;
   const void *embed;      /* bf16 [vocab][hidden]            */
@@ -122,7 +122,7 @@ int vlac_create(const vlac_config* cfg, const vlac_weights* w, vlac_ctx** out);
 int vlac_destroy(vlac_ctx* ctx);
 
 /* Allocate the persistent state of `batch` (1..max_batch) independent sequences: per layer K/V
- * caches of L + n_action - 1 positions (bf16, keys stored after rotation), the previous frame, the
+ * caches of L + n_action positions (bf16, keys stored after rotation), the previous frame, the
  * text-to-vision attention scores saved by the previous step (Sec. 3.3), and the selection buffers.
  * The cache starts cold.  Library-owned device memory; release with vlac_cache_free. */
 int vlac_cache_alloc(vlac_ctx* ctx, int batch, vlac_cache** out);
@@ -176,6 +176,25 @@ int vlac_layer_forward(vlac_ctx* ctx, vlac_cache* cache, int layer, void* hidden
 int vlac_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, const void* vision_feats,
               const int* prompt_ids, const vlac_select_params* params, int force_full,
               int* action_tokens, float* all_logits, const int* forced_tokens, void* stream);
+
+/* One control step whose action tokens all come from ONE parallel pass (the paper applies the method
+ * to OpenVLA-OFT, "a faster variant with action chunking", Sec. 5 main LIBERO results and Table 2,
+ * and prints no equations for that decoder; the reading taken is stated here).  Selection, input rows
+ * and the partial prefill are those of vlac_step.  Then n_action placeholder rows at positions
+ * L .. L+n_action-1, whose input is act_embed[i] for every sequence, go through all layers together:
+ * each sees the whole prompt (reused or fresh K/V, as the prefill left it) and every row of the
+ * chunk, in both directions.  Their K/V are written behind the prompt and overwritten by the next
+ * step.  Token i is the argmax (ties to the lower id) of the logits of row L+i; the prompt's last-row
+ * logits are not formed and nothing is fed back.
+ *   act_embed     device bf16 [n_action][hidden], caller-owned, must stay alive and unchanged while a
+ *                 captured step that read it may be replayed (as for the weights)
+ *   action_tokens device int32 [batch][n_action];  all_logits device fp32 [batch][n_action][vocab] or NULL
+ * The rows of one sequence's chunk are the columns of the single-row kernels, so n_action <= 8 is
+ * required (INVALID_ARG otherwise); sequences of a batch are taken one after the other.  Other
+ * arguments, errors and stream behaviour as for vlac_step. */
+int vlac_step_chunk(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, const void* vision_feats,
+                    const int* prompt_ids, const vlac_select_params* params, int force_full, const void* act_embed,
+                    int* action_tokens, float* all_logits, void* stream);
 
 /* Views of the selection held by the cache (after select / select_import / step). */
 int vlac_selection_view(vlac_cache* cache, vlac_selection* out);

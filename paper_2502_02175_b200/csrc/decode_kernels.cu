@@ -28,6 +28,8 @@ struct GemvArgs {
   bf16 *kc, *vc;           // QKV: [nb][max_seq][N]
   const float *rope_cos, *rope_sin;
   int pos, max_seq, d;
+  int cps;                 // QKV: columns per sequence (0 or 1: one row per sequence at position `pos`; n: column c is
+                           // row pos + c % n of sequence c / n -- an action chunk decoded in parallel)
   float* x_out;            // RESID: [nb][N] +=
   bf16* h_out;             // SWIGLU: [nb][N]
   float* logits;           // LOGITS: [nb][N]
@@ -80,7 +82,8 @@ __device__ __forceinline__ void unit_operands(const GemvArgs& a, const UnitRows&
   if (a.mode == GV_QKV) {
     if (cu.mat < 2) {
       const int half = a.d / 2, j = cu.rowA % a.d;
-      pre[0] = a.rope_cos[(size_t)a.pos * half + j]; pre[1] = a.rope_sin[(size_t)a.pos * half + j];
+      const int p = a.cps > 1 ? a.pos + b % a.cps : a.pos;
+      pre[0] = a.rope_cos[(size_t)p * half + j]; pre[1] = a.rope_sin[(size_t)p * half + j];
     }
   } else if (a.mode == GV_RESID) {
     pre[0] = a.x_out[(size_t)b * a.N + cu.rowA]; pre[1] = a.x_out[(size_t)b * a.N + cu.rowB];
@@ -90,15 +93,17 @@ __device__ __forceinline__ void unit_operands(const GemvArgs& a, const UnitRows&
 __device__ __forceinline__ void store_unit(const GemvArgs& a, const UnitRows& cu, int b, float ya, float yb, const float* pre = nullptr) {
   const int rowA = cu.rowA, rowB = cu.rowB, mat = cu.mat;
   if (a.mode == GV_QKV) {
+    const int p = a.cps > 1 ? a.pos + b % a.cps : a.pos;           // position of column b, and the sequence whose cache takes it
+    const int sb = a.cps > 1 ? b / a.cps : b;
     if (mat == 2) {
-      bf16* dst = a.vc + ((size_t)b * a.max_seq + a.pos) * a.N;
+      bf16* dst = a.vc + ((size_t)sb * a.max_seq + p) * a.N;
       dst[rowA] = __float2bfloat16(ya); dst[rowB] = __float2bfloat16(yb);
     } else {
       const int half = a.d / 2;
       const int j = rowA % a.d;
-      const float c = pre ? pre[0] : a.rope_cos[(size_t)a.pos * half + j], s = pre ? pre[1] : a.rope_sin[(size_t)a.pos * half + j];
+      const float c = pre ? pre[0] : a.rope_cos[(size_t)p * half + j], s = pre ? pre[1] : a.rope_sin[(size_t)p * half + j];
       const float r1 = ya * c - yb * s, r2 = yb * c + ya * s;
-      bf16* dst = mat == 0 ? a.q_out + (size_t)b * a.N : a.kc + ((size_t)b * a.max_seq + a.pos) * a.N;
+      bf16* dst = mat == 0 ? a.q_out + (size_t)b * a.N : a.kc + ((size_t)sb * a.max_seq + p) * a.N;
       dst[rowA] = __float2bfloat16(r1); dst[rowB] = __float2bfloat16(r2);
     }
   } else if (a.mode == GV_SWIGLU) {
@@ -512,14 +517,18 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
 // eight warps, each lane owning d/32 consecutive dimensions, partial sums combined in warp order.
 template <int DPL, int NT>      // dimensions per lane = head_dim / 32; threads of the CTA
 __device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc, const bf16* vc, bf16* out,
-                                                      int pos, int max_seq, int H, int h, int b, float* dsm, float* red) {
+                                                      int pos, int max_seq, int H, int h, int b, float* dsm, float* red,
+                                                      int cps = 1) {
   constexpr int d = 32 * DPL;
   constexpr int NW = NT / 32;
   float* qs = dsm;                 // [d]
   float* p = dsm + d;              // [max_seq]
   float* part = p + max_seq;       // [NW][d]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int D = H * d, nkeys = pos + 1;
+  // cps > 1: query column b is one row of an action chunk of cps rows at positions pos .. pos + cps - 1 of
+  // sequence b / cps, and sees the prompt and the whole chunk
+  const int D = H * d, nkeys = pos + cps;
+  const int sb = b / cps;
   const float scale = rsqrtf((float)d);
   // (q may have been written by another SM earlier in the same kernel: read it past the L1)
   if (tid < d) {
@@ -527,7 +536,7 @@ __device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc
     qs[tid] = __uint_as_float((unsigned)raw << 16) * scale;
   }
   __syncthreads();
-  const bf16* kbase = kc + (size_t)b * max_seq * D + h * d;
+  const bf16* kbase = kc + (size_t)sb * max_seq * D + h * d;
   float mx = -INFINITY;
   for (int j = tid; j < nkeys; j += NT) {
     const uint4* kp = reinterpret_cast<const uint4*>(kbase + (size_t)j * D);
@@ -567,7 +576,7 @@ __device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc
   for (int w = 0; w < NW; ++w) tot += red[w];
   const float inv = 1.f / tot;
   // P * V
-  const bf16* vbase = vc + (size_t)b * max_seq * D + h * d + lane * DPL;
+  const bf16* vbase = vc + (size_t)sb * max_seq * D + h * d + lane * DPL;
   float acc[DPL];
 #pragma unroll
   for (int e = 0; e < DPL; ++e) acc[e] = 0.f;
@@ -605,12 +614,12 @@ __device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc
 
 template <int DPL>
 __global__ void __launch_bounds__(256) decode_attention_kernel(const bf16* q, const bf16* kc, const bf16* vc, bf16* out,
-                                                               int pos, int max_seq, int H) {
+                                                               int pos, int max_seq, int H, int cps) {
   extern __shared__ float dsm[];
   __shared__ float red[8];
   pdl_trigger();
   pdl_wait();
-  decode_attention_body<DPL, 256>(q, kc, vc, out, pos, max_seq, H, blockIdx.x, blockIdx.y, dsm, red);
+  decode_attention_body<DPL, 256>(q, kc, vc, out, pos, max_seq, H, blockIdx.x, blockIdx.y, dsm, red, cps);
 }
 
 // ---- one whole single-row pass as ONE persistent kernel -------------------------------------------
@@ -858,6 +867,14 @@ __global__ void __launch_bounds__(256) embed_token_kernel(const bf16* embed, con
   for (int k = threadIdx.x; k < D; k += blockDim.x) x[(size_t)b * D + k] = bf2f(embed[(size_t)id * D + k]);
 }
 
+// input of an action chunk decoded in parallel: column c starts from placeholder embedding c % n
+__global__ void __launch_bounds__(256) embed_chunk_kernel(const bf16* act_embed, int n, float* x, int D) {
+  const int c = blockIdx.x;
+  pdl_trigger();
+  pdl_wait();
+  for (int k = threadIdx.x; k < D; k += blockDim.x) x[(size_t)c * D + k] = bf2f(act_embed[(size_t)(c % n) * D + k]);
+}
+
 __global__ void __launch_bounds__(256) last_row_kernel(const bf16* hidden, float* x, int L, int D) {
   const int b = blockIdx.x;
   const bf16* src = hidden + ((size_t)b * L + (L - 1)) * D;
@@ -943,9 +960,13 @@ int vlac_decode_setup(vlac_ctx* ctx) {
   const int kmax = ctx->cfg.ffn > ctx->cfg.hidden ? ctx->cfg.ffn : ctx->cfg.hidden;
   const int mb = ctx->cfg.max_batch;
   if (mb > 8) return VLAC_ERR_INVALID_ARG;
-  const int NB = mb <= 1 ? 1 : (mb <= 2 ? 2 : (mb <= 4 ? 4 : 8));
-  const size_t smem = (size_t)NB * kmax * sizeof(bf16);
-  if (smem > 227 * 1024) return VLAC_ERR_INVALID_ARG;
+  const int NB_seq = mb <= 1 ? 1 : (mb <= 2 ? 2 : (mb <= 4 ? 4 : 8));
+  if ((size_t)NB_seq * kmax * sizeof(bf16) > 227 * 1024) return VLAC_ERR_INVALID_ARG;
+  // an action chunk decoded in parallel is one pass with n_action columns: usable if they fit like a batch does
+  const int na = ctx->cfg.n_action;
+  const int NB_chunk = na <= 1 ? 1 : (na <= 2 ? 2 : (na <= 4 ? 4 : 8));
+  ctx->chunk_ok = (na <= 8 && (size_t)NB_chunk * kmax * sizeof(bf16) <= 227 * 1024) ? 1 : 0;
+  const int NB = (ctx->chunk_ok && NB_chunk > NB_seq) ? NB_chunk : NB_seq;
   VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_pair_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(1 * (size_t)kmax * 2)));
   if (NB >= 2) VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_pair_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * (size_t)kmax * 2)));
   if (NB >= 4) VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_pair_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(4 * (size_t)kmax * 2)));
@@ -960,7 +981,7 @@ int vlac_decode_setup(vlac_ctx* ctx) {
   // the per-phase kernels replayed from a graph.  A grid barrier under a saturated memory system costs more
   // than a programmatic kernel boundary, and the ring (19 MB over the GPU) covers under 3 us of streaming.
   if (getenv("VLAC_PASS_KERNEL") != nullptr && ctx->max_seq > 0 && ctx->cfg.hidden % 64 == 0 && ctx->cfg.ffn % 64 == 0) {
-    const size_t psm = pass_smem(ctx, NB);
+    const size_t psm = pass_smem(ctx, NB_seq);
     int per_sm = 0, coop = 0, dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
@@ -1081,10 +1102,10 @@ int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens,
       const bf16 *q = ctx->q_dec, *kc = ph[0].kc, *vc = ph[0].vc;
       cudaError_t e;
       switch (g.head_dim / 32) {
-        case 1: e = launch_pdl(decode_attention_kernel<1>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads); break;
-        case 2: e = launch_pdl(decode_attention_kernel<2>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads); break;
-        case 3: e = launch_pdl(decode_attention_kernel<3>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads); break;
-        default: e = launch_pdl(decode_attention_kernel<4>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads); break;
+        case 1: e = launch_pdl(decode_attention_kernel<1>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, 1); break;
+        case 2: e = launch_pdl(decode_attention_kernel<2>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, 1); break;
+        case 3: e = launch_pdl(decode_attention_kernel<3>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, 1); break;
+        default: e = launch_pdl(decode_attention_kernel<4>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, 1); break;
       }
       VLAC_CUDA_CHECK(e);
       VLAC_LAUNCH_CHECK(ctx);
@@ -1093,6 +1114,62 @@ int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens,
       rc = launch_gemv(ctx, ph[k], s);
       if (rc) return rc;
     }
+  }
+  return VLAC_OK;
+}
+
+// One pass of all n_action placeholder rows of every sequence through all layers (an action chunk decoded in
+// parallel), then the logits and the greedy token of each row.  The rows of a sequence are the columns of the
+// matrix-vector kernels (at most 8); sequences are taken one after the other.
+int vlac_launch_chunk_pass(vlac_ctx* ctx, vlac_cache* c, const void* act_embed, int* tokens_out, float* logits_copy, cudaStream_t s) {
+  const vlac_config& g = ctx->cfg;
+  const int D = g.hidden, B = c->batch, n = g.n_action;
+  if (!ctx->chunk_ok) return VLAC_ERR_INVALID_ARG;
+  for (int b = 0; b < B; ++b) {
+    VLAC_CUDA_CHECK(launch_pdl(embed_chunk_kernel, dim3(n), dim3(256), 0, s, (const bf16*)act_embed, n, ctx->x_dec, D));
+    VLAC_LAUNCH_CHECK(ctx);
+    for (int l = 0; l < g.n_layers; ++l) {
+      GemvArgs ph[4];
+      layer_phases(ctx, c, l, ctx->L, ph);
+      for (int k = 0; k < 4; ++k) ph[k].nb = n;
+      ph[0].cps = n;
+      ph[0].kc += (size_t)b * kv_layer_elems(ctx);
+      ph[0].vc += (size_t)b * kv_layer_elems(ctx);
+      int rc = launch_gemv(ctx, ph[0], s);
+      if (rc) return rc;
+      {
+        const size_t smem = (size_t)(g.head_dim + ctx->max_seq + 8 * g.head_dim) * sizeof(float);
+        const dim3 grid(g.n_heads, n);
+        const bf16 *q = ctx->q_dec, *kc = ph[0].kc, *vc = ph[0].vc;
+        const int pos = ctx->L;
+        cudaError_t e;
+        switch (g.head_dim / 32) {
+          case 1: e = launch_pdl(decode_attention_kernel<1>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, n); break;
+          case 2: e = launch_pdl(decode_attention_kernel<2>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, n); break;
+          case 3: e = launch_pdl(decode_attention_kernel<3>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, n); break;
+          default: e = launch_pdl(decode_attention_kernel<4>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, n); break;
+        }
+        VLAC_CUDA_CHECK(e);
+        VLAC_LAUNCH_CHECK(ctx);
+      }
+      for (int k = 1; k < 4; ++k) {
+        rc = launch_gemv(ctx, ph[k], s);
+        if (rc) return rc;
+      }
+    }
+    GemvArgs a = logits_phase(ctx, c);
+    a.nb = n;
+    int rc = launch_gemv(ctx, a, s);
+    if (rc) return rc;
+    VLAC_CUDA_CHECK(launch_pdl(argmax_partial_kernel, dim3(VLAC_ARGMAX_BLOCKS, n), dim3(256), 0, s, (const float*)ctx->logits, g.vocab,
+                               ctx->argmax_tmp));
+    VLAC_LAUNCH_CHECK(ctx);
+    VLAC_CUDA_CHECK(launch_pdl(argmax_final_kernel, dim3(n), dim3(32), 0, s, (const unsigned long long*)ctx->argmax_tmp,
+                               (int)VLAC_ARGMAX_BLOCKS, tokens_out + (size_t)b * n, 1, 0));
+    VLAC_LAUNCH_CHECK(ctx);
+    if (logits_copy)
+      VLAC_CUDA_CHECK(cudaMemcpyAsync(logits_copy + (size_t)b * n * g.vocab, ctx->logits, sizeof(float) * (size_t)n * g.vocab,
+                                      cudaMemcpyDeviceToDevice, s));
   }
   return VLAC_OK;
 }

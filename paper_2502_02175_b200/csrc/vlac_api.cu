@@ -114,7 +114,7 @@ int vlac_create(const vlac_config* cfg, const vlac_weights* w, vlac_ctx** out) {
   c->w.layers = c->layers;
   c->Lv = g.n_cams * g.grid * g.grid;
   c->L = g.n_text_pre + c->Lv + g.n_text_post;
-  c->max_seq = c->L + g.n_action - 1;
+  c->max_seq = c->L + g.n_action;                 // one cache row per action token behind the prompt
   c->frame_hw = g.grid * g.patch;
   c->rows_max = g.max_batch * c->L;
   int dev = 0;
@@ -126,6 +126,8 @@ int vlac_create(const vlac_config* cfg, const vlac_weights* w, vlac_ctx** out) {
   }
   c->n_sm = prop.multiProcessorCount;
   const size_t R = c->rows_max, D = g.hidden, F = g.ffn, B = g.max_batch;
+  const size_t na8 = (size_t)(g.n_action < 8 ? g.n_action : 8);
+  const size_t R1 = B > na8 ? B : na8;               // columns of the single-row kernels: sequences, or the rows of one action chunk
   const size_t wide = (3 * D > 2 * F ? 3 * D : 2 * F);
   int rc = VLAC_OK;
   if (rc == VLAC_OK) rc = dev_alloc(&c->xn, R * D);
@@ -136,12 +138,12 @@ int vlac_create(const vlac_config* cfg, const vlac_weights* w, vlac_ctx** out) {
   if (rc == VLAC_OK) rc = dev_alloc(&c->scratch, R * wide);
   if (rc == VLAC_OK) rc = dev_alloc(&c->probs, B * (size_t)g.n_text_post * g.n_heads * c->Lv);
   if (rc == VLAC_OK) rc = dev_alloc(&c->hidden, R * D);
-  if (rc == VLAC_OK) rc = dev_alloc(&c->x_dec, B * D);
-  if (rc == VLAC_OK) rc = dev_alloc(&c->q_dec, B * D);
-  if (rc == VLAC_OK) rc = dev_alloc(&c->ao_dec, B * D);
-  if (rc == VLAC_OK) rc = dev_alloc(&c->hm_dec, B * F);
-  if (rc == VLAC_OK) rc = dev_alloc(&c->logits, B * (size_t)g.vocab);
-  if (rc == VLAC_OK) rc = dev_alloc(&c->argmax_tmp, B * VLAC_ARGMAX_BLOCKS);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->x_dec, R1 * D);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->q_dec, R1 * D);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->ao_dec, R1 * D);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->hm_dec, R1 * F);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->logits, R1 * (size_t)g.vocab);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->argmax_tmp, R1 * VLAC_ARGMAX_BLOCKS);
   if (rc == VLAC_OK) rc = dev_alloc(&c->dev_error, 8);
   if (rc == VLAC_OK) rc = dev_alloc(&c->in_frames, B * (size_t)g.n_cams * c->frame_hw * c->frame_hw * 3);
   if (rc == VLAC_OK) rc = dev_alloc(&c->in_feats, B * (size_t)c->Lv * D);
@@ -343,7 +345,7 @@ static int seg_mark(vlac_ctx* ctx, cudaStream_t s) {
 // Enqueue every kernel of one control step on `s` (directly, or into a stream capture).
 static int enqueue_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, const void* vision_feats,
                         const int* prompt_ids, const SelectKernelParams& p, int* action_tokens, float* all_logits,
-                        const int* forced_tokens, cudaStream_t s) {
+                        const int* forced_tokens, const void* act_embed, cudaStream_t s) {
   const vlac_config& g = ctx->cfg;
   const int B = cache->batch, nl = g.n_layers;
   ctx->seg_n = 0;
@@ -368,6 +370,11 @@ static int enqueue_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* f
   TRY(vlac_launch_finalize_norm(ctx, cache, h, nl - 1, n_splits, nl - 1, nullptr, s));
   if (deferred) TRY(vlac_launch_emit_all(ctx, cache, s));
   TRY(seg_mark(ctx, s));
+  if (act_embed) {
+    // 4'. all action tokens from one parallel pass over n_action placeholder rows behind the prompt
+    TRY(vlac_launch_chunk_pass(ctx, cache, act_embed, action_tokens, all_logits, s));
+    TRY(seg_mark(ctx, s));
+  } else {
   // 4. first action token
   TRY(vlac_launch_last_row(ctx, cache, h, s));
   const long long lstride = (long long)g.n_action * g.vocab;
@@ -381,6 +388,7 @@ static int enqueue_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* f
                                   all_logits ? all_logits + (size_t)i * g.vocab : nullptr, lstride, s));
     TRY(seg_mark(ctx, s));
   }
+  }
   // 6. this step becomes "previous"
   const size_t frame = (size_t)B * g.n_cams * ctx->frame_hw * ctx->frame_hw * 3;
   VLAC_CUDA_CHECK(cudaMemcpyAsync(cache->prev_frames, frames, frame, cudaMemcpyDeviceToDevice, s));
@@ -391,9 +399,9 @@ static int enqueue_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* f
   return VLAC_OK;
 }
 
-int vlac_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, const void* vision_feats,
-              const int* prompt_ids, const vlac_select_params* params, int force_full,
-              int* action_tokens, float* all_logits, const int* forced_tokens, void* stream) {
+static int step_impl(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, const void* vision_feats,
+                     const int* prompt_ids, const vlac_select_params* params, int force_full,
+                     int* action_tokens, float* all_logits, const int* forced_tokens, const void* act_embed, void* stream) {
   if (!ctx || !cache || cache->ctx != ctx || !frames || !vision_feats || !action_tokens) return VLAC_ERR_INVALID_ARG;
   const vlac_config& g = ctx->cfg;
   const int n_text = g.n_text_pre + g.n_text_post;
@@ -414,7 +422,7 @@ int vlac_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, con
     if (cap != cudaStreamCaptureStatusNone) direct = true;
   }
   if (direct)
-    return enqueue_step(ctx, cache, frames, vision_feats, prompt_ids, p, action_tokens, all_logits, forced_tokens, s);
+    return enqueue_step(ctx, cache, frames, vision_feats, prompt_ids, p, action_tokens, all_logits, forced_tokens, act_embed, s);
 
   const size_t frame = (size_t)B * g.n_cams * ctx->frame_hw * ctx->frame_hw * 3;
   VLAC_CUDA_CHECK(cudaMemcpyAsync(ctx->in_frames, frames, frame, cudaMemcpyDeviceToDevice, s));
@@ -426,7 +434,7 @@ int vlac_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, con
   for (int i = 0; i < VLAC_MAX_GRAPHS; ++i) {
     StepGraph& e = ctx->graphs[i];
     if (e.used && e.cache == cache && e.force_full == (force_full ? 1 : 0) && e.use_forced == (forced_tokens ? 1 : 0) &&
-        memcmp(&e.p, &p, sizeof(p)) == 0) { entry = &e; break; }
+        e.act_embed == act_embed && memcmp(&e.p, &p, sizeof(p)) == 0) { entry = &e; break; }
   }
   if (!entry) {
     StepGraph& e = ctx->graphs[ctx->graph_next];
@@ -435,7 +443,7 @@ int vlac_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, con
     const unsigned long long l0 = ctx->launches;
     VLAC_CUDA_CHECK(cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal));
     const int rc = enqueue_step(ctx, cache, ctx->in_frames, ctx->in_feats, ctx->in_ids, p, ctx->out_tokens, ctx->logits_all,
-                                forced_tokens ? ctx->in_forced : nullptr, s);
+                                forced_tokens ? ctx->in_forced : nullptr, act_embed, s);
     cudaGraph_t graph = nullptr;
     const cudaError_t ce = cudaStreamEndCapture(s, &graph);
     if (rc != VLAC_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
@@ -444,6 +452,7 @@ int vlac_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, con
     cudaGraphDestroy(graph);
     VLAC_CUDA_CHECK(ie);
     e.used = 1; e.cache = cache; e.force_full = force_full ? 1 : 0; e.use_forced = forced_tokens ? 1 : 0; e.p = p;
+    e.act_embed = act_embed;
     e.launches = ctx->launches - l0;
     ctx->launches = l0;
     entry = &e;
@@ -454,6 +463,22 @@ int vlac_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, con
   if (all_logits)
     VLAC_CUDA_CHECK(cudaMemcpyAsync(all_logits, ctx->logits_all, sizeof(float) * (size_t)B * g.n_action * g.vocab, cudaMemcpyDeviceToDevice, s));
   return VLAC_OK;
+}
+
+int vlac_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, const void* vision_feats,
+              const int* prompt_ids, const vlac_select_params* params, int force_full,
+              int* action_tokens, float* all_logits, const int* forced_tokens, void* stream) {
+  return step_impl(ctx, cache, frames, vision_feats, prompt_ids, params, force_full, action_tokens, all_logits, forced_tokens,
+                   nullptr, stream);
+}
+
+int vlac_step_chunk(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, const void* vision_feats,
+                    const int* prompt_ids, const vlac_select_params* params, int force_full, const void* act_embed,
+                    int* action_tokens, float* all_logits, void* stream) {
+  if (!act_embed) return VLAC_ERR_INVALID_ARG;
+  if (ctx && !ctx->chunk_ok) return VLAC_ERR_INVALID_ARG;
+  return step_impl(ctx, cache, frames, vision_feats, prompt_ids, params, force_full, action_tokens, all_logits, nullptr,
+                   act_embed, stream);
 }
 
 unsigned long long vlac_launch_count(const vlac_ctx* ctx) { return ctx ? ctx->launches : 0ull; }

@@ -34,6 +34,7 @@ struct StepGraph {                     // one captured control step (CUDA graph)
   int used;
   vlac_cache* cache;
   int force_full, use_forced;
+  const void* act_embed;               // chunk steps: the placeholder embeddings the graph reads (NULL: ordinary step)
   SelectKernelParams p;
   cudaGraphExec_t exec;
   unsigned long long launches;
@@ -52,10 +53,11 @@ struct vlac_ctx {
   float *scratch;                    // [rows_max][max(3*hidden, 2*ffn)]   (generic GEMM output)
   float *probs;                      // [max_batch][n_text_post][n_heads][Lv]
   bf16 *hidden;                      // [max_batch][L][hidden]            (used by step)
-  float *x_dec;                      // [max_batch][hidden]
-  bf16 *q_dec, *ao_dec, *hm_dec;     // [max_batch][hidden] x2, [max_batch][ffn]
-  float *logits;                     // [max_batch][vocab]
-  unsigned long long *argmax_tmp;    // [max_batch][VLAC_ARGMAX_BLOCKS]
+  // single-row buffers: one row per column of the matrix-vector kernels, R1 = max(max_batch, min(n_action, 8))
+  float *x_dec;                      // [R1][hidden]
+  bf16 *q_dec, *ao_dec, *hm_dec;     // [R1][hidden] x2, [R1][ffn]
+  float *logits;                     // [R1][vocab]
+  unsigned long long *argmax_tmp;    // [R1][VLAC_ARGMAX_BLOCKS]
   int *dev_error;                    // device ints: [0] nonzero if a bounded wait gave up
   // step staging: the captured graph reads and writes only library-owned buffers
   unsigned char* in_frames; bf16* in_feats; int *in_ids, *in_forced, *out_tokens; float* logits_all;
@@ -68,6 +70,7 @@ struct vlac_ctx {
   int tc_proj;                       // the vision projector has a tensor map (tcgen05 path usable for the input rows)
   int pass_grid;                     // CTAs of the persistent single-row pass kernel (0: not used)
   int gemv_stream;                   // single-row products use the shared-memory-staged kernel
+  int chunk_ok;                      // the n_action rows of a chunk fit the matrix-vector kernels as columns (vlac_step_chunk usable)
   void* tmap_q;                      // device tensor map of the query buffer (tiled attention)
   int attn_tiles;                    // 64-query tiles per sequence, 0: tiled attention not usable
   float* probs_all;                  // [n_layers][max_batch][tiles][n_heads][Lv]: per-tile column sums of every layer of a step
@@ -147,3 +150,5 @@ int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens,
                             int pos, cudaStream_t s);
 int vlac_launch_logits_argmax(vlac_ctx* ctx, vlac_cache* c, int* tokens_out, int tok_stride, int tok_index,
                               float* logits_copy, long long copy_stride, cudaStream_t s);
+int vlac_launch_chunk_pass(vlac_ctx* ctx, vlac_cache* c, const void* act_embed, int* tokens_out /* [batch][n_action] */,
+                           float* logits_copy /* [batch][n_action][vocab] or NULL */, cudaStream_t s);

@@ -100,11 +100,13 @@ def check_selection(got: dict, sel: orc.Selection, seq: int, cfg, where=""):
 
 
 def run_step_pair(sess: Session, frames: np.ndarray, feats: np.ndarray, ids: np.ndarray, params: orc.SelectParams,
-                  force_full=False):
+                  force_full=False, act_embed: np.ndarray = None):
     """One control step on both sides with replay: the checker's selection is computed from the
     library's own saved attention (bit-copied) and the checker is fed the library's tokens.
 
     frames [B, n_cams, H, W, 3] uint8; feats [B, L_v, hidden] bf16 bits; ids [B, n_text] int32.
+    With ``act_embed`` ([n_action, hidden] bf16 bits) both sides decode the action chunk in one parallel
+    pass instead (vlac_step_chunk / step_chunk); the K/V rows of the chunk are compared as well.
     Returns a dict of per-sequence comparison figures.
     """
     cfg, B = sess.cfg, sess.batch
@@ -116,8 +118,14 @@ def run_step_pair(sess: Session, frames: np.ndarray, feats: np.ndarray, ids: np.
     tokens = torch.zeros((B, cfg.n_action), dtype=torch.int32, device="cuda")
     logits = torch.zeros((B, cfg.n_action, cfg.vocab), dtype=torch.float32, device="cuda")
     torch.cuda.synchronize()
+    d_act = vb.upload_bf16(act_embed) if act_embed is not None else None
+    if d_act is not None:
+        sess.keep_alive = getattr(sess, "keep_alive", []) + [d_act]      # a captured step may read it again
     with torch.cuda.stream(sess.stream):
-        vb.vlac_step(sess.ctx, sess.cache, d_frames, d_feats, d_ids, gp, force_full, tokens, logits)
+        if d_act is None:
+            vb.vlac_step(sess.ctx, sess.cache, d_frames, d_feats, d_ids, gp, force_full, tokens, logits)
+        else:
+            vb.vlac_step_chunk(sess.ctx, sess.cache, d_frames, d_feats, d_ids, gp, force_full, d_act, tokens, logits)
     torch.cuda.synchronize()
     assert vb.vlac_device_error(sess.ctx) == 0
     got_sel = vb.selection_to_host(vb.vlac_selection_view(sess.cache))
@@ -132,8 +140,12 @@ def run_step_pair(sess: Session, frames: np.ndarray, feats: np.ndarray, ids: np.
             check_selection(got_sel, sel, b, cfg, where=f"seq {b}")
         else:
             assert np.all(got_sel["M"][b] == cfg.seq_len)
-        res = orc.step(cfg, sess.model, oc, frames[b], feats[b], ids[b], params, force_full,
-                       forced_tokens=g_tokens[b], selection=sel)
+        if act_embed is None:
+            res = orc.step(cfg, sess.model, oc, frames[b], feats[b], ids[b], params, force_full,
+                           forced_tokens=g_tokens[b], selection=sel)
+        else:
+            res = orc.step_chunk(cfg, sess.model, oc, frames[b], feats[b], ids[b], params, act_embed, force_full,
+                                 selection=sel)
         err = max(rel_err(g_logits[b, i], res.logits[i]) for i in range(cfg.n_action))
         abs_err = float(np.max(np.abs(g_logits[b] - res.logits)))
         guarded = 0
@@ -144,6 +156,12 @@ def run_step_pair(sess: Session, frames: np.ndarray, feats: np.ndarray, ids: np.
                 guarded += 1
         g_attn = sess.read_attn(vb.PART_ATTN_PREV, b)
         attn_err = rel_err(g_attn, res.attn_tv)
-        out.append({"logit_err": err, "abs_err": abs_err, "guarded": guarded, "attn_err": attn_err,
+        kv_err = 0.0
+        if act_embed is not None:
+            L, n = cfg.seq_len, cfg.n_action
+            for l in range(cfg.n_layers):
+                kv_err = max(kv_err, rel_err(sess.read_kv(vb.PART_K, l, b)[L:L + n], oc.K[l][L:L + n]),
+                             rel_err(sess.read_kv(vb.PART_V, l, b)[L:L + n], oc.V[l][L:L + n]))
+        out.append({"logit_err": err, "abs_err": abs_err, "guarded": guarded, "attn_err": attn_err, "kv_err": kv_err,
                     "M": sel.M.copy(), "tokens": g_tokens[b].copy(), "selection": sel})
     return out

@@ -278,6 +278,104 @@ def test_step_batch_of_three_ragged(H, vb):
         sess.close()
 
 
+# ------------------------------------------------------------------------------------- action chunk in one pass
+def test_step_chunk_tiny_episode(H, vb):
+    """All action tokens from one parallel pass behind the prefill: cold step, then cached steps."""
+    cfg, model, ids, feats = _tiny_inputs()
+    act = synth.make_action_embed(cfg, 5)
+    prev, cur, changed = synth.rerandomised_pair(cfg, 0, 13)
+    sess = H.Session(cfg, model)
+    try:
+        guarded = 0
+        for t, fr in enumerate([prev, cur, cur]):
+            params = H.oparams(top_k=32, alpha_override=[0.5, 1.0]) if t != 2 else H.oparams(top_k=32, k_ent=50.0)
+            r = H.run_step_pair(sess, fr[None], feats, ids, params, act_embed=act)[0]
+            assert r["logit_err"] <= H.TOL and r["attn_err"] <= H.TOL and r["kv_err"] <= H.TOL, (t, r)
+            if t == 1:
+                assert r["M"][1] < cfg.seq_len
+            guarded += r["guarded"]
+        assert guarded <= 6
+    finally:
+        sess.close()
+
+
+def test_step_chunk_7b_shape_two_layers(H, vb):
+    """7B-shaped layers, vocabulary 32000, 7 chunk rows behind 290 prompt tokens (the wide MLP input does not fit
+    beside the weight ring with 7 columns, so the down projection takes the register-pipelined kernel)."""
+    cfg = synth.llama7b_config(n_layers=2)
+    model = synth.make_model(cfg, 8)
+    ids = synth.make_prompt_ids(cfg, 8)
+    act = synth.make_action_embed(cfg, 8)
+    ep = synth.make_episode(cfg, 8, 2)
+    sess = H.Session(cfg, model)
+    try:
+        for t in range(2):
+            r = H.run_step_pair(sess, ep.frames[t][None], ep.feats[t][None], ids, H.oparams(alpha_override=[0.6, 1.0]), act_embed=act)[0]
+            assert r["logit_err"] <= H.TOL and r["attn_err"] <= H.TOL and r["kv_err"] <= H.TOL, (t, r)
+            if t == 1:
+                assert r["M"][1] < cfg.seq_len
+    finally:
+        sess.close()
+
+
+def test_step_chunk_batch_of_three(H, vb):
+    """A batch takes the chunk pass one sequence after the other; each sequence has its own cache rows."""
+    cfg = synth.tiny_config()
+    model = synth.make_model(cfg, 2)
+    B = 3
+    ids = synth.make_prompt_ids(cfg, 2, batch=B)
+    act = synth.make_action_embed(cfg, 2)
+    pairs = [synth.rerandomised_pair(cfg, 20 + b, n) for b, n in enumerate((5, 30, 60))]
+    rng = np.random.default_rng(7)
+    feats = synth.f32_to_bf16(rng.standard_normal((B, cfg.n_vision, cfg.hidden), dtype=np.float32))
+    sess = H.Session(cfg, model, batch=B)
+    try:
+        p = H.oparams(top_k=64, tau_task=1.0, alpha_override=[1.0, 1.0])
+        r0 = H.run_step_pair(sess, np.stack([q[0] for q in pairs]), feats, ids, p, act_embed=act)
+        r1 = H.run_step_pair(sess, np.stack([q[1] for q in pairs]), feats, ids, p, act_embed=act)
+        for r in r0 + r1:
+            assert r["logit_err"] <= H.TOL and r["attn_err"] <= H.TOL and r["kv_err"] <= H.TOL, r
+        assert len({tuple(r["tokens"].tolist()) for r in r1}) > 1, "sequences must not share one result"
+    finally:
+        sess.close()
+
+
+def test_step_chunk_keeps_the_prompt_state_of_an_ordinary_step(H, vb):
+    """vlac_step_chunk and vlac_step differ only behind the prompt: selection, prompt K/V and the saved
+    text-to-vision scores after two steps are bit-identical."""
+    cfg, model, ids, feats = _tiny_inputs(1)
+    act = synth.make_action_embed(cfg, 1)
+    prev, cur, _ = synth.rerandomised_pair(cfg, 1, 13)
+    L = cfg.seq_len
+    state = []
+    for chunk in (False, True):
+        sess = H.Session(cfg, model)
+        try:
+            gp, keep = H.gparams(H.oparams(top_k=32, alpha_override=[0.5, 1.0]))
+            tok = torch.zeros((1, cfg.n_action), dtype=torch.int32, device="cuda")
+            d_act = vb.upload_bf16(act)
+            args = (vb.upload_bf16(feats), torch.from_numpy(ids).to("cuda"))
+            for fr in (prev, cur):
+                d_fr = torch.from_numpy(fr[None]).to("cuda")
+                if chunk:
+                    vb.vlac_step_chunk(sess.ctx, sess.cache, d_fr, *args, gp, False, d_act, tok)
+                else:
+                    vb.vlac_step(sess.ctx, sess.cache, d_fr, *args, gp, False, tok)
+            torch.cuda.synchronize()
+            sel = vb.selection_to_host(vb.vlac_selection_view(sess.cache))
+            state.append((sel["M"].copy(), sel["rows"].copy(), sess.read_attn(vb.PART_ATTN_PREV),
+                          [sess.read_kv(vb.PART_K, l)[:L] for l in range(cfg.n_layers)],
+                          [sess.read_kv(vb.PART_V, l)[:L] for l in range(cfg.n_layers)]))
+        finally:
+            sess.close()
+    a, b = state
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[2], b[2])
+    for l in range(cfg.n_layers):
+        m = int(a[0][0, l])
+        assert np.array_equal(a[1][0, l, :m], b[1][0, l, :m])
+        assert np.array_equal(a[3][l], b[3][l]) and np.array_equal(a[4][l], b[4][l])
+
+
 def test_step_graph_replay_equals_direct_launch(H, vb):
     """On a non-default stream the step is captured once and replayed as a CUDA graph; on the default
     stream every kernel is launched directly.  Both must give the same bits, step after step."""
