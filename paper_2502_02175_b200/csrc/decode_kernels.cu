@@ -28,6 +28,8 @@ struct GemvArgs {
   bf16 *kc, *vc;           // QKV: [nb][max_seq][N]
   const float *rope_cos, *rope_sin;
   int pos, max_seq, d;
+  int ld;                  // RESID / LOGITS with x_bf16: pitch (elements) of the weight rows and of the rows of x_bf16 when this
+                           // launch covers only K of their columns (0: the pitch is K)
   int cps;                 // QKV: columns per sequence (0 or 1: one row per sequence at position `pos`; n: column c is
                            // row pos + c % n of sequence c / n -- an action chunk decoded in parallel)
   float* x_out;            // RESID: [nb][N] +=
@@ -68,8 +70,9 @@ __device__ __forceinline__ UnitRows unit_rows(const A& a, int u) {
     r.pb = reinterpret_cast<const uint4*>(a.w1 + (size_t)u * K);
   } else {
     r.mat = 0; r.rowA = 2 * u; r.rowB = min(2 * u + 1, a.N - 1);
-    r.pa = reinterpret_cast<const uint4*>(a.w0 + (size_t)r.rowA * K);
-    r.pb = reinterpret_cast<const uint4*>(a.w0 + (size_t)r.rowB * K);
+    const int ld = a.ld ? a.ld : K;
+    r.pa = reinterpret_cast<const uint4*>(a.w0 + (size_t)r.rowA * ld);
+    r.pb = reinterpret_cast<const uint4*>(a.w0 + (size_t)r.rowB * ld);
   }
   return r;
 }
@@ -432,7 +435,7 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
         for (int k = tid; k < K; k += GT_THREADS) xs[(size_t)b * K + k] = __float2bfloat16(x[k] * r * bf2f(a.gain[k]));
       }
     } else {
-      const uint4* src = reinterpret_cast<const uint4*>(a.x_bf16 + (size_t)b * K);
+      const uint4* src = reinterpret_cast<const uint4*>(a.x_bf16 + (size_t)b * (a.ld ? a.ld : K));
       uint4* dst = reinterpret_cast<uint4*>(xs + (size_t)b * K);
       for (int c = tid; c < K / 8; c += GT_THREADS) dst[c] = src[c];
     }
@@ -952,6 +955,27 @@ int launch_gemv(vlac_ctx* ctx, const GemvArgs& a, cudaStream_t s) {
   return VLAC_OK;
 }
 
+// A product whose activations (nb rows of K values) do not fit beside the weight ring is taken as 2 or 4 launches
+// over slices of K, each adding its part to x_out in stream order (RESID with a bf16 input only; the slices are
+// multiples of 64 columns of 16-byte aligned rows).
+int launch_gemv_sliced(vlac_ctx* ctx, const GemvArgs& a, cudaStream_t s) {
+  if (ctx->gemv_stream && a.mode == GV_RESID && a.x_bf16 && !a.ld && a.K % 64 == 0 && gt_smem_bytes(ctx, a) > GT_SMEM_MAX) {
+    for (int n = 2; n <= 4; n *= 2) {
+      if (a.K % (64 * n)) continue;
+      GemvArgs h = a;
+      h.K = a.K / n; h.ld = a.K;
+      if (gt_smem_bytes(ctx, h) > GT_SMEM_MAX) continue;
+      for (int i = 0; i < n; ++i) {
+        h.w0 = a.w0 + (size_t)i * h.K; h.x_bf16 = a.x_bf16 + (size_t)i * h.K;
+        const int rc = launch_gemv(ctx, h, s);
+        if (rc) return rc;
+      }
+      return VLAC_OK;
+    }
+  }
+  return launch_gemv(ctx, a, s);
+}
+
 }  // namespace
 
 static size_t pass_smem(const vlac_ctx* ctx, int NB);
@@ -1111,7 +1135,7 @@ int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens,
       VLAC_LAUNCH_CHECK(ctx);
     }
     for (int k = 1; k < 4; ++k) {
-      rc = launch_gemv(ctx, ph[k], s);
+      rc = launch_gemv_sliced(ctx, ph[k], s);
       if (rc) return rc;
     }
   }
@@ -1153,7 +1177,7 @@ int vlac_launch_chunk_pass(vlac_ctx* ctx, vlac_cache* c, const void* act_embed, 
         VLAC_LAUNCH_CHECK(ctx);
       }
       for (int k = 1; k < 4; ++k) {
-        rc = launch_gemv(ctx, ph[k], s);
+        rc = launch_gemv_sliced(ctx, ph[k], s);
         if (rc) return rc;
       }
     }
