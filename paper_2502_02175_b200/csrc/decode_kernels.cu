@@ -305,6 +305,7 @@ constexpr int GT_DEPTH = GT_DEPTH_N;
 constexpr int GT_SLOT_BYTES = 16 * 128;
 constexpr int GT_RING_BYTES = GT_WARPS * GT_DEPTH * GT_SLOT_BYTES;      // 128 KB
 constexpr int GT_PART_BYTES = 2 * 8 * GT_WARPS * 16 * (int)sizeof(float);  // partial tiles of two rounds: 16 KB
+constexpr int GT_XPAD = 8;                                                 // bf16 elements appended to every activation row in shared memory
 
 __device__ __forceinline__ void cp_async16(unsigned smem_dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(src) : "memory");
@@ -321,9 +322,12 @@ __device__ __forceinline__ void mma_16816(float* c, const unsigned* a, unsigned 
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3]) : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// TEAMS: more than four activation columns (see below); the other instantiation is the single-team kernel.
+template <bool TEAMS>
 __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvArgs a) {
   extern __shared__ __align__(128) unsigned char gt_smem[];
   __shared__ float red[GT_WARPS];
+  __shared__ float red_cols[GT_WARPS * 8];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int K = a.K, nb = a.nb;
   const int n_units = unit_count(a.mode, a.N);
@@ -332,10 +336,20 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
   const int n_groups = (n_local + 7) / 8;
   const unsigned ring_w = (unsigned)__cvta_generic_to_shared(gt_smem) + (unsigned)warp * (GT_DEPTH * GT_SLOT_BYTES);
   float* part = reinterpret_cast<float*>(gt_smem + GT_RING_BYTES);                      // [2][G][GT_WARPS][16][nbp], G * nbp = 8
-  bf16* xs = reinterpret_cast<bf16*>(gt_smem + GT_RING_BYTES + GT_PART_BYTES);            // [nb][K]
+  bf16* xs = reinterpret_cast<bf16*>(gt_smem + GT_RING_BYTES + GT_PART_BYTES);            // [nb][KP]
+  // rows 16 bytes longer than K: the eight columns a warp reads for one MMA then fall into different banks
+  const int KP = K + GT_XPAD;
 
+  // With more than four activation columns the partial-tile buffer holds one group per round, and a barrier of
+  // all 16 warps after every group (128 KB of weights) costs a third of the bandwidth.  The warps then work as
+  // four teams of four: a team owns every fourth group, splits K among its own warps and meets at its own
+  // named barrier, so four groups are in flight and a warp streams four times as much between barriers.
+  constexpr int TW = TEAMS ? 4 : GT_WARPS;                             // warps of a team
+  constexpr int NTm = GT_WARPS / TW;                                   // teams
+  const int team = warp / TW, wt = warp - team * TW;
+  const int n_groups_w = n_groups > team ? (n_groups - team + NTm - 1) / NTm : 0;   // groups of this warp's team
   const int S = K / 64;                                                // sub-stages per row
-  const int ns_w = warp < S ? (S - warp + GT_WARPS - 1) / GT_WARPS : 0;   // ... of this warp
+  const int ns_w = wt < S ? (S - wt + TW - 1) / TW : 0;                // ... of this warp
   // ---- issue side: (group, sub-stage) in order; one copy group per item, empty once the work is exhausted
   int ig = 0, ij = 0, islot = 0;
   const char* rowptr[4];
@@ -348,11 +362,11 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
     rowptr[0] = reinterpret_cast<const char*>(r0.pa); rowptr[1] = reinterpret_cast<const char*>(r1.pa);
     rowptr[2] = reinterpret_cast<const char*>(r0.pb); rowptr[3] = reinterpret_cast<const char*>(r1.pb);
   };
-  if (n_groups > 0 && ns_w > 0) load_rowptrs(0);
+  if (n_groups_w > 0 && ns_w > 0) load_rowptrs(team);
   auto issue = [&]() {
-    if (ig < n_groups && ns_w > 0) {
+    if (ig < n_groups_w && ns_w > 0) {
       const unsigned slotp = ring_w + (unsigned)islot * GT_SLOT_BYTES;
-      const size_t koff = (size_t)(warp + GT_WARPS * ij) * 128 + (size_t)(lane & 7) * 16;
+      const size_t koff = (size_t)(wt + TW * ij) * 128 + (size_t)(lane & 7) * 16;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
         const int row = (lane >> 3) + 4 * i;
@@ -360,7 +374,7 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
       }
       if (++ij == ns_w) {
         ij = 0;
-        if (++ig < n_groups) load_rowptrs(ig);
+        if (++ig < n_groups_w) load_rowptrs(team + NTm * ig);
       }
     }
     cp_async_commit();
@@ -383,7 +397,59 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
   pdl_trigger();
   pdl_wait();
 
-  // ---- activations -> shared memory as bf16 (RMSNorm here if a gain is given); each value is read once
+  // ---- activations -> shared memory as bf16 (RMSNorm here if a gain is given)
+  if (a.x_f32 && nb > 1) {
+    // several columns: all sums of squares in one sweep and one pair of barriers (column by column the CTA would
+    // meet twice per column), then a second sweep over the few KB of inputs to scale and store them
+    float ss[8];
+#pragma unroll
+    for (int b = 0; b < 8; ++b) ss[b] = 0.f;
+    for (int c = tid; c < nchunk; c += GT_THREADS) {
+#pragma unroll
+      for (int b = 0; b < 8; ++b) {
+        if (b < nb) {
+          const float* x = a.x_f32 + (size_t)b * K + (size_t)c * 8;
+          const float4 v0 = *reinterpret_cast<const float4*>(x), v1 = *reinterpret_cast<const float4*>(x + 4);
+          ss[b] += v0.x * v0.x + v0.y * v0.y + v0.z * v0.z + v0.w * v0.w + v1.x * v1.x + v1.y * v1.y + v1.z * v1.z + v1.w * v1.w;
+        }
+      }
+    }
+#pragma unroll
+    for (int b = 0; b < 8; ++b) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) ss[b] += __shfl_xor_sync(0xffffffffu, ss[b], o);
+      if (lane == 0) red_cols[warp * 8 + b] = ss[b];
+    }
+    __syncthreads();
+    float rn[8];
+#pragma unroll
+    for (int b = 0; b < 8; ++b) {
+      float t = 0.f;
+#pragma unroll
+      for (int w = 0; w < GT_WARPS; ++w) t += red_cols[w * 8 + b];
+      rn[b] = rsqrtf(t / (float)K + a.eps);
+    }
+    for (int c = tid; c < nchunk; c += GT_THREADS) {
+      const uint4 gq8 = __ldg(reinterpret_cast<const uint4*>(a.gain) + c);
+      const __nv_bfloat162* g2 = reinterpret_cast<const __nv_bfloat162*>(&gq8);
+#pragma unroll
+      for (int b = 0; b < 8; ++b) {
+        if (b < nb) {
+          const float* x = a.x_f32 + (size_t)b * K + (size_t)c * 8;
+          const float4 v0 = *reinterpret_cast<const float4*>(x), v1 = *reinterpret_cast<const float4*>(x + 4);
+          const float xv[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+          uint4 o;
+          __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float2 gf = __bfloat1622float2(g2[e]);
+            o2[e] = __floats2bfloat162_rn(xv[2 * e] * rn[b] * gf.x, xv[2 * e + 1] * rn[b] * gf.y);
+          }
+          *reinterpret_cast<uint4*>(xs + (size_t)b * KP + (size_t)c * 8) = o;
+        }
+      }
+    }
+  } else
   for (int b = 0; b < nb; ++b) {
     if (a.x_f32) {
       const float* x = a.x_f32 + (size_t)b * K;
@@ -428,15 +494,15 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
               const float2 gf = __bfloat1622float2(g2[e]);
               o2[e] = __floats2bfloat162_rn(xv[2 * e] * r * gf.x, xv[2 * e + 1] * r * gf.y);
             }
-            *reinterpret_cast<uint4*>(xs + (size_t)b * K + (size_t)c * 8) = o;
+            *reinterpret_cast<uint4*>(xs + (size_t)b * KP + (size_t)c * 8) = o;
           }
         }
       } else {
-        for (int k = tid; k < K; k += GT_THREADS) xs[(size_t)b * K + k] = __float2bfloat16(x[k] * r * bf2f(a.gain[k]));
+        for (int k = tid; k < K; k += GT_THREADS) xs[(size_t)b * KP + k] = __float2bfloat16(x[k] * r * bf2f(a.gain[k]));
       }
     } else {
       const uint4* src = reinterpret_cast<const uint4*>(a.x_bf16 + (size_t)b * (a.ld ? a.ld : K));
-      uint4* dst = reinterpret_cast<uint4*>(xs + (size_t)b * K);
+      uint4* dst = reinterpret_cast<uint4*>(xs + (size_t)b * KP);
       for (int c = tid; c < K / 8; c += GT_THREADS) dst[c] = src[c];
     }
   }
@@ -444,7 +510,7 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
 
   // ---- consume side
   const int col_n = lane >> 2;                                         // B column (sequence) this lane feeds
-  const unsigned xw_a = (unsigned)__cvta_generic_to_shared(xs) + (unsigned)((size_t)min(col_n, max(nb - 1, 0)) * K * 2) + (unsigned)(lane & 3) * 4u;
+  const unsigned xw_a = (unsigned)__cvta_generic_to_shared(xs) + (unsigned)((size_t)min(col_n, max(nb - 1, 0)) * KP * 2) + (unsigned)(lane & 3) * 4u;
   const bool col_live = col_n < nb;
   // Partial tiles of G groups are collected before the CTA meets at a barrier: part[2][G][warp][16 rows][nbp]
   const int nbp = nb <= 1 ? 1 : (nb <= 2 ? 2 : (nb <= 4 ? 4 : 8));
@@ -452,18 +518,20 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
   int cslot = 0;
   UnitRows fcu = {nullptr, nullptr, 0, 0, 0};                        // unit this thread finishes in the current round, if any
   float fpre[2] = {0.f, 0.f};
-  int f_ul = -1, f_col = 0;
-  for (int g = 0; g < n_groups; ++g) {
-    if (g % G == 0) {
+  int f_ul = -1, f_col = 0, f_gi = 0;
+  const int tt = tid - team * TW * 32;                                 // thread index inside the team
+  for (int gl = 0; gl < n_groups_w; ++gl) {                            // gl-th group of the team: group team + NTm * gl of the CTA
+    if (gl % G == 0) {
       // start of a round: the threads that will finish its units fetch what the epilogue needs now, so the
       // last round does not end on a dependent global load
-      const int n_gr = min(G, n_groups - g);
+      const int n_gr = min(G, n_groups_w - gl);
       f_ul = -1;
-      if (tid < n_gr * 8 * nb) {
-        const int gi = tid / (8 * nb), rem = tid - gi * 8 * nb;
+      if (tt < n_gr * 8 * nb) {
+        const int gi = tt / (8 * nb), rem = tt - gi * 8 * nb;
         const int uu = rem / nb;
         f_col = rem - uu * nb;
-        const int ul = (g + gi) * 8 + uu;
+        f_gi = gi;
+        const int ul = (team + NTm * (gl + gi)) * 8 + uu;
         if (ul < n_local) { f_ul = ul; fcu = unit_rows(a, u_begin + ul); unit_operands(a, fcu, f_col, fpre); }
       }
     }
@@ -472,7 +540,7 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
       cp_async_wait<GT_DEPTH - 1>();                                   // this lane's copies of the oldest item have landed
       __syncwarp();                                                    // ... and so have the other lanes'
       const unsigned slotp = ring_w + (unsigned)cslot * GT_SLOT_BYTES;
-      const int k0 = (warp + GT_WARPS * j) * 64;
+      const int k0 = (wt + TW * j) * 64;
 #pragma unroll
       for (int kk = 0; kk < 4; ++kk) {
         unsigned af[4];
@@ -486,23 +554,28 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
       issue();
       cslot = (cslot + 1 == GT_DEPTH) ? 0 : cslot + 1;
     }
-    const int round = g / G, gr = g - round * G;
+    const int round = gl / G, gr = gl - round * G;
     {
       float* dst = part + ((size_t)(((round & 1) * G + gr) * GT_WARPS + warp) * 16) * nbp;
       const int r = lane >> 2, n0 = (lane & 3) * 2;
       if (n0 < nb) { dst[r * nbp + n0] = c[0]; dst[(r + 8) * nbp + n0] = c[2]; }
       if (n0 + 1 < nb) { dst[r * nbp + n0 + 1] = c[1]; dst[(r + 8) * nbp + n0 + 1] = c[3]; }
     }
-    if (gr == G - 1 || g == n_groups - 1) {
+    if (gr == G - 1 || gl == n_groups_w - 1) {
       // End of a round: add the warps' partial tiles in warp order and finish these units.  The other half of
       // `part` takes the next round; the barrier that ends it also orders these reads before this half is reused.
-      __syncthreads();
+      if (NTm == 1) __syncthreads();
+      else asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "r"(TW * 32) : "memory");      // the team's own barrier
       if (f_ul >= 0) {                                           // at most 64 units x columns per round: one per thread
-        const int gi = f_ul / 8 - round * G, uu = f_ul & 7, col = f_col;
-        const float* src = part + ((size_t)(((round & 1) * G + gi) * GT_WARPS) * 16) * nbp;
+        const int gi = f_gi, uu = f_ul & 7, col = f_col;
+        const float* src = part + ((size_t)(((round & 1) * G + gi) * GT_WARPS + team * TW) * 16) * nbp;
         float ya = 0.f, yb = 0.f;
+        if (NTm == 1) {
 #pragma unroll
-        for (int w = 0; w < GT_WARPS; ++w) { ya += src[((size_t)w * 16 + uu) * nbp + col]; yb += src[((size_t)w * 16 + uu + 8) * nbp + col]; }
+          for (int w = 0; w < GT_WARPS; ++w) { ya += src[((size_t)w * 16 + uu) * nbp + col]; yb += src[((size_t)w * 16 + uu + 8) * nbp + col]; }
+        } else {
+          for (int w = 0; w < TW; ++w) { ya += src[((size_t)w * 16 + uu) * nbp + col]; yb += src[((size_t)w * 16 + uu + 8) * nbp + col]; }
+        }
         store_unit(a, fcu, col, ya, yb, fpre);
       }
     }
@@ -926,7 +999,7 @@ __global__ void argmax_final_kernel(const unsigned long long* tmp, int n_part, i
 constexpr size_t GT_SMEM_MAX = 226 * 1024;      // dynamic part; the kernel also has a little static shared memory
 size_t gt_smem_bytes(const vlac_ctx* ctx, const GemvArgs& a) {
   (void)ctx;
-  return (size_t)GT_RING_BYTES + GT_PART_BYTES + (size_t)a.nb * a.K * sizeof(bf16);
+  return (size_t)GT_RING_BYTES + GT_PART_BYTES + (size_t)a.nb * (a.K + GT_XPAD) * sizeof(bf16);
 }
 
 int launch_gemv(vlac_ctx* ctx, const GemvArgs& a, cudaStream_t s) {
@@ -938,7 +1011,8 @@ int launch_gemv(vlac_ctx* ctx, const GemvArgs& a, cudaStream_t s) {
   if (timed) VLAC_CUDA_CHECK(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n], s));
   const size_t gt_smem = gt_smem_bytes(ctx, a);
   if (ctx->gemv_stream && a.K % 64 == 0 && nb <= 8 && gt_smem <= GT_SMEM_MAX) {
-    VLAC_CUDA_CHECK(launch_pdl(gemv_mma_kernel, dim3(ctx->n_sm * GT_GRID_PER_SM), dim3(GT_THREADS), gt_smem, s, a));
+    if (nb > 4) VLAC_CUDA_CHECK(launch_pdl(gemv_mma_kernel<true>, dim3(ctx->n_sm * GT_GRID_PER_SM), dim3(GT_THREADS), gt_smem, s, a));
+    else VLAC_CUDA_CHECK(launch_pdl(gemv_mma_kernel<false>, dim3(ctx->n_sm * GT_GRID_PER_SM), dim3(GT_THREADS), gt_smem, s, a));
   } else
   switch (NB) {
     case 1: VLAC_CUDA_CHECK(launch_pdl(gemv_pair_kernel<1>, dim3(grid), dim3(256), smem, s, a)); break;
@@ -997,7 +1071,8 @@ int vlac_decode_setup(vlac_ctx* ctx) {
   if (NB >= 8) VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_pair_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(8 * (size_t)kmax * 2)));
   // tensor-core variant of the weight-streaming kernel (VLAC_GEMV_REG=1 keeps the register-pipelined one)
   ctx->gemv_stream = getenv("VLAC_GEMV_REG") ? 0 : 1;
-  VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GT_SMEM_MAX));
+  VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GT_SMEM_MAX));
+  VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GT_SMEM_MAX));
   // persistent pass kernel: as many CTAs as are guaranteed co-resident
   ctx->pass_grid = 0;
   // Opt-in (VLAC_PASS_KERNEL=1).  Needs every K to be a multiple of 64 (the tensor-core body) and room for

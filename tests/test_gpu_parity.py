@@ -87,6 +87,17 @@ def test_select_7b_shape_episode_frames(H, vb, seed):
     assert got["M"].min() >= cfg.n_text
 
 
+def test_select_noisy_regime_lower_threshold(H, vb):
+    """Sensor noise of sigma 12 and three moving distractors, threshold 0.85 (the paper's real-robot setting):
+    similarities, masks, ratios and row lists bit-exact, with and without the top-k cap."""
+    cfg = synth.llama7b_config(n_layers=32)
+    ep = synth.make_episode(cfg.with_layers(1), 11, 3, n_blobs=3, noise_sigma=12.0)
+    attn = synth.scripted_attention(cfg, 11, hot_tokens=ep.touched[1])
+    for params in (H.oparams(tau=0.85), H.oparams(tau=0.85, top_k=256, k_ent=2.0), H.oparams(tau=0.85, top_k=256, tau_task=0.8, k_ent=3.0)):
+        got = _select_case(H, vb, cfg, [ep.frames[1]], [ep.frames[2]], [attn], params)
+    assert got["static_mask"][0].sum() > 150 and got["M"].min() < cfg.seq_len
+
+
 def test_select_dual_camera_batch(H, vb):
     """Two cameras, three sequences with different change rates: one global top-k per sequence."""
     cfg = synth.dual_camera_config(n_layers=8)
