@@ -473,6 +473,84 @@ def test_step_batch_of_eight_7b_shape(H, vb):
         orc._widen_cache.clear()
 
 
+def test_full_size_32_layers_chunk_step(H, vb):
+    """vlac_step_chunk on the bench configuration (32 layers, device-drawn weights, graph replay on a side
+    stream): run-to-run determinism; selection, prompt K/V and saved scores bit-identical to vlac_step on the
+    same inputs; and the chunk rows' K/V of layer 0, which depend only on the placeholder embeddings and that
+    layer's weights, against the checker."""
+    cfg = synth.llama7b_config(n_layers=32)
+    dev = vb.DeviceModel.random(cfg, seed=78)
+    ep = synth.make_episode(cfg.with_layers(1), 78, 2)
+    ids = torch.from_numpy(synth.make_prompt_ids(cfg, 78)).to("cuda")
+    frames = torch.from_numpy(ep.frames).to("cuda")
+    feats = vb.upload_bf16(ep.feats)
+    act_bits = synth.make_action_embed(cfg, 78)
+    d_act = vb.upload_bf16(act_bits)
+    side = torch.cuda.Stream()
+    ctx = vb.vlac_create(vb.make_config(cfg, 1), dev.weights)
+    L, n = cfg.seq_len, cfg.n_action
+    alpha = [min(1.0, 0.25 + l / 24.0) for l in range(32)]
+
+    def read_kv(cache, part, l):
+        t = torch.empty((cfg.max_seq, cfg.n_heads, cfg.head_dim), dtype=torch.bfloat16, device="cuda")
+        vb.vlac_cache_read(cache, part, 0, l, t)
+        torch.cuda.synchronize()
+        return t.view(torch.int16).cpu().numpy().copy()
+
+    def run(chunk):
+        cache = vb.vlac_cache_alloc(ctx, 1)
+        gp, keep = vb.make_params(alpha_override=alpha)
+        tok = torch.zeros((1, n), dtype=torch.int32, device="cuda")
+        lg = torch.zeros((1, n, cfg.vocab), dtype=torch.float32, device="cuda")
+        torch.cuda.synchronize()
+        with torch.cuda.stream(side):
+            for t in range(2):
+                if chunk:
+                    vb.vlac_step_chunk(ctx, cache, frames[t:t + 1], feats[t:t + 1], ids, gp, False, d_act, tok, lg)
+                else:
+                    vb.vlac_step(ctx, cache, frames[t:t + 1], feats[t:t + 1], ids, gp, False, tok, lg)
+        torch.cuda.synchronize()
+        attn = torch.empty((cfg.n_layers, cfg.n_heads, cfg.n_vision), dtype=torch.float32, device="cuda")
+        vb.vlac_cache_read(cache, vb.PART_ATTN_PREV, 0, 0, attn)
+        sel = vb.selection_to_host(vb.vlac_selection_view(cache))
+        return cache, tok.cpu().numpy().copy(), lg.cpu().numpy().copy(), attn.cpu().numpy().copy(), sel
+
+    caches = []
+    try:
+        ca, tok_a, lg_a, attn_a, sel_a = run(True); caches.append(ca)
+        assert vb.vlac_device_error(ctx) == 0
+        assert sel_a["M"][0, -1] < sel_a["M"][0, 0] < L, "the cached step must reuse tokens"
+        assert np.all(np.isfinite(lg_a)) and np.all((tok_a >= 0) & (tok_a < cfg.vocab))
+        assert np.array_equal(tok_a[0], lg_a[0].argmax(axis=1))
+        cb, tok_b, lg_b, attn_b, _ = run(True); caches.append(cb)
+        assert np.array_equal(tok_a, tok_b) and np.array_equal(lg_a, lg_b)
+        cc, _, _, attn_c, sel_c = run(False); caches.append(cc)
+        assert np.array_equal(sel_a["M"], sel_c["M"]) and np.array_equal(attn_a, attn_c)
+        for l in (0, 13, 31):
+            m = int(sel_a["M"][0, l])
+            assert np.array_equal(sel_a["rows"][0, l, :m], sel_c["rows"][0, l, :m])
+            for part in (vb.PART_K, vb.PART_V):
+                assert np.array_equal(read_kv(ca, part, l)[:L], read_kv(cc, part, l)[:L]), (l, part)
+        # layer 0, chunk rows: k = rope(W_k rmsnorm(e_i)) at position L + i, v = W_v rmsnorm(e_i)
+        lw = {}
+        for name, _ in vb.vlac_layer_w._fields_:
+            ptr = getattr(dev.layer_structs[0], name)
+            t = next(x for x in dev.tensors if x.data_ptr() == ptr)
+            lw[name] = t.view(torch.int16).cpu().numpy().view(np.uint16)
+        cos = next(x for x in dev.tensors if x.data_ptr() == dev.weights.rope_cos).cpu().numpy()
+        sin = next(x for x in dev.tensors if x.data_ptr() == dev.weights.rope_sin).cpu().numpy()
+        xn = orc.rms_norm(orc.widen_bf16(act_bits), orc.widen_bf16(lw["g_attn"]), cfg.rms_eps)
+        k_ref = orc.rope((xn @ orc.widen_bf16(lw["wk"]).T).reshape(n, cfg.n_heads, cfg.head_dim), np.arange(L, L + n), cos, sin)
+        v_ref = (xn @ orc.widen_bf16(lw["wv"]).T).reshape(n, cfg.n_heads, cfg.head_dim)
+        k_got = synth.bf16_to_f64(read_kv(ca, vb.PART_K, 0).view(np.uint16))[L:L + n]
+        v_got = synth.bf16_to_f64(read_kv(ca, vb.PART_V, 0).view(np.uint16))[L:L + n]
+        assert H.rel_err(k_got, k_ref) <= H.TOL and H.rel_err(v_got, v_ref) <= H.TOL
+    finally:
+        for c in caches:
+            vb.vlac_cache_free(c)
+        vb.vlac_destroy(ctx)
+
+
 def test_full_size_32_layers_properties_and_sampled_layer(H, vb):
     """The bench configuration itself: 32 layers of the 7B shape, weights drawn on the device, graph replay
     on a side stream.  Checked at this size: the selection against the checker (bit-exact, from the
