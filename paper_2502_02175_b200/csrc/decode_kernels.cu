@@ -588,6 +588,9 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
 #ifndef DA_KF
 #define DA_KF 20
 #endif
+#ifndef DA_THREADS
+#define DA_THREADS 320   // threads of a single-row attention CTA: every key of a ~300-token context has a thread of its own
+#endif
 // Attention of one new row per sequence over the cache (Sec. 3.1): one CTA per (head, sequence).
 // Scores: one key per thread (whole 16-byte-vectorised dot product); P*V: keys dealt round-robin to the
 // eight warps, each lane owning d/32 consecutive dimensions, partial sums combined in warp order.
@@ -689,13 +692,13 @@ __device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc
 }
 
 template <int DPL>
-__global__ void __launch_bounds__(256) decode_attention_kernel(const bf16* q, const bf16* kc, const bf16* vc, bf16* out,
-                                                               int pos, int max_seq, int H, int cps) {
+__global__ void __launch_bounds__(DA_THREADS) decode_attention_kernel(const bf16* q, const bf16* kc, const bf16* vc, bf16* out,
+                                                                      int pos, int max_seq, int H, int cps) {
   extern __shared__ float dsm[];
-  __shared__ float red[8];
+  __shared__ float red[DA_THREADS / 32];
   pdl_trigger();
   pdl_wait();
-  decode_attention_body<DPL, 256>(q, kc, vc, out, pos, max_seq, H, blockIdx.x, blockIdx.y, dsm, red, cps);
+  decode_attention_body<DPL, DA_THREADS>(q, kc, vc, out, pos, max_seq, H, blockIdx.x, blockIdx.y, dsm, red, cps);
 }
 
 // ---- one whole single-row pass as ONE persistent kernel -------------------------------------------
@@ -1196,15 +1199,15 @@ int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens,
     int rc = launch_gemv(ctx, ph[0], s);
     if (rc) return rc;
     {
-      const size_t smem = (size_t)(g.head_dim + ctx->max_seq + 8 * g.head_dim) * sizeof(float);
+      const size_t smem = (size_t)(g.head_dim + ctx->max_seq + (DA_THREADS / 32) * g.head_dim) * sizeof(float);
       const dim3 grid(g.n_heads, B);
       const bf16 *q = ctx->q_dec, *kc = ph[0].kc, *vc = ph[0].vc;
       cudaError_t e;
       switch (g.head_dim / 32) {
-        case 1: e = launch_pdl(decode_attention_kernel<1>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, 1); break;
-        case 2: e = launch_pdl(decode_attention_kernel<2>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, 1); break;
-        case 3: e = launch_pdl(decode_attention_kernel<3>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, 1); break;
-        default: e = launch_pdl(decode_attention_kernel<4>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, 1); break;
+        case 1: e = launch_pdl(decode_attention_kernel<1>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, 1); break;
+        case 2: e = launch_pdl(decode_attention_kernel<2>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, 1); break;
+        case 3: e = launch_pdl(decode_attention_kernel<3>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, 1); break;
+        default: e = launch_pdl(decode_attention_kernel<4>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, 1); break;
       }
       VLAC_CUDA_CHECK(e);
       VLAC_LAUNCH_CHECK(ctx);
@@ -1237,16 +1240,16 @@ int vlac_launch_chunk_pass(vlac_ctx* ctx, vlac_cache* c, const void* act_embed, 
       int rc = launch_gemv(ctx, ph[0], s);
       if (rc) return rc;
       {
-        const size_t smem = (size_t)(g.head_dim + ctx->max_seq + 8 * g.head_dim) * sizeof(float);
+        const size_t smem = (size_t)(g.head_dim + ctx->max_seq + (DA_THREADS / 32) * g.head_dim) * sizeof(float);
         const dim3 grid(g.n_heads, n);
         const bf16 *q = ctx->q_dec, *kc = ph[0].kc, *vc = ph[0].vc;
         const int pos = ctx->L;
         cudaError_t e;
         switch (g.head_dim / 32) {
-          case 1: e = launch_pdl(decode_attention_kernel<1>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, n); break;
-          case 2: e = launch_pdl(decode_attention_kernel<2>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, n); break;
-          case 3: e = launch_pdl(decode_attention_kernel<3>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, n); break;
-          default: e = launch_pdl(decode_attention_kernel<4>, grid, dim3(256), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, n); break;
+          case 1: e = launch_pdl(decode_attention_kernel<1>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, n); break;
+          case 2: e = launch_pdl(decode_attention_kernel<2>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, n); break;
+          case 3: e = launch_pdl(decode_attention_kernel<3>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, n); break;
+          default: e = launch_pdl(decode_attention_kernel<4>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, n); break;
         }
         VLAC_CUDA_CHECK(e);
         VLAC_LAUNCH_CHECK(ctx);
