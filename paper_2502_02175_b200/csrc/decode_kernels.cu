@@ -586,10 +586,10 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
 #define DA_KL 4
 #endif
 #ifndef DA_KF
-#define DA_KF 20
+#define DA_KF 25
 #endif
 #ifndef DA_THREADS
-#define DA_THREADS 320   // threads of a single-row attention CTA: every key of a ~300-token context has a thread of its own
+#define DA_THREADS 384   // threads of a single-row attention CTA: every key of a ~300-token context has a thread of its own
 #endif
 // Attention of one new row per sequence over the cache (Sec. 3.1): one CTA per (head, sequence).
 // Scores: one key per thread (whole 16-byte-vectorised dot product); P*V: keys dealt round-robin to the
@@ -659,7 +659,7 @@ __device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc
   float acc[DPL];
 #pragma unroll
   for (int e = 0; e < DPL; ++e) acc[e] = 0.f;
-  constexpr int KF = DA_KF;                                      // keys of this warp in flight
+  constexpr int KF = NT >= 512 ? 20 : DA_KF;                     // keys of this warp in flight (the 512-thread persistent pass keeps 20)
   for (int j0 = warp; j0 < nkeys; j0 += NW * KF) {
     float pj[KF];
     __align__(8) bf16 vv[KF][DPL];
