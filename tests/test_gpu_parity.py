@@ -387,6 +387,39 @@ def test_step_chunk_keeps_the_prompt_state_of_an_ordinary_step(H, vb):
         assert np.array_equal(a[3][l], b[3][l]) and np.array_equal(a[4][l], b[4][l])
 
 
+def test_step_chunk_argument_errors(H, vb):
+    """More than 8 chunk rows do not fit the columns of the single-row kernels, and the placeholder
+    embeddings are required: both are refused with INVALID_ARG before anything is launched."""
+    import dataclasses
+    cfg = dataclasses.replace(synth.tiny_config(), n_action=9)
+    sess = H.Session(cfg, None, dev_model=_DummyModel(vb, cfg.n_layers))
+    try:
+        fr = torch.zeros((1, cfg.n_cams, cfg.frame_hw, cfg.frame_hw, 3), dtype=torch.uint8, device="cuda")
+        ft = torch.zeros((1, cfg.n_vision, cfg.hidden), dtype=torch.bfloat16, device="cuda")
+        ids = torch.zeros((1, cfg.n_text), dtype=torch.int32, device="cuda")
+        act = torch.zeros((cfg.n_action, cfg.hidden), dtype=torch.bfloat16, device="cuda")
+        tok = torch.zeros((1, cfg.n_action), dtype=torch.int32, device="cuda")
+        l0 = vb.vlac_launch_count(sess.ctx)
+        with pytest.raises(vb.VlacError):
+            vb.vlac_step_chunk(sess.ctx, sess.cache, fr, ft, ids, None, False, act, tok)
+        assert vb.vlac_launch_count(sess.ctx) == l0
+    finally:
+        sess.close()
+    import ctypes as C
+    cfg = synth.tiny_config()
+    sess = H.Session(cfg, None, dev_model=_DummyModel(vb, cfg.n_layers))
+    try:
+        fr = torch.zeros((1, cfg.n_cams, cfg.frame_hw, cfg.frame_hw, 3), dtype=torch.uint8, device="cuda")
+        ft = torch.zeros((1, cfg.n_vision, cfg.hidden), dtype=torch.bfloat16, device="cuda")
+        ids = torch.zeros((1, cfg.n_text), dtype=torch.int32, device="cuda")
+        tok = torch.zeros((1, cfg.n_action), dtype=torch.int32, device="cuda")
+        rc = vb.lib.vlac_step_chunk(sess.ctx, sess.cache, fr.data_ptr(), ft.data_ptr(), ids.data_ptr(), None, 0, None,
+                                    tok.data_ptr(), None, None)
+        assert rc == -1
+    finally:
+        sess.close()
+
+
 def test_step_graph_replay_equals_direct_launch(H, vb):
     """On a non-default stream the step is captured once and replayed as a CUDA graph; on the default
     stream every kernel is launched directly.  Both must give the same bits, step after step."""
