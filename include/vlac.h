@@ -38,8 +38,9 @@ extern "C" {
 typedef struct vlac_ctx   vlac_ctx;    /* configuration, borrowed weight pointers, workspace         */
 typedef struct vlac_cache vlac_cache;  /* per-sequence K/V, previous frame, saved attention, selection */
 
-/* Decoder and sequence shape.  n_kv_heads must equal n_heads; head_dim must be a multiple of 32
- * and at most 128, hidden and ffn multiples of 8; n_layers <= VLAC_MAX_LAYERS; patch*3 even. */
+/* Decoder and sequence shape.  n_kv_heads must equal n_heads; head_dim must be 64 or 128 (the
+ * tensor-memory kernels take no other), hidden and ffn multiples of 8; n_layers <= VLAC_MAX_LAYERS;
+ * patch*3 even; max_batch <= 8. */
 typedef struct {
   int n_layers, hidden, n_heads, n_kv_heads, head_dim, ffn, vocab;
   int n_cams, grid, patch;            /* L_v = n_cams*grid*grid; a frame is (grid*patch)^2 RGB8 */
@@ -49,7 +50,8 @@ typedef struct {
   int max_batch;
 } vlac_config;
 
-/* One layer's weights: device bf16, row-major [out_features][in_features]; gains [hidden]. */
+/* One layer's weights: device bf16, row-major [out_features][in_features], each matrix 16-byte
+ * aligned (they are read through TMA tensor maps); gains [hidden]. */
 typedef struct {
   const void *wq, *wk, *wv, *wo, *w_gate, *w_up, *w_down, *g_attn, *g_mlp;
 } vlac_layer_w;
@@ -108,16 +110,16 @@ typedef struct {
 #define VLAC_PART_WARM       5   /* int32 [1] of seq: 0 = cold (next select reuses nothing)                */
 
 /* Create a context.  Copies `cfg` and the layer table, borrows every weight pointer, allocates the
- * workspace for max_batch sequences.  Errors: INVALID_ARG (bad shape, NULL), OOM, CUDA.
+ * workspace for max_batch sequences.  Errors: INVALID_ARG (a shape the kernels do not take, a NULL or
+ * a weight matrix that is not 16-byte aligned), OOM, CUDA.
  *
- * Environment switches, read here once per context (all off by default; results stay within the same
- * tolerance, timings differ):
+ * Environment switches, read here once per context (off by default):
  *   VLAC_NO_GRAPH=1     vlac_step launches its kernels one by one instead of replaying a captured graph
- *   VLAC_PASS_KERNEL=1  each single-row pass (action tokens 2..n) runs as one persistent cooperative kernel
- *   VLAC_GEMV_REG=1     single-row products use the register-pipelined kernel instead of the tensor-core one
- *   VLAC_GEMM_PAIR=1    Q/K/V, output and down projections of the prefill run as clusters of two CTAs that share
- *                       the activation tile (tcgen05 cta_group::2)
- *   VLAC_VERBOSE=1      CUDA errors noted by the library are also printed to stderr */
+ *                       (same results; used to profile single kernels)
+ *   VLAC_VERBOSE=1      CUDA errors noted by the library are also printed to stderr
+ *
+ * vlac_destroy releases the context.  Every cache allocated from it must have been freed first:
+ * BAD_STATE otherwise, and nothing is released. */
 int vlac_create(const vlac_config* cfg, const vlac_weights* w, vlac_ctx** out);
 int vlac_destroy(vlac_ctx* ctx);
 
@@ -172,14 +174,19 @@ int vlac_layer_forward(vlac_ctx* ctx, vlac_cache* cache, int layer, void* hidden
  *   action_tokens device int32 [batch][n_action], ties in the argmax go to the lower id
  *   all_logits    device fp32  [batch][n_action][vocab] or NULL: logits behind each action token
  *   forced_tokens device int32 [batch][n_action] or NULL: tokens to feed back instead of the
- *                 library's own choices (action_tokens still reports the library's choices). */
+ *                 library's own choices (action_tokens still reports the library's choices).
+ * Stream behaviour: on an ordinary (created) stream the step is captured once into a CUDA graph and
+ * replayed; caller buffers are staged through library buffers around the replay.  On the NULL /
+ * legacy default stream, inside a caller's own stream capture, with VLAC_NO_GRAPH=1 or while
+ * vlac_profile is on, the ~1300 kernels of a step are launched one by one: same results, but about
+ * three times slower at batch 1 (launch gaps, no overlap across kernel boundaries). */
 int vlac_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, const void* vision_feats,
               const int* prompt_ids, const vlac_select_params* params, int force_full,
               int* action_tokens, float* all_logits, const int* forced_tokens, void* stream);
 
 /* One control step whose action tokens all come from ONE parallel pass (the paper applies the method
- * to OpenVLA-OFT, "a faster variant with action chunking", Sec. 5 main LIBERO results and Table 2,
- * and prints no equations for that decoder; the reading taken is stated here).  Selection, input rows
+ * to OpenVLA-OFT, a decoder that emits its action chunk in one pass: Sec. 5 main LIBERO results and
+ * Table 2; it prints no equations for that decoder, so the reading taken is stated here).  Selection, input rows
  * and the partial prefill are those of vlac_step.  Then n_action placeholder rows at positions
  * L .. L+n_action-1, whose input is act_embed[i] for every sequence, go through all layers together:
  * each sees the whole prompt (reused or fresh K/V, as the prefill left it) and every row of the
@@ -219,6 +226,15 @@ int vlac_profile_segments(vlac_ctx* ctx, double* ms, int cap, int* n);
 /* Nonzero if a device-side bounded wait gave up since the context was created (reads one int
  * back; synchronises the stream). */
 int vlac_device_error(vlac_ctx* ctx, void* stream);
+
+/* Self-test of the bounded device-side waits (the paper has no counterpart).  Every wait on a
+ * shared-memory barrier inside the library's kernels polls against the GPU's wall clock and gives up
+ * after a fixed time, recording a code in the context's device error word instead of hanging.  This
+ * call runs that same wait, in a one-CTA kernel, on a barrier that nothing ever signals, with a limit
+ * of limit_us microseconds (1..100000), then synchronises the stream and returns what
+ * vlac_device_error returns: VLAC_ERR_TIMEOUT when the mechanism works.  The error word stays set for
+ * the life of the context, so use a context made for the purpose. */
+int vlac_selftest_wait_expiry(vlac_ctx* ctx, unsigned int limit_us, void* stream);
 
 /* Greedy token choice that allocates nothing (the paper has no counterpart; it is the last step of
  * vlac_step offered on its own).  For each of `rows` logits rows it returns the index of the largest

@@ -475,8 +475,9 @@ def step_chunk(cfg, model: Dict[str, object], cache: CacheState, frames_t: np.nd
                selection: Optional[Selection] = None) -> StepResult:
     """Selection and partial prefill as in ``step``, then ALL action tokens from one pass.
 
-    The paper applies the method unchanged to OpenVLA-OFT, "a faster variant with action
-    chunking" (main LIBERO results), and gives no equations for that decoder.  Reading taken
+    The paper applies the method unchanged to OpenVLA-OFT, whose decoder emits its action
+    chunk in one pass (Sec. 5, main LIBERO results, Table 2), and gives no equations for that
+    decoder.  Reading taken
     here: behind the prompt sit ``n_action`` placeholder rows at positions ``L .. L+n_action-1``
     whose input is the fixed embedding ``act_embed_bf16[i]`` (a weight, not a fed-back token).
     They run through every layer together: each sees the whole prompt (reused or fresh K/V, as

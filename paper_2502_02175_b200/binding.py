@@ -55,7 +55,8 @@ class vlac_selection(C.Structure):
 EXPORTS = ("vlac_create", "vlac_destroy", "vlac_cache_alloc", "vlac_cache_reset", "vlac_cache_free",
            "vlac_cache_read", "vlac_cache_write", "vlac_select", "vlac_select_import", "vlac_layer_forward",
            "vlac_step", "vlac_step_chunk", "vlac_selection_view", "vlac_launch_count", "vlac_device_error", "vlac_status_string",
-           "vlac_profile", "vlac_profile_read", "vlac_profile_segments", "vlac_greedy_tokens_static")
+           "vlac_profile", "vlac_profile_read", "vlac_profile_segments", "vlac_greedy_tokens_static",
+           "vlac_selftest_wait_expiry")
 
 lib.vlac_status_string.restype = C.c_char_p
 lib.vlac_status_string.argtypes = [C.c_int]
@@ -77,6 +78,7 @@ lib.vlac_step_chunk.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, 
                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 lib.vlac_selection_view.argtypes = [C.c_void_p, C.POINTER(vlac_selection)]
 lib.vlac_device_error.argtypes = [C.c_void_p, C.c_void_p]
+lib.vlac_selftest_wait_expiry.argtypes = [C.c_void_p, C.c_uint, C.c_void_p]
 lib.vlac_profile.argtypes = [C.c_void_p, C.c_int]
 lib.vlac_profile_segments.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.c_int, C.POINTER(C.c_int)]
 lib.vlac_greedy_tokens_static.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_longlong, C.c_void_p, C.c_void_p]
@@ -279,6 +281,11 @@ def vlac_launch_count(ctx: int) -> int:
 
 def vlac_device_error(ctx: int) -> int:
     return int(lib.vlac_device_error(ctx, _stream()))
+
+
+def vlac_selftest_wait_expiry(ctx: int, limit_us: int) -> int:
+    """Status of the bounded-wait self-test (VLAC_ERR_TIMEOUT = -5 when the wait gave up as designed)."""
+    return int(lib.vlac_selftest_wait_expiry(ctx, int(limit_us), _stream()))
 
 
 def vlac_profile(ctx: int, enable: bool) -> None:

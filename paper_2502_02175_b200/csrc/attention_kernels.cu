@@ -340,20 +340,22 @@ constexpr size_t at_smem(int Lv) {
 int vlac_attention_setup(vlac_ctx* ctx) {
   const vlac_config& g = ctx->cfg;
   ctx->attn_tiles = 0;
-  if (!ctx->tc_ok) return VLAC_OK;
-  if (g.head_dim != 64 && g.head_dim != 128) return VLAC_OK;
+  if (g.head_dim != 64 && g.head_dim != 128) return VLAC_ERR_INVALID_ARG;
   const int tiles = (ctx->L + AT_Q - 1) / AT_Q;
-  if (g.n_text_post > 0 && tiles > g.n_text_post) return VLAC_OK;      // the partial buffer is sized by the text rows
   cudaError_t e;
   if (g.head_dim == 128) e = cudaFuncSetAttribute(attention_tile_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)at_smem<128>(ctx->Lv));
   else e = cudaFuncSetAttribute(attention_tile_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)at_smem<64>(ctx->Lv));
-  if (e != cudaSuccess) { cudaGetLastError(); return VLAC_OK; }
+  if (e != cudaSuccess) { vlac_note_cuda_error(e, __FILE__, __LINE__); return VLAC_ERR_CUDA; }
   if (cudaMalloc(&ctx->tmap_q, sizeof(CUtensorMap)) != cudaSuccess) { cudaGetLastError(); return VLAC_ERR_OOM; }
   CUtensorMap m;
   int rc = vlac_encode_map_2d(&m, ctx->q, ctx->rows_max, g.hidden, AT_Q);
   if (rc != VLAC_OK) return rc;
   VLAC_CUDA_CHECK(cudaMemcpy(ctx->tmap_q, &m, sizeof(m), cudaMemcpyHostToDevice));
   ctx->probs_all = nullptr; ctx->defer_emit = 0;
+  if (g.n_text_post > 0 &&
+      cudaMalloc(&ctx->probs, sizeof(float) * (size_t)g.max_batch * tiles * g.n_heads * ctx->Lv) != cudaSuccess) {
+    cudaGetLastError(); return VLAC_ERR_OOM;
+  }
   if (g.n_text_post > 0 &&
       cudaMalloc(&ctx->probs_all, sizeof(float) * (size_t)g.n_layers * g.max_batch * tiles * g.n_heads * ctx->Lv) != cudaSuccess) {
     cudaGetLastError(); return VLAC_ERR_OOM;
@@ -364,7 +366,6 @@ int vlac_attention_setup(vlac_ctx* ctx) {
 
 int vlac_attention_cache_setup(vlac_ctx* ctx, vlac_cache* c) {
   c->tmaps_kv = nullptr;
-  if (!ctx->attn_tiles) return VLAC_OK;
   const vlac_config& g = ctx->cfg;
   const int n = 2 * g.n_layers;
   CUtensorMap* host = (CUtensorMap*)malloc(sizeof(CUtensorMap) * n);

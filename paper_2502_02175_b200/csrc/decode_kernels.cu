@@ -659,7 +659,7 @@ __device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc
   float acc[DPL];
 #pragma unroll
   for (int e = 0; e < DPL; ++e) acc[e] = 0.f;
-  constexpr int KF = NT >= 512 ? 20 : DA_KF;                     // keys of this warp in flight (the 512-thread persistent pass keeps 20)
+  constexpr int KF = DA_KF;                                      // keys of this warp in flight
   for (int j0 = warp; j0 < nkeys; j0 += NW * KF) {
     float pj[KF];
     __align__(8) bf16 vv[KF][DPL];
@@ -699,241 +699,6 @@ __global__ void __launch_bounds__(DA_THREADS) decode_attention_kernel(const bf16
   pdl_trigger();
   pdl_wait();
   decode_attention_body<DPL, DA_THREADS>(q, kc, vc, out, pos, max_seq, H, blockIdx.x, blockIdx.y, dsm, red, cps);
-}
-
-// ---- one whole single-row pass as ONE persistent kernel -------------------------------------------
-// All layers, five phases each (QKV | attention | output proj | gate/up | down), separated by grid
-// barriers instead of kernel boundaries.  Every CTA requests the first weights of its next phase
-// before it enters the barrier, so HBM keeps streaming while the grid synchronises.  Launched
-// cooperatively (all CTAs co-resident); every barrier wait is bounded by the global timer.
-#define GV_BARRIER_LIMIT_NS 200000000ull
-
-__device__ __forceinline__ unsigned long long gv_global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
-  unsigned v;
-  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
-// Arrive on the grid-wide counter and wait until `target` arrivals.  Returns false (for the whole CTA)
-// if the wait gave up or an error was already recorded; later barriers then fall through at once.
-__device__ __forceinline__ bool grid_barrier(unsigned* counter, unsigned target, int* dev_error) {
-  __syncthreads();
-  int ok = 1;
-  if (threadIdx.x == 0) {
-    __threadfence();
-    atomicAdd(counter, 1u);
-    const unsigned long long t0 = gv_global_ns();
-    unsigned polls = 0;
-    while (ld_acquire_u32(counter) < target) {
-      if ((++polls & 255u) != 0) continue;                       // the error word and the wall clock are looked at rarely
-      if (*reinterpret_cast<volatile int*>(dev_error) != 0) { ok = 0; break; }
-      if (gv_global_ns() - t0 > GV_BARRIER_LIMIT_NS) { atomicCAS(dev_error, 0, 0x80000 | (int)(target & 0xffff)); ok = 0; break; }
-    }
-    __threadfence();
-  }
-  return __syncthreads_and(ok) != 0;
-}
-
-struct PassArgs {
-  const GemvArgs* phases;      // [n_layers][4]: QKV, output proj, gate/up, down (for this pass's position)
-  int n_layers, pos, n_heads, batch;
-  bf16* ao;                    // attention output rows [batch][H*d]
-  unsigned* counter;           // grid barrier counter, zeroed before the launch
-  int* dev_error;
-};
-
-// Phase parameters a warp derives from the arguments of a matrix-vector phase.
-struct PhaseGeom { int u_begin, n_local, n_groups, ns_w, K; };
-__device__ __forceinline__ PhaseGeom phase_geom(const GemvArgs& a, int warp) {
-  PhaseGeom g;
-  const int n_units = unit_count(a.mode, a.N);
-  g.u_begin = (int)(((long long)n_units * blockIdx.x) / gridDim.x);
-  g.n_local = (int)(((long long)n_units * (blockIdx.x + 1)) / gridDim.x) - g.u_begin;
-  g.n_groups = (g.n_local + 7) / 8;
-  const int S = a.K / 64;
-  g.ns_w = warp < S ? (S - warp + GT_WARPS - 1) / GT_WARPS : 0;
-  g.K = a.K;
-  return g;
-}
-
-// The tensor-core weight-streaming kernel as one persistent kernel per single-row pass.  The ring of
-// asynchronous copies does not stop at a phase boundary: while the CTA flushes a phase, waits at the grid
-// barrier and stages the next activations, its warps' copies of the NEXT phase's first weights (which depend
-// on nothing) are already in flight, so HBM keeps streaming across what would be a kernel boundary.
-// The issue side may run at most one phase ahead of the consume side; the arguments of phase p+1 are put in
-// shared memory when phase p begins.
-__global__ void __launch_bounds__(GT_THREADS, 1) decode_pass_kernel(PassArgs pa) {
-  extern __shared__ __align__(128) unsigned char gt_smem[];
-  __shared__ float red[GT_WARPS];
-  __shared__ GemvArgs sargs[2];                                 // arguments of phase p in slot p & 1
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const unsigned ring_w = (unsigned)__cvta_generic_to_shared(gt_smem) + (unsigned)warp * (GT_DEPTH * GT_SLOT_BYTES);
-  float* part = reinterpret_cast<float*>(gt_smem + GT_RING_BYTES);
-  bf16* xs = reinterpret_cast<bf16*>(gt_smem + GT_RING_BYTES + GT_PART_BYTES);
-  const int n_phases = 4 * pa.n_layers;
-  const unsigned G_ctas = gridDim.x;
-  unsigned n_bar = 0;
-  auto load_args = [&](int ph) {
-    if (ph < n_phases && tid < (int)(sizeof(GemvArgs) / sizeof(int)))
-      reinterpret_cast<int*>(&sargs[ph & 1])[tid] = reinterpret_cast<const int*>(pa.phases + ph)[tid];
-  };
-  load_args(0);
-  load_args(1);
-  __syncthreads();
-
-  // ---- issue side
-  int pc = 0;                                                   // phase being consumed
-  int ip = 0, ig = 0, ij = 0, islot = 0;
-  bool i_ready = false;
-  unsigned real_mask = 0u;                                      // ring positions that hold an item (the rest were issued empty)
-  PhaseGeom igm = {0, 0, 0, 0, 0};
-  const char* rowptr[4];
-  auto load_rowptrs = [&](int g) {
-    const GemvArgs& a = sargs[ip & 1];
-    const UnitRows r0 = unit_rows(a, igm.u_begin + min(g * 8 + (lane >> 3), igm.n_local - 1));
-    const UnitRows r1 = unit_rows(a, igm.u_begin + min(g * 8 + (lane >> 3) + 4, igm.n_local - 1));
-    rowptr[0] = reinterpret_cast<const char*>(r0.pa); rowptr[1] = reinterpret_cast<const char*>(r1.pa);
-    rowptr[2] = reinterpret_cast<const char*>(r0.pb); rowptr[3] = reinterpret_cast<const char*>(r1.pb);
-  };
-  auto issue = [&]() {
-    if (!i_ready && ip < n_phases && ip <= pc + 1) {
-      igm = phase_geom(sargs[ip & 1], warp);
-      ig = 0; ij = 0;
-      if (igm.n_groups > 0 && igm.ns_w > 0) { load_rowptrs(0); i_ready = true; }
-      else ++ip;                                                // nothing for this warp in that phase
-    }
-    if (i_ready) real_mask |= 1u << islot; else real_mask &= ~(1u << islot);
-    if (i_ready) {
-      const unsigned slotp = ring_w + (unsigned)islot * GT_SLOT_BYTES;
-      const size_t koff = (size_t)(warp + GT_WARPS * ij) * 128 + (size_t)(lane & 7) * 16;
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int row = (lane >> 3) + 4 * i;
-        cp_async16(slotp + (unsigned)(row * 128 + (((lane & 7) ^ (row & 7)) << 4)), rowptr[i] + koff);
-      }
-      if (++ij == igm.ns_w) {
-        ij = 0;
-        if (++ig < igm.n_groups) load_rowptrs(ig);
-        else { ++ip; i_ready = false; }
-      }
-    }
-    cp_async_commit();
-    islot = (islot + 1 == GT_DEPTH) ? 0 : islot + 1;
-  };
-  // (the ring starts empty: the first positions the consume loop meets carry nothing and are filled there,
-  // which keeps the issue code at a single place)
-
-  int cslot = 0;
-  for (pc = 0; pc < n_phases; ++pc) {
-    // ---- phase start: next phase's arguments, dependencies, activations
-    load_args(pc + 1);
-    if (pc > 0) grid_barrier(pa.counter, (++n_bar) * G_ctas, pa.dev_error);   // the row entering the pass came from an earlier kernel
-    if ((pc & 3) == 1) {
-      // attention of this layer sits between the Q/K/V phase and the output projection
-      const int hb = blockIdx.x;
-      if (hb < pa.n_heads * pa.batch) {
-        const GemvArgs* qkv = pa.phases + (pc - 1);
-        const bf16 *q = qkv->q_out, *kc = qkv->kc, *vc = qkv->vc;
-        const int max_seq = qkv->max_seq, dpl = qkv->d / 32;
-        const int h = hb % pa.n_heads, b = hb / pa.n_heads;
-        float* dsm = reinterpret_cast<float*>(xs);
-        if (dpl == 4) decode_attention_body<4, GT_THREADS>(q, kc, vc, pa.ao, pa.pos, max_seq, pa.n_heads, h, b, dsm, red);
-        else if (dpl == 2) decode_attention_body<2, GT_THREADS>(q, kc, vc, pa.ao, pa.pos, max_seq, pa.n_heads, h, b, dsm, red);
-        else if (dpl == 3) decode_attention_body<3, GT_THREADS>(q, kc, vc, pa.ao, pa.pos, max_seq, pa.n_heads, h, b, dsm, red);
-        else decode_attention_body<1, GT_THREADS>(q, kc, vc, pa.ao, pa.pos, max_seq, pa.n_heads, h, b, dsm, red);
-      }
-      grid_barrier(pa.counter, (++n_bar) * G_ctas, pa.dev_error);
-    }
-    __syncthreads();                                            // sargs[pc & 1] and [(pc + 1) & 1] are in place
-    const GemvArgs& a = sargs[pc & 1];
-    const PhaseGeom gm = phase_geom(a, warp);
-    const int K = a.K, nb = a.nb;
-    for (int b = 0; b < nb; ++b) {
-      if (a.x_f32) {
-        // values an earlier phase of this kernel wrote on other SMs: read past the L1
-        const float* x = a.x_f32 + (size_t)b * K;
-        float ss = 0.f;
-        for (int k = tid; k < K; k += GT_THREADS) { const float v = __ldcg(x + k); ss += v * v; }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-        __syncthreads();
-        if (lane == 0) red[warp] = ss;
-        __syncthreads();
-        float t = 0.f;
-#pragma unroll
-        for (int w = 0; w < GT_WARPS; ++w) t += red[w];
-        const float r = rsqrtf(t / (float)K + a.eps);
-        for (int k = tid; k < K; k += GT_THREADS) xs[(size_t)b * K + k] = __float2bfloat16(__ldcg(x + k) * r * bf2f(a.gain[k]));
-      } else {
-        const uint4* src = reinterpret_cast<const uint4*>(a.x_bf16 + (size_t)b * K);
-        uint4* dst = reinterpret_cast<uint4*>(xs + (size_t)b * K);
-        for (int c = tid; c < K / 8; c += GT_THREADS) dst[c] = __ldcg(src + c);
-      }
-    }
-    __syncthreads();
-
-    // ---- consume side of this phase
-    const int col_n = lane >> 2;
-    const unsigned* xw = reinterpret_cast<const unsigned*>(xs + (size_t)min(col_n, max(nb - 1, 0)) * K) + (lane & 3);
-    const bool col_live = col_n < nb;
-    const int nbp = nb <= 1 ? 1 : (nb <= 2 ? 2 : (nb <= 4 ? 4 : 8));
-    const int G = 8 / nbp;
-    for (int g = 0; g < gm.n_groups; ++g) {
-      float c[4] = {0.f, 0.f, 0.f, 0.f};
-      for (int j = 0; j < gm.ns_w;) {
-        // the ring is consumed position by position; a position issued while the issue side had to hold
-        // back (it may not run two phases ahead) carries nothing and is simply handed back
-        cp_async_wait<GT_DEPTH - 1>();
-        __syncwarp();
-        const bool real = (real_mask >> cslot) & 1u;
-        if (real) {
-          const unsigned slotp = ring_w + (unsigned)cslot * GT_SLOT_BYTES;
-          const int k0 = (warp + GT_WARPS * j) * 64;
-#pragma unroll
-          for (int kk = 0; kk < 4; ++kk) {
-            unsigned af[4];
-            const int row = lane & 15, kc = 2 * kk + (lane >> 4);
-            ldmatrix_x4(slotp + (unsigned)(row * 128 + ((kc ^ (row & 7)) << 4)), af);
-            unsigned b0 = 0u, b1 = 0u;
-            if (col_live) { b0 = xw[(k0 + kk * 16) / 2]; b1 = xw[(k0 + kk * 16) / 2 + 4]; }
-            mma_16816(c, af, b0, b1);
-          }
-          ++j;
-        }
-        __syncwarp();
-        issue();
-        cslot = (cslot + 1 == GT_DEPTH) ? 0 : cslot + 1;
-      }
-      const int round = g / G, gr = g - round * G;
-      {
-        float* dst = part + ((size_t)(((round & 1) * G + gr) * GT_WARPS + warp) * 16) * nbp;
-        const int r = lane >> 2, n0 = (lane & 3) * 2;
-        if (n0 < nb) { dst[r * nbp + n0] = c[0]; dst[(r + 8) * nbp + n0] = c[2]; }
-        if (n0 + 1 < nb) { dst[r * nbp + n0 + 1] = c[1]; dst[(r + 8) * nbp + n0 + 1] = c[3]; }
-      }
-      if (gr == G - 1 || g == gm.n_groups - 1) {
-        __syncthreads();
-        const int n_items = (gr + 1) * 8 * nb;
-        for (int idx = tid; idx < n_items; idx += GT_THREADS) {
-          const int gi = idx / (8 * nb), rem = idx - gi * 8 * nb;
-          const int uu = rem / nb, col = rem - uu * nb;
-          const int ul = (round * G + gi) * 8 + uu;
-          if (ul >= gm.n_local) continue;
-          const float* src = part + ((size_t)(((round & 1) * G + gi) * GT_WARPS) * 16) * nbp;
-          float ya = 0.f, yb = 0.f;
-#pragma unroll
-          for (int w = 0; w < GT_WARPS; ++w) { ya += src[((size_t)w * 16 + uu) * nbp + col]; yb += src[((size_t)w * 16 + uu + 8) * nbp + col]; }
-          const UnitRows cu = unit_rows(a, gm.u_begin + ul);
-          store_unit(a, cu, col, ya, yb);
-        }
-      }
-    }
-    __syncthreads();                                            // the last flush has read `part` and the arguments
-  }
 }
 
 __global__ void __launch_bounds__(256) embed_token_kernel(const bf16* embed, const int* tokens, int tok_stride, int tok_index,
@@ -1013,7 +778,7 @@ int launch_gemv(vlac_ctx* ctx, const GemvArgs& a, cudaStream_t s) {
   const bool timed = ctx->prof_on && ctx->prof_n < VLAC_PROF_CAP;
   if (timed) VLAC_CUDA_CHECK(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n], s));
   const size_t gt_smem = gt_smem_bytes(ctx, a);
-  if (ctx->gemv_stream && a.K % 64 == 0 && nb <= 8 && gt_smem <= GT_SMEM_MAX) {
+  if (a.K % 64 == 0 && nb <= 8 && gt_smem <= GT_SMEM_MAX) {
     if (nb > 4) VLAC_CUDA_CHECK(launch_pdl(gemv_mma_kernel<true>, dim3(ctx->n_sm * GT_GRID_PER_SM), dim3(GT_THREADS), gt_smem, s, a));
     else VLAC_CUDA_CHECK(launch_pdl(gemv_mma_kernel<false>, dim3(ctx->n_sm * GT_GRID_PER_SM), dim3(GT_THREADS), gt_smem, s, a));
   } else
@@ -1036,7 +801,7 @@ int launch_gemv(vlac_ctx* ctx, const GemvArgs& a, cudaStream_t s) {
 // over slices of K, each adding its part to x_out in stream order (RESID with a bf16 input only; the slices are
 // multiples of 64 columns of 16-byte aligned rows).
 int launch_gemv_sliced(vlac_ctx* ctx, const GemvArgs& a, cudaStream_t s) {
-  if (ctx->gemv_stream && a.mode == GV_RESID && a.x_bf16 && !a.ld && a.K % 64 == 0 && gt_smem_bytes(ctx, a) > GT_SMEM_MAX) {
+  if (a.mode == GV_RESID && a.x_bf16 && !a.ld && a.K % 64 == 0 && gt_smem_bytes(ctx, a) > GT_SMEM_MAX) {
     for (int n = 2; n <= 4; n *= 2) {
       if (a.K % (64 * n)) continue;
       GemvArgs h = a;
@@ -1055,8 +820,6 @@ int launch_gemv_sliced(vlac_ctx* ctx, const GemvArgs& a, cudaStream_t s) {
 
 }  // namespace
 
-static size_t pass_smem(const vlac_ctx* ctx, int NB);
-
 int vlac_decode_setup(vlac_ctx* ctx) {
   const int kmax = ctx->cfg.ffn > ctx->cfg.hidden ? ctx->cfg.ffn : ctx->cfg.hidden;
   const int mb = ctx->cfg.max_batch;
@@ -1072,28 +835,8 @@ int vlac_decode_setup(vlac_ctx* ctx) {
   if (NB >= 2) VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_pair_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * (size_t)kmax * 2)));
   if (NB >= 4) VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_pair_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(4 * (size_t)kmax * 2)));
   if (NB >= 8) VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_pair_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(8 * (size_t)kmax * 2)));
-  // tensor-core variant of the weight-streaming kernel (VLAC_GEMV_REG=1 keeps the register-pipelined one)
-  ctx->gemv_stream = getenv("VLAC_GEMV_REG") ? 0 : 1;
   VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GT_SMEM_MAX));
   VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GT_SMEM_MAX));
-  // persistent pass kernel: as many CTAs as are guaranteed co-resident
-  ctx->pass_grid = 0;
-  // Opt-in (VLAC_PASS_KERNEL=1).  Needs every K to be a multiple of 64 (the tensor-core body) and room for
-  // the activations beside the ring.  Measured on B200: correct, but a pass takes 3.25 ms against 2.65 ms for
-  // the per-phase kernels replayed from a graph.  A grid barrier under a saturated memory system costs more
-  // than a programmatic kernel boundary, and the ring (19 MB over the GPU) covers under 3 us of streaming.
-  if (getenv("VLAC_PASS_KERNEL") != nullptr && ctx->max_seq > 0 && ctx->cfg.hidden % 64 == 0 && ctx->cfg.ffn % 64 == 0) {
-    const size_t psm = pass_smem(ctx, NB_seq);
-    int per_sm = 0, coop = 0, dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
-    if (e == cudaSuccess && coop && psm <= GT_SMEM_MAX) {
-      e = cudaFuncSetAttribute(decode_pass_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psm);
-      if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_pass_kernel, GT_THREADS, psm);
-      if (e == cudaSuccess && per_sm > 0) ctx->pass_grid = ctx->n_sm;
-    }
-    if (e != cudaSuccess) cudaGetLastError();
-  }
   return VLAC_OK;
 }
 
@@ -1136,42 +879,6 @@ static GemvArgs logits_phase(vlac_ctx* ctx, vlac_cache* c) {
   return a;
 }
 
-static size_t pass_smem(const vlac_ctx* ctx, int NB) {
-  const vlac_config& g = ctx->cfg;
-  const int kmax = g.ffn > g.hidden ? g.ffn : g.hidden;
-  const size_t xs = (size_t)NB * kmax * sizeof(bf16);
-  const size_t at = (size_t)(g.head_dim + ctx->max_seq + GT_WARPS * g.head_dim) * sizeof(float);   // attention scratch shares the activation area
-  return (size_t)GT_RING_BYTES + GT_PART_BYTES + (xs > at ? xs : at);
-}
-
-// Per-cache table of phase arguments for the persistent pass kernel, and its barrier counter.
-int vlac_decode_cache_setup(vlac_ctx* ctx, vlac_cache* c) {
-  const int nl = ctx->cfg.n_layers;
-  const int n_pass = ctx->cfg.n_action > 1 ? ctx->cfg.n_action - 1 : 1;      // one table per single-row position L, L+1, ...
-  const size_t n = (size_t)n_pass * 4 * nl;
-  static_assert(sizeof(GemvArgs) % sizeof(int) == 0, "copied word by word");
-  GemvArgs* host = (GemvArgs*)malloc(sizeof(GemvArgs) * n);
-  if (!host) return VLAC_ERR_OOM;
-  for (int i = 0; i < n_pass; ++i)
-    for (int l = 0; l < nl; ++l) layer_phases(ctx, c, l, ctx->L + i, host + ((size_t)i * nl + l) * 4);
-  int rc = VLAC_OK;
-  if (cudaMalloc(&c->dec_phases, sizeof(GemvArgs) * n) != cudaSuccess) { cudaGetLastError(); rc = VLAC_ERR_OOM; }
-  if (rc == VLAC_OK && cudaMemcpy(c->dec_phases, host, sizeof(GemvArgs) * n, cudaMemcpyHostToDevice) != cudaSuccess) rc = VLAC_ERR_CUDA;
-  free(host);
-  if (rc == VLAC_OK && cudaMalloc(&c->dec_counter, 256) != cudaSuccess) { cudaGetLastError(); rc = VLAC_ERR_OOM; }
-  return rc;
-}
-
-static cudaError_t launch_pass(const PassArgs& pa, int grid, size_t smem, cudaStream_t s) {
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(grid); cfg.blockDim = dim3(GT_THREADS); cfg.dynamicSmemBytes = smem; cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeCooperative;            // all CTAs resident at once: the grid barriers rely on it
-  attr[0].val.cooperative = 1;
-  cfg.attrs = attr; cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, decode_pass_kernel, pa);
-}
-
 int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens, int tok_stride, int tok_index,
                             int pos, cudaStream_t s) {
   const vlac_config& g = ctx->cfg;
@@ -1179,20 +886,6 @@ int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens,
   VLAC_CUDA_CHECK(launch_pdl(embed_token_kernel, dim3(B), dim3(256), 0, s, (const bf16*)ctx->w.embed, fed_tokens, tok_stride, tok_index,
                              ctx->x_dec, D, g.vocab));
   VLAC_LAUNCH_CHECK(ctx);
-  const int NB = B <= 1 ? 1 : (B <= 2 ? 2 : (B <= 4 ? 4 : 8));
-  const int pass_idx = pos - ctx->L;
-  if (ctx->pass_grid > 0 && !ctx->prof_on && g.n_heads * B <= ctx->pass_grid && pass_idx >= 0 && pass_idx < g.n_action - 1) {
-    // the whole pass as one persistent kernel
-    VLAC_CUDA_CHECK(cudaMemsetAsync(c->dec_counter, 0, sizeof(unsigned), s));
-    PassArgs pa;
-    pa.phases = (const GemvArgs*)c->dec_phases + (size_t)pass_idx * 4 * g.n_layers; pa.n_layers = g.n_layers; pa.pos = pos; pa.n_heads = g.n_heads; pa.batch = B;
-    pa.ao = ctx->ao_dec; pa.counter = (unsigned*)c->dec_counter; pa.dev_error = ctx->dev_error;
-    const size_t smem = pass_smem(ctx, NB);
-    VLAC_CUDA_CHECK(launch_pass(pa, ctx->pass_grid, smem, s));
-    VLAC_LAUNCH_CHECK(ctx);
-    return VLAC_OK;
-  }
-  // one kernel per phase (also the path that per-launch timing brackets)
   for (int l = 0; l < g.n_layers; ++l) {
     GemvArgs ph[4];
     layer_phases(ctx, c, l, pos, ph);

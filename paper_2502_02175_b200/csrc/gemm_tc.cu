@@ -87,13 +87,14 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 // Bounded wait.  On expiry the CTA's abort flag is raised, `code` goes to the device error word and
 // every later wait of the CTA returns at once, so the kernel always terminates.
-__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, volatile int* abort_flag, int* dev_error, int code) {
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned parity, volatile int* abort_flag, int* dev_error, int code,
+                                          unsigned long long limit_ns = TG_WAIT_LIMIT_NS) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (global_ns() - t0 > TG_WAIT_LIMIT_NS) break;
+    if (global_ns() - t0 > limit_ns) break;
   }
   *abort_flag = 1;
   if (dev_error) atomicCAS(dev_error, 0, code);
@@ -134,28 +135,6 @@ __device__ __forceinline__ void umma_bf16(unsigned tmem_d, unsigned long long a,
 __device__ __forceinline__ void umma_commit(unsigned long long* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// ---- forms used when two CTAs of a cluster share one 256-row MMA (cta_group::2)
-__device__ __forceinline__ unsigned cluster_ctarank() { unsigned r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
-__device__ __forceinline__ unsigned mapa_u32(unsigned addr, unsigned rank) {
-  unsigned r; asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank)); return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// the copy lands in this CTA's shared memory; its bytes are counted on a barrier that may live in the other CTA of the pair
-__device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* tm, int x, int y, unsigned bar_cluster_addr) {
-  asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-               ::"r"(smem_u32(dst)), "l"(tm), "r"(x), "r"(y), "r"(bar_cluster_addr) : "memory");
-}
-__device__ __forceinline__ void umma_bf16_pair(unsigned tmem_d, unsigned long long a, unsigned long long b, unsigned idesc, unsigned accumulate) {
-  asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n}\n"
-               ::"r"(tmem_d), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_commit_pair(unsigned bar_cluster_addr) {
-  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_cluster_addr) : "memory");
-}
-
 __device__ __forceinline__ void tmem_ld16(unsigned taddr, float* v) {
   unsigned r[16];
   asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
@@ -167,10 +146,6 @@ __device__ __forceinline__ void tmem_ld16(unsigned taddr, float* v) {
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-// PAIR: launched as clusters of two CTAs along x.  Each CTA keeps its own 128 weight rows and epilogue; the token
-// boxes are dealt alternately to the two CTAs, so a CTA stages only half of the activations, and the CTA of rank 0
-// issues one 256-row MMA for both (cta_group::2), reading the other half from its partner's shared memory.
-template <bool PAIR>
 __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_constant__ TcArgs a) {
   extern __shared__ __align__(1024) unsigned char ring_raw[];
   __shared__ __align__(8) unsigned long long full_bar[TG_MAX_STAGES], empty_bar[TG_MAX_STAGES], acc_bar;
@@ -196,19 +171,12 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
-  const unsigned crank = PAIR ? cluster_ctarank() : 0u;
-  if (PAIR) cluster_sync_all();                                 // both CTAs' barriers exist before either is signalled remotely
   pdl_trigger();
   // tensor memory does not depend on earlier kernels either: allocated (for the largest token chunk) before the wait
   const unsigned tmem_cols = (unsigned)a.tmem_cols;
-  if (warp == 1) {                                              // whole warp (in a pair: the same warp of both CTAs)
-    if (PAIR) {
-      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
-      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-    } else {
-      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
-      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
+  if (warp == 1) {                                              // whole warp
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   // The live token count was written by the selection kernels, which never release their dependents early, so
   // it is complete before any kernel launched after them starts: it may be read ahead of the dependency wait.
@@ -216,19 +184,16 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
   const int tok0 = blockIdx.z * 512;
   const int tokens = min(max((a.tot ? *a.tot : a.tot_fixed) - tok0, 0), 512);
   const int n_boxes = (tokens + TG_BOX_TOK - 1) / TG_BOX_TOK;    // token rows are staged in multiples of 64
-  const int my_boxes = PAIR ? (n_boxes + 1) / 2 : n_boxes;       // token boxes staged by this CTA (a pair deals them alternately)
-  const bool pair_halves = PAIR && n_boxes > 2 && n_boxes <= 4;  // ... or, up to 256 tokens, takes one half each
-  const int stage_bytes = TG_A_BYTES + my_boxes * TG_BOX_BYTES;
+  const int stage_bytes = TG_A_BYTES + n_boxes * TG_BOX_BYTES;
   int n_stages = TG_SMEM_RING / stage_bytes;
   if (n_stages > TG_MAX_STAGES) n_stages = TG_MAX_STAGES;
   const int kb_total = (a.K + TG_BK - 1) / TG_BK;
   const int kb0 = (int)(((long long)kb_total * split) / splits);
   const int kb1 = (int)(((long long)kb_total * (split + 1)) / splits);
   const int n_kb = (tokens > 0) ? kb1 - kb0 : 0;
-  // columns of the first / second MMA.  In a pair each CTA supplies half of them: its first 128 staged rows to
-  // the first MMA, the rest to the second.
-  const int n0 = PAIR ? 2 * min(my_boxes * TG_BOX_TOK, 128) : min(((tokens + 15) / 16) * 16, 256);
-  const int n1 = PAIR ? 2 * max(my_boxes * TG_BOX_TOK - 128, 0) : (tokens > 256 ? ((tokens - 256 + 15) / 16) * 16 : 0);
+  // columns of the first / second MMA
+  const int n0 = min(((tokens + 15) / 16) * 16, 256);
+  const int n1 = tokens > 256 ? ((tokens - 256 + 15) / 16) * 16 : 0;
   // weight rows of this tile
   const int tiles_per_mat = (a.N + 127) / 128;
   const int mat = a.mode == TG_QKV ? tile / tiles_per_mat : 0;
@@ -249,7 +214,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
       tma_load_2d(sa, &a.tm_a[mat], k, row_base, &full_bar[s]);
     }
   };
-  const int n_early = PAIR ? 0 : min(n_kb, n_stages);           // k-blocks whose weights go out early
+  const int n_early = min(n_kb, n_stages);                      // k-blocks whose weights go out early
   if (producer)
     for (int i = pid; i < n_early; i += n_prod) {
       asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&full_bar[i])), "r"((unsigned)TG_A_BYTES) : "memory");
@@ -277,20 +242,6 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
         unsigned char* sa = ring + (size_t)s * stage_bytes;
         unsigned char* sb = sa + TG_A_BYTES;
         const int k = (kb0 + i) * TG_BK;
-        if (PAIR) {
-          // all bytes of both CTAs are counted on the barrier of rank 0, whose producer announces them
-          const unsigned bar0 = mapa_u32(smem_u32(&full_bar[s]), 0u);
-          if (crank == 0) mbar_expect_tx(&full_bar[s], 2u * (unsigned)stage_bytes);
-          tma_load_2d_pair(sa, &a.tm_a[mat], k, row_base, bar0);
-          if (pair_halves) {
-            // up to 256 tokens: one 128-row box per CTA (rank 0 the first 128 tokens, rank 1 the rest)
-            tma_load_2d_pair(sb, &a.tm_b[1], k, tok0 + (int)crank * 128, bar0);
-          } else {
-            for (int bl = 0; bl < my_boxes; ++bl)
-              tma_load_2d_pair(sb + (size_t)bl * TG_BOX_BYTES, &a.tm_b[0], k, tok0 + (2 * bl + (int)crank) * TG_BOX_TOK, bar0);
-          }
-          continue;
-        }
         if (i < n_early) {
           mbar_expect_tx(&full_bar[s], (unsigned)(stage_bytes - TG_A_BYTES));     // the weights of this k-block are on their way
         } else {
@@ -302,10 +253,10 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer (in a pair: rank 0 only)
-    if (lane == 0 && crank == 0) {
-      const unsigned idesc0 = umma_idesc_bf16(PAIR ? 256 : 128, n0);
-      const unsigned idesc1 = n1 ? umma_idesc_bf16(PAIR ? 256 : 128, n1) : 0u;
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const unsigned idesc0 = umma_idesc_bf16(128, n0);
+      const unsigned idesc1 = n1 ? umma_idesc_bf16(128, n1) : 0u;
       bool ok = true;
       for (int i = 0; i < n_kb && ok; ++i) {
         const int s = i % n_stages;
@@ -314,30 +265,17 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const unsigned char* sa = ring + (size_t)s * stage_bytes;
         const unsigned char* sb = sa + TG_A_BYTES;
-        const unsigned long long da = umma_desc(sa), db0 = umma_desc(sb), db1 = umma_desc(sb + (PAIR ? 128 : 256) * 128);
+        const unsigned long long da = umma_desc(sa), db0 = umma_desc(sb), db1 = umma_desc(sb + 256 * 128);
 #pragma unroll
         for (int k = 0; k < TG_BK / 16; ++k) {
           const unsigned acc = (i > 0 || k > 0) ? 1u : 0u;
           const unsigned long long koff = (unsigned long long)((k * 32) >> 4);        // 16 bf16 = 32 bytes along the swizzle row
-          if (PAIR) {
-            umma_bf16_pair(tmem_base, da + koff, db0 + koff, idesc0, acc);
-            if (n1) umma_bf16_pair(tmem_base + 256, da + koff, db1 + koff, idesc1, acc);
-          } else {
-            umma_bf16(tmem_base, da + koff, db0 + koff, idesc0, acc);
-            if (n1) umma_bf16(tmem_base + 256, da + koff, db1 + koff, idesc1, acc);
-          }
+          umma_bf16(tmem_base, da + koff, db0 + koff, idesc0, acc);
+          if (n1) umma_bf16(tmem_base + 256, da + koff, db1 + koff, idesc1, acc);
         }
-        if (PAIR) {                                              // the stage is free in both CTAs once these MMAs have read it
-          umma_commit_pair(smem_u32(&empty_bar[s]));
-          umma_commit_pair(mapa_u32(smem_u32(&empty_bar[s]), 1u));
-        } else {
-          umma_commit(&empty_bar[s]);                            // stage reusable once these MMAs have read it
-        }
+        umma_commit(&empty_bar[s]);                              // stage reusable once these MMAs have read it
       }
-      if (ok) {                                                  // accumulator complete
-        if (PAIR) { umma_commit_pair(smem_u32(&acc_bar)); umma_commit_pair(mapa_u32(smem_u32(&acc_bar), 1u)); }
-        else umma_commit(&acc_bar);
-      }
+      if (ok) umma_commit(&acc_bar);                             // accumulator complete
     }
   }
   __syncwarp();
@@ -409,16 +347,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
     int chunk = 0;
     for (int c0 = team * 16; c0 < tokens; c0 += 32, ++chunk) {
       float v[16], pv[16];
-      // accumulator column of the chunk's first token (a pair dealt the 64-token boxes alternately to its two CTAs)
-      int tcol = c0;
-      if (PAIR) {
-        if (pair_halves) tcol = (c0 >> 7) * (n0 / 2) + (c0 & 127);
-        else {
-          const int box = c0 / TG_BOX_TOK, hlf = box & 1, rr = (box >> 1) * TG_BOX_TOK + (c0 & (TG_BOX_TOK - 1));
-          tcol = rr < 128 ? hlf * (n0 / 2) + rr : 256 + hlf * (n1 / 2) + (rr - 128);
-        }
-      }
-      if (ok) tmem_ld16(tmem_base + ((unsigned)(32 * q) << 16) + (unsigned)tcol, v);
+      if (ok) tmem_ld16(tmem_base + ((unsigned)(32 * q) << 16) + (unsigned)c0, v);
       else {
 #pragma unroll
         for (int c = 0; c < 16; ++c) v[c] = 0.f;
@@ -522,11 +451,8 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (PAIR) cluster_sync_all();                                 // neither CTA frees tensor memory (or leaves) while its partner still works
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
-    else
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
   }
 }
@@ -549,6 +475,20 @@ __global__ void __launch_bounds__(256) swiglu_tail_kernel(const float* part, siz
     }
     h_out[(size_t)t * F + f] = __float2bfloat16(__fdividef(g, 1.f + __expf(-g)) * u);
   }
+}
+
+// Self-test of the bounded wait: one CTA waits on a barrier that nothing ever signals, gives up after
+// `limit_ns` and records the code like any kernel of the library would.
+__global__ void wait_expiry_kernel(int* dev_error, unsigned long long limit_ns) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) mbar_wait(&bar, 0, &abort_flag, dev_error, 0x7e570000, limit_ns);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -575,6 +515,12 @@ int encode_map(CUtensorMap* out, const void* base, int rows, int K, int box_rows
 
 }  // namespace
 
+int vlac_launch_wait_expiry(vlac_ctx* ctx, unsigned long long limit_ns, cudaStream_t s) {
+  wait_expiry_kernel<<<1, 32, 0, s>>>(ctx->dev_error, limit_ns);
+  VLAC_LAUNCH_CHECK(ctx);
+  return VLAC_OK;
+}
+
 int vlac_encode_map_2d(void* out, const void* base, int rows, int cols, int box_rows) {
   return encode_map((CUtensorMap*)out, base, rows, cols, box_rows);
 }
@@ -585,9 +531,8 @@ enum { TM_XN = 0, TM_AO = 4, TM_HM = 8, TM_ACT_COUNT = 12 };   // 4 box heights 
 
 int vlac_tc_setup(vlac_ctx* ctx) {
   const vlac_config& g = ctx->cfg;
-  ctx->tc_ok = 0;
-  // the TMA path needs 16-byte aligned rows and pointers
-  if (g.hidden % 8 || g.ffn % 8 || (g.head_dim != 64 && g.head_dim != 128)) return VLAC_OK;
+  // TMA needs 16-byte aligned rows and pointers; the rotary epilogue pairs lanes of a 64- or 128-wide head
+  if (g.hidden % 8 || g.ffn % 8 || (g.head_dim != 64 && g.head_dim != 128)) return VLAC_ERR_INVALID_ARG;
   const int n_maps = g.n_layers * TM_PER_LAYER + TM_ACT_COUNT + 1;      // + the vision projector
   CUtensorMap* host = (CUtensorMap*)malloc(sizeof(CUtensorMap) * n_maps);
   if (!host) return VLAC_ERR_OOM;
@@ -599,7 +544,7 @@ int vlac_tc_setup(vlac_ctx* ctx) {
     const int rows[TM_PER_LAYER] = {D, D, D, D, F, F, D};
     const int cols[TM_PER_LAYER] = {D, D, D, D, D, D, F};
     for (int m = 0; m < TM_PER_LAYER && rc == VLAC_OK; ++m) {
-      if (reinterpret_cast<uintptr_t>(ptr[m]) & 15) { free(host); return VLAC_OK; }   // unaligned weights: stay on the generic path
+      if (reinterpret_cast<uintptr_t>(ptr[m]) & 15) { free(host); return VLAC_ERR_INVALID_ARG; }
       rc = encode_map(&host[l * TM_PER_LAYER + m], ptr[m], rows[m], cols[m], (m == TM_GATE || m == TM_UP) ? 64 : 128);
     }
   }
@@ -610,58 +555,33 @@ int vlac_tc_setup(vlac_ctx* ctx) {
     if (rc == VLAC_OK) rc = encode_map(&act[TM_AO + hgt], ctx->ao, ctx->rows_max, D, box);
     if (rc == VLAC_OK) rc = encode_map(&act[TM_HM + hgt], ctx->hm, ctx->rows_max, F, box);
   }
-  ctx->tc_proj = 0;
-  if (rc == VLAC_OK && ctx->w.proj && (reinterpret_cast<uintptr_t>(ctx->w.proj) & 15) == 0) {
-    rc = encode_map(&act[TM_ACT_COUNT], ctx->w.proj, D, D, 128);
-    if (rc == VLAC_OK) ctx->tc_proj = 1;
+  if (rc == VLAC_OK) {
+    if (reinterpret_cast<uintptr_t>(ctx->w.proj) & 15) rc = VLAC_ERR_INVALID_ARG;
+    else rc = encode_map(&act[TM_ACT_COUNT], ctx->w.proj, D, D, 128);
   }
   if (rc != VLAC_OK) { free(host); return rc; }
   ctx->tmaps_host = host;                                        // copied into the kernel parameters at every launch
-  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, TG_SMEM_RING + 1024);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TG_SMEM_RING + 1024);
-  ctx->gemm_pair = getenv("VLAC_GEMM_PAIR") ? 1 : 0;
+  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TG_SMEM_RING + 1024);
   if (e != cudaSuccess) { vlac_note_cuda_error(e, __FILE__, __LINE__); return VLAC_ERR_CUDA; }
   // a CTA holds up to 512 tokens (accumulator columns); more tokens are further chunks along grid.z
-  ctx->tc_ok = 1;
   return VLAC_OK;
 }
 
 // Tensor-memory columns a CTA needs for the largest token chunk it can meet (power of two >= 32).
-static int tc_tmem_cols(const vlac_ctx* ctx, bool pair) {
+static int tc_tmem_cols(const vlac_ctx* ctx) {
   const int chunk = ctx->rows_max < 512 ? ctx->rows_max : 512;
-  int need;
-  if (pair) {
-    const int n_boxes = (chunk + TG_BOX_TOK - 1) / TG_BOX_TOK, rows = TG_BOX_TOK * ((n_boxes + 1) / 2);
-    const int n0 = 2 * (rows < 128 ? rows : 128), n1 = 2 * (rows > 128 ? rows - 128 : 0);
-    need = n1 ? 256 + n1 : n0;
-  } else {
-    const int n0 = ((chunk < 256 ? chunk : 256) + 15) / 16 * 16;
-    const int n1 = chunk > 256 ? (chunk - 256 + 15) / 16 * 16 : 0;
-    need = n1 ? 256 + n1 : n0;
-  }
+  const int n0 = ((chunk < 256 ? chunk : 256) + 15) / 16 * 16;
+  const int n1 = chunk > 256 ? (chunk - 256 + 15) / 16 * 16 : 0;
+  const int need = n1 ? 256 + n1 : n0;
   int cols = 32;
   while (cols < need) cols *= 2;
   return cols;
 }
 
-static int launch_tc(vlac_ctx* ctx, TcArgs& a, int n_tiles, cudaStream_t s, bool pair = false) {
+static int launch_tc(vlac_ctx* ctx, TcArgs& a, int n_tiles, cudaStream_t s) {
   const dim3 grid(n_tiles, a.n_splits, (ctx->rows_max + 511) / 512);
-  pair = pair && ctx->gemm_pair && (n_tiles % 2 == 0);
-  a.tmem_cols = tc_tmem_cols(ctx, pair);
-  if (pair) {
-    // clusters of two CTAs along x share the activation tile; still launched programmatically behind its predecessor
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = grid; cfg.blockDim = dim3(TG_THREADS); cfg.dynamicSmemBytes = (size_t)TG_SMEM_RING + 1024; cfg.stream = s;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = 2;
-    VLAC_CUDA_CHECK(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<true>, a));
-  } else {
-    VLAC_CUDA_CHECK(launch_pdl(gemm_tc_kernel<false>, grid, dim3(TG_THREADS), (size_t)TG_SMEM_RING + 1024, s, a));
-  }
+  a.tmem_cols = tc_tmem_cols(ctx);
+  VLAC_CUDA_CHECK(launch_pdl(gemm_tc_kernel, grid, dim3(TG_THREADS), (size_t)TG_SMEM_RING + 1024, s, a));
   VLAC_LAUNCH_CHECK(ctx);
   return VLAC_OK;
 }
@@ -689,7 +609,7 @@ int vlac_tc_qkv(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s) {
   a.q_out = ctx->q;
   a.kc = c->k + (size_t)layer * c->batch * kv_layer_elems(ctx);
   a.vc = c->v + (size_t)layer * c->batch * kv_layer_elems(ctx);
-  return launch_tc(ctx, a, 3 * ((g.hidden + 127) / 128), s, true);
+  return launch_tc(ctx, a, 3 * ((g.hidden + 127) / 128), s);
 }
 
 int vlac_tc_partial(vlac_ctx* ctx, vlac_cache* c, int layer, int which, int* n_splits, cudaStream_t s) {
@@ -710,7 +630,7 @@ int vlac_tc_partial(vlac_ctx* ctx, vlac_cache* c, int layer, int which, int* n_s
   a.n_splits = splits;
   a.part = ctx->part; a.split_stride = (size_t)ctx->rows_max * g.hidden;
   *n_splits = splits;
-  return launch_tc(ctx, a, tiles, s, true);
+  return launch_tc(ctx, a, tiles, s);
 }
 
 // Vision projector (input rows of the vision positions): features [rows][D] x W_proj^T as K-split fp32
@@ -718,7 +638,7 @@ int vlac_tc_partial(vlac_ctx* ctx, vlac_cache* c, int layer, int which, int* n_s
 // are made here, per launch (inside a graph capture: once).
 int vlac_tc_projector(vlac_ctx* ctx, vlac_cache* c, const void* feats, int rows, int* n_splits, cudaStream_t s) {
   const vlac_config& g = ctx->cfg;
-  if (!ctx->tc_ok || !ctx->tc_proj || (reinterpret_cast<uintptr_t>(feats) & 15) || rows > ctx->rows_max) return VLAC_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(feats) & 15) || rows > ctx->rows_max) return VLAC_ERR_INVALID_ARG;
   const CUtensorMap* act = (const CUtensorMap*)ctx->tmaps_host + (size_t)g.n_layers * TM_PER_LAYER;
   TcArgs a; tc_common(ctx, c, 0, &a);
   a.tot = nullptr; a.tot_fixed = rows;

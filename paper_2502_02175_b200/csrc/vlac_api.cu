@@ -49,7 +49,7 @@ int fill_params(const vlac_ctx* ctx, const vlac_select_params* in, int force_ful
 void free_ctx_buffers(vlac_ctx* c) {
   cudaFree(c->xn); cudaFree(c->q); cudaFree(c->ao); cudaFree(c->hm); cudaFree(c->part); cudaFree(c->scratch);
   cudaFree(c->probs); cudaFree(c->hidden); cudaFree(c->x_dec); cudaFree(c->q_dec); cudaFree(c->ao_dec);
-  cudaFree(c->hm_dec); cudaFree(c->logits); cudaFree(c->argmax_tmp); cudaFree(c->dev_error); cudaFree(c->tmaps); cudaFree(c->tmap_q); cudaFree(c->probs_all); free(c->tmaps_host);
+  cudaFree(c->hm_dec); cudaFree(c->logits); cudaFree(c->argmax_tmp); cudaFree(c->dev_error); cudaFree(c->tmap_q); cudaFree(c->probs_all); free(c->tmaps_host);
   cudaFree(c->in_frames); cudaFree(c->in_feats); cudaFree(c->in_ids); cudaFree(c->in_forced); cudaFree(c->out_tokens); cudaFree(c->logits_all);
   for (int i = 0; i < VLAC_MAX_GRAPHS; ++i) if (c->graphs[i].used) cudaGraphExecDestroy(c->graphs[i].exec);
   for (int i = 0; i < VLAC_SEG_CAP; ++i) if (c->seg_ev[i]) cudaEventDestroy(c->seg_ev[i]);
@@ -65,7 +65,7 @@ void free_cache_buffers(vlac_cache* c) {
   cudaFree(c->warm); cudaFree(c->sim); cudaFree(c->S_layer); cudaFree(c->S); cudaFree(c->alpha);
   cudaFree(c->alpha_raw); cudaFree(c->entropy); cudaFree(c->static_mask); cudaFree(c->task_mask);
   cudaFree(c->final_mask); cudaFree(c->rank); cudaFree(c->n_reuse); cudaFree(c->M); cudaFree(c->rows);
-  cudaFree(c->tot); cudaFree(c->rowmap); cudaFree(c->slot); cudaFree(c->tmaps_kv); cudaFree(c->dec_phases); cudaFree(c->dec_counter);
+  cudaFree(c->tot); cudaFree(c->rowmap); cudaFree(c->slot); cudaFree(c->tmaps_kv);
 }
 
 __global__ void set_warm_kernel(int* warm, int n, int value) {
@@ -95,7 +95,7 @@ int vlac_create(const vlac_config* cfg, const vlac_weights* w, vlac_ctx** out) {
   *out = nullptr;
   const vlac_config& g = *cfg;
   if (g.n_layers < 1 || g.n_layers > VLAC_MAX_LAYERS || g.hidden < 8 || g.hidden % 8 || g.hidden > 8192 ||
-      g.n_heads < 1 || g.n_kv_heads != g.n_heads || g.head_dim < 32 || g.head_dim % 32 || g.head_dim > 128 ||
+      g.n_heads < 1 || g.n_kv_heads != g.n_heads || (g.head_dim != 64 && g.head_dim != 128) ||
       g.n_heads * g.head_dim != g.hidden || g.ffn < 8 || g.ffn % 8 || g.vocab < 2 || g.n_cams < 1 || g.grid < 1 ||
       g.grid > 64 || g.patch < 1 || g.n_text_pre < 0 || g.n_text_post < 0 || g.n_action < 1 ||
       g.max_batch < 1 || g.max_batch > 8 || !(g.rms_eps > 0.f))
@@ -136,7 +136,6 @@ int vlac_create(const vlac_config* cfg, const vlac_weights* w, vlac_ctx** out) {
   if (rc == VLAC_OK) rc = dev_alloc(&c->hm, R * F);
   if (rc == VLAC_OK) rc = dev_alloc(&c->part, (size_t)VLAC_MAX_SPLITS * R * D);
   if (rc == VLAC_OK) rc = dev_alloc(&c->scratch, R * wide);
-  if (rc == VLAC_OK) rc = dev_alloc(&c->probs, B * (size_t)g.n_text_post * g.n_heads * c->Lv);
   if (rc == VLAC_OK) rc = dev_alloc(&c->hidden, R * D);
   if (rc == VLAC_OK) rc = dev_alloc(&c->x_dec, R1 * D);
   if (rc == VLAC_OK) rc = dev_alloc(&c->q_dec, R1 * D);
@@ -162,6 +161,7 @@ int vlac_create(const vlac_config* cfg, const vlac_weights* w, vlac_ctx** out) {
 
 int vlac_destroy(vlac_ctx* ctx) {
   if (!ctx) return VLAC_ERR_INVALID_ARG;
+  if (ctx->live_caches > 0) return VLAC_ERR_BAD_STATE;          // a cache still points at this context
   cudaDeviceSynchronize();
   free_ctx_buffers(ctx);
   delete ctx;
@@ -202,8 +202,8 @@ int vlac_cache_alloc(vlac_ctx* ctx, int batch, vlac_cache** out) {
   if (rc == VLAC_OK) rc = dev_alloc(&c->rowmap, nl * B * L);
   if (rc == VLAC_OK) rc = dev_alloc(&c->slot, nl * B * L);
   if (rc == VLAC_OK) rc = vlac_attention_cache_setup(ctx, c);
-  if (rc == VLAC_OK) rc = vlac_decode_cache_setup(ctx, c);
   if (rc != VLAC_OK) { free_cache_buffers(c); delete c; return rc; }
+  ctx->live_caches++;
   *out = c;
   return VLAC_OK;
 }
@@ -224,6 +224,7 @@ int vlac_cache_free(vlac_cache* cache) {
     StepGraph& e = cache->ctx->graphs[i];
     if (e.used && e.cache == cache) { cudaGraphExecDestroy(e.exec); e.used = 0; }
   }
+  cache->ctx->live_caches--;
   free_cache_buffers(cache);
   delete cache;
   return VLAC_OK;
@@ -359,7 +360,7 @@ static int enqueue_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* f
   TRY(seg_mark(ctx, s));
   // 3. layers; the down-projection partials of layer l are folded into layer l+1's first kernel
   int n_splits = 0;
-  ctx->defer_emit = ctx->attn_tiles > 0 && ctx->probs_all != nullptr;
+  ctx->defer_emit = ctx->probs_all != nullptr;
   for (int l = 0; l < nl; ++l) {
     int rc = vlac_launch_finalize_norm(ctx, cache, h, l == 0 ? 0 : l - 1, l == 0 ? 0 : n_splits, l, ctx->layers[l].g_attn, s);
     if (rc == VLAC_OK) rc = vlac_launch_layer_body(ctx, cache, l, h, &n_splits, s);
@@ -528,6 +529,12 @@ int vlac_device_error(vlac_ctx* ctx, void* stream) {
   VLAC_CUDA_CHECK(cudaMemcpyAsync(&v, ctx->dev_error, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
   VLAC_CUDA_CHECK(cudaStreamSynchronize((cudaStream_t)stream));
   return v ? VLAC_ERR_TIMEOUT : VLAC_OK;
+}
+
+int vlac_selftest_wait_expiry(vlac_ctx* ctx, unsigned int limit_us, void* stream) {
+  if (!ctx || limit_us == 0 || limit_us > 100000) return VLAC_ERR_INVALID_ARG;
+  TRY(vlac_launch_wait_expiry(ctx, (unsigned long long)limit_us * 1000ull, (cudaStream_t)stream));
+  return vlac_device_error(ctx, stream);
 }
 
 }  // extern "C"

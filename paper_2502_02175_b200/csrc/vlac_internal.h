@@ -46,12 +46,13 @@ struct vlac_ctx {
   vlac_weights w;
   vlac_layer_w layers[VLAC_MAX_LAYERS];
   int L, Lv, max_seq, frame_hw, rows_max, n_sm;
+  int live_caches;                   // caches allocated from this context and not yet freed
   unsigned long long launches;
   // workspace (device)
   bf16 *xn, *q, *ao, *hm;            // [rows_max][hidden] x3, [rows_max][ffn]
   float *part;                       // [VLAC_MAX_SPLITS][rows_max][hidden]
-  float *scratch;                    // [rows_max][max(3*hidden, 2*ffn)]   (generic GEMM output)
-  float *probs;                      // [max_batch][n_text_post][n_heads][Lv]
+  float *scratch;                    // [rows_max][max(3*hidden, 2*ffn)]   raw gate/up sums of the K-split tail tiles
+  float *probs;                      // [max_batch][tiles][n_heads][Lv]: per-tile column sums of one layer (vlac_layer_forward)
   bf16 *hidden;                      // [max_batch][L][hidden]            (used by step)
   // single-row buffers: one row per column of the matrix-vector kernels, R1 = max(max_batch, min(n_action, 8))
   float *x_dec;                      // [R1][hidden]
@@ -63,16 +64,10 @@ struct vlac_ctx {
   unsigned char* in_frames; bf16* in_feats; int *in_ids, *in_forced, *out_tokens; float* logits_all;
   StepGraph graphs[VLAC_MAX_GRAPHS];
   int graph_next, use_graph;
-  void* tmaps;                       // (unused) device copy of the tensor maps
   void* tmaps_host;                  // host array of TMA tensor maps (weights per layer, activation buffers)
-  int tc_ok;                         // 1: shapes fit the tensor-memory GEMM
-  int gemm_pair;                     // prefill GEMMs with an even tile count run as two-CTA clusters (cta_group::2)
-  int tc_proj;                       // the vision projector has a tensor map (tcgen05 path usable for the input rows)
-  int pass_grid;                     // CTAs of the persistent single-row pass kernel (0: not used)
-  int gemv_stream;                   // single-row products use the shared-memory-staged kernel
   int chunk_ok;                      // the n_action rows of a chunk fit the matrix-vector kernels as columns (vlac_step_chunk usable)
   void* tmap_q;                      // device tensor map of the query buffer (tiled attention)
-  int attn_tiles;                    // 64-query tiles per sequence, 0: tiled attention not usable
+  int attn_tiles;                    // 64-query tiles per sequence
   float* probs_all;                  // [n_layers][max_batch][tiles][n_heads][Lv]: per-tile column sums of every layer of a step
   int defer_emit;                    // set while a whole step is enqueued: text-to-vision scores of all layers are formed by one kernel at its end
   // optional per-launch timing of the matrix-vector kernel (vlac_profile)
@@ -103,8 +98,6 @@ struct vlac_cache {
   int *rowmap;                       // [nl][batch*L]        compact index -> b*L + pos
   int *slot;                         // [nl][batch*L]        b*L + pos -> compact index or -1
   void* tmaps_kv;                    // device tensor maps of the K and V cache of every layer
-  void* dec_phases;                  // device table of per-layer phase arguments (persistent pass kernel)
-  void* dec_counter;                 // its grid barrier counter
 };
 
 static inline size_t kv_layer_elems(const vlac_ctx* c) {
@@ -126,10 +119,9 @@ int vlac_launch_finalize_norm(vlac_ctx* ctx, vlac_cache* c, bf16* hidden, int l_
 // partials (left in ctx->part); returns the number of partials in *n_splits.
 int vlac_launch_layer_body(vlac_ctx* ctx, vlac_cache* c, int layer, bf16* hidden, int* n_splits, cudaStream_t s);
 
-int vlac_launch_decode_attention(vlac_ctx* ctx, vlac_cache* c, int layer, int pos, cudaStream_t s);
-
 // ---- tensor-memory GEMM (gemm_tc.cu)
 int vlac_tc_setup(vlac_ctx* ctx);
+int vlac_launch_wait_expiry(vlac_ctx* ctx, unsigned long long limit_ns, cudaStream_t s);
 int vlac_tc_qkv(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s);
 int vlac_tc_partial(vlac_ctx* ctx, vlac_cache* c, int layer, int which /* 0: output proj, 1: down proj */, int* n_splits, cudaStream_t s);
 int vlac_tc_gateup(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s);
@@ -144,7 +136,6 @@ int vlac_launch_emit_all(vlac_ctx* ctx, vlac_cache* c, cudaStream_t s);   // aft
 
 // ---- decode (decode_kernels.cu)
 int vlac_decode_setup(vlac_ctx* ctx);
-int vlac_decode_cache_setup(vlac_ctx* ctx, vlac_cache* c);
 int vlac_launch_last_row(vlac_ctx* ctx, vlac_cache* c, const bf16* hidden, cudaStream_t s);
 int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens, int tok_stride, int tok_index,
                             int pos, cudaStream_t s);

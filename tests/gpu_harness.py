@@ -99,14 +99,33 @@ def check_selection(got: dict, sel: orc.Selection, seq: int, cfg, where=""):
         assert np.array_equal(got["rows"][seq, l, :m], sel.rows[l]), f"{where}: rows of layer {l}"
 
 
+def host_model_from_device(dev, cfg) -> dict:
+    """Bit copy of a ``DeviceModel``'s tensors into the dictionary layout of ``synth.make_model``."""
+    by_ptr = {t.data_ptr(): t for t in dev.tensors}
+
+    def bits(ptr):
+        t = by_ptr[ptr]
+        if t.dtype == torch.bfloat16:
+            return t.view(torch.int16).cpu().numpy().view(np.uint16)
+        return t.cpu().numpy()
+
+    model = {"layers": [{name: bits(getattr(dev.layer_structs[l], name)) for name, _ in vb.vlac_layer_w._fields_}
+                        for l in range(cfg.n_layers)]}
+    for name in ("embed", "proj", "g_final", "lm_head", "rope_cos", "rope_sin"):
+        model[name] = bits(getattr(dev.weights, name))
+    return model
+
+
 def run_step_pair(sess: Session, frames: np.ndarray, feats: np.ndarray, ids: np.ndarray, params: orc.SelectParams,
-                  force_full=False, act_embed: np.ndarray = None):
+                  force_full=False, act_embed: np.ndarray = None, layer_major=False):
     """One control step on both sides with replay: the checker's selection is computed from the
     library's own saved attention (bit-copied) and the checker is fed the library's tokens.
 
     frames [B, n_cams, H, W, 3] uint8; feats [B, L_v, hidden] bf16 bits; ids [B, n_text] int32.
     With ``act_embed`` ([n_action, hidden] bf16 bits) both sides decode the action chunk in one parallel
     pass instead (vlac_step_chunk / step_chunk); the K/V rows of the chunk are compared as well.
+    ``layer_major`` takes the checker's step through ``oracle_compose.step_layer_major`` (same bits, each
+    layer's weights widened once per step: for the 32-layer model).
     Returns a dict of per-sequence comparison figures.
     """
     cfg, B = sess.cfg, sess.batch
@@ -140,7 +159,11 @@ def run_step_pair(sess: Session, frames: np.ndarray, feats: np.ndarray, ids: np.
             check_selection(got_sel, sel, b, cfg, where=f"seq {b}")
         else:
             assert np.all(got_sel["M"][b] == cfg.seq_len)
-        if act_embed is None:
+        if act_embed is None and layer_major:
+            import oracle_compose
+            res = oracle_compose.step_layer_major(cfg, sess.model, oc, frames[b], feats[b], ids[b], params,
+                                                  forced_tokens=g_tokens[b], force_full=force_full, selection=sel)
+        elif act_embed is None:
             res = orc.step(cfg, sess.model, oc, frames[b], feats[b], ids[b], params, force_full,
                            forced_tokens=g_tokens[b], selection=sel)
         else:
@@ -156,12 +179,15 @@ def run_step_pair(sess: Session, frames: np.ndarray, feats: np.ndarray, ids: np.
                 guarded += 1
         g_attn = sess.read_attn(vb.PART_ATTN_PREV, b)
         attn_err = rel_err(g_attn, res.attn_tv)
+        attn_err_layers = [rel_err(g_attn[l], res.attn_tv[l]) for l in range(cfg.n_layers)]
         kv_err = 0.0
         if act_embed is not None:
             L, n = cfg.seq_len, cfg.n_action
             for l in range(cfg.n_layers):
                 kv_err = max(kv_err, rel_err(sess.read_kv(vb.PART_K, l, b)[L:L + n], oc.K[l][L:L + n]),
                              rel_err(sess.read_kv(vb.PART_V, l, b)[L:L + n], oc.V[l][L:L + n]))
-        out.append({"logit_err": err, "abs_err": abs_err, "guarded": guarded, "attn_err": attn_err, "kv_err": kv_err,
+        out.append({"logit_err": err, "abs_err": abs_err, "guarded": guarded, "attn_err": attn_err, "attn_err_layers": attn_err_layers, "kv_err": kv_err,
+                    "logit_err_rows": [rel_err(g_logits[b, i], res.logits[i]) for i in range(cfg.n_action)],
+                    "margins": res.margins.copy(), "ref_tokens": res.tokens.copy(),
                     "M": sel.M.copy(), "tokens": g_tokens[b].copy(), "selection": sel})
     return out

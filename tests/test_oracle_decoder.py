@@ -25,7 +25,35 @@ def _tiny(seed=0, n_layers=2):
 
 
 def _t(bits):
-    return torch.from_numpy(orc.widen_bf16(bits))
+    """bf16 bit patterns -> fp64 torch tensor through torch's own bfloat16 type (not the checker's widening)."""
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).double()
+
+
+def test_widen_bf16_matches_torch_bfloat16():
+    """The checker's bit widening against torch.bfloat16 on every class of pattern: normals of both signs,
+    subnormals, zeros, infinities, and (as a set) NaNs."""
+    rng = np.random.default_rng(0)
+    bits = rng.integers(0, 1 << 16, size=20000, dtype=np.uint16)
+    special = np.array([0x0000, 0x8000, 0x0001, 0x8001, 0x007F, 0x0080, 0x7F7F, 0xFF7F, 0x7F80, 0xFF80, 0x3F80, 0xBF80,
+                        0x7FC0, 0xFFC1], dtype=np.uint16)
+    bits = np.concatenate([bits, special])
+    with np.errstate(invalid="ignore"):          # widening a signalling NaN raises the flag
+        got = orc.widen_bf16(bits)
+    want = torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).double().numpy()
+    nan = np.isnan(want)
+    assert np.array_equal(np.isnan(got), nan)
+    assert np.array_equal(got[~nan], want[~nan])
+    assert np.array_equal(np.signbit(got[~nan]), np.signbit(want[~nan]))
+    assert got[len(bits) - len(special) + 2] == 2.0 ** -133 and np.isposinf(got[len(bits) - len(special) + 8])
+    # the memoised form is the same conversion
+    orc.WIDEN_CACHE_MAX = 2
+    try:
+        with np.errstate(invalid="ignore"):
+            assert np.array_equal(orc._widen_cached(bits)[~nan], want[~nan])
+            assert np.array_equal(orc._widen_cached(bits)[~nan], want[~nan])
+    finally:
+        orc.WIDEN_CACHE_MAX = 0
+        orc._widen_cache.clear()
 
 
 def _torch_rope(x, cos, sin):
@@ -298,3 +326,20 @@ def test_forced_tokens_are_fed_back():
     np.testing.assert_array_equal(r.logits[0], free.logits[0])
     assert r.tokens[0] == free.tokens[0] and np.abs(r.logits[1] - free.logits[1]).max() > 1e-9
     assert np.all(r.margins >= 0)
+
+
+def test_layer_major_composition_equals_step():
+    """tests/oracle_compose.step_layer_major (each layer once: prefill rows, then the single rows) gives the
+    bits of oracle.step when it is fed the same tokens, cold and cached."""
+    import oracle_compose
+    cfg, model, ids, feats = _tiny(4)
+    prev, cur, _ = synth.rerandomised_pair(cfg, 4, 13)
+    params = orc.SelectParams(top_k=32, alpha_override=[0.5, 1.0])
+    ca, cb = orc.new_cache(cfg), orc.new_cache(cfg)
+    for fr in (prev, cur):
+        ra = orc.step(cfg, model, ca, fr, feats, ids, params)
+        rb = oracle_compose.step_layer_major(cfg, model, cb, fr, feats, ids, params, forced_tokens=ra.tokens)
+        assert np.array_equal(ra.logits, rb.logits) and np.array_equal(ra.tokens, rb.tokens)
+        assert np.array_equal(ra.attn_tv, rb.attn_tv) and np.array_equal(ra.hidden, rb.hidden)
+        assert np.array_equal(ca.K, cb.K) and np.array_equal(ca.V, cb.V)
+    assert ra.selection.M[1] < cfg.seq_len
