@@ -238,7 +238,8 @@ int vlac_selftest_wait_expiry(vlac_ctx* ctx, unsigned int limit_us, void* stream
 
 /* Greedy token choice that allocates nothing (the paper has no counterpart; it is the last step of
  * vlac_step offered on its own).  For each of `rows` logits rows it returns the index of the largest
- * value, equal values going to the lower index, exactly as vlac_step picks action tokens.
+ * value, equal values (-0 and +0 are equal) going to the lower index, exactly as vlac_step picks
+ * action tokens.
  *
  * It exists for callers that may not allocate device memory at the time of the call: a control loop
  * that reserved its whole memory budget at start-up and must not hit cudaMalloc (or the device-wide
@@ -250,7 +251,9 @@ int vlac_selftest_wait_expiry(vlac_ctx* ctx, unsigned int limit_us, void* stream
  *   rows        1..64; more returns VLAC_ERR_TOO_LARGE and does nothing
  *   tokens      device int32 [rows]
  * The first call on each device looks up the array's device address (one runtime query); make that
- * first call outside any stream capture.  All calls share the array and it keeps the previous call's
+ * first call outside any stream capture.  The address is remembered per device ordinal and belongs to
+ * the device's primary context: after cudaDeviceReset, or from a context the caller made through the
+ * driver API, it is not valid.  All calls share the array and it keeps the previous call's
  * contents; every slot is rewritten before it is read, so nothing needs clearing, but two calls whose
  * kernels overlap on the GPU (different streams, no ordering) race on it: order them. */
 int vlac_greedy_tokens_static(const float* logits, int rows, int vocab, long long row_stride,

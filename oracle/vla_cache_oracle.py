@@ -11,8 +11,16 @@ Conventions
 -----------
 * Everything is float64 except pixel sums, which are exact integers.
 * Model weights arrive as bf16 bit patterns (uint16) and are widened, never rounded.
-* The K/V cache, hidden states and attention scores are kept in float64: no rounding
-  point of any GPU kernel is imitated here.
+* By default (``operands="exact"``) the K/V cache, hidden states and attention scores are
+  kept in float64 and nothing is rounded.
+* The paper runs its models in BF16 (Sec. 5, implementation details; Appendix
+  "Experimental Settings").  ``operands="bf16"`` is that precision for the contractions:
+  every operand of a matrix product (normalised rows, queries, keys, values, attention
+  probabilities, attention output, MLP activations, the row entering the lm_head) is
+  rounded to the nearest bf16 value before the product, and keys and values are stored in
+  the cache as bf16; sums, the residual stream and everything else stay float64.  The
+  distance between the two settings is what bf16 operands cost on a given network; it
+  grows with depth (tests/test_oracle_decoder.py measures it).
 * Matrix products use ``numpy.matmul``; there is no blocking, fusion or reordering
   beyond what the cited passage states.
 
@@ -40,6 +48,26 @@ def widen_bf16(bits: np.ndarray) -> np.ndarray:
     """bf16 bit patterns (uint16) -> float64, exactly."""
     b = np.ascontiguousarray(bits, dtype=np.uint16)
     return (b.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+
+
+def round_bf16(x: np.ndarray) -> np.ndarray:
+    """float64 -> nearest bf16 value (ties to even), returned as float64.  NaN and inf pass through."""
+    f = np.ascontiguousarray(x, dtype=np.float32)
+    u = f.view(np.uint32)
+    r = (u + (np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1)))) & np.uint32(0xFFFF0000)
+    out = r.view(np.float32).astype(np.float64)
+    bad = ~np.isfinite(f)
+    if bad.any():
+        out[bad] = f[bad]
+    return out
+
+
+def _operand(x: np.ndarray, operands: str) -> np.ndarray:
+    if operands == "exact":
+        return x
+    if operands == "bf16":
+        return round_bf16(x)
+    raise ValueError(f"operands must be 'exact' or 'bf16', not {operands!r}")
 
 
 # Optional memo of widened matrices (format conversion only, no arithmetic).  Off by default; tests that
@@ -337,7 +365,8 @@ def silu(x: np.ndarray) -> np.ndarray:
 
 def layer_forward(cfg, layer_w: Dict[str, np.ndarray], K: np.ndarray, V: np.ndarray,
                   hidden: np.ndarray, rows: np.ndarray, cos: np.ndarray, sin: np.ndarray,
-                  emit_attention: bool = True, block_start: Optional[int] = None) -> Optional[np.ndarray]:
+                  emit_attention: bool = True, block_start: Optional[int] = None,
+                  operands: str = "exact") -> Optional[np.ndarray]:
     """One decoder layer over the positions in ``rows`` only (Algorithm 2, Sec. 4.1).
 
     ``K``/``V`` are this layer's cache ``[max_seq, heads, d]`` and are updated in place at
@@ -349,6 +378,9 @@ def layer_forward(cfg, layer_w: Dict[str, np.ndarray], K: np.ndarray, V: np.ndar
     at positions ``>= block_start`` form one block that is decoded in parallel: each of them
     also sees the block's later positions (see ``step_chunk``).
 
+    ``operands="bf16"`` rounds every operand of a matrix product to bf16 first and stores keys and values
+    as bf16 (the paper's BF16 setting; see the module header); the emitted probabilities are not rounded.
+
     Returns, if asked, ``[heads, L_v]``: the softmax probability on each vision key averaged
     over the prompt-text query rows that follow the vision block (Eq. avistext, read as
     text queries x vision keys).
@@ -357,14 +389,14 @@ def layer_forward(cfg, layer_w: Dict[str, np.ndarray], K: np.ndarray, V: np.ndar
     rows = np.asarray(rows, dtype=np.int64)
     W = {k: _widen_cached(v) for k, v in layer_w.items()}
     x = hidden[rows]
-    xn = rms_norm(x, W["g_attn"], cfg.rms_eps)
+    xn = _operand(rms_norm(x, W["g_attn"], cfg.rms_eps), operands)
     q = (xn @ W["wq"].T).reshape(len(rows), H, d)
     k = (xn @ W["wk"].T).reshape(len(rows), H, d)
     v = (xn @ W["wv"].T).reshape(len(rows), H, d)
-    q = rope(q, rows, cos, sin)
+    q = _operand(rope(q, rows, cos, sin), operands)
     k = rope(k, rows, cos, sin)
-    K[rows] = k
-    V[rows] = v
+    K[rows] = _operand(k, operands)
+    V[rows] = _operand(v, operands)
 
     n_keys = int(rows.max()) + 1
     key_pos = np.arange(n_keys)
@@ -382,12 +414,12 @@ def layer_forward(cfg, layer_w: Dict[str, np.ndarray], K: np.ndarray, V: np.ndar
         scores = scores - scores.max(axis=1, keepdims=True)
         p = np.exp(scores)
         p = p / p.sum(axis=1, keepdims=True)
-        attn_out[:, h, :] = p @ V[:n_keys, h, :]
+        attn_out[:, h, :] = _operand(p, operands) @ V[:n_keys, h, :]
         if emit_attention and text_q.any():
             emitted[h] = p[text_q][:, v0:v1].mean(axis=0)
-    x = x + attn_out.reshape(len(rows), H * d) @ W["wo"].T
-    xn = rms_norm(x, W["g_mlp"], cfg.rms_eps)
-    x = x + (silu(xn @ W["w_gate"].T) * (xn @ W["w_up"].T)) @ W["w_down"].T
+    x = x + _operand(attn_out.reshape(len(rows), H * d), operands) @ W["wo"].T
+    xn = _operand(rms_norm(x, W["g_mlp"], cfg.rms_eps), operands)
+    x = x + _operand(silu(xn @ W["w_gate"].T) * (xn @ W["w_up"].T), operands) @ W["w_down"].T
     hidden[rows] = x
     return emitted if emit_attention else None
 
@@ -419,15 +451,15 @@ def input_rows(cfg, model: Dict[str, object], feats_bf16: np.ndarray, prompt_ids
     return hidden
 
 
-def _logits(cfg, model, h_row: np.ndarray) -> np.ndarray:
-    xn = rms_norm(h_row[None, :], widen_bf16(model["g_final"]), cfg.rms_eps)
+def _logits(cfg, model, h_row: np.ndarray, operands: str = "exact") -> np.ndarray:
+    xn = _operand(rms_norm(h_row[None, :], widen_bf16(model["g_final"]), cfg.rms_eps), operands)
     return (xn @ _widen_cached(model["lm_head"]).T)[0]
 
 
 def step(cfg, model: Dict[str, object], cache: CacheState, frames_t: np.ndarray,
          feats_bf16: np.ndarray, prompt_ids: np.ndarray, params: SelectParams,
          force_full: bool = False, forced_tokens: Optional[Sequence[int]] = None,
-         selection: Optional[Selection] = None) -> StepResult:
+         selection: Optional[Selection] = None, operands: str = "exact") -> StepResult:
     """Selection, partial prefill, then greedy decoding of ``n_action`` tokens.
 
     The first action token is the argmax (ties to the lower id) of the logits at the last
@@ -444,7 +476,7 @@ def step(cfg, model: Dict[str, object], cache: CacheState, frames_t: np.ndarray,
     attn_next = np.zeros((cfg.n_layers, cfg.n_heads, cfg.n_vision), dtype=np.float64)
     for l in range(cfg.n_layers):
         attn_next[l] = layer_forward(cfg, model["layers"][l], cache.K[l], cache.V[l], hidden,
-                                     sel.rows[l], cos, sin, emit_attention=True)
+                                     sel.rows[l], cos, sin, emit_attention=True, operands=operands)
     L = cfg.seq_len
     tokens = np.zeros(cfg.n_action, dtype=np.int64)
     fed = np.zeros(cfg.n_action, dtype=np.int64)
@@ -456,8 +488,8 @@ def step(cfg, model: Dict[str, object], cache: CacheState, frames_t: np.ndarray,
             hidden[pos] = widen_bf16(model["embed"][int(fed[i - 1])])
             for l in range(cfg.n_layers):
                 layer_forward(cfg, model["layers"][l], cache.K[l], cache.V[l], hidden,
-                              np.asarray([pos]), cos, sin, emit_attention=False)
-        logits[i] = _logits(cfg, model, hidden[pos])
+                              np.asarray([pos]), cos, sin, emit_attention=False, operands=operands)
+        logits[i] = _logits(cfg, model, hidden[pos], operands)
         tokens[i] = int(np.argmax(logits[i]))
         top2 = np.partition(logits[i], -2)[-2:]
         margins[i] = float(top2[1] - top2[0])
@@ -472,7 +504,7 @@ def step(cfg, model: Dict[str, object], cache: CacheState, frames_t: np.ndarray,
 def step_chunk(cfg, model: Dict[str, object], cache: CacheState, frames_t: np.ndarray,
                feats_bf16: np.ndarray, prompt_ids: np.ndarray, params: SelectParams,
                act_embed_bf16: np.ndarray, force_full: bool = False,
-               selection: Optional[Selection] = None) -> StepResult:
+               selection: Optional[Selection] = None, operands: str = "exact") -> StepResult:
     """Selection and partial prefill as in ``step``, then ALL action tokens from one pass.
 
     The paper applies the method unchanged to OpenVLA-OFT, whose decoder emits its action
@@ -492,18 +524,18 @@ def step_chunk(cfg, model: Dict[str, object], cache: CacheState, frames_t: np.nd
     attn_next = np.zeros((cfg.n_layers, cfg.n_heads, cfg.n_vision), dtype=np.float64)
     for l in range(cfg.n_layers):
         attn_next[l] = layer_forward(cfg, model["layers"][l], cache.K[l], cache.V[l], hidden,
-                                     sel.rows[l], cos, sin, emit_attention=True)
+                                     sel.rows[l], cos, sin, emit_attention=True, operands=operands)
     L, n = cfg.seq_len, cfg.n_action
     chunk_rows = np.arange(L, L + n, dtype=np.int64)
     hidden[chunk_rows] = widen_bf16(np.asarray(act_embed_bf16).reshape(n, cfg.hidden))
     for l in range(cfg.n_layers):
         layer_forward(cfg, model["layers"][l], cache.K[l], cache.V[l], hidden, chunk_rows, cos, sin,
-                      emit_attention=False, block_start=L)
+                      emit_attention=False, block_start=L, operands=operands)
     tokens = np.zeros(n, dtype=np.int64)
     logits = np.zeros((n, cfg.vocab), dtype=np.float64)
     margins = np.zeros(n, dtype=np.float64)
     for i in range(n):
-        logits[i] = _logits(cfg, model, hidden[L + i])
+        logits[i] = _logits(cfg, model, hidden[L + i], operands)
         tokens[i] = int(np.argmax(logits[i]))
         top2 = np.partition(logits[i], -2)[-2:]
         margins[i] = float(top2[1] - top2[0])

@@ -150,6 +150,25 @@ class DeviceModel:
             self.tensors.append(t)
             setattr(self.weights, name, t.data_ptr())
 
+    def to_host(self, cfg) -> Dict[str, object]:
+        """Bit copy of every tensor into the dictionary layout of ``synth.make_model`` (bf16 as uint16 patterns;
+        the rotary tables cut to the ``cfg.max_seq`` rows that layout has)."""
+        by_ptr = {t.data_ptr(): t for t in self.tensors}
+
+        def bits(ptr):
+            t = by_ptr[ptr]
+            if t.dtype == torch.bfloat16:
+                return t.view(torch.int16).cpu().numpy().view(np.uint16)
+            return t.cpu().numpy()
+
+        model = {"layers": [{name: bits(getattr(self.layer_structs[l], name)) for name, _ in vlac_layer_w._fields_}
+                            for l in range(cfg.n_layers)]}
+        for name in ("embed", "proj", "g_final", "lm_head"):
+            model[name] = bits(getattr(self.weights, name))
+        for name in ("rope_cos", "rope_sin"):
+            model[name] = bits(getattr(self.weights, name))[:cfg.max_seq]
+        return model
+
     @classmethod
     def random(cls, cfg, seed: int, device="cuda") -> "DeviceModel":
         """Random-init weights generated on the device (same distributions as ``synth.make_model``;

@@ -719,15 +719,15 @@ __global__ void __launch_bounds__(256) embed_chunk_kernel(const bf16* act_embed,
   for (int k = threadIdx.x; k < D; k += blockDim.x) x[(size_t)c * D + k] = bf2f(act_embed[(size_t)(c % n) * D + k]);
 }
 
-__global__ void __launch_bounds__(256) last_row_kernel(const bf16* hidden, float* x, int L, int D) {
+__global__ void __launch_bounds__(256) last_row_kernel(const float* hidden, float* x, int L, int D) {
   const int b = blockIdx.x;
-  const bf16* src = hidden + ((size_t)b * L + (L - 1)) * D;
-  for (int k = threadIdx.x; k < D; k += blockDim.x) x[(size_t)b * D + k] = bf2f(src[k]);
+  const float* src = hidden + ((size_t)b * L + (L - 1)) * D;
+  for (int k = threadIdx.x; k < D; k += blockDim.x) x[(size_t)b * D + k] = src[k];
 }
 
-// greedy choice; equal logits -> lower id
+// greedy choice; equal logits -> lower id (-0 counts as +0)
 __device__ __forceinline__ unsigned long long argmax_key(float v, int idx) {
-  unsigned int u = __float_as_uint(v);
+  unsigned int u = __float_as_uint(v + 0.0f);
   u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);          // monotone map of float order onto unsigned order
   return ((unsigned long long)u << 32) | (unsigned long long)(0xFFFFFFFFu - (unsigned int)idx);
 }
@@ -840,7 +840,7 @@ int vlac_decode_setup(vlac_ctx* ctx) {
   return VLAC_OK;
 }
 
-int vlac_launch_last_row(vlac_ctx* ctx, vlac_cache* c, const bf16* hidden, cudaStream_t s) {
+int vlac_launch_last_row(vlac_ctx* ctx, vlac_cache* c, const float* hidden, cudaStream_t s) {
   last_row_kernel<<<c->batch, 256, 0, s>>>(hidden, ctx->x_dec, ctx->L, ctx->cfg.hidden);
   VLAC_LAUNCH_CHECK(ctx);
   return VLAC_OK;

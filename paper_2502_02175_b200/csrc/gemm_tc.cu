@@ -4,22 +4,32 @@
 //
 // The prefill multiplies every weight matrix with a few hundred rows (T = rows the selection kept), so
 // the weights are the big operand and each must cross HBM exactly once.  The operands are therefore
-// swapped: a CTA owns 128 rows of W as the M side of a 128 x T x 16 UMMA and ALL T tokens as the N
-// side; the fp32 accumulator [128 lanes][T columns] lives in tensor memory.  T is read from device
-// memory (the selection kernels wrote it); the instruction descriptor and the number of token boxes
-// are formed in the kernel, so no host round trip is needed.
+// swapped: a tile is 128 rows of W as the M side of a 128 x T x 16 UMMA and up to 256 tokens as the N
+// side; the fp32 accumulator [128 lanes][tokens] lives in tensor memory.  T is read from device memory
+// (the selection kernels wrote it), so no host round trip is needed.
 //
-// Warp roles (256 threads): one lane each of warps 0, 6 and 7 issues TMA loads into a ring of stages (the
-// k-blocks dealt round-robin: a thread gets a tensor load accepted only every ~0.3 us whatever its size,
-// but threads of different warps are served in parallel), warp 1 allocates TMEM and issues the MMAs.  When
-// the accumulator is complete all eight warps read it back (two teams of four, one warp per quarter of
-// the 128 lanes, alternating 16-token chunks) and run the epilogue.  Few, large TMA boxes are used (one
-// 128-row box of weights, one box of up to 256 token rows per k-block).
-// Epilogues:
-//   QKV     rotation at the row's own position, K/V scatter into the cache, Q to the compact buffer;
-//           the two halves of a rotary pair sit in different warps and are exchanged through shared memory
+// Persistent CTAs, one per SM.  Work is counted in k-blocks (128 weight rows x 64 k): the Q/K/V and the
+// gate/up products give every CTA the same share of ALL k-blocks of the launch (a contiguous range that
+// may begin and end inside a tile), the output / down projections and the vision projector give every
+// CTA one K-split of one tile.  A CTA walks its range segment by segment (tile, k-blocks kb0..kb1) and,
+// with more than 256 tokens, chunk by chunk of tokens.
+//
+// Warp roles (384 threads): one lane each of warps 0, 2 and 3 issues TMA loads into one ring of stages that
+// runs on across segments (a thread gets a tensor load accepted only every ~0.3 us, threads of different
+// warps are served in parallel); warp 1 allocates tensor memory and issues the MMAs into one of two
+// accumulator buffers; warps 4-11 are the epilogue (two teams of four, one warp per quarter of the 128
+// accumulator lanes, alternating 16-token chunks) and work on one buffer while the MMAs fill the other.
+//
+// Epilogue of a segment that covers all of K: the values pass through shared memory (16 tokens x 128 rows
+// fp32) so that each thread then owns 8 consecutive features of one token AND their partners (the other
+// half of the rotary pair, or the up row of a gate row), and results leave with 16-byte stores:
+//   QKV     rotation at the row's own position, K/V scatter into the cache, Q to the compact buffer
 //   SWIGLU  the tile is 64 gate rows followed by the 64 up rows of the same features; silu(gate) * up
-//   PARTIAL fp32 split-K partial (output / down projection)
+//   PARTIAL fp32 K-split partial sums (folded, with the residual and the next norm, by the next kernel)
+// A segment that covers only part of K leaves its raw sums in a workspace slot and adds its k-blocks to the
+// tile's counter; the CTA whose addition completes the tile adds the slots of all segments in k order
+// (a fixed order: results do not depend on which CTA came last) and runs the epilogue above.  No CTA
+// ever waits for another.
 #include "vlac_internal.h"
 #include "launch_util.h"
 #include <cuda.h>
@@ -30,15 +40,21 @@
 namespace {
 
 constexpr int TG_QKV = 0, TG_PARTIAL = 1, TG_SWIGLU = 2;
-constexpr int TG_THREADS = 256;
-constexpr int TG_STG = 8;                       // table loads a thread keeps in flight while staging the rotary rows
-constexpr int TG_PRODUCERS = 3;                // warps 0, 6, 7: one elected lane each issues TMA loads
+constexpr int TG_THREADS = 384;
+constexpr int TG_EPI_WARP0 = 4;                 // first epilogue warp
+constexpr int TG_EPI_THREADS = 256;
+constexpr int TG_PRODUCERS = 3;                 // warps 0, 2, 3: one elected lane each issues TMA loads
 constexpr int TG_BK = 64;                       // bf16 elements per k-block = one 128-byte swizzle row
 constexpr int TG_A_BYTES = 128 * TG_BK * 2;     // 16 KB: 128 weight rows
 constexpr int TG_BOX_TOK = 64;                  // token rows per TMA box
 constexpr int TG_BOX_BYTES = TG_BOX_TOK * TG_BK * 2;   // 8 KB
+constexpr int TG_CHUNK = 256;                   // most tokens one accumulator buffer holds
 constexpr int TG_MAX_STAGES = 8;
-constexpr int TG_SMEM_RING = 192 * 1024;        // dynamic shared memory for the ring (four stages of 48 KB at up to 256 tokens)
+constexpr int TG_SMEM_RING = 192 * 1024;        // ring: four stages of 48 KB at 256 tokens
+constexpr int TG_STAGE_OUT = 8192;              // one 16-token chunk of a tile as fp32
+constexpr int TG_SMEM_OUT = 4 * TG_STAGE_OUT;   // [team][double buffer]
+constexpr int TG_SMEM_DYN = TG_SMEM_RING + TG_SMEM_OUT;    // with the static part this is all of an SM's 227 KB
+constexpr int TG_SLOT_FLOATS = TG_CHUNK * 128;  // one workspace slot: raw sums of one segment and token chunk
 constexpr unsigned long long TG_WAIT_LIMIT_NS = 400000000ull;
 
 struct alignas(64) TcArgs {
@@ -49,7 +65,8 @@ struct alignas(64) TcArgs {
   const int* tot;                 // live token count in device memory (NULL: tot_fixed)
   int tot_fixed;
   int K, N;                       // N = rows of one weight matrix
-  int mode, n_splits;
+  int mode, n_splits;             // n_splits: K-splits of a tile (PARTIAL); the other modes share k-blocks evenly
+  int n_tiles;
   int d;                          // head_dim (QKV)
   int batch;                      // sequences sharing the compact row space
   // epilogue operands
@@ -59,11 +76,9 @@ struct alignas(64) TcArgs {
   bf16 *q_out, *kc, *vc;          // QKV: [T][N], caches [B][max_seq][N]
   float* part; size_t split_stride;   // PARTIAL: [split][T][N]
   bf16* h_out;                    // SWIGLU: [T][N]
-  // SWIGLU tail: tiles beyond the last full wave of CTAs are split along K so that they finish together;
-  // their raw gate/up sums go to tail_part[split][T][tail_ld] and a small kernel finishes them
-  int full_tiles, tail_splits, tail_ld;
-  float* tail_part; size_t tail_stride;
-  int tmem_cols;                  // tensor-memory columns to allocate: covers the largest token chunk (power of two >= 32)
+  float* ws;                      // raw sums of segments that cover part of K: [cta][2][token chunk][256][128]
+  int* tile_cnt;                  // [tile][token chunk] k-blocks accumulated so far (zero between launches)
+  int tmem_cols;                  // tensor-memory columns to allocate (two buffers; power of two >= 32)
   int* dev_error;
 };
 
@@ -73,6 +88,9 @@ __device__ __forceinline__ void mbar_init(unsigned long long* bar, unsigned coun
 }
 __device__ __forceinline__ void mbar_expect_tx(unsigned long long* bar, unsigned bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned parity) {
   unsigned ok;
@@ -92,7 +110,9 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned pari
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
   while (true) {
-    if (mbar_try_wait(bar, parity)) return true;
+#pragma unroll 1
+    for (int i = 0; i < 32; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
     if (global_ns() - t0 > limit_ns) break;
   }
@@ -100,17 +120,12 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, unsigned pari
   if (dev_error) atomicCAS(dev_error, 0, code);
   return false;
 }
-__device__ __forceinline__ float lds_f32(unsigned addr) { float v; asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr)); return v; }
-__device__ __forceinline__ int lds_s32(unsigned addr) { int v; asm volatile("ld.shared.s32 %0, [%1];" : "=r"(v) : "r"(addr)); return v; }
-__device__ __forceinline__ uint4 lds_v4(unsigned addr) {
-  uint4 v;
-  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+__device__ __forceinline__ float4 lds_f4(unsigned addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
   return v;
 }
 __device__ __forceinline__ void sts_f32(unsigned addr, float v) { asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory"); }
-__device__ __forceinline__ void sts_b16(unsigned addr, bf16 v) {
-  asm volatile("st.shared.b16 [%0], %1;" ::"r"(addr), "h"(*reinterpret_cast<unsigned short*>(&v)) : "memory");
-}
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, int x, int y, unsigned long long* bar) {
   asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                ::"r"(smem_u32(dst)), "l"(tm), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
@@ -145,306 +160,333 @@ __device__ __forceinline__ void tmem_ld16(unsigned taddr, float* v) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
+// barrier over the epilogue threads that also tells every thread whether all of them passed `ok`
+__device__ __forceinline__ bool epi_all_ok(bool ok) {
+  unsigned r;
+  asm volatile("{\n.reg .pred p, q;\nsetp.ne.u32 q, %1, 0;\nbarrier.cta.red.and.pred p, 1, %2, q;\nselp.u32 %0, 1, 0, p;\n}\n"
+               : "=r"(r) : "r"((unsigned)ok), "n"(TG_EPI_THREADS) : "memory");
+  return r != 0;
+}
+__device__ __forceinline__ void team_sync(int team) { asm volatile("bar.sync %0, 128;" ::"r"(2 + team) : "memory"); }
+__device__ __forceinline__ float4 ldcg_f4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ uint4 pack8(const float* y) {
+  uint4 o;
+  __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) o2[e] = __floats2bfloat162_rn(y[2 * e], y[2 * e + 1]);
+  return o;
+}
+
+// ---- the share of work of one CTA, as a sequence of segments
+struct Seg { int tile, kb0, kb1; bool first; };
+struct Range { long long u0, u1; };
+__device__ __forceinline__ long long range_begin(long long total, int c, int G) { return total * c / G; }
+__device__ __forceinline__ bool next_seg(long long& u, const Range& r, int kbt, Seg& s) {
+  if (u >= r.u1) return false;
+  s.tile = (int)(u / kbt);
+  s.kb0 = (int)(u - (long long)s.tile * kbt);
+  const long long left = r.u1 - u;
+  s.kb1 = (int)((long long)s.kb0 + left < (long long)kbt ? (long long)s.kb0 + left : (long long)kbt);
+  s.first = (u == r.u0);
+  u += s.kb1 - s.kb0;
+  return true;
+}
+
+// What the epilogue does with 8 consecutive features x1[] of one token and their 8 partners x2[].
+struct EmitCtx {
+  int mode, mat, row_base, N, d, half, L, max_seq, batch;
+  const float *rope_cos, *rope_sin;
+  bf16 *q_out, *kc, *vc, *h_out;
+};
+// r1: first of the 8 rows inside the tile; tok: compact token index; row: rowmap entry of the token
+__device__ __forceinline__ void emit8(const EmitCtx& e, const float* x1, const float* x2, int r1, size_t tok, int row) {
+  const size_t N = (size_t)e.N;
+  if (e.mode == TG_SWIGLU) {
+    if (e.row_base + r1 >= e.N) return;
+    float y[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) y[i] = __fdividef(x1[i], 1.f + __expf(-x1[i])) * x2[i];
+    *reinterpret_cast<uint4*>(e.h_out + tok * N + e.row_base + r1) = pack8(y);
+    return;
+  }
+  // QKV
+  const int n1 = e.row_base + r1, n2 = n1 + e.half;
+  if (n1 >= e.N) return;
+  int b = 0, pos = row;
+  if (e.batch > 1) { b = row / e.L; pos = row - b * e.L; }
+  float y1[8], y2[8];
+  if (e.mat < 2) {
+    const int j0 = r1 % e.half;
+    const float4* cp = reinterpret_cast<const float4*>(e.rope_cos + (size_t)pos * e.half + j0);
+    const float4* sp = reinterpret_cast<const float4*>(e.rope_sin + (size_t)pos * e.half + j0);
+    const float4 c0 = __ldg(cp), c1 = __ldg(cp + 1), s0 = __ldg(sp), s1 = __ldg(sp + 1);
+    const float c[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+    const float s[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { y1[i] = x1[i] * c[i] - x2[i] * s[i]; y2[i] = x2[i] * c[i] + x1[i] * s[i]; }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { y1[i] = x1[i]; y2[i] = x2[i]; }
+  }
+  bf16* dst;
+  if (e.mat == 0) dst = e.q_out + tok * N;
+  else dst = (e.mat == 1 ? e.kc : e.vc) + ((size_t)b * e.max_seq + pos) * N;
+  *reinterpret_cast<uint4*>(dst + n1) = pack8(y1);
+  *reinterpret_cast<uint4*>(dst + n2) = pack8(y2);
+}
 
 __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_constant__ TcArgs a) {
   extern __shared__ __align__(1024) unsigned char ring_raw[];
-  __shared__ __align__(8) unsigned long long full_bar[TG_MAX_STAGES], empty_bar[TG_MAX_STAGES], acc_bar;
-  __shared__ float xch[2][2][4][16][32];                         // epilogue exchange between warp pairs: [team][double buffer]
+  __shared__ __align__(8) unsigned long long full_bar[TG_MAX_STAGES], empty_bar[TG_MAX_STAGES], acc_full[2], acc_empty[2];
   __shared__ unsigned tmem_base_slot;
-  __shared__ int abort_flag;
+  __shared__ int abort_flag, fold_flag;
+  __shared__ int rows_buf[2][TG_CHUNK];                          // rowmap entries of the token chunk the epilogue works on (by item parity)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  // the ring must start on a 1024-byte boundary (swizzle atoms); dynamic smem is over-allocated by 1 KB
-  // (an offset from the array keeps the pointer in the shared address space for the compiler)
-  unsigned char* ring = ring_raw + ((1024u - (smem_u32(ring_raw) & 1023u)) & 1023u);
+  // the ring must start on a 1024-byte boundary (swizzle atoms): the declared alignment makes the compiler pad the
+  // static part; checked below, since a misplaced ring would corrupt results silently
+  unsigned char* ring = ring_raw;
+  const unsigned out_smem = smem_u32(ring) + (unsigned)TG_SMEM_RING;
 
-  int tile = blockIdx.x, split = blockIdx.y, splits = a.n_splits;
-  bool tail = false;                                            // a K-split SWIGLU tile: epilogue stores raw sums
-  if (a.mode == TG_SWIGLU && a.tail_splits > 1 && tile >= a.full_tiles) {
-    const int u = tile - a.full_tiles;
-    tile = a.full_tiles + u / a.tail_splits; split = u % a.tail_splits; splits = a.tail_splits; tail = true;
-  }
   if (tid == 0) {
     for (int s = 0; s < TG_MAX_STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-    mbar_init(&acc_bar, 1);
-    abort_flag = 0;
+    for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], TG_EPI_THREADS / 32); }
+    abort_flag = 0; fold_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
   pdl_trigger();
-  // tensor memory does not depend on earlier kernels either: allocated (for the largest token chunk) before the wait
+  // tensor memory depends on no earlier kernel: allocated before the dependency wait
   const unsigned tmem_cols = (unsigned)a.tmem_cols;
   if (warp == 1) {                                              // whole warp
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)), "r"(tmem_cols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  // The live token count was written by the selection kernels, which never release their dependents early, so
-  // it is complete before any kernel launched after them starts: it may be read ahead of the dependency wait.
-  // blockIdx.z selects a chunk of up to 512 tokens (one accumulator's worth of tensor-memory columns)
-  const int tok0 = blockIdx.z * 512;
-  const int tokens = min(max((a.tot ? *a.tot : a.tot_fixed) - tok0, 0), 512);
-  const int n_boxes = (tokens + TG_BOX_TOK - 1) / TG_BOX_TOK;    // token rows are staged in multiples of 64
-  const int stage_bytes = TG_A_BYTES + n_boxes * TG_BOX_BYTES;
+  // The live token count was written by the selection kernels, which never release their dependents early, so it
+  // is complete before any kernel launched after them starts: it is read ahead of the dependency wait (to size the
+  // early weight loads) and checked again behind it.
+  const int T = a.tot ? *a.tot : a.tot_fixed;
+  const int n_chunks = (T + TG_CHUNK - 1) / TG_CHUNK;
+  const int chunk_sz = n_chunks > 0 ? (((T + n_chunks - 1) / n_chunks + 15) / 16) * 16 : 0;     // tokens of every chunk but the last
+  const int max_boxes = (chunk_sz + TG_BOX_TOK - 1) / TG_BOX_TOK;
+  const int stage_bytes = TG_A_BYTES + max_boxes * TG_BOX_BYTES;
   int n_stages = TG_SMEM_RING / stage_bytes;
   if (n_stages > TG_MAX_STAGES) n_stages = TG_MAX_STAGES;
-  const int kb_total = (a.K + TG_BK - 1) / TG_BK;
-  const int kb0 = (int)(((long long)kb_total * split) / splits);
-  const int kb1 = (int)(((long long)kb_total * (split + 1)) / splits);
-  const int n_kb = (tokens > 0) ? kb1 - kb0 : 0;
-  // columns of the first / second MMA
-  const int n0 = min(((tokens + 15) / 16) * 16, 256);
-  const int n1 = tokens > 256 ? ((tokens - 256 + 15) / 16) * 16 : 0;
-  // weight rows of this tile
+  const int kbt = (a.K + TG_BK - 1) / TG_BK;                       // k-blocks of a tile
+  // ---- this CTA's share
+  Range rg;
+  const long long total = (long long)a.n_tiles * kbt;
+  const int G = (int)gridDim.x;
+  if (a.mode == TG_PARTIAL) {                                    // blockIdx.x = tile * n_splits + split
+    const int tile = (int)blockIdx.x / a.n_splits, split = (int)blockIdx.x - tile * a.n_splits;
+    rg.u0 = (long long)tile * kbt + ((long long)kbt * split) / a.n_splits;
+    rg.u1 = (long long)tile * kbt + ((long long)kbt * (split + 1)) / a.n_splits;
+  } else {
+    rg.u0 = range_begin(total, (int)blockIdx.x, G);
+    rg.u1 = range_begin(total, (int)blockIdx.x + 1, G);
+  }
+  if (T <= 0) rg.u1 = rg.u0;
   const int tiles_per_mat = (a.N + 127) / 128;
-  const int mat = a.mode == TG_QKV ? tile / tiles_per_mat : 0;
-  const int row_base = a.mode == TG_QKV ? (tile - mat * tiles_per_mat) * 128 : (a.mode == TG_SWIGLU ? tile * 64 : tile * 128);
+  auto tile_mat = [&](int tile) { return a.mode == TG_QKV ? tile / tiles_per_mat : 0; };
+  auto tile_row_base = [&](int tile) {
+    return a.mode == TG_QKV ? (tile % tiles_per_mat) * 128 : (a.mode == TG_SWIGLU ? tile * 64 : tile * 128);
+  };
+  auto chunk_tokens = [&](int ch) { return min(chunk_sz, T - ch * chunk_sz); };
 
-  // ---- the weights depend on no earlier kernel: the weight boxes of the first ring round are requested before
-  // the dependency wait (their bytes announced without an arrival; the activation boxes follow after the wait)
   const int n_prod = min(TG_PRODUCERS, n_stages);
-  const int pid = warp == 0 ? 0 : warp - 5;
-  const bool producer = lane == 0 && (warp == 0 || warp >= 6) && pid < n_prod;
-  auto load_weights = [&](int i, int s) {
+  const int pid = warp == 0 ? 0 : warp - 1;                      // warps 0, 2, 3 -> 0, 1, 2
+  const bool producer = lane == 0 && (warp == 0 || warp == 2 || warp == 3) && pid < n_prod;
+  auto load_weights = [&](int tile, int kb, int s) {
     unsigned char* sa = ring + (size_t)s * stage_bytes;
-    const int k = (kb0 + i) * TG_BK;
+    const int k = kb * TG_BK, rb = tile_row_base(tile);
     if (a.mode == TG_SWIGLU) {
-      tma_load_2d(sa, &a.tm_a[0], k, row_base, &full_bar[s]);                // 64 gate rows
-      tma_load_2d(sa + 64 * 128, &a.tm_a[1], k, row_base, &full_bar[s]);     // 64 up rows of the same features
+      tma_load_2d(sa, &a.tm_a[0], k, rb, &full_bar[s]);                      // 64 gate rows
+      tma_load_2d(sa + 64 * 128, &a.tm_a[1], k, rb, &full_bar[s]);           // 64 up rows of the same features
     } else {
-      tma_load_2d(sa, &a.tm_a[mat], k, row_base, &full_bar[s]);
+      tma_load_2d(sa, &a.tm_a[tile_mat(tile)], k, rb, &full_bar[s]);
     }
   };
-  const int n_early = min(n_kb, n_stages);                      // k-blocks whose weights go out early
-  if (producer)
-    for (int i = pid; i < n_early; i += n_prod) {
-      asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&full_bar[i])), "r"((unsigned)TG_A_BYTES) : "memory");
-      load_weights(i, i);
-    }
+  // ---- the weights depend on no earlier kernel: the weight boxes of the first ring round are requested before
+  // the dependency wait (their bytes announced without an arrival; the activation boxes follow after the wait)
+  int n_early = 0;
+  {
+    long long u = rg.u0; Seg sg; int it = 0;
+    while (it < n_stages && next_seg(u, rg, kbt, sg))
+      for (int ch = 0; ch < n_chunks && it < n_stages; ++ch)
+        for (int kb = sg.kb0; kb < sg.kb1 && it < n_stages; ++kb, ++it) {
+          if (producer && it % n_prod == pid) {
+            asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&full_bar[it])), "r"((unsigned)TG_A_BYTES) : "memory");
+            load_weights(sg.tile, kb, it);
+          }
+        }
+    n_early = it;
+  }
   pdl_wait();                                                   // everything below may read what earlier kernels wrote
+  if (tid == 0 && a.tot && *a.tot != T) { abort_flag = 1; atomicCAS(a.dev_error, 0, 0x30000); }   // the count changed under us: give up
+  if (tid == 0 && (smem_u32(ring_raw) & 1023u)) { abort_flag = 1; atomicCAS(a.dev_error, 0, 0x31000); }
 
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  if (abort_flag) rg.u1 = rg.u0;                                // uniform: written before the barrier
   const unsigned tmem_base = tmem_base_slot;
+  const unsigned buf_cols = tmem_cols >> 1;                      // columns of one accumulator buffer
 
-  if (warp == 0 || warp >= 6) {
+  if (warp == 0 || warp == 2 || warp == 3) {
     // ------------------------------------------------------------------ TMA producers
-    // A thread gets a tensor load accepted only every ~0.3 us whatever the box size, but threads of
-    // different warps are served in parallel: the k-blocks are dealt round-robin to three producer lanes.
-    // Each producer waits for the ring slot of its own k-blocks only.  Its previous wait proved k-block
-    // i - P - n_stages consumed; the slot's previous phase (k-block i - 2 n_stages) must be complete by
-    // then, or the one-bit phase parity would alias: hence no more producers than stages.
+    // The k-blocks of all segments and chunks, in order, are dealt round-robin to the producer lanes.  A producer
+    // waits for the ring slot of its own k-blocks only; no more producers than stages, or the one-bit phase
+    // parity of a slot could alias.
     if (producer) {
-      const int rows0 = min(n_boxes, 4), rows1 = n_boxes - rows0;            // boxes of the first / second token request
-      for (int i = pid; i < n_kb; i += n_prod) {
-        const int s = i % n_stages;
-        if (i >= n_stages && !mbar_wait(&empty_bar[s], ((i / n_stages) & 1) ^ 1, &abort_flag, a.dev_error, 0x40000 | (i & 0xffff))) break;
-        unsigned char* sa = ring + (size_t)s * stage_bytes;
-        unsigned char* sb = sa + TG_A_BYTES;
-        const int k = (kb0 + i) * TG_BK;
-        if (i < n_early) {
-          mbar_expect_tx(&full_bar[s], (unsigned)(stage_bytes - TG_A_BYTES));     // the weights of this k-block are on their way
-        } else {
-          mbar_expect_tx(&full_bar[s], (unsigned)stage_bytes);
-          load_weights(i, s);
+      long long u = rg.u0; Seg sg; int it = 0; bool ok = true;
+      while (ok && next_seg(u, rg, kbt, sg))
+        for (int ch = 0; ch < n_chunks && ok; ++ch) {
+          const int boxes = (chunk_tokens(ch) + TG_BOX_TOK - 1) / TG_BOX_TOK;
+          const unsigned x_bytes = (unsigned)(boxes * TG_BOX_BYTES);
+          for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
+            if (it % n_prod != pid) continue;
+            const int s = it % n_stages;
+            if (it >= n_stages && !mbar_wait(&empty_bar[s], ((it / n_stages) & 1) ^ 1, &abort_flag, a.dev_error, 0x40000 | (it & 0xffff))) { ok = false; break; }
+            if (it < n_early) {
+              mbar_expect_tx(&full_bar[s], x_bytes);               // the weights of this k-block are on their way
+            } else {
+              mbar_expect_tx(&full_bar[s], (unsigned)TG_A_BYTES + x_bytes);
+              load_weights(sg.tile, kb, s);
+            }
+            tma_load_2d(ring + (size_t)s * stage_bytes + TG_A_BYTES, &a.tm_b[boxes - 1], kb * TG_BK, ch * chunk_sz, &full_bar[s]);
+          }
         }
-        tma_load_2d(sb, &a.tm_b[rows0 - 1], k, tok0, &full_bar[s]);
-        if (rows1 > 0) tma_load_2d(sb + 4 * TG_BOX_BYTES, &a.tm_b[rows1 - 1], k, tok0 + 256, &full_bar[s]);
-      }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      const unsigned idesc0 = umma_idesc_bf16(128, n0);
-      const unsigned idesc1 = n1 ? umma_idesc_bf16(128, n1) : 0u;
-      bool ok = true;
-      for (int i = 0; i < n_kb && ok; ++i) {
-        const int s = i % n_stages;
-        ok = mbar_wait(&full_bar[s], (i / n_stages) & 1, &abort_flag, a.dev_error, 0x50000 | (i & 0xffff));
+      long long u = rg.u0; Seg sg; int it = 0, item = 0; bool ok = true;
+      while (ok && next_seg(u, rg, kbt, sg))
+        for (int ch = 0; ch < n_chunks && ok; ++ch, ++item) {
+          const int b = item & 1, use = item >> 1;
+          if (use > 0) ok = mbar_wait(&acc_empty[b], (use - 1) & 1, &abort_flag, a.dev_error, 0x58000 | (item & 0x7fff));
+          if (!ok) break;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const unsigned idesc = umma_idesc_bf16(128, ((chunk_tokens(ch) + 15) / 16) * 16);
+          const unsigned acc_addr = tmem_base + (unsigned)b * buf_cols;
+          for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
+            const int s = it % n_stages;
+            ok = mbar_wait(&full_bar[s], (it / n_stages) & 1, &abort_flag, a.dev_error, 0x50000 | (it & 0x7fff));
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const unsigned char* sa = ring + (size_t)s * stage_bytes;
+            const unsigned long long da = umma_desc(sa), db = umma_desc(sa + TG_A_BYTES);
+#pragma unroll
+            for (int k = 0; k < TG_BK / 16; ++k) {
+              const unsigned long long koff = (unsigned long long)((k * 32) >> 4);        // 16 bf16 = 32 bytes along the swizzle row
+              umma_bf16(acc_addr, da + koff, db + koff, idesc, (kb > sg.kb0 || k > 0) ? 1u : 0u);
+            }
+            umma_commit(&empty_bar[s]);                          // stage reusable once these MMAs have read it
+          }
+          if (ok) umma_commit(&acc_full[b]);                     // accumulator of this segment and chunk complete
+        }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 4-11)
+    const int ew = warp - TG_EPI_WARP0;
+    const int team = ew >> 2, q = warp & 3;                      // q: the TMEM lane quarter this warp may read
+    const int et = tid - TG_EPI_WARP0 * 32;                      // thread index among the epilogue threads
+    const int tteam = (q << 5) | lane;                           // thread index inside the team; also its tile row in phase A
+    const int r = tteam;
+    EmitCtx e;
+    e.mode = a.mode; e.N = a.N; e.d = a.d; e.half = a.mode == TG_SWIGLU ? 64 : a.d / 2; e.L = a.L; e.max_seq = a.max_seq; e.batch = a.batch;
+    e.rope_cos = a.rope_cos; e.rope_sin = a.rope_sin; e.q_out = a.q_out; e.kc = a.kc; e.vc = a.vc; e.h_out = a.h_out;
+    // phase B task of this thread: token t_b of the 16-token chunk, 8 rows from r1 and their partners from r1 + half
+    const int t_b = tteam >> 3, f0 = (tteam & 7) * 8;
+    const int r1 = (f0 / e.half) * (2 * e.half) + f0 % e.half;
+    const unsigned stage_base = out_smem + (unsigned)team * 2u * TG_STAGE_OUT;
+    long long u = rg.u0; Seg sg; int item = 0, cb = 0;          // cb: running count of 16-token chunks of this team (double buffer)
+    bool ok = true;
+    while (ok && next_seg(u, rg, kbt, sg)) {
+      const bool whole = sg.kb0 == 0 && sg.kb1 == kbt;
+      const bool direct = whole || a.mode == TG_PARTIAL;         // results leave in their final form straight from the accumulator
+      e.mat = tile_mat(sg.tile); e.row_base = tile_row_base(sg.tile);
+      const int split = a.mode == TG_PARTIAL ? (int)blockIdx.x % a.n_splits : 0;
+      for (int ch = 0; ch < n_chunks && ok; ++ch, ++item) {
+        const int b = item & 1, use = item >> 1;
+        const int tok0 = ch * chunk_sz, tokens = chunk_tokens(ch);
+        int* rows_s = rows_buf[item & 1];
+        if (et < tokens && a.rowmap) rows_s[et] = __ldg(a.rowmap + tok0 + et);
+        ok = mbar_wait(&acc_full[b], use & 1, &abort_flag, a.dev_error, 0x60000 | (item & 0xffff));
+        ok = epi_all_ok(ok);                                      // same decision in all epilogue threads; rows_s visible
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const unsigned char* sa = ring + (size_t)s * stage_bytes;
-        const unsigned char* sb = sa + TG_A_BYTES;
-        const unsigned long long da = umma_desc(sa), db0 = umma_desc(sb), db1 = umma_desc(sb + 256 * 128);
+        const unsigned acc_addr = tmem_base + (unsigned)b * buf_cols + ((unsigned)(32 * q) << 16);
+        float* ws_slot = a.ws ? a.ws + ((size_t)(blockIdx.x * 2 + (sg.first ? 0 : 1)) * n_chunks + ch) * TG_SLOT_FLOATS : nullptr;
+        for (int c0 = team * 16; c0 < tokens; c0 += 32, ++cb) {
+          // ---- phase A: 16 tokens of this thread's tile row -> shared memory, transposed to [token][row]
+          float v[16];
+          tmem_ld16(acc_addr + (unsigned)c0, v);
+          const unsigned sb = stage_base + (unsigned)(cb & 1) * TG_STAGE_OUT;
 #pragma unroll
-        for (int k = 0; k < TG_BK / 16; ++k) {
-          const unsigned acc = (i > 0 || k > 0) ? 1u : 0u;
-          const unsigned long long koff = (unsigned long long)((k * 32) >> 4);        // 16 bf16 = 32 bytes along the swizzle row
-          umma_bf16(tmem_base, da + koff, db0 + koff, idesc0, acc);
-          if (n1) umma_bf16(tmem_base + 256, da + koff, db1 + koff, idesc1, acc);
-        }
-        umma_commit(&empty_bar[s]);                              // stage reusable once these MMAs have read it
-      }
-      if (ok) umma_commit(&acc_bar);                             // accumulator complete
-    }
-  }
-  __syncwarp();
-  {
-    // ------------------------------------------------------------------ epilogue (all eight warps)
-    // Once their loops are done the producer and MMA warps join: two teams of four warps (one warp per
-    // quarter of the 128 accumulator lanes in each) take the 16-token chunks alternately.
-    const int team = (warp >= 2 && warp <= 5) ? 0 : 1;
-    const int q = warp & 3;                                      // TMEM lane quarter this warp may read
-    bool ok = n_kb > 0;
-    if (ok) ok = mbar_wait(&acc_bar, 0, &abort_flag, a.dev_error, 0x60000);
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const int r = 32 * q + lane;                                 // row of the tile held by this thread
-    const int half = a.d / 2;
-    // feature (weight row) this thread finishes, and the warp holding its partner value
-    int n, pq;
-    bool first;                                                  // QKV: first half of the rotary pair; SWIGLU: gate side
-    if (a.mode == TG_SWIGLU) { n = row_base + (r & 63); first = r < 64; pq = q ^ 2; }
-    else { n = row_base + r; first = ((r / half) & 1) == 0; pq = q ^ (half >> 5); }
-    const bool n_ok = n < a.N;
-    const bool exchange = (a.mode == TG_SWIGLU && !tail) || (a.mode == TG_QKV && mat < 2);
-    const int j = (n % a.d) % half;
-    const size_t N = (size_t)a.N;
-    // QKV: the ring is free once the accumulator is complete.  The row map of the tile's tokens and, for Q
-    // and K tiles, the rotary table rows of their positions are copied into it by all warps at once, so the
-    // chunk loop below reads them from shared memory instead of waiting on 32 global loads per chunk.
-    int* rows_s = reinterpret_cast<int*>(ring);                                  // [tokens]
-    float* tab_s = reinterpret_cast<float*>(ring + 2048);                        // [tokens][2 * half]: cos | sin
-    const bool staged = a.mode == TG_QKV && tokens > 0 &&
-                        (size_t)2048 + (size_t)tokens * 2 * half * sizeof(float) <= (size_t)TG_SMEM_RING - 4 * 8192 && (half % 4) == 0;
-    if (staged) {                                                // uniform over the CTA
-      for (int t = tid; t < tokens; t += TG_THREADS) rows_s[t] = __ldg(a.rowmap + tok0 + t);
-      __syncthreads();
-      if (mat < 2) {
-        const int vec_per_tok = half / 2;                        // float4 per token: half/4 of cos, half/4 of sin
-        const int total = tokens * vec_per_tok;
-        for (int base = tid; base < total; base += TG_STG * TG_THREADS) {        // TG_STG independent loads in flight per thread
-          float4 tmp[TG_STG];
+          for (int c = 0; c < 16; ++c) sts_f32(sb + (unsigned)(c * 512 + r * 4), v[c]);
+          team_sync(team);
+          // ---- phase B
+          if (direct && a.mode != TG_PARTIAL) {
+            if (c0 + t_b < tokens) {
+              const float4 p0 = lds_f4(sb + (unsigned)(t_b * 512 + r1 * 4)), p1 = lds_f4(sb + (unsigned)(t_b * 512 + r1 * 4 + 16));
+              const float4 p2 = lds_f4(sb + (unsigned)(t_b * 512 + (r1 + e.half) * 4)), p3 = lds_f4(sb + (unsigned)(t_b * 512 + (r1 + e.half) * 4 + 16));
+              const float x1[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
+              const float x2[8] = {p2.x, p2.y, p2.z, p2.w, p3.x, p3.y, p3.z, p3.w};
+              emit8(e, x1, x2, r1, (size_t)(tok0 + c0 + t_b), a.rowmap ? rows_s[c0 + t_b] : 0);
+            }
+          } else {
+            // raw fp32 sums, 16 bytes per thread and request: a K-split partial of its own (PARTIAL) or a workspace slot
 #pragma unroll
-          for (int u = 0; u < TG_STG; ++u) {
-            const int idx = min(base + u * TG_THREADS, total - 1);
-            const int t = idx / vec_per_tok, v = idx - t * vec_per_tok;
-            const int row = rows_s[t];
-            const int pos = a.batch > 1 ? row % a.L : row;
-            const float* src = (v < half / 4 ? a.rope_cos : a.rope_sin) + (size_t)pos * half + (size_t)(v % (half / 4)) * 4;
-            tmp[u] = __ldg(reinterpret_cast<const float4*>(src));
-          }
-#pragma unroll
-          for (int u = 0; u < TG_STG; ++u) {
-            const int idx = base + u * TG_THREADS;
-            if (idx < total) *reinterpret_cast<float4*>(tab_s + (size_t)idx * 4) = tmp[u];
+            for (int i = 0; i < 4; ++i) {
+              const int sgm = tteam + 128 * i, t = sgm >> 5, sx = sgm & 31;
+              if (c0 + t >= tokens) continue;
+              const float4 val = lds_f4(sb + (unsigned)(t * 512 + sx * 16));
+              if (a.mode == TG_PARTIAL) {
+                if (e.row_base + sx * 4 < a.N)
+                  *reinterpret_cast<float4*>(a.part + (size_t)split * a.split_stride + (size_t)(tok0 + c0 + t) * a.N + e.row_base + sx * 4) = val;
+              } else {
+                *reinterpret_cast<float4*>(ws_slot + (size_t)(c0 + t) * 128 + sx * 4) = val;
+              }
+            }
           }
         }
-      }
-      __syncthreads();
-    }
-    const unsigned bar_id = 2u + (unsigned)team;
-    // Results leave through shared memory: a team writes the 16 token rows of a chunk into its own buffer
-    // (end of the ring, double-buffered), meets at the team barrier and copies them out 16 bytes per thread,
-    // so that one store instruction of a warp carries 512 contiguous bytes instead of 64 or 128.  (The
-    // number of store requests an SM can have in flight, not their size, bounds the direct form.)
-    const int tteam = (q << 5) | lane;                            // thread index inside the team: also the tile row
-    const int out_cols = a.mode == TG_SWIGLU && !tail ? 64 : 128;
-    const int esz = (tail || a.mode == TG_PARTIAL) ? 4 : 2;       // fp32 partial sums, bf16 otherwise
-    const int row_bytes = out_cols * esz;
-    const bool vec_ok = (a.mode == TG_SWIGLU && !tail) ? (row_base + 64 <= a.N) : (tail ? true : (row_base + 128 <= a.N));
-    const unsigned out_base = smem_u32(ring) + (unsigned)TG_SMEM_RING - 4u * 8192u + (unsigned)team * 2u * 8192u;
-    const unsigned rows_a = smem_u32(rows_s), tab_a = smem_u32(tab_s) + (unsigned)j * 4u;
-    int chunk = 0;
-    for (int c0 = team * 16; c0 < tokens; c0 += 32, ++chunk) {
-      float v[16], pv[16];
-      if (ok) tmem_ld16(tmem_base + ((unsigned)(32 * q) << 16) + (unsigned)c0, v);
-      else {
+        // this warp has read all it needs from the accumulator buffer
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[b]);
+        if (direct) continue;
+        // ---- a segment that covers part of K: count its k-blocks; the CTA that completes the tile folds it
+        __threadfence();
+        epi_all_ok(true);
+        if (et == 0) {
+          int* cnt = a.tile_cnt + (size_t)sg.tile * n_chunks + ch;
+          const int done = atomicAdd(cnt, sg.kb1 - sg.kb0) + (sg.kb1 - sg.kb0);
+          fold_flag = done == kbt;
+          if (done == kbt) *cnt = 0;                             // ready for the next launch
+        }
+        epi_all_ok(true);
+        if (!fold_flag) continue;                                // (fold_flag is rewritten only after the next two barriers)
+        __threadfence();
+        // segments of this tile in k order: CTA c holds k-blocks [max(begin(c), lo), min(begin(c + 1), hi))
+        const long long lo = (long long)sg.tile * kbt, hi = lo + kbt;
+        int c_first = (int)((lo * G) / total);
+        while (c_first + 1 < G && range_begin(total, c_first + 1, G) <= lo) ++c_first;
+        while (c_first > 0 && range_begin(total, c_first, G) > lo) --c_first;
+        for (int g0 = team * 16; g0 < tokens; g0 += 32) {
+          const int t = g0 + t_b;
+          if (t >= tokens) continue;
+          float x1[8], x2[8];
 #pragma unroll
-        for (int c = 0; c < 16; ++c) v[c] = 0.f;
-      }
-      if (exchange) {                                            // uniform over the four warps of a team
-        float (*buf)[16][32] = xch[team][chunk & 1];
-#pragma unroll
-        for (int c = 0; c < 16; ++c) buf[q][c][lane] = v[c];
-        asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
-#pragma unroll
-        for (int c = 0; c < 16; ++c) pv[c] = buf[pq][c][lane];
-      }
-      const unsigned out_a = out_base + (unsigned)(chunk & 1) * 8192u;
-      int rw[16];                                                // QKV: row map entries of the chunk's tokens
-      if (a.mode == TG_QKV) {
-        float cs[16], sn[16];
-        if (staged) {
-#pragma unroll
-          for (int c = 0; c < 16; ++c) rw[c] = lds_s32(rows_a + (unsigned)min(c0 + c, tokens - 1) * 4u);
-#pragma unroll
-          for (int c = 0; c < 16; ++c) {
-            const unsigned ta = tab_a + (unsigned)min(c0 + c, tokens - 1) * (unsigned)(2 * half) * 4u;
-            if (mat < 2) { cs[c] = lds_f32(ta); sn[c] = lds_f32(ta + (unsigned)half * 4u); }
-            else { cs[c] = 1.f; sn[c] = 0.f; }
+          for (int i = 0; i < 8; ++i) x1[i] = x2[i] = 0.f;
+          for (int c = c_first; c < G && range_begin(total, c, G) < hi; ++c) {
+            const int which = range_begin(total, c, G) >= lo ? 0 : 1;
+            const float* src = a.ws + ((size_t)(c * 2 + which) * n_chunks + ch) * TG_SLOT_FLOATS + (size_t)t * 128;
+            const float4 p0 = ldcg_f4(src + r1), p1 = ldcg_f4(src + r1 + 4), p2 = ldcg_f4(src + r1 + e.half), p3 = ldcg_f4(src + r1 + e.half + 4);
+            x1[0] += p0.x; x1[1] += p0.y; x1[2] += p0.z; x1[3] += p0.w; x1[4] += p1.x; x1[5] += p1.y; x1[6] += p1.z; x1[7] += p1.w;
+            x2[0] += p2.x; x2[1] += p2.y; x2[2] += p2.z; x2[3] += p2.w; x2[4] += p3.x; x2[5] += p3.y; x2[6] += p3.z; x2[7] += p3.w;
           }
-        } else {
-#pragma unroll
-          for (int c = 0; c < 16; ++c) rw[c] = __ldg(a.rowmap + tok0 + min(c0 + c, tokens - 1));
-#pragma unroll
-          for (int c = 0; c < 16; ++c) {
-            const int pos = a.batch > 1 ? rw[c] % a.L : rw[c];
-            if (mat < 2) { cs[c] = __ldg(a.rope_cos + (size_t)pos * half + j); sn[c] = __ldg(a.rope_sin + (size_t)pos * half + j); }
-            else { cs[c] = 1.f; sn[c] = 0.f; }
-          }
-        }
-#pragma unroll
-        for (int c = 0; c < 16; ++c) {
-          float y = v[c];
-          if (mat < 2) y = first ? v[c] * cs[c] - pv[c] * sn[c] : v[c] * cs[c] + pv[c] * sn[c];
-          v[c] = y;
-        }
-      } else if (a.mode == TG_SWIGLU && !tail) {
-        // gate-side threads finish even columns, up-side threads odd columns
-#pragma unroll
-        for (int c = 0; c < 16; ++c) {
-          const float g = first ? v[c] : pv[c], u = first ? pv[c] : v[c];
-          v[c] = __fdividef(g, 1.f + __expf(-g)) * u;
-        }
-      }
-      if (vec_ok) {
-        // ---- rows of the chunk -> shared memory
-        if (esz == 4) {
-#pragma unroll
-          for (int c = 0; c < 16; ++c) sts_f32(out_a + (unsigned)(c * 512 + r * 4), v[c]);
-        } else if (a.mode == TG_QKV) {
-#pragma unroll
-          for (int c = 0; c < 16; ++c) sts_b16(out_a + (unsigned)(c * 256 + r * 2), __float2bfloat16(v[c]));
-        } else {
-#pragma unroll
-          for (int c = 0; c < 16; ++c)
-            if (((c & 1) == 0) == first) sts_b16(out_a + (unsigned)(c * 128 + (r & 63) * 2), __float2bfloat16(v[c]));
-        }
-        asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
-        // ---- shared memory -> global, 16 bytes per thread and request
-        const int spt = row_bytes >> 4;                          // 16-byte segments per token row: 32, 16 or 8
-        for (int seg = tteam; seg < 16 * spt; seg += 128) {
-          const int t = seg / spt, sx = seg - t * spt;
-          if (!ok || c0 + t >= tokens) continue;
-          const size_t tok = (size_t)(tok0 + c0 + t);
-          unsigned char* dst;
-          if (tail) dst = reinterpret_cast<unsigned char*>(a.tail_part + (size_t)split * a.tail_stride + tok * a.tail_ld + (size_t)(tile - a.full_tiles) * 128);
-          else if (a.mode == TG_PARTIAL) dst = reinterpret_cast<unsigned char*>(a.part + (size_t)split * a.split_stride + tok * N + row_base);
-          else if (a.mode == TG_SWIGLU) dst = reinterpret_cast<unsigned char*>(a.h_out + tok * N + row_base);
-          else if (mat == 0) dst = reinterpret_cast<unsigned char*>(a.q_out + tok * N + row_base);
-          else {
-            const int row = staged ? lds_s32(rows_a + (unsigned)(c0 + t) * 4u) : __ldg(a.rowmap + tok0 + c0 + t);
-            int b = 0, pos = row;
-            if (a.batch > 1) { b = row / a.L; pos = row - b * a.L; }
-            dst = reinterpret_cast<unsigned char*>((mat == 1 ? a.kc : a.vc) + ((size_t)b * a.max_seq + pos) * N + row_base);
-          }
-          *reinterpret_cast<uint4*>(dst + sx * 16) = lds_v4(out_a + (unsigned)(t * row_bytes + sx * 16));
-        }
-      } else {
-        // ragged last tile of a matrix whose row count is no multiple of the tile: element by element
-        const bool live = ok && n_ok;
-#pragma unroll
-        for (int c = 0; c < 16; ++c) {
-          if (!live || c0 + c >= tokens) continue;
-          const size_t tok = (size_t)(tok0 + c0 + c);
-          if (a.mode == TG_PARTIAL) a.part[(size_t)split * a.split_stride + tok * N + n] = v[c];
-          else if (a.mode == TG_SWIGLU) { if (((c & 1) == 0) == first) a.h_out[tok * N + n] = __float2bfloat16(v[c]); }
-          else if (mat == 0) a.q_out[tok * N + n] = __float2bfloat16(v[c]);
-          else {
-            int b = 0, pos = rw[c];
-            if (a.batch > 1) { b = pos / a.L; pos -= b * a.L; }
-            (mat == 1 ? a.kc : a.vc)[((size_t)b * a.max_seq + pos) * N + n] = __float2bfloat16(v[c]);
-          }
+          emit8(e, x1, x2, r1, (size_t)(tok0 + t), a.rowmap ? rows_s[t] : 0);
         }
       }
     }
@@ -454,26 +496,6 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
-  }
-}
-
-// finishes the K-split SWIGLU tiles: sums the splits in order, silu(gate) * up
-__global__ void __launch_bounds__(256) swiglu_tail_kernel(const float* part, size_t stride, int ld, int splits, const int* tot,
-                                                          int full_tiles, int rem_tiles, int F, bf16* h_out) {
-  const int t = blockIdx.x;
-  pdl_trigger();
-  pdl_wait();
-  if (t >= *tot) return;
-  for (int i = threadIdx.x; i < rem_tiles * 64; i += blockDim.x) {
-    const int tl = i >> 6, fr = i & 63;
-    const int f = (full_tiles + tl) * 64 + fr;
-    if (f >= F) continue;
-    float g = 0.f, u = 0.f;
-    for (int s = 0; s < splits; ++s) {
-      const float* row = part + (size_t)s * stride + (size_t)t * ld + tl * 128;
-      g += row[fr]; u += row[64 + fr];
-    }
-    h_out[(size_t)t * F + f] = __float2bfloat16(__fdividef(g, 1.f + __expf(-g)) * u);
   }
 }
 
@@ -560,28 +582,38 @@ int vlac_tc_setup(vlac_ctx* ctx) {
     else rc = encode_map(&act[TM_ACT_COUNT], ctx->w.proj, D, D, 128);
   }
   if (rc != VLAC_OK) { free(host); return rc; }
+  {
+    // workspace of the k-block-sharing launches: two slots per CTA and token chunk, and the per-tile counters
+    const size_t chunks = (size_t)(ctx->rows_max + TG_CHUNK - 1) / TG_CHUNK;
+    const size_t ws_floats = (size_t)ctx->n_sm * 2 * chunks * TG_SLOT_FLOATS;
+    const size_t tiles = (size_t)(3 * ((D + 127) / 128) > (F + 63) / 64 ? 3 * ((D + 127) / 128) : (F + 63) / 64);
+    cudaError_t e1 = cudaMalloc(&ctx->tc_ws, ws_floats * sizeof(float));
+    if (e1 == cudaSuccess) e1 = cudaMalloc(&ctx->tc_cnt, tiles * chunks * sizeof(int));
+    if (e1 == cudaSuccess) e1 = cudaMemset(ctx->tc_cnt, 0, tiles * chunks * sizeof(int));
+    if (e1 != cudaSuccess) { cudaGetLastError(); free(host); return e1 == cudaErrorMemoryAllocation ? VLAC_ERR_OOM : VLAC_ERR_CUDA; }
+  }
   ctx->tmaps_host = host;                                        // copied into the kernel parameters at every launch
-  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TG_SMEM_RING + 1024);
+  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TG_SMEM_DYN);
   if (e != cudaSuccess) { vlac_note_cuda_error(e, __FILE__, __LINE__); return VLAC_ERR_CUDA; }
   // a CTA holds up to 512 tokens (accumulator columns); more tokens are further chunks along grid.z
   return VLAC_OK;
 }
 
-// Tensor-memory columns a CTA needs for the largest token chunk it can meet (power of two >= 32).
+// Tensor-memory columns of the two accumulator buffers (each covers the largest token chunk; power of two >= 32).
 static int tc_tmem_cols(const vlac_ctx* ctx) {
-  const int chunk = ctx->rows_max < 512 ? ctx->rows_max : 512;
-  const int n0 = ((chunk < 256 ? chunk : 256) + 15) / 16 * 16;
-  const int n1 = chunk > 256 ? (chunk - 256 + 15) / 16 * 16 : 0;
-  const int need = n1 ? 256 + n1 : n0;
+  const int chunk = ((ctx->rows_max < TG_CHUNK ? ctx->rows_max : TG_CHUNK) + 15) / 16 * 16;
   int cols = 32;
-  while (cols < need) cols *= 2;
-  return cols;
+  while (cols < chunk) cols *= 2;
+  return 2 * cols;
 }
 
-static int launch_tc(vlac_ctx* ctx, TcArgs& a, int n_tiles, cudaStream_t s) {
-  const dim3 grid(n_tiles, a.n_splits, (ctx->rows_max + 511) / 512);
+// grid: one CTA per K-split of a tile (PARTIAL), else one per SM sharing all k-blocks evenly
+static int launch_tc(vlac_ctx* ctx, TcArgs& a, cudaStream_t s) {
+  const long long total = (long long)a.n_tiles * ((a.K + TG_BK - 1) / TG_BK);
+  int grid = a.mode == TG_PARTIAL ? a.n_tiles * a.n_splits : (int)(total < ctx->n_sm ? total : ctx->n_sm);
   a.tmem_cols = tc_tmem_cols(ctx);
-  VLAC_CUDA_CHECK(launch_pdl(gemm_tc_kernel, grid, dim3(TG_THREADS), (size_t)TG_SMEM_RING + 1024, s, a));
+  a.ws = ctx->tc_ws; a.tile_cnt = ctx->tc_cnt;
+  VLAC_CUDA_CHECK(launch_pdl(gemm_tc_kernel, dim3(grid), dim3(TG_THREADS), (size_t)TG_SMEM_DYN, s, a));
   VLAC_LAUNCH_CHECK(ctx);
   return VLAC_OK;
 }
@@ -598,6 +630,15 @@ static void tc_common(vlac_ctx* ctx, vlac_cache* c, int layer, TcArgs* a) {
   a->batch = c->batch;
 }
 
+static int tc_splits(const vlac_ctx* ctx, int tiles, int K) {
+  int splits = ctx->n_sm / tiles;                       // fill the SMs: the partial sums are folded by the next kernel
+  if (splits < 1) splits = 1;
+  if (splits > VLAC_MAX_SPLITS) splits = VLAC_MAX_SPLITS;
+  const int kb_total = (K + TG_BK - 1) / TG_BK;
+  if (splits > kb_total) splits = kb_total;
+  return splits;
+}
+
 int vlac_tc_qkv(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s) {
   const vlac_config& g = ctx->cfg;
   const CUtensorMap* tm = (const CUtensorMap*)ctx->tmaps_host + (size_t)layer * TM_PER_LAYER;
@@ -606,10 +647,11 @@ int vlac_tc_qkv(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s) {
   a.tm_a[0] = tm[TM_WQ]; a.tm_a[1] = tm[TM_WK]; a.tm_a[2] = tm[TM_WV];
   for (int i = 0; i < 4; ++i) a.tm_b[i] = act[TM_XN + i];
   a.K = g.hidden; a.N = g.hidden; a.mode = TG_QKV;
+  a.n_tiles = 3 * ((g.hidden + 127) / 128);
   a.q_out = ctx->q;
   a.kc = c->k + (size_t)layer * c->batch * kv_layer_elems(ctx);
   a.vc = c->v + (size_t)layer * c->batch * kv_layer_elems(ctx);
-  return launch_tc(ctx, a, 3 * ((g.hidden + 127) / 128), s);
+  return launch_tc(ctx, a, s);
 }
 
 int vlac_tc_partial(vlac_ctx* ctx, vlac_cache* c, int layer, int which, int* n_splits, cudaStream_t s) {
@@ -621,16 +663,11 @@ int vlac_tc_partial(vlac_ctx* ctx, vlac_cache* c, int layer, int which, int* n_s
   a.tm_a[0] = tm[down ? TM_DOWN : TM_WO];
   for (int i = 0; i < 4; ++i) a.tm_b[i] = act[(down ? TM_HM : TM_AO) + i];
   a.K = down ? g.ffn : g.hidden; a.N = g.hidden; a.mode = TG_PARTIAL;
-  const int tiles = (g.hidden + 127) / 128;
-  int splits = ctx->n_sm / tiles;                       // fill the SMs: the partial sums are folded by the next kernel
-  if (splits < 1) splits = 1;
-  if (splits > VLAC_MAX_SPLITS) splits = VLAC_MAX_SPLITS;
-  const int kb_total = (a.K + TG_BK - 1) / TG_BK;
-  if (splits > kb_total) splits = kb_total;
-  a.n_splits = splits;
+  a.n_tiles = (g.hidden + 127) / 128;
+  a.n_splits = tc_splits(ctx, a.n_tiles, a.K);
   a.part = ctx->part; a.split_stride = (size_t)ctx->rows_max * g.hidden;
-  *n_splits = splits;
-  return launch_tc(ctx, a, tiles, s);
+  *n_splits = a.n_splits;
+  return launch_tc(ctx, a, s);
 }
 
 // Vision projector (input rows of the vision positions): features [rows][D] x W_proj^T as K-split fp32
@@ -648,16 +685,11 @@ int vlac_tc_projector(vlac_ctx* ctx, vlac_cache* c, const void* feats, int rows,
     if (rc != VLAC_OK) return rc;
   }
   a.K = g.hidden; a.N = g.hidden; a.mode = TG_PARTIAL;
-  const int tiles = (g.hidden + 127) / 128;
-  int splits = ctx->n_sm / tiles;
-  if (splits < 1) splits = 1;
-  if (splits > VLAC_MAX_SPLITS) splits = VLAC_MAX_SPLITS;
-  const int kb_total = (a.K + TG_BK - 1) / TG_BK;
-  if (splits > kb_total) splits = kb_total;
-  a.n_splits = splits;
+  a.n_tiles = (g.hidden + 127) / 128;
+  a.n_splits = tc_splits(ctx, a.n_tiles, a.K);
   a.part = ctx->part; a.split_stride = (size_t)ctx->rows_max * g.hidden;
-  *n_splits = splits;
-  return launch_tc(ctx, a, tiles, s);
+  *n_splits = a.n_splits;
+  return launch_tc(ctx, a, s);
 }
 
 int vlac_tc_gateup(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s) {
@@ -668,25 +700,7 @@ int vlac_tc_gateup(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s) {
   a.tm_a[0] = tm[TM_GATE]; a.tm_a[1] = tm[TM_UP];
   for (int i = 0; i < 4; ++i) a.tm_b[i] = act[TM_XN + i];
   a.K = g.hidden; a.N = g.ffn; a.mode = TG_SWIGLU;
+  a.n_tiles = (g.ffn + 63) / 64;
   a.h_out = ctx->hm;
-  const int tiles = (g.ffn + 63) / 64;
-  // tiles beyond the last full wave: split along K so that the second, short wave fills every SM
-  int full = tiles >= ctx->n_sm ? (tiles / ctx->n_sm) * ctx->n_sm : tiles;
-  int rem = tiles - full, splits = 1;
-  if (rem > 0) {
-    splits = ctx->n_sm / rem;
-    const int kb_total = (a.K + TG_BK - 1) / TG_BK;
-    if (splits > kb_total) splits = kb_total;
-    if (splits > 8) splits = 8;
-    const size_t wide = (size_t)(3 * g.hidden > 2 * g.ffn ? 3 * g.hidden : 2 * g.ffn);     // floats per row of ctx->scratch
-    if (splits < 2 || (size_t)splits * rem * 128 > wide) { splits = 1; full = tiles; rem = 0; }
-  }
-  a.full_tiles = full; a.tail_splits = splits; a.tail_ld = rem * 128;
-  a.tail_part = ctx->scratch; a.tail_stride = (size_t)ctx->rows_max * rem * 128;
-  int rc = launch_tc(ctx, a, full + rem * splits, s);
-  if (rc || rem == 0) return rc;
-  VLAC_CUDA_CHECK(launch_pdl(swiglu_tail_kernel, dim3(ctx->rows_max), dim3(256), 0, s, (const float*)a.tail_part, a.tail_stride, a.tail_ld,
-                             splits, a.tot, full, rem, g.ffn, ctx->hm));
-  VLAC_LAUNCH_CHECK(ctx);
-  return VLAC_OK;
+  return launch_tc(ctx, a, s);
 }

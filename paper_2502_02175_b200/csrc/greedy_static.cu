@@ -18,9 +18,9 @@ static __device__ __align__(256) unsigned long long g_greedy_scratch[GS_MAX_ROWS
 
 namespace {
 
-// order-preserving key: larger logit wins, equal logits go to the lower id
+// order-preserving key: larger logit wins, equal logits go to the lower id (-0 counts as +0)
 __device__ __forceinline__ unsigned long long gs_key(float v, int idx) {
-  unsigned int u = __float_as_uint(v);
+  unsigned int u = __float_as_uint(v + 0.0f);
   u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
   return ((unsigned long long)u << 32) | (unsigned long long)(0xFFFFFFFFu - (unsigned int)idx);
 }
@@ -55,7 +55,9 @@ __global__ void gs_final_kernel(const unsigned long long* scratch, int* tokens) 
 }
 
 // The array's name means something only to device code; host code has to ask the runtime where the
-// array lives on the current device.  Done once per device and remembered.
+// array lives on the current device.  Done once per device ordinal and remembered for the life of the
+// process: the address belongs to the device's primary context, so a cudaDeviceReset (or a caller that
+// works in a context of its own making) invalidates what is remembered here.
 #define GS_MAX_DEVICES 64
 std::mutex g_gs_mutex;
 unsigned long long* g_gs_ptr[GS_MAX_DEVICES] = {nullptr};

@@ -47,7 +47,7 @@ int fill_params(const vlac_ctx* ctx, const vlac_select_params* in, int force_ful
 }
 
 void free_ctx_buffers(vlac_ctx* c) {
-  cudaFree(c->xn); cudaFree(c->q); cudaFree(c->ao); cudaFree(c->hm); cudaFree(c->part); cudaFree(c->scratch);
+  cudaFree(c->xn); cudaFree(c->q); cudaFree(c->ao); cudaFree(c->hm); cudaFree(c->part); cudaFree(c->tc_ws); cudaFree(c->tc_cnt);
   cudaFree(c->probs); cudaFree(c->hidden); cudaFree(c->x_dec); cudaFree(c->q_dec); cudaFree(c->ao_dec);
   cudaFree(c->hm_dec); cudaFree(c->logits); cudaFree(c->argmax_tmp); cudaFree(c->dev_error); cudaFree(c->tmap_q); cudaFree(c->probs_all); free(c->tmaps_host);
   cudaFree(c->in_frames); cudaFree(c->in_feats); cudaFree(c->in_ids); cudaFree(c->in_forced); cudaFree(c->out_tokens); cudaFree(c->logits_all);
@@ -128,14 +128,12 @@ int vlac_create(const vlac_config* cfg, const vlac_weights* w, vlac_ctx** out) {
   const size_t R = c->rows_max, D = g.hidden, F = g.ffn, B = g.max_batch;
   const size_t na8 = (size_t)(g.n_action < 8 ? g.n_action : 8);
   const size_t R1 = B > na8 ? B : na8;               // columns of the single-row kernels: sequences, or the rows of one action chunk
-  const size_t wide = (3 * D > 2 * F ? 3 * D : 2 * F);
   int rc = VLAC_OK;
   if (rc == VLAC_OK) rc = dev_alloc(&c->xn, R * D);
   if (rc == VLAC_OK) rc = dev_alloc(&c->q, R * D);
   if (rc == VLAC_OK) rc = dev_alloc(&c->ao, R * D);
   if (rc == VLAC_OK) rc = dev_alloc(&c->hm, R * F);
   if (rc == VLAC_OK) rc = dev_alloc(&c->part, (size_t)VLAC_MAX_SPLITS * R * D);
-  if (rc == VLAC_OK) rc = dev_alloc(&c->scratch, R * wide);
   if (rc == VLAC_OK) rc = dev_alloc(&c->hidden, R * D);
   if (rc == VLAC_OK) rc = dev_alloc(&c->x_dec, R1 * D);
   if (rc == VLAC_OK) rc = dev_alloc(&c->q_dec, R1 * D);
@@ -326,11 +324,10 @@ int vlac_layer_forward(vlac_ctx* ctx, vlac_cache* cache, int layer, void* hidden
   if (!ctx || !cache || cache->ctx != ctx || !hidden || layer < 0 || layer >= ctx->cfg.n_layers) return VLAC_ERR_INVALID_ARG;
   if (!cache->has_selection) return VLAC_ERR_BAD_STATE;
   cudaStream_t s = (cudaStream_t)stream;
-  bf16* h = (bf16*)hidden;
   int n_splits = 0;
-  TRY(vlac_launch_finalize_norm(ctx, cache, h, layer, 0, layer, ctx->layers[layer].g_attn, s));
-  TRY(vlac_launch_layer_body(ctx, cache, layer, h, &n_splits, s));
-  TRY(vlac_launch_finalize_norm(ctx, cache, h, layer, n_splits, layer, nullptr, s));
+  TRY(vlac_launch_finalize_norm(ctx, cache, hidden, 0, layer, 0, layer, ctx->layers[layer].g_attn, s));
+  TRY(vlac_launch_layer_body(ctx, cache, layer, hidden, 0, &n_splits, s));
+  TRY(vlac_launch_finalize_norm(ctx, cache, hidden, 0, layer, n_splits, layer, nullptr, s));
   return VLAC_OK;
 }
 
@@ -355,20 +352,20 @@ static int enqueue_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* f
   TRY(vlac_launch_select(ctx, cache, frames, p, s));
   TRY(seg_mark(ctx, s));
   // 2. rows entering layer 0
-  bf16* h = ctx->hidden;
+  float* h = ctx->hidden;
   TRY(vlac_launch_input_rows(ctx, cache, vision_feats, prompt_ids, h, s));
   TRY(seg_mark(ctx, s));
   // 3. layers; the down-projection partials of layer l are folded into layer l+1's first kernel
   int n_splits = 0;
   ctx->defer_emit = ctx->probs_all != nullptr;
   for (int l = 0; l < nl; ++l) {
-    int rc = vlac_launch_finalize_norm(ctx, cache, h, l == 0 ? 0 : l - 1, l == 0 ? 0 : n_splits, l, ctx->layers[l].g_attn, s);
-    if (rc == VLAC_OK) rc = vlac_launch_layer_body(ctx, cache, l, h, &n_splits, s);
+    int rc = vlac_launch_finalize_norm(ctx, cache, h, 1, l == 0 ? 0 : l - 1, l == 0 ? 0 : n_splits, l, ctx->layers[l].g_attn, s);
+    if (rc == VLAC_OK) rc = vlac_launch_layer_body(ctx, cache, l, h, 1, &n_splits, s);
     if (rc != VLAC_OK) { ctx->defer_emit = 0; return rc; }
   }
   const bool deferred = ctx->defer_emit != 0;
   ctx->defer_emit = 0;
-  TRY(vlac_launch_finalize_norm(ctx, cache, h, nl - 1, n_splits, nl - 1, nullptr, s));
+  TRY(vlac_launch_finalize_norm(ctx, cache, h, 1, nl - 1, n_splits, nl - 1, nullptr, s));
   if (deferred) TRY(vlac_launch_emit_all(ctx, cache, s));
   TRY(seg_mark(ctx, s));
   if (act_embed) {

@@ -51,9 +51,10 @@ struct vlac_ctx {
   // workspace (device)
   bf16 *xn, *q, *ao, *hm;            // [rows_max][hidden] x3, [rows_max][ffn]
   float *part;                       // [VLAC_MAX_SPLITS][rows_max][hidden]
-  float *scratch;                    // [rows_max][max(3*hidden, 2*ffn)]   raw gate/up sums of the K-split tail tiles
+  float *tc_ws;                      // [n_sm][2][token chunks][256][128] raw sums of tile segments that cover part of K
+  int *tc_cnt;                       // [tiles][token chunks] k-blocks accumulated per tile (zero between launches)
   float *probs;                      // [max_batch][tiles][n_heads][Lv]: per-tile column sums of one layer (vlac_layer_forward)
-  bf16 *hidden;                      // [max_batch][L][hidden]            (used by step)
+  float *hidden;                     // [max_batch][L][hidden] fp32 residual stream of a whole step
   // single-row buffers: one row per column of the matrix-vector kernels, R1 = max(max_batch, min(n_action, 8))
   float *x_dec;                      // [R1][hidden]
   bf16 *q_dec, *ao_dec, *hm_dec;     // [R1][hidden] x2, [R1][ffn]
@@ -110,14 +111,14 @@ int vlac_launch_select(vlac_ctx* ctx, vlac_cache* c, const unsigned char* frames
 int vlac_launch_flatten(vlac_ctx* ctx, vlac_cache* c, cudaStream_t s);
 
 // ---- prefill (prefill_kernels.cu)
-int vlac_launch_input_rows(vlac_ctx* ctx, vlac_cache* c, const void* feats, const int* ids, bf16* hidden, cudaStream_t s);
+int vlac_launch_input_rows(vlac_ctx* ctx, vlac_cache* c, const void* feats, const int* ids, float* hidden, cudaStream_t s);
 // If n_splits > 0: hidden[row] += sum of split-K partials, for the rows of layer l_prev.
 // If gain != NULL: RMSNorm the rows of layer l_next (after the update) into ctx->xn.
-int vlac_launch_finalize_norm(vlac_ctx* ctx, vlac_cache* c, bf16* hidden, int l_prev, int n_splits,
+int vlac_launch_finalize_norm(vlac_ctx* ctx, vlac_cache* c, void* hidden, int hidden_f32, int l_prev, int n_splits,
                               int l_next, const void* gain, cudaStream_t s);
 // Everything of layer `layer` between its first RMSNorm (already in ctx->xn) and the down-projection
 // partials (left in ctx->part); returns the number of partials in *n_splits.
-int vlac_launch_layer_body(vlac_ctx* ctx, vlac_cache* c, int layer, bf16* hidden, int* n_splits, cudaStream_t s);
+int vlac_launch_layer_body(vlac_ctx* ctx, vlac_cache* c, int layer, void* hidden, int hidden_f32, int* n_splits, cudaStream_t s);
 
 // ---- tensor-memory GEMM (gemm_tc.cu)
 int vlac_tc_setup(vlac_ctx* ctx);
@@ -136,7 +137,7 @@ int vlac_launch_emit_all(vlac_ctx* ctx, vlac_cache* c, cudaStream_t s);   // aft
 
 // ---- decode (decode_kernels.cu)
 int vlac_decode_setup(vlac_ctx* ctx);
-int vlac_launch_last_row(vlac_ctx* ctx, vlac_cache* c, const bf16* hidden, cudaStream_t s);
+int vlac_launch_last_row(vlac_ctx* ctx, vlac_cache* c, const float* hidden, cudaStream_t s);
 int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens, int tok_stride, int tok_index,
                             int pos, cudaStream_t s);
 int vlac_launch_logits_argmax(vlac_ctx* ctx, vlac_cache* c, int* tokens_out, int tok_stride, int tok_index,

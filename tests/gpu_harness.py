@@ -2,7 +2,13 @@
 seeded inputs and compare them.
 
 Index sets must agree bit for bit; floating-point outputs within ``TOL`` = 2e-2 of the largest
-reference magnitude (bf16 storage of hidden states, K/V and weights bounds the error well below it).
+reference magnitude, against the checker in exact arithmetic (``OPERANDS`` = "exact").  That bound holds
+for the shallow models of most tests.  Through 32 layers two computations that both round their
+matrix-product operands to bf16 drift apart by more than 2e-2, however faithful each is (a difference
+far below one bf16 unit in a value that is about to be rounded moves the result by a whole unit with
+the matching probability, so differences do not stay small); the 32-layer test therefore measures, on
+the CPU alone, how far the checker's own bf16-operand setting is from its exact setting and scales its
+tolerance by that figure.
 """
 from __future__ import annotations
 
@@ -14,6 +20,7 @@ from paper_2502_02175_b200 import binding as vb
 from paper_2502_02175_b200 import synth
 
 TOL = 2e-2
+OPERANDS = "exact"
 
 
 def rel_err(got: np.ndarray, ref: np.ndarray) -> float:
@@ -101,19 +108,7 @@ def check_selection(got: dict, sel: orc.Selection, seq: int, cfg, where=""):
 
 def host_model_from_device(dev, cfg) -> dict:
     """Bit copy of a ``DeviceModel``'s tensors into the dictionary layout of ``synth.make_model``."""
-    by_ptr = {t.data_ptr(): t for t in dev.tensors}
-
-    def bits(ptr):
-        t = by_ptr[ptr]
-        if t.dtype == torch.bfloat16:
-            return t.view(torch.int16).cpu().numpy().view(np.uint16)
-        return t.cpu().numpy()
-
-    model = {"layers": [{name: bits(getattr(dev.layer_structs[l], name)) for name, _ in vb.vlac_layer_w._fields_}
-                        for l in range(cfg.n_layers)]}
-    for name in ("embed", "proj", "g_final", "lm_head", "rope_cos", "rope_sin"):
-        model[name] = bits(getattr(dev.weights, name))
-    return model
+    return dev.to_host(cfg)
 
 
 def run_step_pair(sess: Session, frames: np.ndarray, feats: np.ndarray, ids: np.ndarray, params: orc.SelectParams,
@@ -162,21 +157,29 @@ def run_step_pair(sess: Session, frames: np.ndarray, feats: np.ndarray, ids: np.
         if act_embed is None and layer_major:
             import oracle_compose
             res = oracle_compose.step_layer_major(cfg, sess.model, oc, frames[b], feats[b], ids[b], params,
-                                                  forced_tokens=g_tokens[b], force_full=force_full, selection=sel)
+                                                  forced_tokens=g_tokens[b], force_full=force_full, selection=sel, operands=OPERANDS)
         elif act_embed is None:
             res = orc.step(cfg, sess.model, oc, frames[b], feats[b], ids[b], params, force_full,
-                           forced_tokens=g_tokens[b], selection=sel)
+                           forced_tokens=g_tokens[b], selection=sel, operands=OPERANDS)
         else:
             res = orc.step_chunk(cfg, sess.model, oc, frames[b], feats[b], ids[b], params, act_embed, force_full,
-                                 selection=sel)
+                                 selection=sel, operands=OPERANDS)
         err = max(rel_err(g_logits[b, i], res.logits[i]) for i in range(cfg.n_action))
         abs_err = float(np.max(np.abs(g_logits[b] - res.logits)))
-        guarded = 0
+        # Tokens: identical wherever the checker's top-2 margin exceeds twice the measured logit error.  Below that
+        # margin ("guarded") the two may differ, but only as a near-tie: the library's token must then score within
+        # the same bound of the checker's best logit ("flipped").  Both counts are reported; the tests bound them.
+        guarded = flipped = 0
         for i in range(cfg.n_action):
+            same = int(g_tokens[b, i]) == int(res.tokens[i])
             if res.margins[i] > 2.0 * abs_err:
-                assert int(g_tokens[b, i]) == int(res.tokens[i]), f"seq {b} token {i}"
+                assert same, f"seq {b} token {i}: {int(g_tokens[b, i])} != {int(res.tokens[i])} at margin {res.margins[i]:.3g}"
             else:
                 guarded += 1
+                if not same:
+                    flipped += 1
+                    gap = float(res.logits[i].max() - res.logits[i][int(g_tokens[b, i])])
+                    assert gap <= 2.0 * abs_err, f"seq {b} token {i}: the library's token is {gap:.3g} below the best logit"
         g_attn = sess.read_attn(vb.PART_ATTN_PREV, b)
         attn_err = rel_err(g_attn, res.attn_tv)
         attn_err_layers = [rel_err(g_attn[l], res.attn_tv[l]) for l in range(cfg.n_layers)]
@@ -186,8 +189,8 @@ def run_step_pair(sess: Session, frames: np.ndarray, feats: np.ndarray, ids: np.
             for l in range(cfg.n_layers):
                 kv_err = max(kv_err, rel_err(sess.read_kv(vb.PART_K, l, b)[L:L + n], oc.K[l][L:L + n]),
                              rel_err(sess.read_kv(vb.PART_V, l, b)[L:L + n], oc.V[l][L:L + n]))
-        out.append({"logit_err": err, "abs_err": abs_err, "guarded": guarded, "attn_err": attn_err, "attn_err_layers": attn_err_layers, "kv_err": kv_err,
+        out.append({"logit_err": err, "abs_err": abs_err, "guarded": guarded, "flipped": flipped, "attn_err": attn_err, "attn_err_layers": attn_err_layers, "kv_err": kv_err,
                     "logit_err_rows": [rel_err(g_logits[b, i], res.logits[i]) for i in range(cfg.n_action)],
-                    "margins": res.margins.copy(), "ref_tokens": res.tokens.copy(),
+                    "margins": res.margins.copy(), "ref_tokens": res.tokens.copy(), "ref_logits": res.logits, "got_logits": g_logits[b],
                     "M": sel.M.copy(), "tokens": g_tokens[b].copy(), "selection": sel})
     return out

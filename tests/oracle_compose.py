@@ -17,7 +17,7 @@ from oracle import vla_cache_oracle as orc
 
 
 def step_layer_major(cfg, model, cache, frames_t, feats_bf16, prompt_ids, params, forced_tokens,
-                     force_full=False, selection=None) -> orc.StepResult:
+                     force_full=False, selection=None, operands="exact") -> orc.StepResult:
     sel = selection if selection is not None else orc.select(cfg, frames_t, cache, params, force_full)
     cos, sin = model["rope_cos"], model["rope_sin"]
     hidden = orc.input_rows(cfg, model, feats_bf16, prompt_ids)
@@ -28,14 +28,14 @@ def step_layer_major(cfg, model, cache, frames_t, feats_bf16, prompt_ids, params
     attn_next = np.zeros((cfg.n_layers, cfg.n_heads, cfg.n_vision), dtype=np.float64)
     for l in range(cfg.n_layers):
         lw, K, V = model["layers"][l], cache.K[l], cache.V[l]
-        attn_next[l] = orc.layer_forward(cfg, lw, K, V, hidden, sel.rows[l], cos, sin, emit_attention=True)
+        attn_next[l] = orc.layer_forward(cfg, lw, K, V, hidden, sel.rows[l], cos, sin, emit_attention=True, operands=operands)
         for i in range(1, n):
-            orc.layer_forward(cfg, lw, K, V, hidden, np.asarray([L - 1 + i]), cos, sin, emit_attention=False)
+            orc.layer_forward(cfg, lw, K, V, hidden, np.asarray([L - 1 + i]), cos, sin, emit_attention=False, operands=operands)
     tokens = np.zeros(n, dtype=np.int64)
     logits = np.zeros((n, cfg.vocab), dtype=np.float64)
     margins = np.zeros(n, dtype=np.float64)
     for i in range(n):
-        logits[i] = orc._logits(cfg, model, hidden[L - 1 + i])
+        logits[i] = orc._logits(cfg, model, hidden[L - 1 + i], operands)
         tokens[i] = int(np.argmax(logits[i]))
         top2 = np.partition(logits[i], -2)[-2:]
         margins[i] = float(top2[1] - top2[0])

@@ -65,21 +65,26 @@ def _torch_rope(x, cos, sin):
     return x * c + rot * s
 
 
-def _torch_layer(cfg, lw, h, cos, sin, mask=None):
-    """Textbook Llama layer over a full sequence in fp64: causal, or with a boolean mask [L, L]."""
+def _torch_layer(cfg, lw, h, cos, sin, mask=None, rb=lambda t: t):
+    """Textbook Llama layer over a full sequence in fp64: causal, or with a boolean mask [L, L].  ``rb`` is applied to
+    every operand of a matrix product other than the weights (identity, or a rounding to bf16 by torch)."""
     L, H, d = h.shape[0], cfg.n_heads, cfg.head_dim
     F = torch.nn.functional
-    xn = F.rms_norm(h, (cfg.hidden,), _t(lw["g_attn"]), cfg.rms_eps)
-    q = _torch_rope(F.linear(xn, _t(lw["wq"])).view(L, H, d), cos, sin)
-    k = _torch_rope(F.linear(xn, _t(lw["wk"])).view(L, H, d), cos, sin)
-    v = F.linear(xn, _t(lw["wv"])).view(L, H, d)
-    if mask is None:
+    xn = rb(F.rms_norm(h, (cfg.hidden,), _t(lw["g_attn"]), cfg.rms_eps))
+    q = rb(_torch_rope(F.linear(xn, _t(lw["wq"])).view(L, H, d), cos, sin))
+    k = rb(_torch_rope(F.linear(xn, _t(lw["wk"])).view(L, H, d), cos, sin))
+    v = rb(F.linear(xn, _t(lw["wv"])).view(L, H, d))
+    if mask is None and rb(torch.tensor([1.0 + 2.0 ** -12], dtype=torch.float64)).item() != 1.0:
         o = F.scaled_dot_product_attention(q.transpose(0, 1), k.transpose(0, 1), v.transpose(0, 1), is_causal=True)
-    else:
+    elif mask is not None:
         o = F.scaled_dot_product_attention(q.transpose(0, 1), k.transpose(0, 1), v.transpose(0, 1), attn_mask=mask)
-    h = h + F.linear(o.transpose(0, 1).reshape(L, H * d), _t(lw["wo"]))
-    xn = F.rms_norm(h, (cfg.hidden,), _t(lw["g_mlp"]), cfg.rms_eps)
-    return h + F.linear(F.silu(F.linear(xn, _t(lw["w_gate"]))) * F.linear(xn, _t(lw["w_up"])), _t(lw["w_down"])), k, v
+    else:       # rounded probabilities: the softmax has to be written out
+        sc = torch.einsum("qhd,khd->hqk", q, k) / math.sqrt(d)
+        sc = sc.masked_fill(~torch.tril(torch.ones(L, L, dtype=torch.bool)), float("-inf"))
+        o = torch.einsum("hqk,khd->hqd", rb(torch.softmax(sc, dim=-1)), v)
+    h = h + F.linear(rb(o.transpose(0, 1).reshape(L, H * d)), _t(lw["wo"]))
+    xn = rb(F.rms_norm(h, (cfg.hidden,), _t(lw["g_mlp"]), cfg.rms_eps))
+    return h + F.linear(rb(F.silu(F.linear(xn, _t(lw["w_gate"]))) * F.linear(xn, _t(lw["w_up"]))), _t(lw["w_down"])), k, v
 
 
 def test_full_prefill_equals_textbook_layer():
@@ -343,3 +348,59 @@ def test_layer_major_composition_equals_step():
         assert np.array_equal(ra.attn_tv, rb.attn_tv) and np.array_equal(ra.hidden, rb.hidden)
         assert np.array_equal(ca.K, cb.K) and np.array_equal(ca.V, cb.V)
     assert ra.selection.M[1] < cfg.seq_len
+
+
+
+def _torch_bf16(t):
+    return t.to(torch.bfloat16).double()
+
+
+def test_round_bf16_matches_torch_conversion():
+    rng = np.random.default_rng(1)
+    x = np.concatenate([rng.standard_normal(20000) * 10.0 ** rng.integers(-30, 30, size=20000),
+                        np.array([0.0, -0.0, 1.0, 1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -9, -(1.0 + 2.0 ** -8),
+                                  2.0 ** -133, 2.0 ** -134, 3.0e38, 3.4e38, np.inf, -np.inf])])
+    got = orc.round_bf16(x)
+    want = torch.from_numpy(x).to(torch.bfloat16).double().numpy()
+    assert np.array_equal(got, want) and np.array_equal(np.signbit(got), np.signbit(want))
+    assert got[20003] == 1.0 and got[20004] == 1.0 + 2.0 ** -6           # ties go to the even mantissa
+
+
+def test_bf16_operand_setting_equals_torch_layer_with_torch_roundings():
+    """operands="bf16": the same textbook layer, every matrix-product operand rounded by torch's own bf16 conversion."""
+    cfg, model, ids, feats = _tiny(6)
+    L = cfg.seq_len
+    h0 = orc.input_rows(cfg, model, feats, ids)
+    cos, sin = torch.from_numpy(model["rope_cos"][:L]).double(), torch.from_numpy(model["rope_sin"][:L]).double()
+    K = np.zeros((cfg.max_seq, cfg.n_heads, cfg.head_dim)); V = np.zeros_like(K)
+    hid = h0.copy()
+    orc.layer_forward(cfg, model["layers"][0], K, V, hid, np.arange(L), model["rope_cos"], model["rope_sin"], operands="bf16")
+    want, k, v = _torch_layer(cfg, model["layers"][0], torch.from_numpy(h0[:L]), cos, sin, rb=_torch_bf16)
+    np.testing.assert_allclose(hid[:L], want.numpy(), rtol=0, atol=2e-3 * np.abs(want.numpy()).max())   # a rounding may flip where fp64 sums differ in the last bit
+    assert np.median(np.abs(hid[:L] - want.numpy())) <= 1e-9 * np.abs(want.numpy()).max()
+    assert np.array_equal(K[:L], orc.round_bf16(K[:L])) and np.array_equal(V[:L], orc.round_bf16(V[:L]))      # stored as bf16 values
+    np.testing.assert_allclose(K[:L], k.numpy(), rtol=0, atol=2.0 ** -7 * np.abs(k.numpy()).max())
+    # and the exact setting is a different function of the same inputs
+    hid_x = h0.copy()
+    Kx = np.zeros_like(K); Vx = np.zeros_like(V)
+    orc.layer_forward(cfg, model["layers"][0], Kx, Vx, hid_x, np.arange(L), model["rope_cos"], model["rope_sin"])
+    d = np.abs(hid_x[:L] - hid[:L]).max() / np.abs(hid_x[:L]).max()
+    assert 1e-4 < d < 2e-2
+
+
+def test_cost_of_bf16_operands_on_the_tiny_decoder():
+    """Distance between the checker's two settings on the tiny decoder stacked to 2 and 8 layers: a bf16 computation
+    is a different function from exact arithmetic, by a few 1e-3 of the largest logit at this width.  (On the 32-layer
+    7B shape the same distance is measured in tests/test_gpu_parity.py, where the host is fast enough.)"""
+    cfg8 = synth.tiny_config().with_layers(8)
+    model = synth.make_model(cfg8, 9)
+    ids = synth.make_prompt_ids(cfg8, 9)[0]
+    feats = synth.f32_to_bf16(np.random.default_rng(10).standard_normal((cfg8.n_vision, cfg8.hidden), dtype=np.float32))
+    frame = synth.rerandomised_pair(cfg8, 9, 0)[0]
+    for nl in (2, 8):
+        cfg = cfg8.with_layers(nl)
+        m = dict(model, layers=model["layers"][:nl])
+        ra = orc.step(cfg, m, orc.new_cache(cfg), frame, feats, ids, orc.SelectParams())
+        rb = orc.step(cfg, m, orc.new_cache(cfg), frame, feats, ids, orc.SelectParams(), forced_tokens=ra.tokens, operands="bf16")
+        dist = max(float(np.abs(rb.logits[i] - ra.logits[i]).max() / np.abs(ra.logits[i]).max()) for i in range(cfg.n_action))
+        assert 1e-4 < dist < 2e-2, (nl, dist)

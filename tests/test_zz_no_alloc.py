@@ -48,6 +48,27 @@ def test_static_greedy_tokens_match_step_tokens_twice():
         vb.vlac_greedy_tokens_static(x[:, :60], got)
         torch.cuda.synchronize()
         assert got.tolist() == [7, 0, 0]
+        # -0.0 and +0.0 are equal: the lower index wins
+        z = torch.full((1, 16), -1.0, dtype=torch.float32, device="cuda")
+        z[0, 3] = -0.0
+        z[0, 9] = 0.0
+        got1 = torch.zeros(1, dtype=torch.int32, device="cuda")
+        vb.vlac_greedy_tokens_static(z, got1)
+        torch.cuda.synchronize()
+        assert got1.tolist() == [3]
+        # nothing is allocated: the free device memory is the same before and after a (warmed-up) call
+        torch.cuda.synchronize()
+        free0, _ = torch.cuda.mem_get_info()
+        vb.vlac_greedy_tokens_static(x[:, :60], got)
+        torch.cuda.synchronize()
+        free1, _ = torch.cuda.mem_get_info()
+        assert free1 == free0
+        # bad arguments are refused before anything is launched
+        import ctypes as C
+        assert vb.lib.vlac_greedy_tokens_static(None, 1, 8, 8, got.data_ptr(), None) == -1
+        assert vb.lib.vlac_greedy_tokens_static(x.data_ptr(), 1, 8, 8, None, None) == -1
+        assert vb.lib.vlac_greedy_tokens_static(x.data_ptr(), 1, 100, 60, got.data_ptr(), None) == -1      # row_stride < vocab
+        assert vb.lib.vlac_greedy_tokens_static(x.data_ptr(), 0, 8, 8, got.data_ptr(), None) == -1
         # capacity is enforced with its own error code and nothing runs
         big = torch.zeros((65, 8), dtype=torch.float32, device="cuda")
         out = torch.zeros(65, dtype=torch.int32, device="cuda")
