@@ -48,13 +48,13 @@ constexpr int TG_BK = 64;                       // bf16 elements per k-block = o
 constexpr int TG_A_BYTES = 128 * TG_BK * 2;     // 16 KB: 128 weight rows
 constexpr int TG_BOX_TOK = 64;                  // token rows per TMA box
 constexpr int TG_BOX_BYTES = TG_BOX_TOK * TG_BK * 2;   // 8 KB
-constexpr int TG_CHUNK = 256;                   // most tokens one accumulator buffer holds
+constexpr int TG_CHUNK = 256;                   // most tokens of a chunk while two accumulator buffers alternate
+constexpr int TG_CHUNK_MAX = 512;               // ... and with one buffer (more than 256 live tokens): all 512 tensor-memory columns
 constexpr int TG_MAX_STAGES = 8;
 constexpr int TG_SMEM_RING = 192 * 1024;        // ring: four stages of 48 KB at 256 tokens
 constexpr int TG_STAGE_OUT = 8192;              // one 16-token chunk of a tile as fp32
 constexpr int TG_SMEM_OUT = 4 * TG_STAGE_OUT;   // [team][double buffer]
 constexpr int TG_SMEM_DYN = TG_SMEM_RING + TG_SMEM_OUT;    // with the static part this is all of an SM's 227 KB
-constexpr int TG_SLOT_FLOATS = TG_CHUNK * 128;  // one workspace slot: raw sums of one segment and token chunk
 constexpr unsigned long long TG_WAIT_LIMIT_NS = 400000000ull;
 
 struct alignas(64) TcArgs {
@@ -240,7 +240,8 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
   __shared__ __align__(8) unsigned long long full_bar[TG_MAX_STAGES], empty_bar[TG_MAX_STAGES], acc_full[2], acc_empty[2];
   __shared__ unsigned tmem_base_slot;
   __shared__ int abort_flag, fold_flag;
-  __shared__ int rows_buf[2][TG_CHUNK];                          // rowmap entries of the token chunk the epilogue works on (by item parity)
+  __shared__ int rows_buf[2][TG_CHUNK];                          // rowmap entries of the token chunk the epilogue works on (by item parity;
+                                                                 // one 512-entry array when a single accumulator buffer is in use)
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // the ring must start on a 1024-byte boundary (swizzle atoms): the declared alignment makes the compiler pad the
   // static part; checked below, since a misplaced ring would corrupt results silently
@@ -266,7 +267,11 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
   // is complete before any kernel launched after them starts: it is read ahead of the dependency wait (to size the
   // early weight loads) and checked again behind it.
   const int T = a.tot ? *a.tot : a.tot_fixed;
-  const int n_chunks = (T + TG_CHUNK - 1) / TG_CHUNK;
+  // Up to 256 live tokens: one chunk, two accumulator buffers, the epilogue of a segment overlaps the next one's MMAs.
+  // More: chunks of up to 512 tokens in one buffer (half as many passes over the weights as 256-token chunks need).
+  const int cap = T <= TG_CHUNK ? TG_CHUNK : TG_CHUNK_MAX;
+  const int n_bufs = T <= TG_CHUNK ? 2 : 1;
+  const int n_chunks = (T + cap - 1) / cap;
   const int chunk_sz = n_chunks > 0 ? (((T + n_chunks - 1) / n_chunks + 15) / 16) * 16 : 0;     // tokens of every chunk but the last
   const int max_boxes = (chunk_sz + TG_BOX_TOK - 1) / TG_BOX_TOK;
   const int stage_bytes = TG_A_BYTES + max_boxes * TG_BOX_BYTES;
@@ -330,7 +335,8 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   if (abort_flag) rg.u1 = rg.u0;                                // uniform: written before the barrier
   const unsigned tmem_base = tmem_base_slot;
-  const unsigned buf_cols = tmem_cols >> 1;                      // columns of one accumulator buffer
+  const unsigned buf_cols = tmem_cols >> 1;                      // columns of one accumulator buffer when two are in use
+  const size_t slot_floats = (size_t)cap * 128;                  // one workspace slot: raw sums of one segment and token chunk
 
   if (warp == 0 || warp == 2 || warp == 3) {
     // ------------------------------------------------------------------ TMA producers
@@ -353,7 +359,10 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
               mbar_expect_tx(&full_bar[s], (unsigned)TG_A_BYTES + x_bytes);
               load_weights(sg.tile, kb, s);
             }
-            tma_load_2d(ring + (size_t)s * stage_bytes + TG_A_BYTES, &a.tm_b[boxes - 1], kb * TG_BK, ch * chunk_sz, &full_bar[s]);
+            unsigned char* sb = ring + (size_t)s * stage_bytes + TG_A_BYTES;
+            const int rows0 = min(boxes, 4), rows1 = boxes - rows0;     // boxes of the first / second request
+            tma_load_2d(sb, &a.tm_b[rows0 - 1], kb * TG_BK, ch * chunk_sz, &full_bar[s]);
+            if (rows1 > 0) tma_load_2d(sb + 4 * TG_BOX_BYTES, &a.tm_b[rows1 - 1], kb * TG_BK, ch * chunk_sz + 256, &full_bar[s]);
           }
         }
     }
@@ -363,25 +372,48 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
       long long u = rg.u0; Seg sg; int it = 0, item = 0; bool ok = true;
       while (ok && next_seg(u, rg, kbt, sg))
         for (int ch = 0; ch < n_chunks && ok; ++ch, ++item) {
-          const int b = item & 1, use = item >> 1;
+          const int b = n_bufs == 2 ? item & 1 : 0, use = n_bufs == 2 ? item >> 1 : item;
           if (use > 0) ok = mbar_wait(&acc_empty[b], (use - 1) & 1, &abort_flag, a.dev_error, 0x58000 | (item & 0x7fff));
           if (!ok) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const unsigned idesc = umma_idesc_bf16(128, ((chunk_tokens(ch) + 15) / 16) * 16);
+          const int ncols = ((chunk_tokens(ch) + 15) / 16) * 16;
+          const unsigned idesc0 = umma_idesc_bf16(128, min(ncols, 256));
+          const unsigned idesc1 = ncols > 256 ? umma_idesc_bf16(128, ncols - 256) : 0u;
           const unsigned acc_addr = tmem_base + (unsigned)b * buf_cols;
-          for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
-            const int s = it % n_stages;
-            ok = mbar_wait(&full_bar[s], (it / n_stages) & 1, &abort_flag, a.dev_error, 0x50000 | (it & 0x7fff));
-            if (!ok) break;
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const unsigned char* sa = ring + (size_t)s * stage_bytes;
-            const unsigned long long da = umma_desc(sa), db = umma_desc(sa + TG_A_BYTES);
+          if (idesc1 == 0u) {
+            // up to 256 tokens: the loop the step spends its prefill in, kept free of anything it does not need
+            for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
+              const int s = it % n_stages;
+              ok = mbar_wait(&full_bar[s], (it / n_stages) & 1, &abort_flag, a.dev_error, 0x50000 | (it & 0x7fff));
+              if (!ok) break;
+              asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+              const unsigned char* sa = ring + (size_t)s * stage_bytes;
+              const unsigned long long da = umma_desc(sa), db = umma_desc(sa + TG_A_BYTES);
 #pragma unroll
-            for (int k = 0; k < TG_BK / 16; ++k) {
-              const unsigned long long koff = (unsigned long long)((k * 32) >> 4);        // 16 bf16 = 32 bytes along the swizzle row
-              umma_bf16(acc_addr, da + koff, db + koff, idesc, (kb > sg.kb0 || k > 0) ? 1u : 0u);
+              for (int k = 0; k < TG_BK / 16; ++k) {
+                const unsigned long long koff = (unsigned long long)((k * 32) >> 4);        // 16 bf16 = 32 bytes along the swizzle row
+                umma_bf16(acc_addr, da + koff, db + koff, idesc0, (kb > sg.kb0 || k > 0) ? 1u : 0u);
+              }
+              umma_commit(&empty_bar[s]);                          // stage reusable once these MMAs have read it
             }
-            umma_commit(&empty_bar[s]);                          // stage reusable once these MMAs have read it
+          } else {
+            // 257..512 tokens: a second MMA per k-step fills columns 256.. of the one accumulator buffer
+            for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
+              const int s = it % n_stages;
+              ok = mbar_wait(&full_bar[s], (it / n_stages) & 1, &abort_flag, a.dev_error, 0x50000 | (it & 0x7fff));
+              if (!ok) break;
+              asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+              const unsigned char* sa = ring + (size_t)s * stage_bytes;
+              const unsigned long long da = umma_desc(sa), db0 = umma_desc(sa + TG_A_BYTES), db1 = umma_desc(sa + TG_A_BYTES + 256 * 128);
+#pragma unroll
+              for (int k = 0; k < TG_BK / 16; ++k) {
+                const unsigned long long koff = (unsigned long long)((k * 32) >> 4);
+                const unsigned acc = (kb > sg.kb0 || k > 0) ? 1u : 0u;
+                umma_bf16(acc_addr, da + koff, db0 + koff, idesc0, acc);
+                umma_bf16(acc_addr + 256, da + koff, db1 + koff, idesc1, acc);
+              }
+              umma_commit(&empty_bar[s]);
+            }
           }
           if (ok) umma_commit(&acc_full[b]);                     // accumulator of this segment and chunk complete
         }
@@ -408,16 +440,18 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
       e.mat = tile_mat(sg.tile); e.row_base = tile_row_base(sg.tile);
       const int split = a.mode == TG_PARTIAL ? (int)blockIdx.x % a.n_splits : 0;
       for (int ch = 0; ch < n_chunks && ok; ++ch, ++item) {
-        const int b = item & 1, use = item >> 1;
+        const int b = n_bufs == 2 ? item & 1 : 0, use = n_bufs == 2 ? item >> 1 : item;
         const int tok0 = ch * chunk_sz, tokens = chunk_tokens(ch);
-        int* rows_s = rows_buf[item & 1];
-        if (et < tokens && a.rowmap) rows_s[et] = __ldg(a.rowmap + tok0 + et);
+        int* rows_s = n_bufs == 2 ? rows_buf[item & 1] : rows_buf[0];
+        if (n_bufs == 1 && item > 0) epi_all_ok(true);             // one row list: not rewritten while a thread may still read it
+        if (a.rowmap)
+          for (int i = et; i < tokens; i += TG_EPI_THREADS) rows_s[i] = __ldg(a.rowmap + tok0 + i);
         ok = mbar_wait(&acc_full[b], use & 1, &abort_flag, a.dev_error, 0x60000 | (item & 0xffff));
         ok = epi_all_ok(ok);                                      // same decision in all epilogue threads; rows_s visible
         if (!ok) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const unsigned acc_addr = tmem_base + (unsigned)b * buf_cols + ((unsigned)(32 * q) << 16);
-        float* ws_slot = a.ws ? a.ws + ((size_t)(blockIdx.x * 2 + (sg.first ? 0 : 1)) * n_chunks + ch) * TG_SLOT_FLOATS : nullptr;
+        float* ws_slot = a.ws ? a.ws + ((size_t)(blockIdx.x * 2 + (sg.first ? 0 : 1)) * n_chunks + ch) * slot_floats : nullptr;
         for (int c0 = team * 16; c0 < tokens; c0 += 32, ++cb) {
           // ---- phase A: 16 tokens of this thread's tile row -> shared memory, transposed to [token][row]
           float v[16];
@@ -481,7 +515,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
           for (int i = 0; i < 8; ++i) x1[i] = x2[i] = 0.f;
           for (int c = c_first; c < G && range_begin(total, c, G) < hi; ++c) {
             const int which = range_begin(total, c, G) >= lo ? 0 : 1;
-            const float* src = a.ws + ((size_t)(c * 2 + which) * n_chunks + ch) * TG_SLOT_FLOATS + (size_t)t * 128;
+            const float* src = a.ws + ((size_t)(c * 2 + which) * n_chunks + ch) * slot_floats + (size_t)t * 128;
             const float4 p0 = ldcg_f4(src + r1), p1 = ldcg_f4(src + r1 + 4), p2 = ldcg_f4(src + r1 + e.half), p3 = ldcg_f4(src + r1 + e.half + 4);
             x1[0] += p0.x; x1[1] += p0.y; x1[2] += p0.z; x1[3] += p0.w; x1[4] += p1.x; x1[5] += p1.y; x1[6] += p1.z; x1[7] += p1.w;
             x2[0] += p2.x; x2[1] += p2.y; x2[2] += p2.z; x2[3] += p2.w; x2[4] += p3.x; x2[5] += p3.y; x2[6] += p3.z; x2[7] += p3.w;
@@ -584,8 +618,8 @@ int vlac_tc_setup(vlac_ctx* ctx) {
   if (rc != VLAC_OK) { free(host); return rc; }
   {
     // workspace of the k-block-sharing launches: two slots per CTA and token chunk, and the per-tile counters
-    const size_t chunks = (size_t)(ctx->rows_max + TG_CHUNK - 1) / TG_CHUNK;
-    const size_t ws_floats = (size_t)ctx->n_sm * 2 * chunks * TG_SLOT_FLOATS;
+    const size_t chunks = (size_t)(ctx->rows_max + TG_CHUNK - 1) / TG_CHUNK + 1;     // in units of 256 tokens: covers ceil(T / 512) chunks of 512
+    const size_t ws_floats = (size_t)ctx->n_sm * 2 * chunks * TG_CHUNK * 128;
     const size_t tiles = (size_t)(3 * ((D + 127) / 128) > (F + 63) / 64 ? 3 * ((D + 127) / 128) : (F + 63) / 64);
     cudaError_t e1 = cudaMalloc(&ctx->tc_ws, ws_floats * sizeof(float));
     if (e1 == cudaSuccess) e1 = cudaMalloc(&ctx->tc_cnt, tiles * chunks * sizeof(int));
@@ -601,7 +635,8 @@ int vlac_tc_setup(vlac_ctx* ctx) {
 
 // Tensor-memory columns of the two accumulator buffers (each covers the largest token chunk; power of two >= 32).
 static int tc_tmem_cols(const vlac_ctx* ctx) {
-  const int chunk = ((ctx->rows_max < TG_CHUNK ? ctx->rows_max : TG_CHUNK) + 15) / 16 * 16;
+  if (ctx->rows_max > TG_CHUNK) return 512;
+  const int chunk = (ctx->rows_max + 15) / 16 * 16;
   int cols = 32;
   while (cols < chunk) cols *= 2;
   return 2 * cols;
