@@ -438,16 +438,27 @@ class StepResult:
     attn_tv: np.ndarray              # [n_layers, heads, L_v] emitted by this step's prefill
 
 
-def input_rows(cfg, model: Dict[str, object], feats_bf16: np.ndarray, prompt_ids: np.ndarray) -> np.ndarray:
+def input_rows(cfg, model: Dict[str, object], feats_bf16: np.ndarray, prompt_ids: np.ndarray,
+               rows0: Optional[np.ndarray] = None) -> np.ndarray:
     """Hidden rows entering layer 0: token embeddings at the text positions, projected
-    vision features (one linear map) at the vision positions."""
+    vision features (one linear map) at the vision positions.
+
+    With ``rows0`` (the positions layer 0 recomputes) only those vision positions are
+    projected (Sec. 4.1: ``H_t`` is needed for the tokens that are not reused); the other
+    vision rows stay zero.  The reuse sets are nested over depth, so a row that layer 0
+    skips is read by no layer."""
     hidden = np.zeros((cfg.max_seq, cfg.hidden), dtype=np.float64)
     embed = model["embed"]
     v0, v1 = cfg.n_text_pre, cfg.n_text_pre + cfg.n_vision
     ids = np.asarray(prompt_ids, dtype=np.int64)
     hidden[:v0] = widen_bf16(embed[ids[:v0]])
     hidden[v1:cfg.seq_len] = widen_bf16(embed[ids[v0:]])
-    hidden[v0:v1] = widen_bf16(feats_bf16) @ widen_bf16(model["proj"]).T
+    if rows0 is None:
+        hidden[v0:v1] = widen_bf16(feats_bf16) @ widen_bf16(model["proj"]).T
+    else:
+        vis = np.asarray([p for p in np.asarray(rows0, dtype=np.int64) if v0 <= p < v1], dtype=np.int64)
+        if len(vis):
+            hidden[vis] = widen_bf16(np.asarray(feats_bf16)[vis - v0]) @ widen_bf16(model["proj"]).T
     return hidden
 
 
@@ -472,7 +483,7 @@ def step(cfg, model: Dict[str, object], cache: CacheState, frames_t: np.ndarray,
     """
     sel = selection if selection is not None else select(cfg, frames_t, cache, params, force_full)
     cos, sin = model["rope_cos"], model["rope_sin"]
-    hidden = input_rows(cfg, model, feats_bf16, prompt_ids)
+    hidden = input_rows(cfg, model, feats_bf16, prompt_ids, rows0=sel.rows[0])
     attn_next = np.zeros((cfg.n_layers, cfg.n_heads, cfg.n_vision), dtype=np.float64)
     for l in range(cfg.n_layers):
         attn_next[l] = layer_forward(cfg, model["layers"][l], cache.K[l], cache.V[l], hidden,
@@ -520,7 +531,7 @@ def step_chunk(cfg, model: Dict[str, object], cache: CacheState, frames_t: np.nd
     """
     sel = selection if selection is not None else select(cfg, frames_t, cache, params, force_full)
     cos, sin = model["rope_cos"], model["rope_sin"]
-    hidden = input_rows(cfg, model, feats_bf16, prompt_ids)
+    hidden = input_rows(cfg, model, feats_bf16, prompt_ids, rows0=sel.rows[0])
     attn_next = np.zeros((cfg.n_layers, cfg.n_heads, cfg.n_vision), dtype=np.float64)
     for l in range(cfg.n_layers):
         attn_next[l] = layer_forward(cfg, model["layers"][l], cache.K[l], cache.V[l], hidden,

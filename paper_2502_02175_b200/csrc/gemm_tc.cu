@@ -705,20 +705,14 @@ int vlac_tc_partial(vlac_ctx* ctx, vlac_cache* c, int layer, int which, int* n_s
   return launch_tc(ctx, a, s);
 }
 
-// Vision projector (input rows of the vision positions): features [rows][D] x W_proj^T as K-split fp32
-// partial sums in ctx->part; the caller folds them.  The feature buffer is the caller's, so its tensor maps
-// are made here, per launch (inside a graph capture: once).
-int vlac_tc_projector(vlac_ctx* ctx, vlac_cache* c, const void* feats, int rows, int* n_splits, cudaStream_t s) {
+// Vision projector: the gathered features of layer 0's vision rows (compact rows of ctx->xn; text rows hold stale values
+// whose products are never used) x W_proj^T as K-split fp32 partial sums in ctx->part; the caller folds them.
+int vlac_tc_projector(vlac_ctx* ctx, vlac_cache* c, int* n_splits, cudaStream_t s) {
   const vlac_config& g = ctx->cfg;
-  if ((reinterpret_cast<uintptr_t>(feats) & 15) || rows > ctx->rows_max) return VLAC_ERR_INVALID_ARG;
   const CUtensorMap* act = (const CUtensorMap*)ctx->tmaps_host + (size_t)g.n_layers * TM_PER_LAYER;
   TcArgs a; tc_common(ctx, c, 0, &a);
-  a.tot = nullptr; a.tot_fixed = rows;
   a.tm_a[0] = act[TM_ACT_COUNT];
-  for (int i = 0; i < 4; ++i) {
-    const int rc = encode_map(&a.tm_b[i], feats, rows, g.hidden, 64 * (i + 1));
-    if (rc != VLAC_OK) return rc;
-  }
+  for (int i = 0; i < 4; ++i) a.tm_b[i] = act[TM_XN + i];
   a.K = g.hidden; a.N = g.hidden; a.mode = TG_PARTIAL;
   a.n_tiles = (g.hidden + 127) / 128;
   a.n_splits = tc_splits(ctx, a.n_tiles, a.K);

@@ -43,12 +43,29 @@ __global__ void __launch_bounds__(128) embed_rows_kernel(const bf16* embed, cons
   }
 }
 
-// fp32 [splits][B*Lv][D] (K-split partial sums, added in split order) -> rows at the vision positions
+// Only the vision rows that layer 0 recomputes need an input row (Sec. 4.1: H_t of the tokens that are not reused; a token
+// reused in layer 0 is reused in every layer, so its hidden row is never read).  Their features are gathered into the
+// compact row space of layer 0 -- the projector GEMM then runs over the live row count like every other product.
+__global__ void __launch_bounds__(256) gather_vision_feats_kernel(const bf16* feats, const int* tot0, const int* rowmap0, bf16* xn,
+                                                                  int n_text_pre, int Lv, int L, int D) {
+  const int i = blockIdx.x;
+  if (i >= *tot0) return;
+  const int row = rowmap0[i], b = row / L, v = row - b * L - n_text_pre;
+  if (v < 0 || v >= Lv) return;                                 // a text position: its row comes from the embedding table
+  const uint4* src = reinterpret_cast<const uint4*>(feats + ((size_t)b * Lv + v) * D);
+  uint4* dst = reinterpret_cast<uint4*>(xn + (size_t)i * D);
+  for (int c = threadIdx.x; c < D / 8; c += blockDim.x) dst[c] = src[c];
+}
+
+// fp32 [splits][compact rows of layer 0][D] (K-split partial sums, added in split order) -> rows at their vision positions
 __global__ void __launch_bounds__(256) place_vision_rows_kernel(const float* src, int n_splits, size_t split_stride, float* hidden,
-                                                                int n_text_pre, int Lv, int L, int D) {
-  const int r = blockIdx.x, b = r / Lv, v = r % Lv;
-  const float* s = src + (size_t)r * D;
-  float* d = hidden + ((size_t)b * L + n_text_pre + v) * D;
+                                                                const int* tot0, const int* rowmap0, int n_text_pre, int Lv, int L, int D) {
+  const int i = blockIdx.x;
+  if (i >= *tot0) return;
+  const int row = rowmap0[i], b = row / L, v = row - b * L - n_text_pre;
+  if (v < 0 || v >= Lv) return;
+  const float* s = src + (size_t)i * D;
+  float* d = hidden + (size_t)row * D;
   for (int c = threadIdx.x; c < D; c += blockDim.x) {
     float acc = s[c];
     for (int k = 1; k < n_splits; ++k) acc += s[(size_t)k * split_stride + c];
@@ -144,11 +161,15 @@ int vlac_launch_input_rows(vlac_ctx* ctx, vlac_cache* c, const void* feats, cons
                                                  ctx->Lv, ctx->L, D, g.vocab);
     VLAC_LAUNCH_CHECK(ctx);
   }
+  if (reinterpret_cast<uintptr_t>(feats) & 15) return VLAC_ERR_INVALID_ARG;
+  const int BL = B * ctx->L;
+  gather_vision_feats_kernel<<<BL, 256, 0, s>>>((const bf16*)feats, c->tot, c->rowmap, ctx->xn, g.n_text_pre, ctx->Lv, ctx->L, D);
+  VLAC_LAUNCH_CHECK(ctx);
   int n_splits = 1;
-  const int rc = vlac_tc_projector(ctx, c, feats, B * ctx->Lv, &n_splits, s);
+  const int rc = vlac_tc_projector(ctx, c, &n_splits, s);
   if (rc) return rc;
-  const float* src = ctx->part;
-  place_vision_rows_kernel<<<B * ctx->Lv, 256, 0, s>>>(src, n_splits, (size_t)ctx->rows_max * D, hidden, g.n_text_pre, ctx->Lv, ctx->L, D);
+  place_vision_rows_kernel<<<BL, 256, 0, s>>>((const float*)ctx->part, n_splits, (size_t)ctx->rows_max * D, hidden, c->tot, c->rowmap,
+                                              g.n_text_pre, ctx->Lv, ctx->L, D);
   VLAC_LAUNCH_CHECK(ctx);
   return VLAC_OK;
 }

@@ -126,7 +126,7 @@ int vlac_launch_wait_expiry(vlac_ctx* ctx, unsigned long long limit_ns, cudaStre
 int vlac_tc_qkv(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s);
 int vlac_tc_partial(vlac_ctx* ctx, vlac_cache* c, int layer, int which /* 0: output proj, 1: down proj */, int* n_splits, cudaStream_t s);
 int vlac_tc_gateup(vlac_ctx* ctx, vlac_cache* c, int layer, cudaStream_t s);
-int vlac_tc_projector(vlac_ctx* ctx, vlac_cache* c, const void* feats, int rows, int* n_splits, cudaStream_t s);
+int vlac_tc_projector(vlac_ctx* ctx, vlac_cache* c, int* n_splits, cudaStream_t s);
 
 // ---- tiled prefill attention (attention_kernels.cu)
 int vlac_encode_map_2d(void* out, const void* base, int rows, int cols, int box_rows);

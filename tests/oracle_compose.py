@@ -20,7 +20,7 @@ def step_layer_major(cfg, model, cache, frames_t, feats_bf16, prompt_ids, params
                      force_full=False, selection=None, operands="exact") -> orc.StepResult:
     sel = selection if selection is not None else orc.select(cfg, frames_t, cache, params, force_full)
     cos, sin = model["rope_cos"], model["rope_sin"]
-    hidden = orc.input_rows(cfg, model, feats_bf16, prompt_ids)
+    hidden = orc.input_rows(cfg, model, feats_bf16, prompt_ids, rows0=sel.rows[0])
     L, n = cfg.seq_len, cfg.n_action
     fed = np.asarray(forced_tokens, dtype=np.int64).reshape(n)
     for i in range(1, n):

@@ -210,6 +210,32 @@ def test_step_tiny_episode(H, vb):
         sess.close()
 
 
+def test_step_input_rows_only_for_recomputed_positions(H, vb):
+    """Only the vision rows layer 0 recomputes are projected: the features of the tokens it reuses are never read, so
+    replacing them by garbage changes no bit of the step's outputs (and the step still matches the checker)."""
+    cfg, model, ids, feats = _tiny_inputs(5)
+    prev, cur, _ = synth.rerandomised_pair(cfg, 5, 13)
+    params = H.oparams(top_k=32, alpha_override=[0.5, 1.0])
+    outs = []
+    for poison in (False, True):
+        sess = H.Session(cfg, model)
+        try:
+            H.run_step_pair(sess, prev[None], feats, ids, params)
+            f2 = feats.copy()
+            if poison:
+                sel = orc.select(cfg, cur, sess.ocache[0], params)
+                v0 = cfg.n_text_pre
+                skipped = np.setdiff1d(np.arange(v0, v0 + cfg.n_vision), sel.rows[0]) - v0
+                assert len(skipped) > 0
+                f2[0, skipped] = synth.f32_to_bf16(np.full((len(skipped), cfg.hidden), 1000.0, dtype=np.float32))
+            r = H.run_step_pair(sess, cur[None], f2, ids, params)[0]
+            assert r["logit_err"] <= H.TOL and r["M"][0] < cfg.seq_len
+            outs.append((r["tokens"], r["got_logits"].copy(), sess.read_attn(vb.PART_ATTN_PREV)))
+        finally:
+            sess.close()
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1]) and np.array_equal(outs[0][2], outs[1][2])
+
+
 def test_step_force_full_equals_cold_step(H, vb):
     """The no-reuse step of the same library equals a cold step on the same inputs, bit for bit."""
     cfg, model, ids, feats = _tiny_inputs(1)

@@ -117,6 +117,38 @@ def test_input_rows_layout():
     assert np.all(h[cfg.seq_len:] == 0)
 
 
+def test_input_rows_of_the_recomputed_positions_only():
+    """Projecting only the vision rows layer 0 recomputes: those rows equal the full projection, every other vision row
+    stays zero, and a whole cached step gives the same bits either way (a row skipped in layer 0 is skipped everywhere)."""
+    cfg, model, ids, feats = _tiny(5)
+    v0, v1 = cfg.n_text_pre, cfg.n_text_pre + cfg.n_vision
+    rows0 = np.asarray([0, v0 + 3, v0 + 4, v0 + 40, v1, v1 + 2])
+    full = orc.input_rows(cfg, model, feats, ids)
+    part = orc.input_rows(cfg, model, feats, ids, rows0=rows0)
+    vis = rows0[(rows0 >= v0) & (rows0 < v1)]
+    assert np.array_equal(part[vis], full[vis]) and np.array_equal(part[:v0], full[:v0]) and np.array_equal(part[v1:], full[v1:])
+    rest = np.setdiff1d(np.arange(v0, v1), vis)
+    assert np.all(part[rest] == 0.0) and np.any(full[rest] != 0.0)
+    # brute force on one row: dot products in Python floats
+    w = orc.widen_bf16(model["proj"]); x = orc.widen_bf16(feats[3])
+    assert np.allclose(part[v0 + 3], [float(np.dot(w[n], x)) for n in range(cfg.hidden)], rtol=1e-12, atol=1e-12)
+    # a cached step whose unselected feature rows are garbage gives the same result
+    prev, cur, changed = synth.rerandomised_pair(cfg, 5, 13)
+    params = orc.SelectParams(top_k=32, alpha_override=[0.5, 1.0])
+    outs = []
+    for poison in (False, True):
+        cache = orc.new_cache(cfg)
+        orc.step(cfg, model, cache, prev, feats, ids, params)
+        sel = orc.select(cfg, cur, cache, params)
+        f2 = feats.copy()
+        if poison:
+            skipped = np.setdiff1d(np.arange(v0, v1), sel.rows[0]) - v0
+            assert len(skipped) > 0
+            f2[skipped] = synth.f32_to_bf16(np.full((len(skipped), cfg.hidden), 1000.0, dtype=np.float32))
+        outs.append(orc.step(cfg, model, cache, cur, f2, ids, params, selection=sel).logits)
+    assert np.array_equal(outs[0], outs[1])
+
+
 def test_rope_complex_form_and_relative_property():
     cfg = synth.tiny_config()
     cos, sin = synth.rope_tables(cfg)
