@@ -108,6 +108,7 @@ typedef struct {
 #define VLAC_PART_ATTN_PREV  3   /* fp32 [n_layers][n_heads][L_v] of seq: scores saved by the previous step */
 #define VLAC_PART_ATTN_NEXT  4   /* same layout: scores being written by the current prefill               */
 #define VLAC_PART_WARM       5   /* int32 [1] of seq: 0 = cold (next select reuses nothing)                */
+#define VLAC_PART_PREV_FRAME_BF16 6 /* bf16 [n_cams][H][W][3] of seq: previous frame of vlac_select_bf16   */
 
 /* Create a context.  Copies `cfg` and the layer table, borrows every weight pointer, allocates the
  * workspace for max_batch sequences.  Errors: INVALID_ARG (a shape the kernels do not take, a NULL or
@@ -144,6 +145,16 @@ int vlac_cache_write(vlac_cache* cache, int part, int seq, int layer, const void
  * Runs entirely on the device; no host synchronisation. */
 int vlac_select(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames,
                 const vlac_select_params* params, vlac_selection* out, void* stream);
+
+/* The same selection from frames given as bf16 values (normalised pixels, the form a vision encoder takes; the
+ * Appendix "Experimental Settings" lowers tau to 0.85 for noisy real-robot frames).  Eq. (sim) is evaluated on those
+ * values with fp32 sums in a fixed order, so the similarities are reproducible but not exact: they agree with exact
+ * arithmetic to about 1e-6, and a caller who needs index sets that do not depend on the last bits keeps tau and the
+ * top-k boundary 1e-5 away from any similarity.  The previous frame is the cache part VLAC_PART_PREV_FRAME_BF16
+ * (written by the caller with vlac_cache_write; vlac_step maintains only the byte frame).
+ *   frames_bf16: device bf16 [batch][n_cams][H][W][3]. */
+int vlac_select_bf16(vlac_ctx* ctx, vlac_cache* cache, const void* frames_bf16,
+                     const vlac_select_params* params, vlac_selection* out, void* stream);
 
 /* Install a caller-made selection instead: HOST arrays M[batch][n_layers] and
  * rows[batch][n_layers][L] (ascending positions).  For each sequence the row sets must shrink with

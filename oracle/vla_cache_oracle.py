@@ -169,6 +169,30 @@ def patch_similarity(frames_t: np.ndarray, frames_prev: np.ndarray, grid: int, p
     return sim
 
 
+def patch_similarity_values(frames_t: np.ndarray, frames_prev: np.ndarray, grid: int, patch: int) -> np.ndarray:
+    """Eq. (sim) on frames given as real values ``[n_cams, H, W, 3]`` (normalised pixels rather than raw bytes; the
+    Appendix's noisy real-robot setting): the same patch layout and 0/0 readings as ``patch_similarity``, sums in
+    float64.  Values may be negative, so the similarity ranges over [-1, 1]."""
+    ft = np.asarray(frames_t, dtype=np.float64)
+    fp = np.asarray(frames_prev, dtype=np.float64)
+    n_cams = ft.shape[0]
+    sim = np.empty(n_cams * grid * grid, dtype=np.float64)
+    for cam in range(n_cams):
+        for i in range(grid):
+            for j in range(grid):
+                a = ft[cam, i * patch:(i + 1) * patch, j * patch:(j + 1) * patch, :].reshape(-1)
+                b = fp[cam, i * patch:(i + 1) * patch, j * patch:(j + 1) * patch, :].reshape(-1)
+                dot, na, nb = math.fsum(a * b), math.fsum(a * a), math.fsum(b * b)
+                if na == 0.0 and nb == 0.0:
+                    s = 1.0
+                elif na == 0.0 or nb == 0.0:
+                    s = 0.0
+                else:
+                    s = dot / math.sqrt(na * nb)
+                sim[cam * grid * grid + i * grid + j] = s
+    return sim
+
+
 def static_tokens(sim: np.ndarray, tau: float, top_k: int) -> np.ndarray:
     """Eq. (topk): of the tokens with ``sim >= tau`` keep the ``top_k`` most similar.
 
@@ -293,7 +317,7 @@ def reuse_order(final_mask: np.ndarray, S: np.ndarray) -> np.ndarray:
 
 
 def select(cfg, frames_t: np.ndarray, cache: CacheState, params: SelectParams,
-           force_full: bool = False) -> Selection:
+           force_full: bool = False, frame_values: bool = False) -> Selection:
     """Algorithm 1 followed by line 3 of Algorithm 2: which positions each layer recomputes.
 
     Layer ``l`` reuses the first ``floor(alpha_bar^l * |P_final|)`` tokens of ``reuse_order``;
@@ -309,7 +333,10 @@ def select(cfg, frames_t: np.ndarray, cache: CacheState, params: SelectParams,
                          ratio=np.zeros(nl), alpha=np.zeros(nl), alpha_bar=np.zeros(nl),
                          n_reuse=np.zeros(nl, dtype=np.int64), reuse_order=np.zeros(0, dtype=np.int64),
                          rows=[all_rows.copy() for _ in range(nl)], M=np.full(nl, L, dtype=np.int64))
-    sim = patch_similarity(frames_t, cache.prev_frames, cfg.grid, cfg.patch)
+    if frame_values:      # frames and cache.prev_frames hold real values (normalised pixels), not bytes
+        sim = patch_similarity_values(frames_t, cache.prev_frames, cfg.grid, cfg.patch)
+    else:
+        sim = patch_similarity(frames_t, cache.prev_frames, cfg.grid, cfg.patch)
     static_mask = static_tokens(sim, params.tau, params.top_k)
     S_layer, S = task_relevance(cache.attn_tv, params.layer_mask)
     task_mask = task_relevant_tokens(S, params.tau_task, params.task_mode)

@@ -22,7 +22,7 @@ if not os.path.exists(LIB_PATH):
 lib = C.CDLL(LIB_PATH)
 
 VLAC_OK = 0
-PART_K, PART_V, PART_PREV_FRAME, PART_ATTN_PREV, PART_ATTN_NEXT, PART_WARM = range(6)
+PART_K, PART_V, PART_PREV_FRAME, PART_ATTN_PREV, PART_ATTN_NEXT, PART_WARM, PART_PREV_FRAME_BF16 = range(7)
 MAX_LAYERS = 64
 
 
@@ -53,7 +53,7 @@ class vlac_selection(C.Structure):
 
 
 EXPORTS = ("vlac_create", "vlac_destroy", "vlac_cache_alloc", "vlac_cache_reset", "vlac_cache_free",
-           "vlac_cache_read", "vlac_cache_write", "vlac_select", "vlac_select_import", "vlac_layer_forward",
+           "vlac_cache_read", "vlac_cache_write", "vlac_select", "vlac_select_bf16", "vlac_select_import", "vlac_layer_forward",
            "vlac_step", "vlac_step_chunk", "vlac_selection_view", "vlac_launch_count", "vlac_device_error", "vlac_status_string",
            "vlac_profile", "vlac_profile_read", "vlac_profile_segments", "vlac_greedy_tokens_static",
            "vlac_selftest_wait_expiry")
@@ -70,6 +70,7 @@ lib.vlac_cache_free.argtypes = [C.c_void_p]
 lib.vlac_cache_read.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_ulonglong, C.c_void_p]
 lib.vlac_cache_write.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_ulonglong, C.c_void_p]
 lib.vlac_select.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(vlac_select_params), C.POINTER(vlac_selection), C.c_void_p]
+lib.vlac_select_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(vlac_select_params), C.POINTER(vlac_selection), C.c_void_p]
 lib.vlac_select_import.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 lib.vlac_layer_forward.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
 lib.vlac_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(vlac_select_params), C.c_int,
@@ -246,6 +247,13 @@ def vlac_select(ctx: int, cache: int, frames: torch.Tensor, params: vlac_select_
     assert frames.is_cuda and frames.dtype == torch.uint8 and frames.is_contiguous()
     out = vlac_selection()
     _check(lib.vlac_select(ctx, cache, frames.data_ptr(), C.byref(params), C.byref(out), _stream()), "vlac_select")
+    return out
+
+
+def vlac_select_bf16(ctx: int, cache: int, frames_bf16: torch.Tensor, params: vlac_select_params) -> vlac_selection:
+    assert frames_bf16.is_cuda and frames_bf16.dtype == torch.bfloat16 and frames_bf16.is_contiguous()
+    out = vlac_selection()
+    _check(lib.vlac_select_bf16(ctx, cache, frames_bf16.data_ptr(), C.byref(params), C.byref(out), _stream()), "vlac_select_bf16")
     return out
 
 

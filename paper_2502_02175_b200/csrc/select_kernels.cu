@@ -100,6 +100,51 @@ __global__ void __launch_bounds__(256) select_stage1_kernel(Stage1Args a) {
   }
 }
 
+// Stage 1 for frames given as bf16 values (normalised pixels, as a vision encoder takes them) instead of raw bytes: the
+// same Eq. (sim), sums in fp32.  One warp per patch; a lane adds the patch's elements lane, lane + 32, ... in that order
+// and the warp combines the lanes in a fixed tree, so the result does not depend on launch shape or timing.  The final
+// divide and square root are fp64.  (The similarities are no longer exact: decisions made on them need a margin.)
+__global__ void __launch_bounds__(256) select_stage1_bf16_kernel(const bf16* frames, const bf16* prev, double* sim,
+                                                                 int n_cams, int grid, int patch, int HW, int Lv) {
+  const int strip = blockIdx.x;
+  const int i = strip % grid, cam = (strip / grid) % n_cams, b = strip / (grid * n_cams);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int RB = HW * 3, PB = patch * 3, n = patch * PB;
+  const size_t base = ((size_t)(b * n_cams + cam) * HW + (size_t)i * patch) * RB;
+  for (int j = warp; j < grid; j += 8) {
+    float d = 0.f, na = 0.f, nb = 0.f;
+    for (int e = lane; e < n; e += 32) {
+      const int r = e / PB, c = e - r * PB;
+      const size_t off = base + (size_t)r * RB + (size_t)j * PB + c;
+      const float x = __bfloat162float(frames[off]), y = __bfloat162float(prev[off]);
+      d = fmaf(x, y, d); na = fmaf(x, x, na); nb = fmaf(y, y, nb);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      d += __shfl_xor_sync(0xffffffffu, d, o); na += __shfl_xor_sync(0xffffffffu, na, o); nb += __shfl_xor_sync(0xffffffffu, nb, o);
+    }
+    if (lane == 0) {
+      double s;
+      if (na == 0.f && nb == 0.f) s = 1.0;
+      else if (na == 0.f || nb == 0.f) s = 0.0;
+      else s = (double)d / sqrt((double)na * (double)nb);
+      sim[(size_t)b * Lv + (size_t)cam * grid * grid + i * grid + j] = s;
+    }
+  }
+}
+
+// head means only (the other half of stage 1), for the bf16-frame path
+__global__ void __launch_bounds__(256) head_mean_kernel(const float* attn_prev, double* S_layer, int nl, int H, int Lv) {
+  const int b = blockIdx.x / nl, l = blockIdx.x % nl;
+  const float* src = attn_prev + ((size_t)(b * nl + l) * H) * Lv;
+  double* dst = S_layer + (size_t)(b * nl + l) * Lv;
+  for (int v = threadIdx.x; v < Lv; v += blockDim.x) {
+    double s = 0.0;
+    for (int h = 0; h < H; ++h) s += (double)src[(size_t)h * Lv + v];
+    dst[v] = s / (double)H;
+  }
+}
+
 // ------------------------------------------------------------------------------------------------
 // Stage 2
 // ------------------------------------------------------------------------------------------------
@@ -369,7 +414,7 @@ __global__ void __launch_bounds__(256) flatten_rows_kernel(const int* M, const i
 }  // namespace
 
 int vlac_launch_select(vlac_ctx* ctx, vlac_cache* c, const unsigned char* frames,
-                       const SelectKernelParams& p, cudaStream_t s) {
+                       const SelectKernelParams& p, cudaStream_t s, const void* frames_bf16) {
   const vlac_config& g = ctx->cfg;
   Stage1Args a1;
   a1.frames = frames; a1.prev = c->prev_frames; a1.attn_prev = c->attn_prev;
@@ -379,7 +424,13 @@ int vlac_launch_select(vlac_ctx* ctx, vlac_cache* c, const unsigned char* frames
   a1.n_strips = c->batch * g.n_cams * g.grid;
   a1.vec_ok = ((ctx->frame_hw * 3) % 16 == 0) && ((g.patch * 3) % 2 == 0) && (g.patch * 3 >= 16) &&
               ((reinterpret_cast<uintptr_t>(frames) & 15u) == 0);
-  if (!p.force_full) {
+  if (!p.force_full && frames_bf16) {
+    select_stage1_bf16_kernel<<<a1.n_strips, 256, 0, s>>>((const bf16*)frames_bf16, c->prev_frames_bf16, c->sim, g.n_cams, g.grid, g.patch,
+                                                          ctx->frame_hw, ctx->Lv);
+    VLAC_LAUNCH_CHECK(ctx);
+    head_mean_kernel<<<c->batch * g.n_layers, 256, 0, s>>>(c->attn_prev, c->S_layer, g.n_layers, g.n_heads, ctx->Lv);
+    VLAC_LAUNCH_CHECK(ctx);
+  } else if (!p.force_full) {
     const int blocks = a1.n_strips + c->batch * g.n_layers;
     select_stage1_kernel<<<blocks, 256, 3 * g.grid * sizeof(unsigned int), s>>>(a1);
     VLAC_LAUNCH_CHECK(ctx);

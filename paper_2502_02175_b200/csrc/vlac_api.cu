@@ -61,7 +61,7 @@ void free_ctx_buffers(vlac_ctx* c) {
 }
 
 void free_cache_buffers(vlac_cache* c) {
-  cudaFree(c->k); cudaFree(c->v); cudaFree(c->prev_frames); cudaFree(c->attn_prev); cudaFree(c->attn_next);
+  cudaFree(c->k); cudaFree(c->v); cudaFree(c->prev_frames); cudaFree(c->prev_frames_bf16); cudaFree(c->attn_prev); cudaFree(c->attn_next);
   cudaFree(c->warm); cudaFree(c->sim); cudaFree(c->S_layer); cudaFree(c->S); cudaFree(c->alpha);
   cudaFree(c->alpha_raw); cudaFree(c->entropy); cudaFree(c->static_mask); cudaFree(c->task_mask);
   cudaFree(c->final_mask); cudaFree(c->rank); cudaFree(c->n_reuse); cudaFree(c->M); cudaFree(c->rows);
@@ -180,6 +180,7 @@ int vlac_cache_alloc(vlac_ctx* ctx, int batch, vlac_cache** out) {
   if (rc == VLAC_OK) rc = dev_alloc(&c->k, nl * B * kv_layer_elems(ctx));
   if (rc == VLAC_OK) rc = dev_alloc(&c->v, nl * B * kv_layer_elems(ctx));
   if (rc == VLAC_OK) rc = dev_alloc(&c->prev_frames, B * frame);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->prev_frames_bf16, B * frame);
   if (rc == VLAC_OK) rc = dev_alloc(&c->attn_prev, B * nl * g.n_heads * Lv);
   if (rc == VLAC_OK) rc = dev_alloc(&c->attn_next, B * nl * g.n_heads * Lv);
   if (rc == VLAC_OK) rc = dev_alloc(&c->warm, B);
@@ -246,6 +247,7 @@ static int cache_part(vlac_cache* c, int part, int seq, int layer, void** ptr, s
     case VLAC_PART_ATTN_PREV: *ptr = c->attn_prev + seq * attn; *bytes = attn * sizeof(float); return VLAC_OK;
     case VLAC_PART_ATTN_NEXT: *ptr = c->attn_next + seq * attn; *bytes = attn * sizeof(float); return VLAC_OK;
     case VLAC_PART_WARM: *ptr = c->warm + seq; *bytes = sizeof(int); return VLAC_OK;
+    case VLAC_PART_PREV_FRAME_BF16: *ptr = c->prev_frames_bf16 + seq * frame; *bytes = frame * sizeof(bf16); return VLAC_OK;
     default: return VLAC_ERR_INVALID_ARG;
   }
 }
@@ -281,6 +283,17 @@ int vlac_select(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, c
   SelectKernelParams p;
   TRY(fill_params(ctx, params, 0, &p));
   TRY(vlac_launch_select(ctx, cache, frames, p, (cudaStream_t)stream));
+  cache->has_selection = 1;
+  if (out) vlac_selection_view(cache, out);
+  return VLAC_OK;
+}
+
+int vlac_select_bf16(vlac_ctx* ctx, vlac_cache* cache, const void* frames_bf16, const vlac_select_params* params,
+                     vlac_selection* out, void* stream) {
+  if (!ctx || !cache || cache->ctx != ctx || !frames_bf16 || !params) return VLAC_ERR_INVALID_ARG;
+  SelectKernelParams p;
+  TRY(fill_params(ctx, params, 0, &p));
+  TRY(vlac_launch_select(ctx, cache, nullptr, p, (cudaStream_t)stream, frames_bf16));
   cache->has_selection = 1;
   if (out) vlac_selection_view(cache, out);
   return VLAC_OK;

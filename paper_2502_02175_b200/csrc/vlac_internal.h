@@ -88,6 +88,7 @@ struct vlac_cache {
   // persistent state (device)
   bf16 *k, *v;                       // [n_layers][batch][max_seq][n_heads][head_dim]
   unsigned char* prev_frames;        // [batch][n_cams][H][W][3]
+  bf16* prev_frames_bf16;            // same shape: previous frame of the bf16-frame selection (vlac_select_bf16)
   float *attn_prev, *attn_next;      // [batch][n_layers][n_heads][Lv]
   int* warm;                         // [batch]
   // selection state (device)
@@ -107,7 +108,7 @@ static inline size_t kv_layer_elems(const vlac_ctx* c) {
 
 // ---- selection (select_kernels.cu)
 int vlac_launch_select(vlac_ctx* ctx, vlac_cache* c, const unsigned char* frames,
-                       const SelectKernelParams& p, cudaStream_t s);
+                       const SelectKernelParams& p, cudaStream_t s, const void* frames_bf16 = nullptr);
 int vlac_launch_flatten(vlac_ctx* ctx, vlac_cache* c, cudaStream_t s);
 
 // ---- prefill (prefill_kernels.cu)

@@ -98,6 +98,47 @@ def test_select_noisy_regime_lower_threshold(H, vb):
     assert got["static_mask"][0].sum() > 150 and got["M"].min() < cfg.seq_len
 
 
+def test_select_bf16_normalised_frames(H, vb):
+    """Selection from bf16 frames of normalised pixels (7B shape, noisy regime, tau 0.85): similarities within 1e-5 of
+    the checker's exact sums on the same bf16 values, and -- with tau and the top-k boundary kept 1e-5 away from every
+    similarity -- the same index sets, ratios and row lists."""
+    cfg = synth.llama7b_config(n_layers=4)
+    ep = synth.make_episode(cfg.with_layers(1), 31, 2, n_blobs=3, noise_sigma=12.0)
+    norm = lambda f: synth.f32_to_bf16(((f.astype(np.float32) / 255.0) - 0.45) / 0.225)
+    prev_b, cur_b = norm(ep.frames[0]), norm(ep.frames[1])
+    prev_v, cur_v = synth.bf16_to_f64(prev_b), synth.bf16_to_f64(cur_b)
+    attn = synth.scripted_attention(cfg, 31, ep.touched[1])
+    sess = H.Session(cfg, None, dev_model=_DummyModel(vb, cfg.n_layers))
+    try:
+        oc = sess.ocache[0]
+        oc.prev_frames, oc.attn_tv, oc.warm = prev_v, attn.astype(np.float64), True
+        sim = orc.patch_similarity_values(cur_v, prev_v, cfg.grid, cfg.patch)
+        tau = 0.85
+        assert np.min(np.abs(sim - tau)) >= 1e-5
+        order = np.sort(sim[sim >= tau])[::-1]
+        k = next(k for k in range(100, len(order)) if order[k - 1] - order[k] >= 1e-5)      # a top-k boundary with a margin
+        params = H.oparams(tau=tau, top_k=k, k_ent=3.0)
+        want = orc.select(cfg, cur_v, oc, params, frame_values=True)
+        vb.vlac_cache_write(sess.cache, vb.PART_PREV_FRAME_BF16, 0, 0, vb.upload_bf16(prev_b))
+        vb.vlac_cache_write(sess.cache, vb.PART_ATTN_PREV, 0, 0, torch.from_numpy(attn).to("cuda").contiguous())
+        vb.vlac_cache_write(sess.cache, vb.PART_WARM, 0, 0, torch.ones(1, dtype=torch.int32, device="cuda"))
+        gp, keep = H.gparams(params)
+        got = vb.selection_to_host(vb.vlac_select_bf16(sess.ctx, sess.cache, vb.upload_bf16(cur_b[None]), gp))
+        assert np.max(np.abs(got["sim"][0] - want.sim)) <= 1e-5
+        assert np.array_equal(got["static_mask"][0].astype(bool), want.static_mask)
+        assert np.array_equal(got["S"][0], want.S) and np.array_equal(got["task_mask"][0].astype(bool), want.task_mask)
+        assert np.array_equal(got["final_mask"][0].astype(bool), want.final_mask)
+        assert 0 < want.final_mask.sum() < cfg.n_vision
+        for l in range(cfg.n_layers):
+            m = int(want.M[l])
+            assert int(got["M"][0, l]) == m and np.array_equal(got["rows"][0, l, :m], want.rows[l])
+        # run to run the similarities are the same bits
+        again = vb.selection_to_host(vb.vlac_select_bf16(sess.ctx, sess.cache, vb.upload_bf16(cur_b[None]), gp))
+        assert np.array_equal(again["sim"], got["sim"])
+    finally:
+        sess.close()
+
+
 def test_select_dual_camera_batch(H, vb):
     """Two cameras, three sequences with different change rates: one global top-k per sequence."""
     cfg = synth.dual_camera_config(n_layers=8)

@@ -267,3 +267,38 @@ def test_noisy_regime_needs_the_lower_threshold():
     capped = orc.static_tokens(sim, 0.85, 100)
     assert capped.sum() == 100 and sim[capped].min() >= np.sort(sim)[-100]
     assert capped[touched].sum() <= 0.2 * touched.sum() + 10
+
+
+def test_similarity_of_real_valued_frames():
+    """patch_similarity_values: closed forms, the integer path on byte frames, and torch's cosine_similarity."""
+    import torch
+    cfg = synth.tiny_config()
+    prev, cur, changed = synth.rerandomised_pair(cfg, 11, 13)
+    # on byte frames the two functions are the same quantity
+    a = orc.patch_similarity(cur, prev, cfg.grid, cfg.patch)
+    b = orc.patch_similarity_values(cur.astype(np.float64), prev.astype(np.float64), cfg.grid, cfg.patch)
+    np.testing.assert_allclose(b, a, rtol=0, atol=1e-15)
+    # normalised frames: centred pixels change the values (and allow negative similarities)
+    x = (cur.astype(np.float64) / 255.0 - 0.5) / 0.25
+    y = (prev.astype(np.float64) / 255.0 - 0.5) / 0.25
+    s = orc.patch_similarity_values(x, y, cfg.grid, cfg.patch)
+    unchanged = np.setdiff1d(np.arange(cfg.n_vision), changed)
+    assert np.all(s[unchanged] == 1.0) and np.all(np.abs(s[changed]) < 0.2)
+    p = cfg.patch
+    for v in (0, int(changed[0]), cfg.n_vision - 1):
+        i, j = divmod(v, cfg.grid)
+        ta = torch.from_numpy(x[0, i * p:(i + 1) * p, j * p:(j + 1) * p, :].reshape(1, -1))
+        tb = torch.from_numpy(y[0, i * p:(i + 1) * p, j * p:(j + 1) * p, :].reshape(1, -1))
+        assert abs(float(torch.nn.functional.cosine_similarity(ta, tb)) - s[v]) < 1e-12
+    assert np.all(orc.patch_similarity_values(x, -x, cfg.grid, cfg.patch) == -1.0)
+    z = np.zeros_like(x)
+    assert np.all(orc.patch_similarity_values(z, z, cfg.grid, cfg.patch) == 1.0)
+    assert np.all(orc.patch_similarity_values(x, z, cfg.grid, cfg.patch) == 0.0)
+    # select() on values: same sets as on bytes when only the scale changes (cosine is scale-free)
+    cache = orc.new_cache(cfg)
+    cache.warm, cache.prev_frames = True, prev
+    cache.attn_tv = synth.scripted_attention(cfg, 11).astype(np.float64)
+    want = orc.select(cfg, cur, cache, orc.SelectParams(top_k=32))
+    cache.prev_frames = prev.astype(np.float64) / 255.0
+    got = orc.select(cfg, cur.astype(np.float64) / 255.0, cache, orc.SelectParams(top_k=32), frame_values=True)
+    assert np.array_equal(got.final_mask, want.final_mask) and np.array_equal(got.M, want.M)
