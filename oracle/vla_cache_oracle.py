@@ -393,7 +393,7 @@ def silu(x: np.ndarray) -> np.ndarray:
 def layer_forward(cfg, layer_w: Dict[str, np.ndarray], K: np.ndarray, V: np.ndarray,
                   hidden: np.ndarray, rows: np.ndarray, cos: np.ndarray, sin: np.ndarray,
                   emit_attention: bool = True, block_start: Optional[int] = None,
-                  operands: str = "exact") -> Optional[np.ndarray]:
+                  operands: str = "exact", hidden_keys: Optional[np.ndarray] = None) -> Optional[np.ndarray]:
     """One decoder layer over the positions in ``rows`` only (Algorithm 2, Sec. 4.1).
 
     ``K``/``V`` are this layer's cache ``[max_seq, heads, d]`` and are updated in place at
@@ -404,6 +404,9 @@ def layer_forward(cfg, layer_w: Dict[str, np.ndarray], K: np.ndarray, V: np.ndar
     K/V are fresh or reused.  Keys are stored after rotation.  With ``block_start`` the rows
     at positions ``>= block_start`` form one block that is decoded in parallel: each of them
     also sees the block's later positions (see ``step_chunk``).
+
+    ``hidden_keys`` (bool ``[max_seq]``) marks cache positions no query may attend to (tokens
+    removed from the sequence by ``step_pruned``).
 
     ``operands="bf16"`` rounds every operand of a matrix product to bf16 first and stores keys and values
     as bf16 (the paper's BF16 setting; see the module header); the emitted probabilities are not rounded.
@@ -430,6 +433,8 @@ def layer_forward(cfg, layer_w: Dict[str, np.ndarray], K: np.ndarray, V: np.ndar
     visible = key_pos[None, :] <= rows[:, None]                      # [rows, keys]
     if block_start is not None:
         visible = visible | ((rows[:, None] >= block_start) & (key_pos[None, :] >= block_start))
+    if hidden_keys is not None:
+        visible = visible & ~np.asarray(hidden_keys, dtype=bool)[None, :n_keys]
     v0 = cfg.n_text_pre
     v1 = v0 + cfg.n_vision
     text_q = (rows >= v1) & (rows < cfg.seq_len)
@@ -581,4 +586,81 @@ def step_chunk(cfg, model: Dict[str, object], cache: CacheState, frames_t: np.nd
     cache.prev_frames = np.array(frames_t, copy=True)
     cache.warm = True
     return StepResult(tokens=tokens, fed_tokens=tokens.copy(), logits=logits, margins=margins,
+                      selection=sel, hidden=hidden, attn_tv=attn_next)
+
+
+# --------------------------------------------------------------------------- #
+# comparison baseline: intra-frame pruning after layer K (FastV-style)
+# --------------------------------------------------------------------------- #
+def pruned_vision_tokens(score: np.ndarray, n_keep: int) -> np.ndarray:
+    """The ``n_keep`` vision tokens with the highest score (ties to the lower index) as a bool mask."""
+    order = sorted(range(len(score)), key=lambda v: (-score[v], v))
+    keep = np.zeros(len(score), dtype=bool)
+    for v in order[:max(min(n_keep, len(score)), 0)]:
+        keep[v] = True
+    return keep
+
+
+def step_pruned(cfg, model: Dict[str, object], cache: CacheState, frames_t: np.ndarray,
+                feats_bf16: np.ndarray, prompt_ids: np.ndarray, prune_layer: int, n_keep: int,
+                forced_tokens: Optional[Sequence[int]] = None, operands: str = "exact") -> StepResult:
+    """The baseline the paper compares with in its main LIBERO table (row "+FastV"; Sec. 5, baselines): no reuse
+    across frames; instead, inside one frame, vision tokens that receive little attention are dropped part-way
+    through the decoder.  The paper gives no equations for it; reading taken here (that of the FastV method):
+
+    * layers ``0 .. prune_layer-1`` run over the whole sequence;
+    * every vision token gets the score ``mean over heads and over the prompt-text query rows behind the vision
+      block`` of the attention probability it received in layer ``prune_layer-1`` (the text-to-vision scores of
+      Eq. (avistext) that every prefill emits); the ``n_keep`` best are kept, ties to the lower index;
+    * from layer ``prune_layer`` on, the dropped tokens are gone: their rows are not computed and no query attends
+      to their positions, in the prefill and in the single-row passes of the action tokens; kept tokens and text
+      keep their original positions (and so their rotary angles).
+
+    ``prune_layer >= n_layers`` or ``n_keep >= L_v`` is the plain full step.  The cache is used as scratch for this
+    step's K/V and is left warm like after ``step`` (previous frame, emitted scores); ``selection.M`` reports the
+    rows per layer.
+    """
+    nl, L, lv = cfg.n_layers, cfg.seq_len, cfg.n_vision
+    sel = select(cfg, frames_t, cache, SelectParams(), force_full=True)
+    cos, sin = model["rope_cos"], model["rope_sin"]
+    hidden = input_rows(cfg, model, feats_bf16, prompt_ids)
+    attn_next = np.zeros((nl, cfg.n_heads, lv), dtype=np.float64)
+    hidden_keys = None
+    rows = np.arange(L, dtype=np.int64)
+    v0 = cfg.n_text_pre
+    kept = np.ones(lv, dtype=bool)
+    for l in range(nl):
+        if l == prune_layer and l > 0 and n_keep < lv:
+            score = np.zeros(lv, dtype=np.float64)
+            for h in range(cfg.n_heads):
+                score = score + attn_next[l - 1, h]
+            kept = pruned_vision_tokens(score / np.float64(cfg.n_heads), n_keep)
+            hidden_keys = np.zeros(cfg.max_seq, dtype=bool)
+            hidden_keys[v0:v0 + lv] = ~kept
+            rows = np.asarray([p for p in range(L) if not hidden_keys[p]], dtype=np.int64)
+        sel.rows[l], sel.M[l] = rows, len(rows)
+        attn_next[l] = layer_forward(cfg, model["layers"][l], cache.K[l], cache.V[l], hidden, rows, cos, sin,
+                                     emit_attention=True, operands=operands, hidden_keys=hidden_keys)
+    tokens = np.zeros(cfg.n_action, dtype=np.int64)
+    fed = np.zeros(cfg.n_action, dtype=np.int64)
+    logits = np.zeros((cfg.n_action, cfg.vocab), dtype=np.float64)
+    margins = np.zeros(cfg.n_action, dtype=np.float64)
+    for i in range(cfg.n_action):
+        pos = L - 1 + i
+        if i > 0:
+            hidden[pos] = widen_bf16(model["embed"][int(fed[i - 1])])
+            for l in range(nl):
+                hk = hidden_keys if (hidden_keys is not None and l >= prune_layer) else None
+                layer_forward(cfg, model["layers"][l], cache.K[l], cache.V[l], hidden, np.asarray([pos]), cos, sin,
+                              emit_attention=False, operands=operands, hidden_keys=hk)
+        logits[i] = _logits(cfg, model, hidden[pos], operands)
+        tokens[i] = int(np.argmax(logits[i]))
+        top2 = np.partition(logits[i], -2)[-2:]
+        margins[i] = float(top2[1] - top2[0])
+        fed[i] = tokens[i] if forced_tokens is None else int(forced_tokens[i])
+    cache.attn_tv = attn_next
+    cache.prev_frames = np.array(frames_t, copy=True)
+    cache.warm = True
+    sel.final_mask = ~kept                    # reported for inspection: the dropped vision tokens
+    return StepResult(tokens=tokens, fed_tokens=fed, logits=logits, margins=margins,
                       selection=sel, hidden=hidden, attn_tv=attn_next)

@@ -436,3 +436,52 @@ def test_cost_of_bf16_operands_on_the_tiny_decoder():
         rb = orc.step(cfg, m, orc.new_cache(cfg), frame, feats, ids, orc.SelectParams(), forced_tokens=ra.tokens, operands="bf16")
         dist = max(float(np.abs(rb.logits[i] - ra.logits[i]).max() / np.abs(ra.logits[i]).max()) for i in range(cfg.n_action))
         assert 1e-4 < dist < 2e-2, (nl, dist)
+
+
+def test_pruned_tokens_match_a_brute_force_sort():
+    rng = np.random.default_rng(3)
+    score = np.round(rng.random(40), 1)                       # many ties
+    for n_keep in (0, 1, 7, 39, 40, 50):
+        keep = orc.pruned_vision_tokens(score, n_keep)
+        order = np.lexsort((np.arange(40), -score))          # by score descending, then index ascending
+        want = np.zeros(40, dtype=bool); want[order[:min(n_keep, 40)]] = True
+        assert np.array_equal(keep, want)
+
+
+def test_pruned_step_special_cases_and_textbook_model_on_the_reduced_sequence():
+    """step_pruned: keeping every token (or pruning behind the last layer) is the plain step, bit for bit; and with
+    tokens dropped after layer 0, layer 1 equals a textbook layer run on the REDUCED sequence (dropped tokens removed,
+    the others at their original rotary positions)."""
+    cfg, model, ids, feats = _tiny(7)
+    frame = synth.rerandomised_pair(cfg, 7, 0)[0]
+    L, v0, lv = cfg.seq_len, cfg.n_text_pre, cfg.n_vision
+    full = orc.step(cfg, model, orc.new_cache(cfg), frame, feats, ids, orc.SelectParams())
+    for args in ((1, lv), (cfg.n_layers, 10)):
+        same = orc.step_pruned(cfg, model, orc.new_cache(cfg), frame, feats, ids, *args)
+        assert np.array_equal(same.logits, full.logits) and np.array_equal(same.tokens, full.tokens)
+    n_keep = 24
+    cache = orc.new_cache(cfg)
+    res = orc.step_pruned(cfg, model, cache, frame, feats, ids, 1, n_keep)
+    assert list(res.selection.M) == [L, L - (lv - n_keep)]
+    assert not np.array_equal(res.logits, full.logits)
+    # layer 0 by the textbook layer, scores from its softmax, kept set by sorting
+    h0 = torch.from_numpy(orc.input_rows(cfg, model, feats, ids)[:L])
+    cos, sin = torch.from_numpy(model["rope_cos"][:L]).double(), torch.from_numpy(model["rope_sin"][:L]).double()
+    h1, k0, v0_ = _torch_layer(cfg, model["layers"][0], h0, cos, sin)
+    xn = torch.nn.functional.rms_norm(h0, (cfg.hidden,), _t(model["layers"][0]["g_attn"]), cfg.rms_eps)
+    q = _torch_rope(torch.nn.functional.linear(xn, _t(model["layers"][0]["wq"])).view(L, cfg.n_heads, cfg.head_dim), cos, sin)
+    sc = torch.einsum("qhd,khd->hqk", q, k0) / math.sqrt(cfg.head_dim)
+    sc = sc.masked_fill(~torch.tril(torch.ones(L, L, dtype=torch.bool)), float("-inf"))
+    p = torch.softmax(sc, dim=-1)
+    score = p[:, v0 + lv:L, v0:v0 + lv].mean(dim=1).mean(dim=0).numpy()
+    kept = np.zeros(lv, dtype=bool); kept[np.lexsort((np.arange(lv), -score))[:n_keep]] = True
+    assert np.array_equal(~res.selection.final_mask, kept)
+    rows = np.asarray([p_ for p_ in range(L) if not (v0 <= p_ < v0 + lv and not kept[p_ - v0])])
+    assert np.array_equal(res.selection.rows[1], rows)
+    h2, k1, v1 = _torch_layer(cfg, model["layers"][1], h1[rows], cos[rows], sin[rows])
+    np.testing.assert_allclose(res.hidden[rows], h2.numpy(), rtol=1e-9, atol=1e-9)
+    np.testing.assert_allclose(cache.K[1][rows], k1.numpy(), rtol=1e-9, atol=1e-9)
+    np.testing.assert_allclose(cache.V[1][rows], v1.numpy(), rtol=1e-9, atol=1e-9)
+    # the first logits row is the lm_head of the last reduced row
+    xf = torch.nn.functional.rms_norm(h2[-1:], (cfg.hidden,), _t(model["g_final"]), cfg.rms_eps)
+    np.testing.assert_allclose(res.logits[0], torch.nn.functional.linear(xf, _t(model["lm_head"]))[0].numpy(), rtol=1e-9, atol=1e-9)
