@@ -214,6 +214,20 @@ int vlac_step_chunk(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frame
                     const int* prompt_ids, const vlac_select_params* params, int force_full, const void* act_embed,
                     int* action_tokens, float* all_logits, void* stream);
 
+/* Comparison baseline, not part of the method: one control step WITHOUT reuse across frames in which, instead, vision
+ * tokens that receive little attention are dropped inside the frame after layer prune_layer - 1 (the FastV row of the
+ * paper's Table 2; Sec. 5 "Baselines"; the paper prints no equations for it, the reading is that of the FastV method).
+ * Layers 0 .. prune_layer-1 run over the whole sequence.  Each vision token is then scored by the text-to-vision
+ * attention it received in layer prune_layer-1 of this step (mean over heads and over the prompt-text queries behind the
+ * vision block, the scores of Eq. avistext that every prefill records); the n_keep best stay (ties to the lower
+ * index).  From layer prune_layer on the other vision tokens are gone: their rows are not computed and no query attends to
+ * their positions, in the prefill and in the single-row passes; kept tokens keep their positions.  prune_layer >= n_layers
+ * or n_keep >= L_v gives the plain no-reuse step.  Afterwards vlac_selection_view shows the rows per layer, and the cache
+ * is warm as after vlac_step.  prune_layer < 1: INVALID_ARG.  Other arguments and stream behaviour as for vlac_step. */
+int vlac_step_pruned(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, const void* vision_feats,
+                     const int* prompt_ids, int prune_layer, int n_keep, int* action_tokens, float* all_logits,
+                     const int* forced_tokens, void* stream);
+
 /* Views of the selection held by the cache (after select / select_import / step). */
 int vlac_selection_view(vlac_cache* cache, vlac_selection* out);
 

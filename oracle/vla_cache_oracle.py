@@ -603,7 +603,8 @@ def pruned_vision_tokens(score: np.ndarray, n_keep: int) -> np.ndarray:
 
 def step_pruned(cfg, model: Dict[str, object], cache: CacheState, frames_t: np.ndarray,
                 feats_bf16: np.ndarray, prompt_ids: np.ndarray, prune_layer: int, n_keep: int,
-                forced_tokens: Optional[Sequence[int]] = None, operands: str = "exact") -> StepResult:
+                forced_tokens: Optional[Sequence[int]] = None, operands: str = "exact",
+                prune_scores: Optional[np.ndarray] = None) -> StepResult:
     """The baseline the paper compares with in its main LIBERO table (row "+FastV"; Sec. 5, baselines): no reuse
     across frames; instead, inside one frame, vision tokens that receive little attention are dropped part-way
     through the decoder.  The paper gives no equations for it; reading taken here (that of the FastV method):
@@ -616,6 +617,8 @@ def step_pruned(cfg, model: Dict[str, object], cache: CacheState, frames_t: np.n
       to their positions, in the prefill and in the single-row passes of the action tokens; kept tokens and text
       keep their original positions (and so their rotary angles).
 
+    ``prune_scores`` (``[heads, L_v]``) replaces this run's own layer ``prune_layer-1`` scores in the ranking (a
+    replayed comparison ranks by another implementation's scores so that the kept sets can be compared exactly).
     ``prune_layer >= n_layers`` or ``n_keep >= L_v`` is the plain full step.  The cache is used as scratch for this
     step's K/V and is left warm like after ``step`` (previous frame, emitted scores); ``selection.M`` reports the
     rows per layer.
@@ -632,8 +635,9 @@ def step_pruned(cfg, model: Dict[str, object], cache: CacheState, frames_t: np.n
     for l in range(nl):
         if l == prune_layer and l > 0 and n_keep < lv:
             score = np.zeros(lv, dtype=np.float64)
+            src = attn_next[l - 1] if prune_scores is None else np.asarray(prune_scores, dtype=np.float64)
             for h in range(cfg.n_heads):
-                score = score + attn_next[l - 1, h]
+                score = score + src[h]
             kept = pruned_vision_tokens(score / np.float64(cfg.n_heads), n_keep)
             hidden_keys = np.zeros(cfg.max_seq, dtype=bool)
             hidden_keys[v0:v0 + lv] = ~kept

@@ -54,7 +54,7 @@ class vlac_selection(C.Structure):
 
 EXPORTS = ("vlac_create", "vlac_destroy", "vlac_cache_alloc", "vlac_cache_reset", "vlac_cache_free",
            "vlac_cache_read", "vlac_cache_write", "vlac_select", "vlac_select_bf16", "vlac_select_import", "vlac_layer_forward",
-           "vlac_step", "vlac_step_chunk", "vlac_selection_view", "vlac_launch_count", "vlac_device_error", "vlac_status_string",
+           "vlac_step", "vlac_step_chunk", "vlac_step_pruned", "vlac_selection_view", "vlac_launch_count", "vlac_device_error", "vlac_status_string",
            "vlac_profile", "vlac_profile_read", "vlac_profile_segments", "vlac_greedy_tokens_static",
            "vlac_selftest_wait_expiry")
 
@@ -77,6 +77,8 @@ lib.vlac_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_vo
                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 lib.vlac_step_chunk.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(vlac_select_params), C.c_int,
                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+lib.vlac_step_pruned.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
+                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 lib.vlac_selection_view.argtypes = [C.c_void_p, C.POINTER(vlac_selection)]
 lib.vlac_device_error.argtypes = [C.c_void_p, C.c_void_p]
 lib.vlac_selftest_wait_expiry.argtypes = [C.c_void_p, C.c_uint, C.c_void_p]
@@ -294,6 +296,18 @@ def vlac_step_chunk(ctx: int, cache: int, frames: torch.Tensor, vision_feats: to
     _check(lib.vlac_step_chunk(ctx, cache, frames.data_ptr(), vision_feats.data_ptr(), prompt_ids.data_ptr(),
                                C.byref(params) if params is not None else None, int(bool(force_full)),
                                act_embed.data_ptr(), action_tokens.data_ptr(), _ptr(all_logits), _stream()), "vlac_step_chunk")
+
+
+def vlac_step_pruned(ctx: int, cache: int, frames: torch.Tensor, vision_feats: torch.Tensor, prompt_ids: torch.Tensor,
+                     prune_layer: int, n_keep: int, action_tokens: torch.Tensor, all_logits: Optional[torch.Tensor] = None,
+                     forced_tokens: Optional[torch.Tensor] = None) -> None:
+    assert frames.is_cuda and frames.dtype == torch.uint8 and frames.is_contiguous()
+    assert vision_feats.is_cuda and vision_feats.dtype == torch.bfloat16 and vision_feats.is_contiguous()
+    assert prompt_ids.is_cuda and prompt_ids.dtype == torch.int32 and prompt_ids.is_contiguous()
+    assert action_tokens.is_cuda and action_tokens.dtype == torch.int32 and action_tokens.is_contiguous()
+    assert all_logits is None or (all_logits.is_cuda and all_logits.dtype == torch.float32 and all_logits.is_contiguous())
+    _check(lib.vlac_step_pruned(ctx, cache, frames.data_ptr(), vision_feats.data_ptr(), prompt_ids.data_ptr(), int(prune_layer),
+                                int(n_keep), action_tokens.data_ptr(), _ptr(all_logits), _ptr(forced_tokens), _stream()), "vlac_step_pruned")
 
 
 def vlac_selection_view(cache: int) -> vlac_selection:

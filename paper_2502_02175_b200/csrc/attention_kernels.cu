@@ -32,6 +32,7 @@ struct AttnTileArgs {
   const int* rowmap;                      // [B*L] compact index -> b*L + pos (this layer)
   bf16* out;                              // [rows][H*d]
   float* partial;                         // [B][tiles][H][Lv] column sums over text rows, or NULL
+  const unsigned char* hidden_keys;       // [B][max_seq] 1 = position removed from the sequence (no query attends to it), or NULL
   int* dev_error;
   int layer, nl, B, L, max_seq, H, v0, Lv, tiles;
 };
@@ -193,6 +194,7 @@ __global__ void __launch_bounds__(AT_THREADS, 1) attention_tile_kernel(AttnTileA
   const int pos_lo = r_lo < n_valid ? a.rowmap[row0 + r_lo] - b * a.L : -1;
   const int pos_hi = r_hi < n_valid ? a.rowmap[row0 + r_hi] - b * a.L : -1;
   const float scale = rsqrtf((float)DH) * 1.44269504088896f;     // softmax in base 2
+  const unsigned char* hk = a.hidden_keys ? a.hidden_keys + (size_t)b * a.max_seq : nullptr;
 
   bool ok = mbar_wait(&q_bar, 0, &abort_flag, a.dev_error, 0x71000);
   unsigned qf[DH / 16][4];
@@ -221,10 +223,12 @@ __global__ void __launch_bounds__(AT_THREADS, 1) attention_tile_kernel(AttnTileA
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       const int key = i * AT_KB + j * 8 + 2 * t;
-      sc[j][0] = key <= pos_lo ? sc[j][0] * scale : -INFINITY;
-      sc[j][1] = key + 1 <= pos_lo ? sc[j][1] * scale : -INFINITY;
-      sc[j][2] = key <= pos_hi ? sc[j][2] * scale : -INFINITY;
-      sc[j][3] = key + 1 <= pos_hi ? sc[j][3] * scale : -INFINITY;
+      bool v0k = true, v1k = true;                                // key, key + 1 still part of the sequence
+      if (hk) { v0k = key < a.max_seq && !hk[key]; v1k = key + 1 < a.max_seq && !hk[key + 1]; }
+      sc[j][0] = (key <= pos_lo && v0k) ? sc[j][0] * scale : -INFINITY;
+      sc[j][1] = (key + 1 <= pos_lo && v1k) ? sc[j][1] * scale : -INFINITY;
+      sc[j][2] = (key <= pos_hi && v0k) ? sc[j][2] * scale : -INFINITY;
+      sc[j][3] = (key + 1 <= pos_hi && v1k) ? sc[j][3] * scale : -INFINITY;
       bm_lo = fmaxf(bm_lo, fmaxf(sc[j][0], sc[j][1]));
       bm_hi = fmaxf(bm_hi, fmaxf(sc[j][2], sc[j][3]));
     }
@@ -294,9 +298,12 @@ __global__ void __launch_bounds__(AT_THREADS, 1) attention_tile_kernel(AttnTileA
     for (int j = 0; j < 8; ++j) {
       const int key = kb * AT_KB + j * 8 + 2 * t;
       float c0 = 0.f, c1 = 0.f;
-      // text rows sit behind the vision block, so they see every vision key: no mask needed here
+      // text rows sit behind the vision block, so they see every vision key still in the sequence
+      const bool v0k = !hk || (key < a.max_seq && !hk[key]), v1k = !hk || (key + 1 < a.max_seq && !hk[key + 1]);
       if (text_lo) { c0 += exp2f(sc[j][0] * scale - m_lo) * inv_lo; c1 += exp2f(sc[j][1] * scale - m_lo) * inv_lo; }
       if (text_hi) { c0 += exp2f(sc[j][2] * scale - m_hi) * inv_hi; c1 += exp2f(sc[j][3] * scale - m_hi) * inv_hi; }
+      if (!v0k) c0 = 0.f;
+      if (!v1k) c1 = 0.f;
 #pragma unroll
       for (int sh = 4; sh <= 16; sh <<= 1) { c0 += __shfl_xor_sync(0xffffffffu, c0, sh); c1 += __shfl_xor_sync(0xffffffffu, c1, sh); }
       if (g == 0) {
@@ -395,13 +402,23 @@ int vlac_launch_prefill_attention(vlac_ctx* ctx, vlac_cache* c, int layer, cudaS
   const size_t layer_stride = (size_t)B * ctx->attn_tiles * g.n_heads * ctx->Lv;
   a.partial = g.n_text_post > 0 ? (defer ? ctx->probs_all + (size_t)layer * layer_stride : ctx->probs) : nullptr;
   a.dev_error = ctx->dev_error;
+  a.hidden_keys = (ctx->prune_layer > 0 && layer >= ctx->prune_layer) ? c->hidden_keys : nullptr;
   a.layer = layer; a.nl = g.n_layers; a.B = B; a.L = ctx->L; a.max_seq = ctx->max_seq; a.H = g.n_heads;
   a.v0 = g.n_text_pre; a.Lv = ctx->Lv; a.tiles = ctx->attn_tiles;
   const dim3 grid(ctx->attn_tiles, B, g.n_heads);
   if (g.head_dim == 128) VLAC_CUDA_CHECK(launch_pdl(attention_tile_kernel<128>, grid, dim3(AT_THREADS), at_smem<128>(ctx->Lv), s, a));
   else VLAC_CUDA_CHECK(launch_pdl(attention_tile_kernel<64>, grid, dim3(AT_THREADS), at_smem<64>(ctx->Lv), s, a));
   VLAC_LAUNCH_CHECK(ctx);
-  if (defer) return VLAC_OK;
+  if (defer) {
+    // the pruning baseline ranks the tokens by this layer's scores before the next layer starts
+    if (ctx->prune_layer > 0 && layer == ctx->prune_layer - 1) {
+      VLAC_CUDA_CHECK(launch_pdl(emit_from_tiles_kernel, dim3(g.n_heads, B), dim3(256), 0, s, (const float*)a.partial,
+                                 c->attn_next + (size_t)layer * g.n_heads * ctx->Lv, (size_t)g.n_layers * g.n_heads * ctx->Lv, ctx->attn_tiles,
+                                 g.n_text_post, g.n_heads, ctx->Lv, (size_t)0));
+      VLAC_LAUNCH_CHECK(ctx);
+    }
+    return VLAC_OK;
+  }
   float* dst = c->attn_next + (size_t)layer * g.n_heads * ctx->Lv;
   VLAC_CUDA_CHECK(launch_pdl(emit_from_tiles_kernel, dim3(g.n_heads, B), dim3(256), 0, s, (const float*)ctx->probs, dst,
                              (size_t)g.n_layers * g.n_heads * ctx->Lv, ctx->attn_tiles, g.n_text_post, g.n_heads, ctx->Lv, (size_t)0));

@@ -597,7 +597,7 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
 template <int DPL, int NT>      // dimensions per lane = head_dim / 32; threads of the CTA
 __device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc, const bf16* vc, bf16* out,
                                                       int pos, int max_seq, int H, int h, int b, float* dsm, float* red,
-                                                      int cps = 1) {
+                                                      int cps = 1, const unsigned char* hidden_keys = nullptr) {
   constexpr int d = 32 * DPL;
   constexpr int NW = NT / 32;
   float* qs = dsm;                 // [d]
@@ -633,6 +633,7 @@ __device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc
         for (int e = 0; e < 8; ++e) dot += qs[(c0 + c) * 8 + e] * bf2f(kb[e]);
       }
     }
+    if (hidden_keys && hidden_keys[(size_t)sb * max_seq + j]) dot = -INFINITY;      // position removed from the sequence
     p[j] = dot;
     mx = fmaxf(mx, dot);
   }
@@ -693,12 +694,12 @@ __device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc
 
 template <int DPL>
 __global__ void __launch_bounds__(DA_THREADS) decode_attention_kernel(const bf16* q, const bf16* kc, const bf16* vc, bf16* out,
-                                                                      int pos, int max_seq, int H, int cps) {
+                                                                      int pos, int max_seq, int H, int cps, const unsigned char* hidden_keys) {
   extern __shared__ float dsm[];
   __shared__ float red[DA_THREADS / 32];
   pdl_trigger();
   pdl_wait();
-  decode_attention_body<DPL, DA_THREADS>(q, kc, vc, out, pos, max_seq, H, blockIdx.x, blockIdx.y, dsm, red, cps);
+  decode_attention_body<DPL, DA_THREADS>(q, kc, vc, out, pos, max_seq, H, blockIdx.x, blockIdx.y, dsm, red, cps, hidden_keys);
 }
 
 __global__ void __launch_bounds__(256) embed_token_kernel(const bf16* embed, const int* tokens, int tok_stride, int tok_index,
@@ -895,12 +896,11 @@ int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens,
       const size_t smem = (size_t)(g.head_dim + ctx->max_seq + (DA_THREADS / 32) * g.head_dim) * sizeof(float);
       const dim3 grid(g.n_heads, B);
       const bf16 *q = ctx->q_dec, *kc = ph[0].kc, *vc = ph[0].vc;
+      const unsigned char* hk = (ctx->prune_layer > 0 && l >= ctx->prune_layer) ? c->hidden_keys : nullptr;
       cudaError_t e;
       switch (g.head_dim / 32) {
-        case 1: e = launch_pdl(decode_attention_kernel<1>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, 1); break;
-        case 2: e = launch_pdl(decode_attention_kernel<2>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, 1); break;
-        case 3: e = launch_pdl(decode_attention_kernel<3>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, 1); break;
-        default: e = launch_pdl(decode_attention_kernel<4>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, 1); break;
+        case 2: e = launch_pdl(decode_attention_kernel<2>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, 1, hk); break;
+        default: e = launch_pdl(decode_attention_kernel<4>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, 1, hk); break;
       }
       VLAC_CUDA_CHECK(e);
       VLAC_LAUNCH_CHECK(ctx);
@@ -939,10 +939,8 @@ int vlac_launch_chunk_pass(vlac_ctx* ctx, vlac_cache* c, const void* act_embed, 
         const int pos = ctx->L;
         cudaError_t e;
         switch (g.head_dim / 32) {
-          case 1: e = launch_pdl(decode_attention_kernel<1>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, n); break;
-          case 2: e = launch_pdl(decode_attention_kernel<2>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, n); break;
-          case 3: e = launch_pdl(decode_attention_kernel<3>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, n); break;
-          default: e = launch_pdl(decode_attention_kernel<4>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, n); break;
+          case 2: e = launch_pdl(decode_attention_kernel<2>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, n, (const unsigned char*)nullptr); break;
+          default: e = launch_pdl(decode_attention_kernel<4>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, n, (const unsigned char*)nullptr); break;
         }
         VLAC_CUDA_CHECK(e);
         VLAC_LAUNCH_CHECK(ctx);

@@ -411,7 +411,68 @@ __global__ void __launch_bounds__(256) flatten_rows_kernel(const int* M, const i
   if (tid == 0) tot[l] = off;
 }
 
+// Intra-frame pruning after a layer (the FastV-style baseline of the paper's Table 2): rank the vision tokens by the
+// text-to-vision score they received in layer `layer_from - 1` of THIS step (mean over heads in fixed order, fp64), keep
+// the n_keep best (ties to the lower index), and rewrite the row lists of layers >= layer_from to text + kept tokens.
+// hidden_keys marks the dropped positions for the attention kernels.  One CTA per sequence.
+__global__ void __launch_bounds__(1024) prune_rows_kernel(const float* attn_layer, size_t seq_stride, int H, int Lv, int L, int nl,
+                                                          int n_text_pre, int layer_from, int n_keep, int B, int max_seq,
+                                                          int* M, int* rows, int* tot, int* rowmap, int* slot, unsigned char* hidden_keys) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);            // [Lv]
+  unsigned int* hist = reinterpret_cast<unsigned int*>(keys + Lv);                       // [256]
+  int* sh = reinterpret_cast<int*>(hist + 256);                                          // [8]
+  unsigned char* cand = reinterpret_cast<unsigned char*>(sh + 8);                        // [Lv]
+  unsigned char* keep = cand + Lv;                                                       // [Lv]
+  unsigned char* live = keep + Lv;                                                       // [L]: position is computed from layer_from on
+  const int tid = threadIdx.x, b = blockIdx.x;
+  const float* src = attn_layer + (size_t)b * seq_stride;
+  for (int v = tid; v < Lv; v += blockDim.x) {
+    double s = 0.0;
+    for (int h = 0; h < H; ++h) s += (double)src[(size_t)h * Lv + v];
+    s /= (double)H;
+    keys[v] = (unsigned long long)__double_as_longlong(s);      // probabilities: non-negative, so the bit patterns are ordered
+    cand[v] = 1;
+  }
+  __syncthreads();
+  block_topk(keys, cand, Lv, n_keep, keep, hist, sh);
+  for (int p = tid; p < max_seq; p += blockDim.x) {
+    const int v = p - n_text_pre;
+    const unsigned char hidden = (v >= 0 && v < Lv && !keep[v]) ? 1 : 0;
+    hidden_keys[(size_t)b * max_seq + p] = hidden;
+    if (p < L) live[p] = !hidden;
+  }
+  __syncthreads();
+  for (int p = tid; p < L; p += blockDim.x) {
+    int idx = 0;
+    for (int q = 0; q < p; ++q) idx += live[q];
+    int count = idx;
+    if (p == L - 1) count += live[p];
+    for (int l = layer_from; l < nl; ++l) {
+      if (live[p]) rows[((size_t)b * nl + l) * L + idx] = p;
+      if (p == L - 1) M[(size_t)b * nl + l] = count;
+      if (B == 1) {
+        if (live[p]) rowmap[(size_t)l * L + idx] = p;
+        slot[(size_t)l * L + p] = live[p] ? idx : -1;
+        if (p == L - 1) tot[l] = count;
+      }
+    }
+  }
+}
+
 }  // namespace
+
+int vlac_launch_prune(vlac_ctx* ctx, vlac_cache* c, int layer_from, int n_keep, cudaStream_t s) {
+  const vlac_config& g = ctx->cfg;
+  const size_t smem = (size_t)ctx->Lv * 8 + 256 * 4 + 8 * 4 + 2 * (size_t)ctx->Lv + ctx->L + 16;
+  const float* attn_layer = c->attn_next + (size_t)(layer_from - 1) * g.n_heads * ctx->Lv;
+  prune_rows_kernel<<<c->batch, 1024, smem, s>>>(attn_layer, (size_t)g.n_layers * g.n_heads * ctx->Lv, g.n_heads, ctx->Lv, ctx->L, g.n_layers,
+                                                 g.n_text_pre, layer_from, n_keep, c->batch, ctx->max_seq, c->M, c->rows, c->tot, c->rowmap,
+                                                 c->slot, c->hidden_keys);
+  VLAC_LAUNCH_CHECK(ctx);
+  if (c->batch > 1) return vlac_launch_flatten(ctx, c, s);
+  return VLAC_OK;
+}
 
 int vlac_launch_select(vlac_ctx* ctx, vlac_cache* c, const unsigned char* frames,
                        const SelectKernelParams& p, cudaStream_t s, const void* frames_bf16) {

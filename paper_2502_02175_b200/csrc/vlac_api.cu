@@ -65,7 +65,7 @@ void free_cache_buffers(vlac_cache* c) {
   cudaFree(c->warm); cudaFree(c->sim); cudaFree(c->S_layer); cudaFree(c->S); cudaFree(c->alpha);
   cudaFree(c->alpha_raw); cudaFree(c->entropy); cudaFree(c->static_mask); cudaFree(c->task_mask);
   cudaFree(c->final_mask); cudaFree(c->rank); cudaFree(c->n_reuse); cudaFree(c->M); cudaFree(c->rows);
-  cudaFree(c->tot); cudaFree(c->rowmap); cudaFree(c->slot); cudaFree(c->tmaps_kv);
+  cudaFree(c->tot); cudaFree(c->hidden_keys); cudaFree(c->rowmap); cudaFree(c->slot); cudaFree(c->tmaps_kv);
 }
 
 __global__ void set_warm_kernel(int* warm, int n, int value) {
@@ -198,6 +198,7 @@ int vlac_cache_alloc(vlac_ctx* ctx, int batch, vlac_cache** out) {
   if (rc == VLAC_OK) rc = dev_alloc(&c->M, B * nl);
   if (rc == VLAC_OK) rc = dev_alloc(&c->rows, B * nl * L);
   if (rc == VLAC_OK) rc = dev_alloc(&c->tot, nl);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->hidden_keys, B * (size_t)ctx->max_seq);
   if (rc == VLAC_OK) rc = dev_alloc(&c->rowmap, nl * B * L);
   if (rc == VLAC_OK) rc = dev_alloc(&c->slot, nl * B * L);
   if (rc == VLAC_OK) rc = vlac_attention_cache_setup(ctx, c);
@@ -356,7 +357,7 @@ static int seg_mark(vlac_ctx* ctx, cudaStream_t s) {
 // Enqueue every kernel of one control step on `s` (directly, or into a stream capture).
 static int enqueue_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, const void* vision_feats,
                         const int* prompt_ids, const SelectKernelParams& p, int* action_tokens, float* all_logits,
-                        const int* forced_tokens, const void* act_embed, cudaStream_t s) {
+                        const int* forced_tokens, const void* act_embed, int prune_layer, int n_keep, cudaStream_t s) {
   const vlac_config& g = ctx->cfg;
   const int B = cache->batch, nl = g.n_layers;
   ctx->seg_n = 0;
@@ -371,10 +372,15 @@ static int enqueue_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* f
   // 3. layers; the down-projection partials of layer l are folded into layer l+1's first kernel
   int n_splits = 0;
   ctx->defer_emit = ctx->probs_all != nullptr;
+  ctx->prune_layer = (prune_layer > 0 && prune_layer < nl && n_keep < ctx->Lv && g.n_text_post > 0) ? prune_layer : 0;
   for (int l = 0; l < nl; ++l) {
-    int rc = vlac_launch_finalize_norm(ctx, cache, h, 1, l == 0 ? 0 : l - 1, l == 0 ? 0 : n_splits, l, ctx->layers[l].g_attn, s);
+    int rc = VLAC_OK;
+    // pruning baseline: the scores layer l - 1 just emitted decide which vision tokens layers l.. still see
+    if (ctx->prune_layer > 0 && l == ctx->prune_layer) rc = vlac_launch_prune(ctx, cache, l, n_keep, s);
+    if (rc != VLAC_OK) { ctx->defer_emit = 0; ctx->prune_layer = 0; return rc; }
+    rc = vlac_launch_finalize_norm(ctx, cache, h, 1, l == 0 ? 0 : l - 1, l == 0 ? 0 : n_splits, l, ctx->layers[l].g_attn, s);
     if (rc == VLAC_OK) rc = vlac_launch_layer_body(ctx, cache, l, h, 1, &n_splits, s);
-    if (rc != VLAC_OK) { ctx->defer_emit = 0; return rc; }
+    if (rc != VLAC_OK) { ctx->defer_emit = 0; ctx->prune_layer = 0; return rc; }
   }
   const bool deferred = ctx->defer_emit != 0;
   ctx->defer_emit = 0;
@@ -406,13 +412,15 @@ static int enqueue_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* f
   VLAC_CUDA_CHECK(cudaMemcpyAsync(cache->attn_prev, cache->attn_next, sizeof(float) * (size_t)B * nl * g.n_heads * ctx->Lv,
                                   cudaMemcpyDeviceToDevice, s));
   set_warm_kernel<<<1, 32, 0, s>>>(cache->warm, B, 1);
+  ctx->prune_layer = 0;
   VLAC_LAUNCH_CHECK(ctx);
   return VLAC_OK;
 }
 
 static int step_impl(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, const void* vision_feats,
                      const int* prompt_ids, const vlac_select_params* params, int force_full,
-                     int* action_tokens, float* all_logits, const int* forced_tokens, const void* act_embed, void* stream) {
+                     int* action_tokens, float* all_logits, const int* forced_tokens, const void* act_embed,
+                     int prune_layer, int n_keep, void* stream) {
   if (!ctx || !cache || cache->ctx != ctx || !frames || !vision_feats || !action_tokens) return VLAC_ERR_INVALID_ARG;
   const vlac_config& g = ctx->cfg;
   const int n_text = g.n_text_pre + g.n_text_post;
@@ -433,7 +441,8 @@ static int step_impl(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* fram
     if (cap != cudaStreamCaptureStatusNone) direct = true;
   }
   if (direct)
-    return enqueue_step(ctx, cache, frames, vision_feats, prompt_ids, p, action_tokens, all_logits, forced_tokens, act_embed, s);
+    return enqueue_step(ctx, cache, frames, vision_feats, prompt_ids, p, action_tokens, all_logits, forced_tokens, act_embed,
+                        prune_layer, n_keep, s);
 
   const size_t frame = (size_t)B * g.n_cams * ctx->frame_hw * ctx->frame_hw * 3;
   VLAC_CUDA_CHECK(cudaMemcpyAsync(ctx->in_frames, frames, frame, cudaMemcpyDeviceToDevice, s));
@@ -445,7 +454,7 @@ static int step_impl(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* fram
   for (int i = 0; i < VLAC_MAX_GRAPHS; ++i) {
     StepGraph& e = ctx->graphs[i];
     if (e.used && e.cache == cache && e.force_full == (force_full ? 1 : 0) && e.use_forced == (forced_tokens ? 1 : 0) &&
-        e.act_embed == act_embed && memcmp(&e.p, &p, sizeof(p)) == 0) { entry = &e; break; }
+        e.act_embed == act_embed && e.prune_layer == prune_layer && e.n_keep == n_keep && memcmp(&e.p, &p, sizeof(p)) == 0) { entry = &e; break; }
   }
   if (!entry) {
     StepGraph& e = ctx->graphs[ctx->graph_next];
@@ -454,7 +463,7 @@ static int step_impl(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* fram
     const unsigned long long l0 = ctx->launches;
     VLAC_CUDA_CHECK(cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal));
     const int rc = enqueue_step(ctx, cache, ctx->in_frames, ctx->in_feats, ctx->in_ids, p, ctx->out_tokens, ctx->logits_all,
-                                forced_tokens ? ctx->in_forced : nullptr, act_embed, s);
+                                forced_tokens ? ctx->in_forced : nullptr, act_embed, prune_layer, n_keep, s);
     cudaGraph_t graph = nullptr;
     const cudaError_t ce = cudaStreamEndCapture(s, &graph);
     if (rc != VLAC_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
@@ -463,7 +472,7 @@ static int step_impl(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* fram
     cudaGraphDestroy(graph);
     VLAC_CUDA_CHECK(ie);
     e.used = 1; e.cache = cache; e.force_full = force_full ? 1 : 0; e.use_forced = forced_tokens ? 1 : 0; e.p = p;
-    e.act_embed = act_embed;
+    e.act_embed = act_embed; e.prune_layer = prune_layer; e.n_keep = n_keep;
     e.launches = ctx->launches - l0;
     ctx->launches = l0;
     entry = &e;
@@ -480,7 +489,15 @@ int vlac_step(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, con
               const int* prompt_ids, const vlac_select_params* params, int force_full,
               int* action_tokens, float* all_logits, const int* forced_tokens, void* stream) {
   return step_impl(ctx, cache, frames, vision_feats, prompt_ids, params, force_full, action_tokens, all_logits, forced_tokens,
-                   nullptr, stream);
+                   nullptr, 0, 0, stream);
+}
+
+int vlac_step_pruned(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, const void* vision_feats,
+                     const int* prompt_ids, int prune_layer, int n_keep, int* action_tokens, float* all_logits,
+                     const int* forced_tokens, void* stream) {
+  if (prune_layer < 1 || n_keep < 0) return VLAC_ERR_INVALID_ARG;
+  return step_impl(ctx, cache, frames, vision_feats, prompt_ids, nullptr, 1, action_tokens, all_logits, forced_tokens,
+                   nullptr, prune_layer, n_keep, stream);
 }
 
 int vlac_step_chunk(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frames, const void* vision_feats,
@@ -489,7 +506,7 @@ int vlac_step_chunk(vlac_ctx* ctx, vlac_cache* cache, const unsigned char* frame
   if (!act_embed) return VLAC_ERR_INVALID_ARG;
   if (ctx && !ctx->chunk_ok) return VLAC_ERR_INVALID_ARG;
   return step_impl(ctx, cache, frames, vision_feats, prompt_ids, params, force_full, action_tokens, all_logits, nullptr,
-                   act_embed, stream);
+                   act_embed, 0, 0, stream);
 }
 
 unsigned long long vlac_launch_count(const vlac_ctx* ctx) { return ctx ? ctx->launches : 0ull; }

@@ -35,6 +35,7 @@ struct StepGraph {                     // one captured control step (CUDA graph)
   vlac_cache* cache;
   int force_full, use_forced;
   const void* act_embed;               // chunk steps: the placeholder embeddings the graph reads (NULL: ordinary step)
+  int prune_layer, n_keep;             // pruning-baseline steps (0: not one)
   SelectKernelParams p;
   cudaGraphExec_t exec;
   unsigned long long launches;
@@ -70,6 +71,7 @@ struct vlac_ctx {
   void* tmap_q;                      // device tensor map of the query buffer (tiled attention)
   int attn_tiles;                    // 64-query tiles per sequence
   float* probs_all;                  // [n_layers][max_batch][tiles][n_heads][Lv]: per-tile column sums of every layer of a step
+  int prune_layer;                   // > 0 while a pruning-baseline step is enqueued: layers >= it skip the positions in hidden_keys
   int defer_emit;                    // set while a whole step is enqueued: text-to-vision scores of all layers are formed by one kernel at its end
   // optional per-launch timing of the matrix-vector kernel (vlac_profile)
   int prof_on, prof_n;
@@ -96,6 +98,7 @@ struct vlac_cache {
   unsigned char *static_mask, *task_mask, *final_mask;       // [b][Lv]
   int *rank, *n_reuse;               // [b][Lv], [b][nl]
   int *M, *rows;                     // [b][nl], [b][nl][L]
+  unsigned char* hidden_keys;        // [batch][max_seq]     1 = position dropped by the pruning baseline (vlac_step_pruned)
   int *tot;                          // [nl]                 total rows over the batch
   int *rowmap;                       // [nl][batch*L]        compact index -> b*L + pos
   int *slot;                         // [nl][batch*L]        b*L + pos -> compact index or -1
@@ -110,6 +113,7 @@ static inline size_t kv_layer_elems(const vlac_ctx* c) {
 int vlac_launch_select(vlac_ctx* ctx, vlac_cache* c, const unsigned char* frames,
                        const SelectKernelParams& p, cudaStream_t s, const void* frames_bf16 = nullptr);
 int vlac_launch_flatten(vlac_ctx* ctx, vlac_cache* c, cudaStream_t s);
+int vlac_launch_prune(vlac_ctx* ctx, vlac_cache* c, int layer_from, int n_keep, cudaStream_t s);
 
 // ---- prefill (prefill_kernels.cu)
 int vlac_launch_input_rows(vlac_ctx* ctx, vlac_cache* c, const void* feats, const int* ids, float* hidden, cudaStream_t s);

@@ -340,6 +340,77 @@ def test_step_batch_of_three_ragged(H, vb):
         sess.close()
 
 
+# ------------------------------------------------------------------------------------- intra-frame pruning baseline
+def _pruned_case(H, vb, cfg, model, ids, frames, feats, prune_layer, n_keep):
+    sess = H.Session(cfg, model)
+    try:
+        tok = torch.zeros((1, cfg.n_action), dtype=torch.int32, device="cuda")
+        lg = torch.zeros((1, cfg.n_action, cfg.vocab), dtype=torch.float32, device="cuda")
+        with torch.cuda.stream(sess.stream):
+            vb.vlac_step_pruned(sess.ctx, sess.cache, torch.from_numpy(frames[None]).to("cuda"), vb.upload_bf16(feats[None]),
+                                torch.from_numpy(ids).to("cuda"), prune_layer, n_keep, tok, lg)
+        torch.cuda.synchronize()
+        assert vb.vlac_device_error(sess.ctx) == 0
+        g_attn = sess.read_attn(vb.PART_ATTN_PREV)
+        got = vb.selection_to_host(vb.vlac_selection_view(sess.cache))
+        g_tok, g_log = tok.cpu().numpy()[0], lg.cpu().numpy()[0].astype(np.float64)
+        res = orc.step_pruned(cfg, model, sess.ocache[0], frames, feats, ids[0], prune_layer, n_keep, forced_tokens=g_tok,
+                              prune_scores=g_attn[prune_layer - 1].astype(np.float64) if 0 < prune_layer < cfg.n_layers else None)
+        for l in range(cfg.n_layers):                     # kept sets and row lists: exact
+            m = int(res.selection.M[l])
+            assert int(got["M"][0, l]) == m, (l, got["M"][0, l], m)
+            assert np.array_equal(got["rows"][0, l, :m], res.selection.rows[l])
+        err = max(H.rel_err(g_log[i], res.logits[i]) for i in range(cfg.n_action))
+        abs_err = float(np.max(np.abs(g_log - res.logits)))
+        for i in range(cfg.n_action):
+            if res.margins[i] > 2.0 * abs_err:
+                assert int(g_tok[i]) == int(res.tokens[i])
+        attn_err = max(H.rel_err(g_attn[l], res.attn_tv[l]) for l in range(cfg.n_layers))
+        return err, attn_err, res, g_log
+    finally:
+        sess.close()
+
+
+def test_step_pruned_tiny(H, vb):
+    """The FastV-style baseline against the checker on the tiny decoder: tokens dropped after layer 0, kept sets exact."""
+    cfg, model, ids, feats = _tiny_inputs(6)
+    frame = synth.rerandomised_pair(cfg, 6, 0)[0]
+    err, attn_err, res, g_log = _pruned_case(H, vb, cfg, model, ids, frame, feats[0], 1, 24)
+    assert err <= H.TOL and attn_err <= H.TOL
+    assert list(res.selection.M) == [cfg.seq_len, cfg.seq_len - (cfg.n_vision - 24)]
+    # nothing dropped: the plain no-reuse step, bit for bit
+    err_all, _, _, g_all = _pruned_case(H, vb, cfg, model, ids, frame, feats[0], 1, cfg.n_vision)
+    sess = H.Session(cfg, model)
+    try:
+        tok = torch.zeros((1, cfg.n_action), dtype=torch.int32, device="cuda")
+        lg = torch.zeros((1, cfg.n_action, cfg.vocab), dtype=torch.float32, device="cuda")
+        with torch.cuda.stream(sess.stream):
+            vb.vlac_step(sess.ctx, sess.cache, torch.from_numpy(frame[None]).to("cuda"), vb.upload_bf16(feats), torch.from_numpy(ids).to("cuda"),
+                         None, True, tok, lg)
+        torch.cuda.synchronize()
+        assert np.array_equal(lg.cpu().numpy()[0].astype(np.float64), g_all)
+    finally:
+        sess.close()
+    assert not np.array_equal(g_log, g_all)
+
+
+def test_step_pruned_7b_shape(H, vb):
+    """7B-shaped layers (3 of them), half of the 256 vision tokens dropped after layer 1."""
+    cfg = synth.llama7b_config(n_layers=3)
+    model = synth.make_model(cfg, 15)
+    ids = synth.make_prompt_ids(cfg, 15)
+    ep = synth.make_episode(cfg.with_layers(1), 15, 1)
+    orc.WIDEN_CACHE_MAX = 40
+    try:
+        err, attn_err, res, _ = _pruned_case(H, vb, cfg, model, ids, ep.frames[0], ep.feats[0], 2, 128)
+        print(f"pruned step, 7B shape: logit err {err:.2e}, attn err {attn_err:.2e}, rows per layer {list(res.selection.M)}")
+        assert err <= H.TOL and attn_err <= H.TOL
+        assert list(res.selection.M) == [290, 290, 162]
+    finally:
+        orc.WIDEN_CACHE_MAX = 0
+        orc._widen_cache.clear()
+
+
 # ------------------------------------------------------------------------------------- action chunk in one pass
 def test_step_chunk_tiny_episode(H, vb):
     """All action tokens from one parallel pass behind the prefill: cold step, then cached steps."""
