@@ -460,6 +460,31 @@ def run_ours(args):
             sweep.append({"reused": n_reuse, "rows": m, "us_per_layer": us, "floor_us_measured": f_meas,
                           "frac_of_roofline_measured": f_meas / us, "frac_of_roofline_nominal": f_nom / us})
         check_ctx(ctx, tokens, cfg.vocab, "layer sweep")
+
+        # ---------------------------------------------------------------- the paper's intra-frame pruning baseline (Table 2, +FastV)
+        def pruned_step(t):
+            vb.vlac_step_pruned(ctx, cache, frames_d[t:t + 1], feats_d[t:t + 1], ids_d, 2, cfg.n_vision // 2, tokens)
+        for i in range(3):
+            pruned_step(1 + i)
+        tot_p, _ = timed_loop(lambda i: pruned_step(2 + W + i), Kx)
+        got = vb.selection_to_host(vb.vlac_selection_view(cache))
+        extra["pruning_baseline"] = {
+            "note": "vlac_step_pruned: no reuse across frames; half of the vision tokens dropped after layer 1 by the attention they received "
+                    "(FastV-style, the comparison row of the paper's Table 2), on the same kernels",
+            "prune_layer": 2, "n_keep": cfg.n_vision // 2, "ms_per_step": tot_p / Kx, "rows_per_layer_first_last": [int(got["M"][0, 0]), int(got["M"][0, -1])]}
+        check_ctx(ctx, tokens, cfg.vocab, "pruning baseline")
+
+        # ---------------------------------------------------------------- selection alone: byte frames and bf16 normalised frames
+        fb = (((frames_d[1:3].float() / 255.0) - 0.45) / 0.225).to(torch.bfloat16)
+        vb.vlac_cache_write(cache, vb.PART_PREV_FRAME_BF16, 0, 0, fb[0].contiguous())
+        sel_us = {}
+        for name, fn in (("byte_frames", lambda i: vb.vlac_select(ctx, cache, frames_d[2:3], params)),
+                         ("bf16_frames", lambda i: vb.vlac_select_bf16(ctx, cache, fb[1:2].contiguous(), params))):
+            for i in range(3):
+                fn(i)
+            tot_s, _ = timed_loop(fn, 50)
+            sel_us[name] = 1e3 * tot_s / 50
+        extra["selection_alone_us"] = dict(sel_us, note="vlac_select / vlac_select_bf16, direct launches (2-3 kernels), 50 calls each")
         extra["cfg2_single_layer_sweep"] = {
             "note": "one 7B-shaped layer through vlac_layer_forward (7 direct launches: norm, Q/K/V, attention, output projection, norm, "
                     "gate/up, down + fold), reused vision tokens swept as in the paper's Table 4; floor = max(weights+K/V bytes / HBM, flops / "

@@ -320,6 +320,261 @@ __global__ void __launch_bounds__(AT_THREADS, 1) attention_tile_kernel(AttnTileA
   for (int v = tid; v < a.Lv; v += 128) dst[v] = ((colsum[v] + colsum[a.Lv + v]) + colsum[2 * a.Lv + v]) + colsum[3 * a.Lv + v];
 }
 
+// ------------------------------------------------------------------------------------------------
+// The same attention on the 5th-generation tensor cores (tcgen05 + tensor memory), used whenever a
+// query tile can see at most TA_MAXK = 320 keys (sequences of up to 320 positions; longer ones take the
+// warp-level kernel above).  One CTA per (128-query tile, sequence, head):
+//   warp 4, one lane: TMA loads of Q, K, V (64-row boxes, 128-byte swizzle), then the MMAs
+//       S[128 q x keys]  = Q K^T    A = Q (K-major), B = K (K-major), accumulator columns 0 .. keys-1
+//       O[128 q x d]     = P V      A = P (bf16, written by the softmax warps over the K tile, K-major),
+//                                   B = V as it lies in the cache, keys x d: the MN-major operand form
+//   warps 0-3: one query row per thread (TMEM lane = row).  Exact softmax in two sweeps over the row's
+//       scores (maximum; then exponentials, row sum and P), then O / row sum -> bf16 output row.
+//   Text rows behind the vision block add their normalised probabilities per vision key (a fixed shuffle tree
+//   per warp, warps added in order) into the per-tile partial that emit_from_tiles_kernel folds.
+constexpr int TA_Q = 128;
+constexpr int TA_MAXK = 320;                    // most score columns of a tile: Q + K/P + V tiles of that many keys fill the shared memory
+constexpr int TA_THREADS = 160;
+constexpr int TA_O_COL = 384;                   // accumulator columns of O behind the score columns
+
+__device__ __forceinline__ unsigned long long ta_desc(unsigned addr, unsigned lbo_bytes, unsigned sbo_bytes) {
+  unsigned long long d = 0;
+  d |= (unsigned long long)((addr & 0x3FFFFu) >> 4);
+  d |= (unsigned long long)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (unsigned long long)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= (unsigned long long)1 << 46;               // descriptor version of this architecture
+  d |= (unsigned long long)2 << 61;               // SWIZZLE_128B
+  return d;
+}
+// f32 accumulate, bf16 x bf16; A K-major; B K-major or MN-major
+__device__ __forceinline__ unsigned ta_idesc(int M, int N, bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) | ((unsigned)(N >> 3) << 17) | ((unsigned)(M >> 4) << 24);
+}
+__device__ __forceinline__ void ta_mma(unsigned tmem_d, unsigned long long a, unsigned long long b, unsigned idesc, unsigned accumulate) {
+  asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+               ::"r"(tmem_d), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void ta_commit(unsigned long long* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void ta_ld16(unsigned taddr, float* v) {
+  unsigned r[16];
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                 "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+               : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+template <int DH>
+__global__ void __launch_bounds__(TA_THREADS, 1) attention_tc_kernel(AttnTileArgs a) {
+  extern __shared__ __align__(1024) unsigned char ta_raw[];
+  __shared__ __align__(8) unsigned long long bar_qk, bar_v, bar_s, bar_o;
+  __shared__ unsigned tmem_slot;
+  __shared__ int abort_flag;
+  constexpr int HALVES = DH / 64;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tile = blockIdx.x, b = blockIdx.y, h = blockIdx.z;
+  if (tid == 0) {
+    mbar_init(&bar_qk, 1); mbar_init(&bar_v, 1); mbar_init(&bar_s, 1); mbar_init(&bar_o, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+  pdl_trigger();
+  pdl_wait();                                                   // the row lists, Q and the caches come from earlier kernels
+
+  int off = 0;
+  for (int bb = 0; bb < b; ++bb) off += a.M[(size_t)bb * a.nl + a.layer];
+  const int Mb = a.M[(size_t)b * a.nl + a.layer];
+  const int n_valid = min(TA_Q, Mb - tile * TA_Q);
+  if (n_valid <= 0) {                                           // no rows: the partial of this tile must still read as zero
+    if (a.partial)
+      for (int v = tid; v < a.Lv; v += TA_THREADS) a.partial[(((size_t)b * a.tiles + tile) * a.H + h) * a.Lv + v] = 0.f;
+    return;
+  }
+  const int row0 = off + tile * TA_Q;
+  const int pos_last = a.rowmap[row0 + n_valid - 1] - b * a.L;
+  const int n_keys = ((pos_last + 1 + 15) / 16) * 16;            // score columns (those behind pos_last are masked)
+  const int n_kb = (n_keys + 63) / 64;                           // 64-row boxes of K and of V per half of the head
+  const int v1 = a.v0 + a.Lv;
+  const bool has_text = a.partial != nullptr && pos_last >= v1;
+
+  // shared memory: Q | K, later overwritten by P | V | column sums
+  const unsigned kv_half = (unsigned)n_kb * 64u * 128u;          // bytes of one half (64 dims) of K or V
+  const unsigned kp_bytes = max(kv_half * HALVES, (unsigned)n_kb * (TA_Q * 128u));   // K tile, or P: 64-key chunks of 128 rows
+  unsigned char* q_s = ta_raw;
+  unsigned char* k_s = q_s + HALVES * TA_Q * 128;
+  unsigned char* v_s = k_s + kp_bytes;
+  float* colsum = reinterpret_cast<float*>(v_s + kv_half * HALVES);      // [4 warps][Lv]
+  if ((smem_u32(ta_raw) & 1023u) && tid == 0) { abort_flag = 1; if (a.dev_error) atomicCAS(a.dev_error, 0, 0x74000); }
+
+  if (warp == 4) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const unsigned tmem = tmem_slot;
+  bool ok = abort_flag == 0;
+
+  if (warp == 4) {
+    if (lane == 0 && ok) {
+      // ---- loads
+      mbar_expect_tx(&bar_qk, (unsigned)(HALVES * TA_Q * 128) + kv_half * HALVES);
+      const int yk = b * a.max_seq;
+#pragma unroll
+      for (int hf = 0; hf < HALVES; ++hf) {
+        tma_load_2d(q_s + hf * TA_Q * 128, a.tm_q, h * DH + hf * 64, row0, &bar_qk);
+        tma_load_2d(q_s + hf * TA_Q * 128 + 64 * 128, a.tm_q, h * DH + hf * 64, row0 + 64, &bar_qk);
+        for (int i = 0; i < n_kb; ++i) tma_load_2d(k_s + hf * kv_half + i * 64 * 128, a.tm_k, h * DH + hf * 64, yk + i * 64, &bar_qk);
+      }
+      mbar_expect_tx(&bar_v, kv_half * HALVES);
+#pragma unroll
+      for (int hf = 0; hf < HALVES; ++hf)
+        for (int i = 0; i < n_kb; ++i) tma_load_2d(v_s + hf * kv_half + i * 64 * 128, a.tm_v, h * DH + hf * 64, yk + i * 64, &bar_v);
+      // ---- S = Q K^T
+      ok = mbar_wait(&bar_qk, 0, &abort_flag, a.dev_error, 0x75000);
+      if (ok) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const int n0 = min(n_keys, 256), n1 = n_keys - n0;
+        const unsigned id0 = ta_idesc(128, n0, false), id1 = n1 ? ta_idesc(128, n1, false) : 0u;
+#pragma unroll
+        for (int ks = 0; ks < DH / 16; ++ks) {
+          const unsigned koff = (unsigned)(ks >> 2) , kin = (unsigned)(ks & 3) * 32u;
+          const unsigned long long da = ta_desc(smem_u32(q_s) + koff * (TA_Q * 128) + kin, 16, 1024);
+          const unsigned kb_addr = smem_u32(k_s) + koff * kv_half + kin;
+          ta_mma(tmem, da, ta_desc(kb_addr, 16, 1024), id0, ks > 0);
+          if (n1) ta_mma(tmem + 256, da, ta_desc(kb_addr + 256 * 128, 16, 1024), id1, ks > 0);
+        }
+        ta_commit(&bar_s);
+      }
+    }
+  }
+  // ---- softmax warps: thread = query row
+  const int r = tid;                                             // valid for warps 0-3
+  int pos = -1;
+  float m = 0.f, inv_l = 0.f;
+  const float scale = rsqrtf((float)DH) * 1.44269504088896f;     // softmax in base 2
+  const unsigned char* hk = a.hidden_keys ? a.hidden_keys + (size_t)b * a.max_seq : nullptr;
+  if (warp < 4) {
+    if (r < n_valid) pos = a.rowmap[row0 + r] - b * a.L;
+    if (ok) ok = mbar_wait(&bar_s, 0, &abort_flag, a.dev_error, 0x76000);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const unsigned trow = tmem + ((unsigned)(32 * warp) << 16);
+    if (ok) {
+      float mx = -INFINITY;
+      for (int c0 = 0; c0 < n_keys; c0 += 16) {
+        float v[16];
+        ta_ld16(trow + (unsigned)c0, v);
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          const int key = c0 + c;
+          const bool vis = key <= pos && !(hk && hk[key]);
+          if (vis) mx = fmaxf(mx, v[c] * scale);
+        }
+      }
+      m = mx == -INFINITY ? 0.f : mx;
+      float l = 0.f;
+      // P (bf16) over the K tile: 64-key chunks of [128 rows][128 bytes], 16-byte pieces XOR-swizzled by the row
+      for (int c0 = 0; c0 < n_keys; c0 += 16) {
+        float v[16];
+        ta_ld16(trow + (unsigned)c0, v);
+        unsigned pk[8];
+#pragma unroll
+        for (int c = 0; c < 16; c += 2) {
+          const int key = c0 + c;
+          const bool vis0 = key <= pos && !(hk && hk[key]), vis1 = key + 1 <= pos && !(hk && hk[key + 1]);
+          const float p0 = vis0 ? exp2f(v[c] * scale - m) : 0.f, p1 = vis1 ? exp2f(v[c + 1] * scale - m) : 0.f;
+          l += p0 + p1;
+          pk[c >> 1] = pack_bf16(p0, p1);
+        }
+        const unsigned chunk = (unsigned)(c0 >> 6), piece = (unsigned)((c0 & 63) >> 3);
+        const unsigned base = smem_u32(k_s) + chunk * (TA_Q * 128u) + (unsigned)r * 128u;
+        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(base + (((piece) ^ ((unsigned)r & 7u)) << 4)), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
+        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(base + (((piece + 1u) ^ ((unsigned)r & 7u)) << 4)), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]) : "memory");
+      }
+      inv_l = l > 0.f ? 1.f / l : 0.f;
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // P was written by ordinary stores, the MMA reads it through the async proxy
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  }
+  __syncthreads();                                               // P complete (all rows), also orders the score reads before O's columns are written
+  if (warp == 4 && lane == 0 && ok && !abort_flag) {
+    // ---- O = P V
+    bool okv = mbar_wait(&bar_v, 0, &abort_flag, a.dev_error, 0x77000);
+    if (okv) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const unsigned ido = ta_idesc(128, DH, true);
+      for (int j = 0; j < n_keys / 16; ++j) {
+        const unsigned long long da = ta_desc(smem_u32(k_s) + (unsigned)(j >> 2) * (TA_Q * 128u) + (unsigned)(j & 3) * 32u, 16, 1024);
+        // V block: 16 key rows of 128 bytes from row 16 j; the second 64 dims lie kv_half bytes further (leading offset)
+        const unsigned long long db = ta_desc(smem_u32(v_s) + (unsigned)j * 16u * 128u, kv_half, 1024);
+        ta_mma(tmem + TA_O_COL, da, db, ido, j > 0);
+      }
+      ta_commit(&bar_o);
+    }
+  }
+  if (warp < 4) {
+    if (ok) ok = mbar_wait(&bar_o, 0, &abort_flag, a.dev_error, 0x78000);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const unsigned trow = tmem + ((unsigned)(32 * warp) << 16);
+    if (ok) {
+      bf16* dst = a.out + (size_t)(row0 + min(r, n_valid - 1)) * ((size_t)a.H * DH) + (size_t)h * DH;
+#pragma unroll
+      for (int c0 = 0; c0 < DH; c0 += 16) {
+        float v[16];
+        ta_ld16(trow + (unsigned)(TA_O_COL + c0), v);              // (collective load: every lane of the warp takes part)
+        if (r >= n_valid) continue;
+        uint4 o0, o1;
+        o0.x = pack_bf16(v[0] * inv_l, v[1] * inv_l); o0.y = pack_bf16(v[2] * inv_l, v[3] * inv_l);
+        o0.z = pack_bf16(v[4] * inv_l, v[5] * inv_l); o0.w = pack_bf16(v[6] * inv_l, v[7] * inv_l);
+        o1.x = pack_bf16(v[8] * inv_l, v[9] * inv_l); o1.y = pack_bf16(v[10] * inv_l, v[11] * inv_l);
+        o1.z = pack_bf16(v[12] * inv_l, v[13] * inv_l); o1.w = pack_bf16(v[14] * inv_l, v[15] * inv_l);
+        *reinterpret_cast<uint4*>(dst + c0) = o0;
+        *reinterpret_cast<uint4*>(dst + c0 + 8) = o1;
+      }
+    }
+    // ---- text-to-vision scores of this tile: normalised probabilities of the text rows, summed per vision key
+    if (a.partial != nullptr) {
+      const bool text_row = ok && pos >= v1;
+      const bool warp_has = __any_sync(0xffffffffu, text_row);
+      for (int v = lane; v < a.Lv; v += 32) colsum[warp * a.Lv + v] = 0.f;
+      __syncwarp();
+      if (has_text && warp_has) {
+        const int c_lo = (a.v0 / 16) * 16, c_hi = min(n_keys, ((v1 + 15) / 16) * 16);
+        for (int c0 = c_lo; c0 < c_hi; c0 += 16) {
+          float v[16];
+          ta_ld16(trow + (unsigned)c0, v);
+#pragma unroll
+          for (int c = 0; c < 16; ++c) {
+            const int key = c0 + c;
+            float p = 0.f;
+            if (text_row && !(hk && key < a.max_seq && hk[key])) p = exp2f(v[c] * scale - m) * inv_l;     // text rows see every vision key still in the sequence
+#pragma unroll
+            for (int sh = 16; sh > 0; sh >>= 1) p += __shfl_xor_sync(0xffffffffu, p, sh);
+            const int vv = key - a.v0;
+            if (lane == 0 && vv >= 0 && vv < a.Lv) colsum[warp * a.Lv + vv] = p;
+          }
+        }
+      }
+      asm volatile("bar.sync 1, 128;");
+      float* dstp = a.partial + (((size_t)b * a.tiles + tile) * a.H + h) * a.Lv;
+      for (int v = tid; v < a.Lv; v += 128) dstp[v] = ((colsum[v] + colsum[a.Lv + v]) + colsum[2 * a.Lv + v]) + colsum[3 * a.Lv + v];
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  }
+  __syncthreads();
+  if (warp == 4) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+  }
+}
+
 // sum of the per-tile partials in tile order, divided by the number of text rows
 __global__ void __launch_bounds__(256) emit_from_tiles_kernel(const float* partial, float* attn_next_layer, size_t seq_stride,
                                                               int tiles, int n_tp, int H, int Lv, size_t layer_stride_in) {
@@ -342,14 +597,28 @@ constexpr size_t at_smem(int Lv) {
   return 1024 + (size_t)(DH / 64) * AT_Q * 128 + (size_t)AT_STAGES * 2 * (DH / 64) * AT_KB * 128 + (size_t)4 * Lv * sizeof(float);
 }
 
+// dynamic shared memory of the tensor-memory kernel for sequences of L positions
+static size_t ta_smem(int dh, int L, int Lv) {
+  const size_t halves = dh / 64, n_kb = ((size_t)((L + 15) / 16 * 16) + 63) / 64;
+  const size_t kv = n_kb * 64 * 128 * halves, p = n_kb * TA_Q * 128;
+  return halves * TA_Q * 128 + (kv > p ? kv : p) + kv + (size_t)4 * Lv * sizeof(float);
+}
+
 }  // namespace
 
 int vlac_attention_setup(vlac_ctx* ctx) {
   const vlac_config& g = ctx->cfg;
   ctx->attn_tiles = 0;
   if (g.head_dim != 64 && g.head_dim != 128) return VLAC_ERR_INVALID_ARG;
-  const int tiles = (ctx->L + AT_Q - 1) / AT_Q;
+  // the tensor-memory kernel holds all keys a tile can see in shared memory at once
+  ctx->attn_tc = ((ctx->L + 15) / 16) * 16 <= TA_MAXK ? 1 : 0;
+  const int tiles = ctx->attn_tc ? (ctx->L + TA_Q - 1) / TA_Q : (ctx->L + AT_Q - 1) / AT_Q;
   cudaError_t e;
+  if (ctx->attn_tc) {
+    if (g.head_dim == 128) e = cudaFuncSetAttribute(attention_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ta_smem(128, ctx->L, ctx->Lv));
+    else e = cudaFuncSetAttribute(attention_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ta_smem(64, ctx->L, ctx->Lv));
+    if (e != cudaSuccess) { vlac_note_cuda_error(e, __FILE__, __LINE__); return VLAC_ERR_CUDA; }
+  }
   if (g.head_dim == 128) e = cudaFuncSetAttribute(attention_tile_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)at_smem<128>(ctx->Lv));
   else e = cudaFuncSetAttribute(attention_tile_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)at_smem<64>(ctx->Lv));
   if (e != cudaSuccess) { vlac_note_cuda_error(e, __FILE__, __LINE__); return VLAC_ERR_CUDA; }
@@ -406,6 +675,10 @@ int vlac_launch_prefill_attention(vlac_ctx* ctx, vlac_cache* c, int layer, cudaS
   a.layer = layer; a.nl = g.n_layers; a.B = B; a.L = ctx->L; a.max_seq = ctx->max_seq; a.H = g.n_heads;
   a.v0 = g.n_text_pre; a.Lv = ctx->Lv; a.tiles = ctx->attn_tiles;
   const dim3 grid(ctx->attn_tiles, B, g.n_heads);
+  if (ctx->attn_tc) {
+    if (g.head_dim == 128) VLAC_CUDA_CHECK(launch_pdl(attention_tc_kernel<128>, grid, dim3(TA_THREADS), ta_smem(128, ctx->L, ctx->Lv), s, a));
+    else VLAC_CUDA_CHECK(launch_pdl(attention_tc_kernel<64>, grid, dim3(TA_THREADS), ta_smem(64, ctx->L, ctx->Lv), s, a));
+  } else
   if (g.head_dim == 128) VLAC_CUDA_CHECK(launch_pdl(attention_tile_kernel<128>, grid, dim3(AT_THREADS), at_smem<128>(ctx->Lv), s, a));
   else VLAC_CUDA_CHECK(launch_pdl(attention_tile_kernel<64>, grid, dim3(AT_THREADS), at_smem<64>(ctx->Lv), s, a));
   VLAC_LAUNCH_CHECK(ctx);

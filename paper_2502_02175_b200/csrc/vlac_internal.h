@@ -69,7 +69,8 @@ struct vlac_ctx {
   void* tmaps_host;                  // host array of TMA tensor maps (weights per layer, activation buffers)
   int chunk_ok;                      // the n_action rows of a chunk fit the matrix-vector kernels as columns (vlac_step_chunk usable)
   void* tmap_q;                      // device tensor map of the query buffer (tiled attention)
-  int attn_tiles;                    // 64-query tiles per sequence
+  int attn_tc;                       // 1: prefill attention on tcgen05 (every key of a tile fits shared memory at once)
+  int attn_tiles;                    // query tiles per sequence (128 queries with attn_tc, else 64)
   float* probs_all;                  // [n_layers][max_batch][tiles][n_heads][Lv]: per-tile column sums of every layer of a step
   int prune_layer;                   // > 0 while a pruning-baseline step is enqueued: layers >= it skip the positions in hidden_keys
   int defer_emit;                    // set while a whole step is enqueued: text-to-vision scores of all layers are formed by one kernel at its end
