@@ -324,17 +324,18 @@ __global__ void __launch_bounds__(AT_THREADS, 1) attention_tile_kernel(AttnTileA
 // The same attention on the 5th-generation tensor cores (tcgen05 + tensor memory), used whenever a
 // query tile can see at most TA_MAXK = 320 keys (sequences of up to 320 positions; longer ones take the
 // warp-level kernel above).  One CTA per (128-query tile, sequence, head):
-//   warp 4, one lane: TMA loads of Q, K, V (64-row boxes, 128-byte swizzle), then the MMAs
+//   warp 8, one lane: TMA loads of Q, K, V (64-row boxes, 128-byte swizzle), then the MMAs
 //       S[128 q x keys]  = Q K^T    A = Q (K-major), B = K (K-major), accumulator columns 0 .. keys-1
 //       O[128 q x d]     = P V      A = P (bf16, written by the softmax warps over the K tile, K-major),
 //                                   B = V as it lies in the cache, keys x d: the MN-major operand form
-//   warps 0-3: one query row per thread (TMEM lane = row).  Exact softmax in two sweeps over the row's
-//       scores (maximum; then exponentials, row sum and P), then O / row sum -> bf16 output row.
+//   warps 0-7: a query row per PAIR of threads (TMEM lane = row; warps w and w + 4 share the rows of quarter w and take
+//       alternate 64-column chunks).  Exact softmax in two sweeps over the row's scores (maximum; then exponentials,
+//       row sum and P; the halves meet through shared memory), then O / row sum -> bf16 output row.
 //   Text rows behind the vision block add their normalised probabilities per vision key (a fixed shuffle tree
 //   per warp, warps added in order) into the per-tile partial that emit_from_tiles_kernel folds.
 constexpr int TA_Q = 128;
 constexpr int TA_MAXK = 320;                    // most score columns of a tile: Q + K/P + V tiles of that many keys fill the shared memory
-constexpr int TA_THREADS = 160;
+constexpr int TA_THREADS = 288;                 // warps 0-7: softmax / epilogue (two warps per quarter of the rows), warp 8: TMA + MMA
 constexpr int TA_O_COL = 384;                   // accumulator columns of O behind the score columns
 
 __device__ __forceinline__ unsigned long long ta_desc(unsigned addr, unsigned lbo_bytes, unsigned sbo_bytes) {
@@ -368,12 +369,39 @@ __device__ __forceinline__ void ta_ld16(unsigned taddr, float* v) {
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+__device__ __forceinline__ float ta_ex2(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+// barrier over the 256 softmax threads that also makes `ok` the same in all of them (a wait that gave up in one thread
+// must not leave the others standing at a later barrier)
+__device__ __forceinline__ bool ta_all_ok(bool ok) {
+  unsigned r;
+  asm volatile("{\n.reg .pred p, q;\nsetp.ne.u32 q, %1, 0;\nbarrier.cta.red.and.pred p, 2, 256, q;\nselp.u32 %0, 1, 0, p;\n}\n"
+               : "=r"(r) : "r"((unsigned)ok) : "memory");
+  return r != 0;
+}
+// 32 accumulator columns of this thread's row with one wait.  The loops that use it are kept rolled on purpose: a launch
+// starts with a cold instruction cache, and straight-line code of several KB per sweep cost more in instruction fetches
+// than the arithmetic it held.
+__device__ __forceinline__ void ta_ld32(unsigned taddr, float* v) {
+  unsigned r[32];
+#pragma unroll
+  for (int g = 0; g < 2; ++g)
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : "=r"(r[16 * g + 0]), "=r"(r[16 * g + 1]), "=r"(r[16 * g + 2]), "=r"(r[16 * g + 3]), "=r"(r[16 * g + 4]), "=r"(r[16 * g + 5]),
+                   "=r"(r[16 * g + 6]), "=r"(r[16 * g + 7]), "=r"(r[16 * g + 8]), "=r"(r[16 * g + 9]), "=r"(r[16 * g + 10]), "=r"(r[16 * g + 11]),
+                   "=r"(r[16 * g + 12]), "=r"(r[16 * g + 13]), "=r"(r[16 * g + 14]), "=r"(r[16 * g + 15])
+                 : "r"(taddr + 16u * g));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
 template <int DH>
 __global__ void __launch_bounds__(TA_THREADS, 1) attention_tc_kernel(AttnTileArgs a) {
   extern __shared__ __align__(1024) unsigned char ta_raw[];
   __shared__ __align__(8) unsigned long long bar_qk, bar_v, bar_s, bar_o;
   __shared__ unsigned tmem_slot;
-  __shared__ int abort_flag;
+  __shared__ int abort_flag, first_text;
+  __shared__ float red_m[2][TA_Q], red_l[2][TA_Q];
   constexpr int HALVES = DH / 64;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int tile = blockIdx.x, b = blockIdx.y, h = blockIdx.z;
@@ -412,7 +440,7 @@ __global__ void __launch_bounds__(TA_THREADS, 1) attention_tc_kernel(AttnTileArg
   float* colsum = reinterpret_cast<float*>(v_s + kv_half * HALVES);      // [4 warps][Lv]
   if ((smem_u32(ta_raw) & 1023u) && tid == 0) { abort_flag = 1; if (a.dev_error) atomicCAS(a.dev_error, 0, 0x74000); }
 
-  if (warp == 4) {
+  if (warp == 8) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(512u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -422,7 +450,7 @@ __global__ void __launch_bounds__(TA_THREADS, 1) attention_tc_kernel(AttnTileArg
   const unsigned tmem = tmem_slot;
   bool ok = abort_flag == 0;
 
-  if (warp == 4) {
+  if (warp == 8) {
     if (lane == 0 && ok) {
       // ---- loads
       mbar_expect_tx(&bar_qk, (unsigned)(HALVES * TA_Q * 128) + kv_half * HALVES);
@@ -455,56 +483,70 @@ __global__ void __launch_bounds__(TA_THREADS, 1) attention_tc_kernel(AttnTileArg
       }
     }
   }
-  // ---- softmax warps: thread = query row
-  const int r = tid;                                             // valid for warps 0-3
+  // ---- softmax warps: thread = (query row, half of the 64-column chunks)
+  const int q4 = warp & 3, hf = warp >> 2;                       // row quarter (the TMEM lanes this warp may read); chunk parity
+  const int r = 32 * q4 + lane;                                  // valid for warps 0-7
   int pos = -1;
   float m = 0.f, inv_l = 0.f;
   const float scale = rsqrtf((float)DH) * 1.44269504088896f;     // softmax in base 2
   const unsigned char* hk = a.hidden_keys ? a.hidden_keys + (size_t)b * a.max_seq : nullptr;
-  if (warp < 4) {
+  if (warp < 8) {
     if (r < n_valid) pos = a.rowmap[row0 + r] - b * a.L;
     if (ok) ok = mbar_wait(&bar_s, 0, &abort_flag, a.dev_error, 0x76000);
+    ok = ta_all_ok(ok);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const unsigned trow = tmem + ((unsigned)(32 * warp) << 16);
+    const unsigned trow = tmem + ((unsigned)(32 * q4) << 16);
     if (ok) {
+      // (columns are read 32 at a time; those at and behind n_keys hold stale values and are masked like any key > pos)
       float mx = -INFINITY;
-      for (int c0 = 0; c0 < n_keys; c0 += 16) {
-        float v[16];
-        ta_ld16(trow + (unsigned)c0, v);
+#pragma unroll 1
+      for (int g = 0; g < 2 * n_kb; ++g) {
+        const int c0 = (g >> 1) * 64 + (g & 1) * 32;
+        if (((g >> 1) & 1) != hf) continue;
+        float v[32];
+        ta_ld32(trow + (unsigned)c0, v);
 #pragma unroll
-        for (int c = 0; c < 16; ++c) {
+        for (int c = 0; c < 32; ++c) {
           const int key = c0 + c;
           const bool vis = key <= pos && !(hk && hk[key]);
           if (vis) mx = fmaxf(mx, v[c] * scale);
         }
       }
+      red_m[hf][r] = mx;
+      asm volatile("bar.sync 1, 256;");
+      mx = fmaxf(red_m[0][r], red_m[1][r]);
       m = mx == -INFINITY ? 0.f : mx;
       float l = 0.f;
       // P (bf16) over the K tile: 64-key chunks of [128 rows][128 bytes], 16-byte pieces XOR-swizzled by the row
-      for (int c0 = 0; c0 < n_keys; c0 += 16) {
-        float v[16];
-        ta_ld16(trow + (unsigned)c0, v);
-        unsigned pk[8];
+#pragma unroll 1
+      for (int g = 0; g < 2 * n_kb; ++g) {                          // half of a 64-key chunk of P = 64 bytes of this row
+        if (((g >> 1) & 1) != hf) continue;
+        const int c0 = (g >> 1) * 64 + (g & 1) * 32;
+        float v[32];
+        ta_ld32(trow + (unsigned)c0, v);
+        unsigned char* prow = k_s + (size_t)(g >> 1) * (TA_Q * 128u) + (size_t)r * 128u;
 #pragma unroll
-        for (int c = 0; c < 16; c += 2) {
-          const int key = c0 + c;
-          const bool vis0 = key <= pos && !(hk && hk[key]), vis1 = key + 1 <= pos && !(hk && hk[key + 1]);
-          const float p0 = vis0 ? exp2f(v[c] * scale - m) : 0.f, p1 = vis1 ? exp2f(v[c + 1] * scale - m) : 0.f;
-          l += p0 + p1;
-          pk[c >> 1] = pack_bf16(p0, p1);
+        for (int pc = 0; pc < 4; ++pc) {
+          unsigned pk[4];
+#pragma unroll
+          for (int c = 0; c < 8; c += 2) {
+            const int key = c0 + pc * 8 + c;
+            const bool vis0 = key <= pos && !(hk && hk[key]), vis1 = key + 1 <= pos && !(hk && hk[key + 1]);
+            const float p0 = vis0 ? ta_ex2(v[pc * 8 + c] * scale - m) : 0.f, p1 = vis1 ? ta_ex2(v[pc * 8 + c + 1] * scale - m) : 0.f;
+            l += p0 + p1;
+            pk[c >> 1] = pack_bf16(p0, p1);
+          }
+          const unsigned piece = (unsigned)((g & 1) * 4 + pc);
+          *reinterpret_cast<uint4*>(prow + ((piece ^ ((unsigned)r & 7u)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
         }
-        const unsigned chunk = (unsigned)(c0 >> 6), piece = (unsigned)((c0 & 63) >> 3);
-        const unsigned base = smem_u32(k_s) + chunk * (TA_Q * 128u) + (unsigned)r * 128u;
-        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(base + (((piece) ^ ((unsigned)r & 7u)) << 4)), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
-        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(base + (((piece + 1u) ^ ((unsigned)r & 7u)) << 4)), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]) : "memory");
       }
-      inv_l = l > 0.f ? 1.f / l : 0.f;
+      red_l[hf][r] = l;
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // P was written by ordinary stores, the MMA reads it through the async proxy
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   }
   __syncthreads();                                               // P complete (all rows), also orders the score reads before O's columns are written
-  if (warp == 4 && lane == 0 && ok && !abort_flag) {
+  if (warp == 8 && lane == 0 && ok && !abort_flag) {
     // ---- O = P V
     bool okv = mbar_wait(&bar_v, 0, &abort_flag, a.dev_error, 0x77000);
     if (okv) {
@@ -519,14 +561,16 @@ __global__ void __launch_bounds__(TA_THREADS, 1) attention_tc_kernel(AttnTileArg
       ta_commit(&bar_o);
     }
   }
-  if (warp < 4) {
+  if (warp < 8) {
+    { const float l = red_l[0][r] + red_l[1][r]; inv_l = l > 0.f ? 1.f / l : 0.f; }      // (written before the barrier above)
     if (ok) ok = mbar_wait(&bar_o, 0, &abort_flag, a.dev_error, 0x78000);
+    ok = ta_all_ok(ok);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const unsigned trow = tmem + ((unsigned)(32 * warp) << 16);
+    const unsigned trow = tmem + ((unsigned)(32 * q4) << 16);
     if (ok) {
       bf16* dst = a.out + (size_t)(row0 + min(r, n_valid - 1)) * ((size_t)a.H * DH) + (size_t)h * DH;
 #pragma unroll
-      for (int c0 = 0; c0 < DH; c0 += 16) {
+      for (int c0 = hf * (DH / 2); c0 < (hf + 1) * (DH / 2); c0 += 16) {
         float v[16];
         ta_ld16(trow + (unsigned)(TA_O_COL + c0), v);              // (collective load: every lane of the warp takes part)
         if (r >= n_valid) continue;
@@ -539,37 +583,62 @@ __global__ void __launch_bounds__(TA_THREADS, 1) attention_tc_kernel(AttnTileArg
         *reinterpret_cast<uint4*>(dst + c0 + 8) = o1;
       }
     }
-    // ---- text-to-vision scores of this tile: normalised probabilities of the text rows, summed per vision key
+    // ---- text-to-vision scores of this tile: normalised probabilities of the text rows, summed per vision key.
+    // The text rows (the last rows of the tile) put their probabilities into the shared memory the K / P tile no longer
+    // needs, a batch of rows at a time; then every thread adds up two columns over the batch in row order.
     if (a.partial != nullptr) {
-      const bool text_row = ok && pos >= v1;
-      const bool warp_has = __any_sync(0xffffffffu, text_row);
-      for (int v = lane; v < a.Lv; v += 32) colsum[warp * a.Lv + v] = 0.f;
-      __syncwarp();
-      if (has_text && warp_has) {
-        const int c_lo = (a.v0 / 16) * 16, c_hi = min(n_keys, ((v1 + 15) / 16) * 16);
-        for (int c0 = c_lo; c0 < c_hi; c0 += 16) {
-          float v[16];
-          ta_ld16(trow + (unsigned)c0, v);
+      float* dstp = a.partial + (((size_t)b * a.tiles + tile) * a.H + h) * a.Lv;
+      if (!has_text || !ok) {
+        for (int v = tid; v < a.Lv; v += 256) dstp[v] = 0.f;
+      } else {
+        const bool text_row = pos >= v1;
+        if (hf == 0 && text_row && (r == 0 || a.rowmap[row0 + r - 1] - b * a.L < v1)) first_text = r;       // exactly one thread
+        asm volatile("bar.sync 1, 256;");
+        const int t0 = first_text, n_text = n_valid - t0;
+        const int pitch = a.Lv + 4;                                 // floats per row of the staging area
+        float* stage = reinterpret_cast<float*>(k_s);
+        const int cap = max(1, (int)(kp_bytes / (pitch * sizeof(float))));
+        float tot[2] = {0.f, 0.f};                                 // columns tid, tid + 256 (L_v <= 512)
+        const int c_lo = (a.v0 / 64) * 64, c_hi = min(n_kb * 64, ((v1 + 63) / 64) * 64);
+        for (int b0 = 0; b0 < n_text; b0 += cap) {
+          const int ti = r - t0 - b0;                               // this thread's row inside the batch
+          const bool mine = text_row && ti >= 0 && ti < cap;
+          if (__any_sync(0xffffffffu, mine)) {
+#pragma unroll 1
+            for (int c0 = c_lo + 32 * hf; c0 < c_hi; c0 += 64) {
+              float v[32];
+              ta_ld32(trow + (unsigned)c0, v);
+              if (mine) {
 #pragma unroll
-          for (int c = 0; c < 16; ++c) {
-            const int key = c0 + c;
-            float p = 0.f;
-            if (text_row && !(hk && key < a.max_seq && hk[key])) p = exp2f(v[c] * scale - m) * inv_l;     // text rows see every vision key still in the sequence
-#pragma unroll
-            for (int sh = 16; sh > 0; sh >>= 1) p += __shfl_xor_sync(0xffffffffu, p, sh);
-            const int vv = key - a.v0;
-            if (lane == 0 && vv >= 0 && vv < a.Lv) colsum[warp * a.Lv + vv] = p;
+                for (int c = 0; c < 32; ++c) {
+                  const int key = c0 + c, vv = key - a.v0;
+                  if (vv >= 0 && vv < a.Lv)
+                    stage[(size_t)ti * pitch + vv] = (hk && hk[key]) ? 0.f : ta_ex2(v[c] * scale - m) * inv_l;   // text rows see every vision key still in the sequence
+                }
+              }
+            }
           }
+          asm volatile("bar.sync 1, 256;");
+          const int nb = min(cap, n_text - b0);
+#pragma unroll
+          for (int k = 0; k < 2; ++k) {
+            const int v = tid + 256 * k;
+            if (v < a.Lv)
+              for (int i = 0; i < nb; ++i) tot[k] += stage[(size_t)i * pitch + v];
+          }
+          asm volatile("bar.sync 1, 256;");
+        }
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+          const int v = tid + 256 * k;
+          if (v < a.Lv) dstp[v] = tot[k];
         }
       }
-      asm volatile("bar.sync 1, 128;");
-      float* dstp = a.partial + (((size_t)b * a.tiles + tile) * a.H + h) * a.Lv;
-      for (int v = tid; v < a.Lv; v += 128) dstp[v] = ((colsum[v] + colsum[a.Lv + v]) + colsum[2 * a.Lv + v]) + colsum[3 * a.Lv + v];
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   }
   __syncthreads();
-  if (warp == 4) {
+  if (warp == 8) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
   }
