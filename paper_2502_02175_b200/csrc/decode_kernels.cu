@@ -15,6 +15,7 @@ namespace {
 __device__ __forceinline__ float bf2f(bf16 x) { return __bfloat162float(x); }
 
 enum { GV_QKV = 0, GV_RESID = 1, GV_SWIGLU = 2, GV_LOGITS = 3 };
+constexpr int DS_MAX_SPLITS = 8;         // key splits per (head, query row) of the single-row attention at most
 
 struct GemvArgs {
   const float* x_f32;      // [nb][K] fp32 source (normalised with `gain`), or NULL
@@ -32,6 +33,10 @@ struct GemvArgs {
                            // launch covers only K of their columns (0: the pitch is K)
   int cps;                 // QKV: columns per sequence (0 or 1: one row per sequence at position `pos`; n: column c is
                            // row pos + c % n of sequence c / n -- an action chunk decoded in parallel)
+  // RESID fed by the single-row attention: x is the combination of `ns` key splits per head (decode_attention_split_kernel):
+  // x[b][h d + e] = sum_s w_s o[b][h][s][e] / sum_s w_s l_s with w_s = exp(m_s - max_s m_s); parts_ml holds (m_s, l_s)
+  const float *parts_o, *parts_ml;
+  int ns, col0;            // splits; first column of x this launch covers (a launch over a slice of K)
   float* x_out;            // RESID: [nb][N] +=
   bf16* h_out;             // SWIGLU: [nb][N]
   float* logits;           // LOGITS: [nb][N]
@@ -383,6 +388,8 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
   // weights depend on no earlier kernel: fill the ring before the dependency wait
 #pragma unroll
   for (int i = 0; i < GT_DEPTH; ++i) issue();
+  // (Requesting further weights into L2 from here, so that the memory stays busy while every CTA stands at a
+  // dependency, was measured and made the pass 5 to 11 per cent slower.)
   // the norm gains are constants too: two 8-element chunks per thread cover K <= 8192
   const int nchunk = K / 8;
   const bool x_cached = a.x_f32 != nullptr && nchunk <= 2 * GT_THREADS;
@@ -398,6 +405,7 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
   pdl_wait();
 
   // ---- activations -> shared memory as bf16 (RMSNorm here if a gain is given)
+  bool late_scale = false;
   if (a.x_f32 && nb > 1) {
     // several columns: all sums of squares in one sweep and one pair of barriers (column by column the CTA would
     // meet twice per column), then a second sweep over the few KB of inputs to scale and store them
@@ -453,52 +461,96 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
   for (int b = 0; b < nb; ++b) {
     if (a.x_f32) {
       const float* x = a.x_f32 + (size_t)b * K;
-      float4 xq[2][2];
-      float ss = 0.f;
       if (x_cached) {
+        // One column: the products are taken with gain * x and scaled by 1 / rms afterwards (the scale is common to the
+        // whole column), so the sum of squares is off the path to the first MMA: no barrier of its own, and the
+        // warps' sums are added up after the barrier that ends the staging.
+        float ss = 0.f;
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
           const int c = tid + i * GT_THREADS;
           if (c < nchunk) {
-            xq[i][0] = *reinterpret_cast<const float4*>(x + (size_t)c * 8);
-            xq[i][1] = *reinterpret_cast<const float4*>(x + (size_t)c * 8 + 4);
-          } else {
-            xq[i][0] = xq[i][1] = make_float4(0.f, 0.f, 0.f, 0.f);
-          }
-          ss += xq[i][0].x * xq[i][0].x + xq[i][0].y * xq[i][0].y + xq[i][0].z * xq[i][0].z + xq[i][0].w * xq[i][0].w;
-          ss += xq[i][1].x * xq[i][1].x + xq[i][1].y * xq[i][1].y + xq[i][1].z * xq[i][1].z + xq[i][1].w * xq[i][1].w;
-        }
-      } else {
-        for (int k = tid; k < K; k += GT_THREADS) { const float v = x[k]; ss += v * v; }
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-      __syncthreads();
-      if (lane == 0) red[warp] = ss;
-      __syncthreads();
-      float t = 0.f;
-#pragma unroll
-      for (int w = 0; w < GT_WARPS; ++w) t += red[w];
-      const float r = rsqrtf(t / (float)K + a.eps);
-      if (x_cached) {
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          const int c = tid + i * GT_THREADS;
-          if (c < nchunk) {
+            const float4 x0 = *reinterpret_cast<const float4*>(x + (size_t)c * 8), x1 = *reinterpret_cast<const float4*>(x + (size_t)c * 8 + 4);
+            ss += x0.x * x0.x + x0.y * x0.y + x0.z * x0.z + x0.w * x0.w + x1.x * x1.x + x1.y * x1.y + x1.z * x1.z + x1.w * x1.w;
             const __nv_bfloat162* g2 = reinterpret_cast<const __nv_bfloat162*>(&gq[i]);
-            const float xv[8] = {xq[i][0].x, xq[i][0].y, xq[i][0].z, xq[i][0].w, xq[i][1].x, xq[i][1].y, xq[i][1].z, xq[i][1].w};
+            const float xv[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
             uint4 o;
             __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&o);
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
               const float2 gf = __bfloat1622float2(g2[e]);
-              o2[e] = __floats2bfloat162_rn(xv[2 * e] * r * gf.x, xv[2 * e + 1] * r * gf.y);
+              o2[e] = __floats2bfloat162_rn(xv[2 * e] * gf.x, xv[2 * e + 1] * gf.y);
             }
-            *reinterpret_cast<uint4*>(xs + (size_t)b * KP + (size_t)c * 8) = o;
+            *reinterpret_cast<uint4*>(xs + (size_t)c * 8) = o;
           }
         }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        if (lane == 0) red[warp] = ss;
+        late_scale = true;
       } else {
+        float ss = 0.f;
+        for (int k = tid; k < K; k += GT_THREADS) { const float v = x[k]; ss += v * v; }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+        __syncthreads();
+        if (lane == 0) red[warp] = ss;
+        __syncthreads();
+        float t = 0.f;
+#pragma unroll
+        for (int w = 0; w < GT_WARPS; ++w) t += red[w];
+        const float r = rsqrtf(t / (float)K + a.eps);
         for (int k = tid; k < K; k += GT_THREADS) xs[(size_t)b * KP + k] = __float2bfloat16(x[k] * r * bf2f(a.gain[k]));
+      }
+    } else if (a.parts_o) {
+      const int d = a.d, ns = a.ns, H = (a.ld ? a.ld : K) / d;
+      for (int c = tid; c < K / 8; c += GT_THREADS) {
+        const int col = a.col0 + c * 8, h = col / d, e0 = col - h * d;
+        const float* ml = a.parts_ml + (size_t)(b * H + h) * ns * 2;
+        const float* po = a.parts_o + (size_t)(b * H + h) * ns * d + e0;
+        // every load of a batch of four splits is issued before anything is computed: the projection's first weights
+        // are waiting in the ring meanwhile
+        float2 mlv[DS_MAX_SPLITS];
+#pragma unroll
+        for (int i = 0; i < DS_MAX_SPLITS; ++i)
+          mlv[i] = i < ns ? __ldcg(reinterpret_cast<const float2*>(ml) + i) : make_float2(-INFINITY, 0.f);
+        float4 pv[4][2];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float4* src = reinterpret_cast<const float4*>(po + (size_t)min(i, ns - 1) * d);
+          pv[i][0] = __ldcg(src); pv[i][1] = __ldcg(src + 1);
+        }
+        float M = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < DS_MAX_SPLITS; ++i) M = fmaxf(M, mlv[i].x);
+        float den = 0.f, o[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) o[e] = 0.f;
+#pragma unroll
+        for (int i0 = 0; i0 < DS_MAX_SPLITS; i0 += 4) {
+          if (i0 >= ns) break;
+          if (i0 > 0) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float4* src = reinterpret_cast<const float4*>(po + (size_t)min(i0 + i, ns - 1) * d);
+              pv[i][0] = __ldcg(src); pv[i][1] = __ldcg(src + 1);
+            }
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const float mi = mlv[i0 + i].x;
+            const float w = (i0 + i < ns && mi != -INFINITY) ? __expf(mi - M) : 0.f;      // (a split without a visible key has weight 0)
+            den += w * mlv[i0 + i].y;
+            o[0] += w * pv[i][0].x; o[1] += w * pv[i][0].y; o[2] += w * pv[i][0].z; o[3] += w * pv[i][0].w;
+            o[4] += w * pv[i][1].x; o[5] += w * pv[i][1].y; o[6] += w * pv[i][1].z; o[7] += w * pv[i][1].w;
+          }
+        }
+        const float inv = den > 0.f ? 1.f / den : 0.f;
+        uint4 v;
+        __nv_bfloat162* v2 = reinterpret_cast<__nv_bfloat162*>(&v);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) v2[e] = __floats2bfloat162_rn(o[2 * e] * inv, o[2 * e + 1] * inv);
+        *reinterpret_cast<uint4*>(xs + (size_t)b * KP + (size_t)c * 8) = v;
       }
     } else {
       const uint4* src = reinterpret_cast<const uint4*>(a.x_bf16 + (size_t)b * (a.ld ? a.ld : K));
@@ -507,6 +559,13 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
     }
   }
   __syncthreads();
+  float rscale = 1.f;
+  if (late_scale) {
+    float t = 0.f;
+#pragma unroll
+    for (int w = 0; w < GT_WARPS; ++w) t += red[w];
+    rscale = rsqrtf(t / (float)K + a.eps);
+  }
 
   // ---- consume side
   const int col_n = lane >> 2;                                         // B column (sequence) this lane feeds
@@ -576,65 +635,86 @@ __global__ void __launch_bounds__(GT_THREADS, GT_MIN_CTAS) gemv_mma_kernel(GemvA
         } else {
           for (int w = 0; w < TW; ++w) { ya += src[((size_t)w * 16 + uu) * nbp + col]; yb += src[((size_t)w * 16 + uu + 8) * nbp + col]; }
         }
-        store_unit(a, fcu, col, ya, yb, fpre);
+        store_unit(a, fcu, col, ya * rscale, yb * rscale, fpre);
       }
     }
   }
 }
 
-#ifndef DA_KL
-#define DA_KL 4
-#endif
-#ifndef DA_KF
-#define DA_KF 25
-#endif
-#ifndef DA_THREADS
-#define DA_THREADS 384   // threads of a single-row attention CTA: every key of a ~300-token context has a thread of its own
-#endif
-// Attention of one new row per sequence over the cache (Sec. 3.1): one CTA per (head, sequence).
-// Scores: one key per thread (whole 16-byte-vectorised dot product); P*V: keys dealt round-robin to the
-// eight warps, each lane owning d/32 consecutive dimensions, partial sums combined in warp order.
-template <int DPL, int NT>      // dimensions per lane = head_dim / 32; threads of the CTA
-__device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc, const bf16* vc, bf16* out,
-                                                      int pos, int max_seq, int H, int h, int b, float* dsm, float* red,
-                                                      int cps = 1, const unsigned char* hidden_keys = nullptr) {
-  constexpr int d = 32 * DPL;
-  constexpr int NW = NT / 32;
-  float* qs = dsm;                 // [d]
-  float* p = dsm + d;              // [max_seq]
-  float* part = p + max_seq;       // [NW][d]
+constexpr int DS_THREADS = 128;          // threads of a single-row attention CTA
+constexpr int DS_SMEM_MAX = 200 * 1024;  // dynamic shared memory of a CTA at most
+
+struct DecAttnArgs {
+  const bf16 *q, *kc, *vc;               // q: [cols][H d]; caches of this layer: [sequences][max_seq][H d]
+  float *parts_o, *parts_ml;             // [cols][H][ns][d] unnormalised outputs; [cols][H][ns][2] (max score, sum of exponentials)
+  int pos, max_seq, H, cps, ns, kps;     // kps: keys per split
+  const unsigned char* hidden_keys;      // [sequences][max_seq] positions removed from the sequence, or NULL
+};
+
+__host__ __device__ constexpr int ds_row_bytes(int d) { return 2 * d + 16; }   // a cached row in shared memory; the pad spreads rows over the banks
+static size_t ds_smem_bytes(int d, int kps) {
+  return (size_t)2 * kps * ds_row_bytes(d) + sizeof(float) * (size_t)(d + kps + DS_THREADS * 2);
+}
+
+// Attention of one new row per sequence over the cache (Sec. 3.1), keys split over `ns` CTAs per (head, query row) so
+// that a single sequence still covers the GPU.  A CTA copies its slice of K and V (rows of earlier positions: written
+// before this pass began, hence fetched ahead of the dependency wait) to shared memory, takes the scores one key per
+// thread, and leaves an unnormalised partial output with its maximum and sum; the output projection combines the
+// splits while it stages its input.
+template <int DPL>      // dimensions per lane = head_dim / 32
+__global__ void __launch_bounds__(DS_THREADS) decode_attention_split_kernel(DecAttnArgs a) {
+  extern __shared__ __align__(16) unsigned char ds_raw[];
+  __shared__ float red[DS_THREADS / 32];
+  constexpr int d = 32 * DPL, RS = ds_row_bytes(d), CPR = d / 8;
+  constexpr int NW = DS_THREADS / 32, NG = DS_THREADS / (d / 2);   // warps; key groups of the P V phase
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int h = blockIdx.x, b = blockIdx.y, sp = blockIdx.z;
   // cps > 1: query column b is one row of an action chunk of cps rows at positions pos .. pos + cps - 1 of
   // sequence b / cps, and sees the prompt and the whole chunk
-  const int D = H * d, nkeys = pos + cps;
-  const int sb = b / cps;
-  const float scale = rsqrtf((float)d);
-  // (q may have been written by another SM earlier in the same kernel: read it past the L1)
+  const int D = a.H * d, nkeys = a.pos + a.cps, sb = b / a.cps;
+  const int j0 = sp * a.kps, j1 = min(nkeys, j0 + a.kps), n = max(j1 - j0, 0);
+  unsigned char* Ks = ds_raw;
+  unsigned char* Vs = Ks + (size_t)a.kps * RS;
+  float* qs = reinterpret_cast<float*>(Vs + (size_t)a.kps * RS);   // [d]
+  float* ps = qs + d;                                              // [kps]
+  float* acc = ps + a.kps;                                         // [NG][d]
+  const bf16* kbase = a.kc + (size_t)sb * a.max_seq * D + h * d;
+  const bf16* vbase = a.vc + (size_t)sb * a.max_seq * D + h * d;
+  const unsigned ks_u = (unsigned)__cvta_generic_to_shared(Ks), vs_u = (unsigned)__cvta_generic_to_shared(Vs);
+  auto fetch = [&](int ja, int jb) {                               // rows [ja, jb) of K and of V, 16 bytes per copy
+    const int cnt = max(jb - ja, 0) * CPR;
+    for (int i = tid; i < 2 * cnt; i += DS_THREADS) {
+      const int which = i >= cnt, rem = i - which * cnt, r = ja - j0 + rem / CPR, c = rem % CPR;
+      cp_async16((which ? vs_u : ks_u) + (unsigned)(r * RS + c * 16), (which ? vbase : kbase) + (size_t)(j0 + r) * D + c * 8);
+    }
+  };
+  pdl_trigger();
+  fetch(j0, min(j1, a.pos));                                       // rows of earlier passes and of the prefill
+  cp_async_commit();
+  pdl_wait();
+  fetch(max(j0, a.pos), j1);                                       // rows the projection just before this kernel wrote
+  cp_async_commit();
   if (tid < d) {
-    const unsigned short raw = __ldcg(reinterpret_cast<const unsigned short*>(q) + (size_t)b * D + h * d + tid);
-    qs[tid] = __uint_as_float((unsigned)raw << 16) * scale;
+    const unsigned short raw = __ldcg(reinterpret_cast<const unsigned short*>(a.q) + (size_t)b * D + h * d + tid);
+    qs[tid] = __uint_as_float((unsigned)raw << 16) * rsqrtf((float)d);
   }
+  cp_async_wait<0>();
   __syncthreads();
-  const bf16* kbase = kc + (size_t)sb * max_seq * D + h * d;
   float mx = -INFINITY;
-  for (int j = tid; j < nkeys; j += NT) {
-    const uint4* kp = reinterpret_cast<const uint4*>(kbase + (size_t)j * D);
+  for (int j = tid; j < n; j += DS_THREADS) {
+    const uint4* kr = reinterpret_cast<const uint4*>(Ks + (size_t)j * RS);
     float dot = 0.f;
 #pragma unroll
-    for (int c0 = 0; c0 < d / 8; c0 += DA_KL) {                // DA_KL 16-byte loads in flight at a time
-      uint4 raw[DA_KL];
-#pragma unroll
-      for (int c = 0; c < DA_KL; ++c) raw[c] = kp[min(c0 + c, d / 8 - 1)];
-#pragma unroll
-      for (int c = 0; c < DA_KL; ++c) {
-        if (c0 + c >= d / 8) break;
-        const bf16* kb = reinterpret_cast<const bf16*>(&raw[c]);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) dot += qs[(c0 + c) * 8 + e] * bf2f(kb[e]);
-      }
+    for (int c = 0; c < CPR; ++c) {
+      const uint4 raw = kr[c];
+      const float4 q0 = *reinterpret_cast<const float4*>(qs + c * 8), q1 = *reinterpret_cast<const float4*>(qs + c * 8 + 4);
+      const __nv_bfloat162* k2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+      const float2 f0 = __bfloat1622float2(k2[0]), f1 = __bfloat1622float2(k2[1]), f2 = __bfloat1622float2(k2[2]), f3 = __bfloat1622float2(k2[3]);
+      dot += q0.x * f0.x; dot += q0.y * f0.y; dot += q0.z * f1.x; dot += q0.w * f1.y;
+      dot += q1.x * f2.x; dot += q1.y * f2.y; dot += q1.z * f3.x; dot += q1.w * f3.y;
     }
-    if (hidden_keys && hidden_keys[(size_t)sb * max_seq + j]) dot = -INFINITY;      // position removed from the sequence
-    p[j] = dot;
+    if (a.hidden_keys && a.hidden_keys[(size_t)sb * a.max_seq + j0 + j]) dot = -INFINITY;      // position removed from the sequence
+    ps[j] = dot;
     mx = fmaxf(mx, dot);
   }
 #pragma unroll
@@ -644,68 +724,82 @@ __device__ __noinline__ void decode_attention_body(const bf16* q, const bf16* kc
   mx = red[0];
 #pragma unroll
   for (int w = 1; w < NW; ++w) mx = fmaxf(mx, red[w]);
+  float* out_o = a.parts_o + ((size_t)(b * a.H + h) * a.ns + sp) * d;
+  float* out_ml = a.parts_ml + ((size_t)(b * a.H + h) * a.ns + sp) * 2;
+  if (mx == -INFINITY) {                                           // no visible key in this split (the same in every thread)
+    if (tid < d) out_o[tid] = 0.f;
+    if (tid == 0) { out_ml[0] = -INFINITY; out_ml[1] = 0.f; }
+    return;
+  }
   float sum = 0.f;
-  for (int j = tid; j < nkeys; j += NT) { const float e = __expf(p[j] - mx); p[j] = e; sum += e; }
+  for (int j = tid; j < n; j += DS_THREADS) { const float e = __expf(ps[j] - mx); ps[j] = e; sum += e; }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-  __syncthreads();
+  __syncthreads();                                                 // red read by everyone; ps complete
   if (lane == 0) red[warp] = sum;
-  __syncthreads();
-  float tot = 0.f;
-#pragma unroll
-  for (int w = 0; w < NW; ++w) tot += red[w];
-  const float inv = 1.f / tot;
-  // P * V
-  const bf16* vbase = vc + (size_t)sb * max_seq * D + h * d + lane * DPL;
-  float acc[DPL];
-#pragma unroll
-  for (int e = 0; e < DPL; ++e) acc[e] = 0.f;
-  constexpr int KF = DA_KF;                                      // keys of this warp in flight
-  for (int j0 = warp; j0 < nkeys; j0 += NW * KF) {
-    float pj[KF];
-    __align__(8) bf16 vv[KF][DPL];
-#pragma unroll
-    for (int u = 0; u < KF; ++u) {
-      const int j = j0 + NW * u;
-      pj[u] = j < nkeys ? p[j] : 0.f;
-      const bf16* vp = vbase + (size_t)min(j, nkeys - 1) * D;
-      if (DPL == 4) *reinterpret_cast<uint2*>(vv[u]) = *reinterpret_cast<const uint2*>(vp);
-      else if (DPL == 2) *reinterpret_cast<unsigned*>(vv[u]) = *reinterpret_cast<const unsigned*>(vp);
-      else {
-#pragma unroll
-        for (int e = 0; e < DPL; ++e) vv[u][e] = vp[e];
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < KF; ++u)
-#pragma unroll
-      for (int e = 0; e < DPL; ++e) acc[e] += pj[u] * bf2f(vv[u][e]);
+  // P V: a thread owns two neighbouring dimensions and every NG-th key
+  const int dp = tid % (d / 2), kg = tid / (d / 2);
+  float a0 = 0.f, a1 = 0.f;
+  for (int j = kg; j < n; j += NG) {
+    const float p = ps[j];
+    const float2 v = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(Vs + (size_t)j * RS + dp * 4));
+    a0 += p * v.x; a1 += p * v.y;
   }
-#pragma unroll
-  for (int e = 0; e < DPL; ++e) part[warp * d + lane * DPL + e] = acc[e];
+  acc[kg * d + 2 * dp] = a0; acc[kg * d + 2 * dp + 1] = a1;
   __syncthreads();
   if (tid < d) {
     float o = 0.f;
 #pragma unroll
-    for (int w = 0; w < NW; ++w) o += part[w * d + tid];
-    out[(size_t)b * D + h * d + tid] = __float2bfloat16(o * inv);
+    for (int g = 0; g < NG; ++g) o += acc[g * d + tid];
+    out_o[tid] = o;
+  }
+  if (tid == 0) {
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < NW; ++w) tot += red[w];
+    out_ml[0] = mx; out_ml[1] = tot;
   }
 }
 
-template <int DPL>
-__global__ void __launch_bounds__(DA_THREADS) decode_attention_kernel(const bf16* q, const bf16* kc, const bf16* vc, bf16* out,
-                                                                      int pos, int max_seq, int H, int cps, const unsigned char* hidden_keys) {
-  extern __shared__ float dsm[];
-  __shared__ float red[DA_THREADS / 32];
-  pdl_trigger();
-  pdl_wait();
-  decode_attention_body<DPL, DA_THREADS>(q, kc, vc, out, pos, max_seq, H, blockIdx.x, blockIdx.y, dsm, red, cps, hidden_keys);
+// Key splits of the single-row attention for `cols` query rows over `nkeys` keys: enough CTAs to cover the GPU, and
+// slices small enough for shared memory; 0 if even the largest split count does not fit.
+static int ds_splits(const vlac_ctx* ctx, int cols, int nkeys, int* kps_out) {
+  const int d = ctx->cfg.head_dim;
+  int want = ctx->n_sm / (ctx->cfg.n_heads * cols);
+  int ns = 1;
+  while (ns * 2 <= want && ns * 2 <= DS_MAX_SPLITS) ns *= 2;
+  for (; ns <= DS_MAX_SPLITS; ns *= 2) {
+    const int kps = (nkeys + ns - 1) / ns;
+    if (ds_smem_bytes(d, kps) <= (size_t)DS_SMEM_MAX) { *kps_out = kps; return ns; }
+  }
+  return 0;
+}
+
+static int launch_decode_attention(vlac_ctx* ctx, const bf16* kc, const bf16* vc, int cols, int cps, int pos, const unsigned char* hk,
+                                   int* ns_out, cudaStream_t s) {
+  const vlac_config& g = ctx->cfg;
+  DecAttnArgs a = {};
+  a.q = ctx->q_dec; a.kc = kc; a.vc = vc; a.parts_o = ctx->da_o; a.parts_ml = ctx->da_ml;
+  a.pos = pos; a.max_seq = ctx->max_seq; a.H = g.n_heads; a.cps = cps; a.hidden_keys = hk;
+  a.ns = ds_splits(ctx, cols, pos + cps, &a.kps);
+  if (a.ns == 0) return VLAC_ERR_INVALID_ARG;
+  const size_t smem = ds_smem_bytes(g.head_dim, a.kps);
+  const dim3 grid(g.n_heads, cols, a.ns);
+  cudaError_t e;
+  if (g.head_dim == 64) e = launch_pdl(decode_attention_split_kernel<2>, grid, dim3(DS_THREADS), smem, s, a);
+  else e = launch_pdl(decode_attention_split_kernel<4>, grid, dim3(DS_THREADS), smem, s, a);
+  VLAC_CUDA_CHECK(e);
+  VLAC_LAUNCH_CHECK(ctx);
+  *ns_out = a.ns;
+  return VLAC_OK;
 }
 
 __global__ void __launch_bounds__(256) embed_token_kernel(const bf16* embed, const int* tokens, int tok_stride, int tok_index,
                                                           float* x, int D, int vocab) {
   const int b = blockIdx.x;
-  pdl_trigger();
+  // First kernel of a pass, and deliberately without an early launch of its dependents: when it ends, every kernel
+  // before it has ended, so the kernels of this pass may read what earlier passes wrote (cached K/V rows) ahead of
+  // their own dependency wait.
   pdl_wait();
   int id = tokens[(size_t)b * tok_stride + tok_index];
   id = min(max(id, 0), vocab - 1);
@@ -715,8 +809,7 @@ __global__ void __launch_bounds__(256) embed_token_kernel(const bf16* embed, con
 // input of an action chunk decoded in parallel: column c starts from placeholder embedding c % n
 __global__ void __launch_bounds__(256) embed_chunk_kernel(const bf16* act_embed, int n, float* x, int D) {
   const int c = blockIdx.x;
-  pdl_trigger();
-  pdl_wait();
+  pdl_wait();                                                      // (no early launch of dependents: see embed_token_kernel)
   for (int k = threadIdx.x; k < D; k += blockDim.x) x[(size_t)c * D + k] = bf2f(act_embed[(size_t)(c % n) * D + k]);
 }
 
@@ -779,7 +872,9 @@ int launch_gemv(vlac_ctx* ctx, const GemvArgs& a, cudaStream_t s) {
   const bool timed = ctx->prof_on && ctx->prof_n < VLAC_PROF_CAP;
   if (timed) VLAC_CUDA_CHECK(cudaEventRecord(ctx->prof_ev[2 * ctx->prof_n], s));
   const size_t gt_smem = gt_smem_bytes(ctx, a);
-  if (a.K % 64 == 0 && nb <= 8 && gt_smem <= GT_SMEM_MAX) {
+  const bool mma_path = a.K % 64 == 0 && nb <= 8 && gt_smem <= GT_SMEM_MAX;
+  if (a.parts_o && !mma_path) return VLAC_ERR_INVALID_ARG;       // (vlac_decode_setup refuses such shapes)
+  if (mma_path) {
     if (nb > 4) VLAC_CUDA_CHECK(launch_pdl(gemv_mma_kernel<true>, dim3(ctx->n_sm * GT_GRID_PER_SM), dim3(GT_THREADS), gt_smem, s, a));
     else VLAC_CUDA_CHECK(launch_pdl(gemv_mma_kernel<false>, dim3(ctx->n_sm * GT_GRID_PER_SM), dim3(GT_THREADS), gt_smem, s, a));
   } else
@@ -802,14 +897,15 @@ int launch_gemv(vlac_ctx* ctx, const GemvArgs& a, cudaStream_t s) {
 // over slices of K, each adding its part to x_out in stream order (RESID with a bf16 input only; the slices are
 // multiples of 64 columns of 16-byte aligned rows).
 int launch_gemv_sliced(vlac_ctx* ctx, const GemvArgs& a, cudaStream_t s) {
-  if (a.mode == GV_RESID && a.x_bf16 && !a.ld && a.K % 64 == 0 && gt_smem_bytes(ctx, a) > GT_SMEM_MAX) {
+  if (a.mode == GV_RESID && (a.x_bf16 || a.parts_o) && !a.ld && a.K % 64 == 0 && gt_smem_bytes(ctx, a) > GT_SMEM_MAX) {
     for (int n = 2; n <= 4; n *= 2) {
       if (a.K % (64 * n)) continue;
       GemvArgs h = a;
       h.K = a.K / n; h.ld = a.K;
       if (gt_smem_bytes(ctx, h) > GT_SMEM_MAX) continue;
       for (int i = 0; i < n; ++i) {
-        h.w0 = a.w0 + (size_t)i * h.K; h.x_bf16 = a.x_bf16 + (size_t)i * h.K;
+        h.w0 = a.w0 + (size_t)i * h.K; h.col0 = i * h.K;
+        if (a.x_bf16) h.x_bf16 = a.x_bf16 + (size_t)i * h.K;
         const int rc = launch_gemv(ctx, h, s);
         if (rc) return rc;
       }
@@ -838,6 +934,18 @@ int vlac_decode_setup(vlac_ctx* ctx) {
   if (NB >= 8) VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_pair_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(8 * (size_t)kmax * 2)));
   VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_mma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GT_SMEM_MAX));
   VLAC_CUDA_CHECK(cudaFuncSetAttribute(gemv_mma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)GT_SMEM_MAX));
+  VLAC_CUDA_CHECK(cudaFuncSetAttribute(decode_attention_split_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, DS_SMEM_MAX));
+  VLAC_CUDA_CHECK(cudaFuncSetAttribute(decode_attention_split_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, DS_SMEM_MAX));
+  // the single-row attention hands its key splits to the output projection, which must therefore run on the
+  // tensor-core matrix-vector kernel (whole, or over 2 or 4 slices of K), and the longest sequence must fit the splits
+  {
+    const int D = ctx->cfg.hidden, cols = NB;
+    bool fits = false;
+    for (int n = 1; n <= 4 && !fits; n *= 2)
+      fits = D % (64 * n) == 0 && (size_t)GT_RING_BYTES + GT_PART_BYTES + (size_t)cols * (D / n + GT_XPAD) * sizeof(bf16) <= GT_SMEM_MAX;
+    int kps = 0;
+    if (!fits || ds_splits(ctx, 1, ctx->max_seq, &kps) == 0) return VLAC_ERR_INVALID_ARG;
+  }
   return VLAC_OK;
 }
 
@@ -862,7 +970,7 @@ static void layer_phases(vlac_ctx* ctx, vlac_cache* c, int l, int pos, GemvArgs*
   a.rope_cos = ctx->w.rope_cos; a.rope_sin = ctx->w.rope_sin;
   a.pos = pos; a.max_seq = ctx->max_seq; a.d = g.head_dim;
   GemvArgs o = {};
-  o.x_bf16 = ctx->ao_dec; o.w0 = (const bf16*)w.wo; o.mode = GV_RESID; o.nb = B; o.K = D; o.N = D; o.x_out = ctx->x_dec; o.d = g.head_dim;
+  o.parts_o = ctx->da_o; o.parts_ml = ctx->da_ml; o.ns = 1; o.w0 = (const bf16*)w.wo; o.mode = GV_RESID; o.nb = B; o.K = D; o.N = D; o.x_out = ctx->x_dec; o.d = g.head_dim;
   GemvArgs gu = {};
   gu.x_f32 = ctx->x_dec; gu.gain = (const bf16*)w.g_mlp; gu.eps = g.rms_eps;
   gu.w0 = (const bf16*)w.w_gate; gu.w1 = (const bf16*)w.w_up; gu.mode = GV_SWIGLU; gu.nb = B; gu.K = D; gu.N = F;
@@ -893,17 +1001,9 @@ int vlac_launch_decode_pass(vlac_ctx* ctx, vlac_cache* c, const int* fed_tokens,
     int rc = launch_gemv(ctx, ph[0], s);
     if (rc) return rc;
     {
-      const size_t smem = (size_t)(g.head_dim + ctx->max_seq + (DA_THREADS / 32) * g.head_dim) * sizeof(float);
-      const dim3 grid(g.n_heads, B);
-      const bf16 *q = ctx->q_dec, *kc = ph[0].kc, *vc = ph[0].vc;
       const unsigned char* hk = (ctx->prune_layer > 0 && l >= ctx->prune_layer) ? c->hidden_keys : nullptr;
-      cudaError_t e;
-      switch (g.head_dim / 32) {
-        case 2: e = launch_pdl(decode_attention_kernel<2>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, 1, hk); break;
-        default: e = launch_pdl(decode_attention_kernel<4>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, 1, hk); break;
-      }
-      VLAC_CUDA_CHECK(e);
-      VLAC_LAUNCH_CHECK(ctx);
+      rc = launch_decode_attention(ctx, ph[0].kc, ph[0].vc, B, 1, pos, hk, &ph[1].ns, s);
+      if (rc) return rc;
     }
     for (int k = 1; k < 4; ++k) {
       rc = launch_gemv_sliced(ctx, ph[k], s);
@@ -932,19 +1032,8 @@ int vlac_launch_chunk_pass(vlac_ctx* ctx, vlac_cache* c, const void* act_embed, 
       ph[0].vc += (size_t)b * kv_layer_elems(ctx);
       int rc = launch_gemv(ctx, ph[0], s);
       if (rc) return rc;
-      {
-        const size_t smem = (size_t)(g.head_dim + ctx->max_seq + (DA_THREADS / 32) * g.head_dim) * sizeof(float);
-        const dim3 grid(g.n_heads, n);
-        const bf16 *q = ctx->q_dec, *kc = ph[0].kc, *vc = ph[0].vc;
-        const int pos = ctx->L;
-        cudaError_t e;
-        switch (g.head_dim / 32) {
-          case 2: e = launch_pdl(decode_attention_kernel<2>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, n, (const unsigned char*)nullptr); break;
-          default: e = launch_pdl(decode_attention_kernel<4>, grid, dim3(DA_THREADS), smem, s, q, kc, vc, ctx->ao_dec, pos, ctx->max_seq, g.n_heads, n, (const unsigned char*)nullptr); break;
-        }
-        VLAC_CUDA_CHECK(e);
-        VLAC_LAUNCH_CHECK(ctx);
-      }
+      rc = launch_decode_attention(ctx, ph[0].kc, ph[0].vc, n, n, ctx->L, nullptr, &ph[1].ns, s);
+      if (rc) return rc;
       for (int k = 1; k < 4; ++k) {
         rc = launch_gemv_sliced(ctx, ph[k], s);
         if (rc) return rc;

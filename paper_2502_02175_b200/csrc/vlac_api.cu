@@ -48,7 +48,7 @@ int fill_params(const vlac_ctx* ctx, const vlac_select_params* in, int force_ful
 
 void free_ctx_buffers(vlac_ctx* c) {
   cudaFree(c->xn); cudaFree(c->q); cudaFree(c->ao); cudaFree(c->hm); cudaFree(c->part); cudaFree(c->tc_ws); cudaFree(c->tc_cnt);
-  cudaFree(c->probs); cudaFree(c->hidden); cudaFree(c->x_dec); cudaFree(c->q_dec); cudaFree(c->ao_dec);
+  cudaFree(c->probs); cudaFree(c->hidden); cudaFree(c->x_dec); cudaFree(c->q_dec); cudaFree(c->da_o); cudaFree(c->da_ml);
   cudaFree(c->hm_dec); cudaFree(c->logits); cudaFree(c->argmax_tmp); cudaFree(c->dev_error); cudaFree(c->tmap_q); cudaFree(c->probs_all); free(c->tmaps_host);
   cudaFree(c->in_frames); cudaFree(c->in_feats); cudaFree(c->in_ids); cudaFree(c->in_forced); cudaFree(c->out_tokens); cudaFree(c->logits_all);
   for (int i = 0; i < VLAC_MAX_GRAPHS; ++i) if (c->graphs[i].used) cudaGraphExecDestroy(c->graphs[i].exec);
@@ -137,7 +137,8 @@ int vlac_create(const vlac_config* cfg, const vlac_weights* w, vlac_ctx** out) {
   if (rc == VLAC_OK) rc = dev_alloc(&c->hidden, R * D);
   if (rc == VLAC_OK) rc = dev_alloc(&c->x_dec, R1 * D);
   if (rc == VLAC_OK) rc = dev_alloc(&c->q_dec, R1 * D);
-  if (rc == VLAC_OK) rc = dev_alloc(&c->ao_dec, R1 * D);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->da_o, R1 * D * 8);
+  if (rc == VLAC_OK) rc = dev_alloc(&c->da_ml, R1 * (size_t)g.n_heads * 8 * 2);
   if (rc == VLAC_OK) rc = dev_alloc(&c->hm_dec, R1 * F);
   if (rc == VLAC_OK) rc = dev_alloc(&c->logits, R1 * (size_t)g.vocab);
   if (rc == VLAC_OK) rc = dev_alloc(&c->argmax_tmp, R1 * VLAC_ARGMAX_BLOCKS);

@@ -58,7 +58,8 @@ struct vlac_ctx {
   float *hidden;                     // [max_batch][L][hidden] fp32 residual stream of a whole step
   // single-row buffers: one row per column of the matrix-vector kernels, R1 = max(max_batch, min(n_action, 8))
   float *x_dec;                      // [R1][hidden]
-  bf16 *q_dec, *ao_dec, *hm_dec;     // [R1][hidden] x2, [R1][ffn]
+  bf16 *q_dec, *hm_dec;              // [R1][hidden], [R1][ffn]
+  float *da_o, *da_ml;               // single-row attention per key split: [R1][n_heads][8][head_dim] outputs, [R1][n_heads][8][2] (max, sum)
   float *logits;                     // [R1][vocab]
   unsigned long long *argmax_tmp;    // [R1][VLAC_ARGMAX_BLOCKS]
   int *dev_error;                    // device ints: [0] nonzero if a bounded wait gave up
