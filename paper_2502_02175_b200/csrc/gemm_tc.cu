@@ -507,18 +507,49 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
         int c_first = (int)((lo * G) / total);
         while (c_first + 1 < G && range_begin(total, c_first + 1, G) <= lo) ++c_first;
         while (c_first > 0 && range_begin(total, c_first, G) > lo) --c_first;
+        // the slots of the first four contributors, worked out once per tile: inside the token loop all their loads are
+        // then issued together (the loop is a chain of L2 round trips otherwise, and it is the tail of the launch)
+        const float* base[4] = {nullptr, nullptr, nullptr, nullptr};
+        int nsrc = 0;
+        for (int c = c_first; c < G && range_begin(total, c, G) < hi; ++c) ++nsrc;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int c = min(c_first + i, G - 1);
+          base[i] = a.ws + ((size_t)(c * 2 + (range_begin(total, c, G) >= lo ? 0 : 1)) * n_chunks + ch) * slot_floats;
+        }
         for (int g0 = team * 16; g0 < tokens; g0 += 32) {
           const int t = g0 + t_b;
           if (t >= tokens) continue;
           float x1[8], x2[8];
 #pragma unroll
           for (int i = 0; i < 8; ++i) x1[i] = x2[i] = 0.f;
-          for (int c = c_first; c < G && range_begin(total, c, G) < hi; ++c) {
-            const int which = range_begin(total, c, G) >= lo ? 0 : 1;
-            const float* src = a.ws + ((size_t)(c * 2 + which) * n_chunks + ch) * slot_floats + (size_t)t * 128;
-            const float4 p0 = ldcg_f4(src + r1), p1 = ldcg_f4(src + r1 + 4), p2 = ldcg_f4(src + r1 + e.half), p3 = ldcg_f4(src + r1 + e.half + 4);
-            x1[0] += p0.x; x1[1] += p0.y; x1[2] += p0.z; x1[3] += p0.w; x1[4] += p1.x; x1[5] += p1.y; x1[6] += p1.z; x1[7] += p1.w;
-            x2[0] += p2.x; x2[1] += p2.y; x2[2] += p2.z; x2[3] += p2.w; x2[4] += p3.x; x2[5] += p3.y; x2[6] += p3.z; x2[7] += p3.w;
+          float4 pv[4][4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            if (i < nsrc) {
+              const float* src = base[i] + (size_t)t * 128;
+              pv[i][0] = ldcg_f4(src + r1); pv[i][1] = ldcg_f4(src + r1 + 4); pv[i][2] = ldcg_f4(src + r1 + e.half); pv[i][3] = ldcg_f4(src + r1 + e.half + 4);
+            }
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            if (i < nsrc) {
+              x1[0] += pv[i][0].x; x1[1] += pv[i][0].y; x1[2] += pv[i][0].z; x1[3] += pv[i][0].w;
+              x1[4] += pv[i][1].x; x1[5] += pv[i][1].y; x1[6] += pv[i][1].z; x1[7] += pv[i][1].w;
+              x2[0] += pv[i][2].x; x2[1] += pv[i][2].y; x2[2] += pv[i][2].z; x2[3] += pv[i][2].w;
+              x2[4] += pv[i][3].x; x2[5] += pv[i][3].y; x2[6] += pv[i][3].z; x2[7] += pv[i][3].w;
+            }
+          }
+          if (nsrc > 4) {                                          // further contributors (short shares of k-blocks), still in k order
+            int c = c_first;
+            for (int k = 0; k < 4; ++k) ++c;
+            for (; c < G && range_begin(total, c, G) < hi; ++c) {
+              const int which = range_begin(total, c, G) >= lo ? 0 : 1;
+              const float* src = a.ws + ((size_t)(c * 2 + which) * n_chunks + ch) * slot_floats + (size_t)t * 128;
+              const float4 p0 = ldcg_f4(src + r1), p1 = ldcg_f4(src + r1 + 4), p2 = ldcg_f4(src + r1 + e.half), p3 = ldcg_f4(src + r1 + e.half + 4);
+              x1[0] += p0.x; x1[1] += p0.y; x1[2] += p0.z; x1[3] += p0.w; x1[4] += p1.x; x1[5] += p1.y; x1[6] += p1.z; x1[7] += p1.w;
+              x2[0] += p2.x; x2[1] += p2.y; x2[2] += p2.z; x2[3] += p2.w; x2[4] += p3.x; x2[5] += p3.y; x2[6] += p3.z; x2[7] += p3.w;
+            }
           }
           emit8(e, x1, x2, r1, (size_t)(tok0 + t), a.rowmap ? rows_s[t] : 0);
         }
