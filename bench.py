@@ -219,7 +219,7 @@ def run_reference(args):
     from paper_2502_02175_b200 import synth
     K, W = max(1, args.steps), max(0, args.warmup)
     full = _workload(args.layers)
-    sec_per_layer = 125.0 / 32.0                                 # a 32-layer step of the checker measured on this machine's hosts
+    sec_per_layer = 125.0 / 32.0                                 # a 32-layer step of the checker takes about two minutes on a 16-core host
     n_s = int(max(1, min(full.n_layers, (240.0 / (K + W)) // sec_per_layer)))
     cfg = _workload(n_s)
     t_setup = time.perf_counter()
