@@ -12,7 +12,9 @@
 // gate/up products give every CTA the same share of ALL k-blocks of the launch (a contiguous range that
 // may begin and end inside a tile), the output / down projections and the vision projector give every
 // CTA one K-split of one tile.  A CTA walks its range segment by segment (tile, k-blocks kb0..kb1) and,
-// with more than 256 tokens, chunk by chunk of tokens.
+// with more than 256 tokens, chunk by chunk of tokens.  Contexts that can meet more than 512 rows (a batch,
+// two cameras) deal (tile, 256-token chunk) pairs to the CTAs instead, so that the CTAs which need the same
+// weight tile read it at the same time.
 //
 // Warp roles (384 threads): one lane each of warps 0, 2 and 3 issues TMA loads into one ring of stages that
 // runs on across segments (a thread gets a tensor load accepted only every ~0.3 us, threads of different
@@ -50,6 +52,10 @@ constexpr int TG_BOX_TOK = 64;                  // token rows per TMA box
 constexpr int TG_BOX_BYTES = TG_BOX_TOK * TG_BK * 2;   // 8 KB
 constexpr int TG_CHUNK = 256;                   // most tokens of a chunk while two accumulator buffers alternate
 constexpr int TG_CHUNK_MAX = 512;               // ... and with one buffer (more than 256 live tokens): all 512 tensor-memory columns
+#ifndef TG_SPREAD_MIN_N
+#define TG_SPREAD_MIN_N 256
+#endif
+constexpr int TG_SPREAD_MIN = TG_SPREAD_MIN_N;  // more live tokens than this: (tile, chunk) pairs are spread over the CTAs
 constexpr int TG_MAX_STAGES = 8;
 constexpr int TG_SMEM_RING = 192 * 1024;        // ring: four stages of 48 KB at 256 tokens
 constexpr int TG_STAGE_OUT = 8192;              // one 16-token chunk of a tile as fp32
@@ -179,10 +185,11 @@ __device__ __forceinline__ uint4 pack8(const float* y) {
 
 // ---- the share of work of one CTA, as a sequence of segments
 struct Seg { int tile, kb0, kb1; bool first; };
-struct Range { long long u0, u1; };
+struct Range { long long u0, u1; int step; };     // step 0: k-blocks u0..u1 of the launch; step > 0: the whole tiles u0, u0 + step, ... < u1
 __device__ __forceinline__ long long range_begin(long long total, int c, int G) { return total * c / G; }
 __device__ __forceinline__ bool next_seg(long long& u, const Range& r, int kbt, Seg& s) {
   if (u >= r.u1) return false;
+  if (r.step > 0) { s.tile = (int)u; s.kb0 = 0; s.kb1 = kbt; s.first = true; u += r.step; return true; }
   s.tile = (int)(u / kbt);
   s.kb0 = (int)(u - (long long)s.tile * kbt);
   const long long left = r.u1 - u;
@@ -235,6 +242,11 @@ __device__ __forceinline__ void emit8(const EmitCtx& e, const float* x1, const f
   *reinterpret_cast<uint4*>(dst + n2) = pack8(y2);
 }
 
+// MULTI: the instantiation for contexts that can meet more than 512 recomputed rows (a batch, two cameras); it differs
+// only in the schedule described at `spread` below.  (A single 290-position sequence recomputed in full is faster on
+// the k-block-sharing schedule with one 512-column accumulator: 96 and 172 tiles in two chunks balance badly.)  The single-sequence instantiation is kept free of that logic:
+// the kernel sits at its register limit and the k-loop's code is sensitive to what else is live.
+template <bool MULTI>
 __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_constant__ TcArgs a) {
   extern __shared__ __align__(1024) unsigned char ring_raw[];
   __shared__ __align__(8) unsigned long long full_bar[TG_MAX_STAGES], empty_bar[TG_MAX_STAGES], acc_full[2], acc_empty[2];
@@ -269,8 +281,14 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
   const int T = a.tot ? *a.tot : a.tot_fixed;
   // Up to 256 live tokens: one chunk, two accumulator buffers, the epilogue of a segment overlaps the next one's MMAs.
   // More: chunks of up to 512 tokens in one buffer (half as many passes over the weights as 256-token chunks need).
-  const int cap = T <= TG_CHUNK ? TG_CHUNK : TG_CHUNK_MAX;
-  const int n_bufs = T <= TG_CHUNK ? 2 : 1;
+  // MULTI and more than 256: the k-block-sharing launches deal (tile, 256-token chunk) pairs instead.  CTA c owns chunk
+  // c % n_chunks of the tiles c / n_chunks, c / n_chunks + slots, ...: the CTAs that need the same weight tile ask for
+  // it at the same time, so it crosses HBM once and comes out of L2 for the others (a CTA that walks the chunks of
+  // its tiles one after the other re-reads every tile from HBM per chunk: measured 6 x the weight bytes at 2320
+  // tokens), every segment covers all of K (no raw tiles, no fold) and the two accumulators alternate.
+  const bool spread = MULTI && a.mode != TG_PARTIAL && T > TG_SPREAD_MIN && (T + TG_CHUNK - 1) / TG_CHUNK <= (int)gridDim.x;
+  const int cap = (T <= TG_CHUNK || spread) ? TG_CHUNK : TG_CHUNK_MAX;
+  const int n_bufs = cap == TG_CHUNK ? 2 : 1;
   const int n_chunks = (T + cap - 1) / cap;
   const int chunk_sz = n_chunks > 0 ? (((T + n_chunks - 1) / n_chunks + 15) / 16) * 16 : 0;     // tokens of every chunk but the last
   const int max_boxes = (chunk_sz + TG_BOX_TOK - 1) / TG_BOX_TOK;
@@ -289,6 +307,13 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
   } else {
     rg.u0 = range_begin(total, (int)blockIdx.x, G);
     rg.u1 = range_begin(total, (int)blockIdx.x + 1, G);
+  }
+  rg.step = 0;
+  int ch_lo = 0, ch_hi = n_chunks;                                // token chunks this CTA works on
+  if (MULTI && spread) {
+    const int slots = G / n_chunks, slot = (int)blockIdx.x / n_chunks;
+    ch_lo = (int)blockIdx.x % n_chunks; ch_hi = ch_lo + 1;
+    rg.step = slots; rg.u0 = slot; rg.u1 = slot < slots ? a.n_tiles : slot;       // (CTAs beyond the last full group of chunks stay idle)
   }
   if (T <= 0) rg.u1 = rg.u0;
   const int tiles_per_mat = (a.N + 127) / 128;
@@ -317,7 +342,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
   {
     long long u = rg.u0; Seg sg; int it = 0;
     while (it < n_stages && next_seg(u, rg, kbt, sg))
-      for (int ch = 0; ch < n_chunks && it < n_stages; ++ch)
+      for (int ch = ch_lo; ch < ch_hi && it < n_stages; ++ch)
         for (int kb = sg.kb0; kb < sg.kb1 && it < n_stages; ++kb, ++it) {
           if (producer && it % n_prod == pid) {
             asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(&full_bar[it])), "r"((unsigned)TG_A_BYTES) : "memory");
@@ -346,7 +371,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
     if (producer) {
       long long u = rg.u0; Seg sg; int it = 0; bool ok = true;
       while (ok && next_seg(u, rg, kbt, sg))
-        for (int ch = 0; ch < n_chunks && ok; ++ch) {
+        for (int ch = ch_lo; ch < ch_hi && ok; ++ch) {
           const int boxes = (chunk_tokens(ch) + TG_BOX_TOK - 1) / TG_BOX_TOK;
           const unsigned x_bytes = (unsigned)(boxes * TG_BOX_BYTES);
           for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
@@ -371,7 +396,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
     if (lane == 0) {
       long long u = rg.u0; Seg sg; int it = 0, item = 0; bool ok = true;
       while (ok && next_seg(u, rg, kbt, sg))
-        for (int ch = 0; ch < n_chunks && ok; ++ch, ++item) {
+        for (int ch = ch_lo; ch < ch_hi && ok; ++ch, ++item) {
           const int b = n_bufs == 2 ? item & 1 : 0, use = n_bufs == 2 ? item >> 1 : item;
           if (use > 0) ok = mbar_wait(&acc_empty[b], (use - 1) & 1, &abort_flag, a.dev_error, 0x58000 | (item & 0x7fff));
           if (!ok) break;
@@ -439,7 +464,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
       const bool direct = whole || a.mode == TG_PARTIAL;         // results leave in their final form straight from the accumulator
       e.mat = tile_mat(sg.tile); e.row_base = tile_row_base(sg.tile);
       const int split = a.mode == TG_PARTIAL ? (int)blockIdx.x % a.n_splits : 0;
-      for (int ch = 0; ch < n_chunks && ok; ++ch, ++item) {
+      for (int ch = ch_lo; ch < ch_hi && ok; ++ch, ++item) {
         const int b = n_bufs == 2 ? item & 1 : 0, use = n_bufs == 2 ? item >> 1 : item;
         const int tok0 = ch * chunk_sz, tokens = chunk_tokens(ch);
         int* rows_s = n_bufs == 2 ? rows_buf[item & 1] : rows_buf[0];
@@ -658,7 +683,8 @@ int vlac_tc_setup(vlac_ctx* ctx) {
     if (e1 != cudaSuccess) { cudaGetLastError(); free(host); return e1 == cudaErrorMemoryAllocation ? VLAC_ERR_OOM : VLAC_ERR_CUDA; }
   }
   ctx->tmaps_host = host;                                        // copied into the kernel parameters at every launch
-  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TG_SMEM_DYN);
+  cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, TG_SMEM_DYN);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, TG_SMEM_DYN);
   if (e != cudaSuccess) { vlac_note_cuda_error(e, __FILE__, __LINE__); return VLAC_ERR_CUDA; }
   // a CTA holds up to 512 tokens (accumulator columns); more tokens are further chunks along grid.z
   return VLAC_OK;
@@ -679,7 +705,9 @@ static int launch_tc(vlac_ctx* ctx, TcArgs& a, cudaStream_t s) {
   int grid = a.mode == TG_PARTIAL ? a.n_tiles * a.n_splits : (int)(total < ctx->n_sm ? total : ctx->n_sm);
   a.tmem_cols = tc_tmem_cols(ctx);
   a.ws = ctx->tc_ws; a.tile_cnt = ctx->tc_cnt;
-  VLAC_CUDA_CHECK(launch_pdl(gemm_tc_kernel, dim3(grid), dim3(TG_THREADS), (size_t)TG_SMEM_DYN, s, a));
+  // the instantiation with the spread schedule for contexts that can meet more than 512 rows
+  if (ctx->rows_max > TG_CHUNK_MAX) VLAC_CUDA_CHECK(launch_pdl(gemm_tc_kernel<true>, dim3(grid), dim3(TG_THREADS), (size_t)TG_SMEM_DYN, s, a));
+  else VLAC_CUDA_CHECK(launch_pdl(gemm_tc_kernel<false>, dim3(grid), dim3(TG_THREADS), (size_t)TG_SMEM_DYN, s, a));
   VLAC_LAUNCH_CHECK(ctx);
   return VLAC_OK;
 }
