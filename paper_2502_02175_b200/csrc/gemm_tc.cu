@@ -84,6 +84,7 @@ struct alignas(64) TcArgs {
   bf16* h_out;                    // SWIGLU: [T][N]
   float* ws;                      // raw sums of segments that cover part of K: [cta][2][token chunk][256][128]
   int* tile_cnt;                  // [tile][token chunk] k-blocks accumulated so far (zero between launches)
+  int partial_spread;             // PARTIAL over whole K (n_splits == 1) with (tile, chunk) pairs dealt to the CTAs of a full grid
   int tmem_cols;                  // tensor-memory columns to allocate (two buffers; power of two >= 32)
   int* dev_error;
 };
@@ -286,7 +287,7 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
   // it at the same time, so it crosses HBM once and comes out of L2 for the others (a CTA that walks the chunks of
   // its tiles one after the other re-reads every tile from HBM per chunk: measured 6 x the weight bytes at 2320
   // tokens), every segment covers all of K (no raw tiles, no fold) and the two accumulators alternate.
-  const bool spread = MULTI && a.mode != TG_PARTIAL && T > TG_SPREAD_MIN && (T + TG_CHUNK - 1) / TG_CHUNK <= (int)gridDim.x;
+  const bool spread = MULTI && (a.mode != TG_PARTIAL ? T > TG_SPREAD_MIN : a.partial_spread != 0) && (T + TG_CHUNK - 1) / TG_CHUNK <= (int)gridDim.x;
   const int cap = (T <= TG_CHUNK || spread) ? TG_CHUNK : TG_CHUNK_MAX;
   const int n_bufs = cap == TG_CHUNK ? 2 : 1;
   const int n_chunks = (T + cap - 1) / cap;
@@ -300,10 +301,11 @@ __global__ void __launch_bounds__(TG_THREADS, 1) gemm_tc_kernel(const __grid_con
   Range rg;
   const long long total = (long long)a.n_tiles * kbt;
   const int G = (int)gridDim.x;
-  if (a.mode == TG_PARTIAL) {                                    // blockIdx.x = tile * n_splits + split
+  if (a.mode == TG_PARTIAL && !spread) {                         // blockIdx.x = tile * n_splits + split
     const int tile = (int)blockIdx.x / a.n_splits, split = (int)blockIdx.x - tile * a.n_splits;
     rg.u0 = (long long)tile * kbt + ((long long)kbt * split) / a.n_splits;
     rg.u1 = (long long)tile * kbt + ((long long)kbt * (split + 1)) / a.n_splits;
+    if (tile >= a.n_tiles) rg.u1 = rg.u0;                          // (a grid larger than tiles x splits: nothing to do)
   } else {
     rg.u0 = range_begin(total, (int)blockIdx.x, G);
     rg.u1 = range_begin(total, (int)blockIdx.x + 1, G);
@@ -702,7 +704,7 @@ static int tc_tmem_cols(const vlac_ctx* ctx) {
 // grid: one CTA per K-split of a tile (PARTIAL), else one per SM sharing all k-blocks evenly
 static int launch_tc(vlac_ctx* ctx, TcArgs& a, cudaStream_t s) {
   const long long total = (long long)a.n_tiles * ((a.K + TG_BK - 1) / TG_BK);
-  int grid = a.mode == TG_PARTIAL ? a.n_tiles * a.n_splits : (int)(total < ctx->n_sm ? total : ctx->n_sm);
+  int grid = (a.mode == TG_PARTIAL && !a.partial_spread) ? a.n_tiles * a.n_splits : (int)(total < ctx->n_sm ? total : ctx->n_sm);
   a.tmem_cols = tc_tmem_cols(ctx);
   a.ws = ctx->tc_ws; a.tile_cnt = ctx->tc_cnt;
   // the instantiation with the spread schedule for contexts that can meet more than 512 rows
@@ -759,6 +761,10 @@ int vlac_tc_partial(vlac_ctx* ctx, vlac_cache* c, int layer, int which, int* n_s
   a.K = down ? g.ffn : g.hidden; a.N = g.hidden; a.mode = TG_PARTIAL;
   a.n_tiles = (g.hidden + 127) / 128;
   a.n_splits = tc_splits(ctx, a.n_tiles, a.K);
+  // A batch whose text rows alone (always recomputed) exceed 256 live rows: whole-K tiles with (tile, 256-token chunk)
+  // pairs dealt to a full grid, ONE partial for the fold kernel to read instead of four, and a weight tile's readers
+  // running together (five chunks walked one after the other by a K-split's CTA re-read it from HBM).
+  if (ctx->rows_max > TG_CHUNK_MAX && c->batch * (g.n_text_pre + g.n_text_post) > TG_CHUNK) { a.n_splits = 1; a.partial_spread = 1; }
   a.part = ctx->part; a.split_stride = (size_t)ctx->rows_max * g.hidden;
   *n_splits = a.n_splits;
   return launch_tc(ctx, a, s);
