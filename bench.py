@@ -63,7 +63,31 @@ class ClockSampler:
     def __init__(self, index: int):
         self.index, self.samples, self.stop_flag, self.thread = index, [], False, None
 
+    def _run_nvml(self) -> bool:
+        """Read-only NVML queries every 20 ms (an nvidia-smi process per sample yields one or two samples per timed region)."""
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            h = nv.nvmlDeviceGetHandleByIndex(self.index)
+            mx = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+            bits = (("hw_slowdown", nv.nvmlClocksThrottleReasonHwSlowdown), ("hw_thermal_slowdown", nv.nvmlClocksThrottleReasonHwThermalSlowdown),
+                    ("sw_thermal_slowdown", nv.nvmlClocksThrottleReasonSwThermalSlowdown), ("sw_power_cap", nv.nvmlClocksThrottleReasonSwPowerCap))
+            nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM); nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+        except Exception:
+            return False
+        while not self.stop_flag:
+            try:
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                self.samples.append([str(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)), str(mx), str(nv.nvmlDeviceGetPowerUsage(h) / 1e3)]
+                                    + ["Active" if r & b else "Not Active" for _, b in bits])
+            except Exception:
+                pass
+            time.sleep(0.02)
+        return True
+
     def _run(self):
+        if self._run_nvml():
+            return
         while not self.stop_flag:
             try:
                 out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-i", str(self.index)],
